@@ -1,0 +1,299 @@
+"""CPU oracle for the bidirectional Mamba-2 mixer of DiffuMamba's denoising step.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, fp64 statement of what the hot path
+computes.  Only the tests, the smoke check and the benchmark's `cpu_baseline` / reference arm may
+import it; the product (the CUDA library and its Python binding) never does, and this file imports
+nothing from the product.
+
+Everything is written token by token, in the order the paper states its model:
+
+  * Sec. 3.2 / App. A.1: a BiMamba block is two independent Mamba layers, one run left-to-right and
+    one right-to-left, fused by addition (Eq. "Mamba(x_i) = h_i-> + h_i<-").
+  * App. C (per-token FLOPs table): one direction is in_proj (d -> D_in), a short depthwise Conv1d
+    over conv_ch channels, the SSM scan with d_state states per channel, and out_proj (d_inner -> d).
+    D_in combines gate, input, B, C and the per-head step size.
+  * Sec. 4.3 (block-autoregressive inference): the left-to-right state is cached and carried from one
+    committed block to the next; the right-to-left pass only sees the active block.
+  * App. A.1: the stack is Embed -> N blocks (pre-norm, residual) -> OutputProj.
+
+The paper does not print the discretisation of the Mamba-2 layer it uses; the reading taken here
+(the usual Mamba-2 one: scalar decay per head, a = exp(Delta * A), input scaled by Delta, B and C
+shared by the heads of a group, depthwise conv then SiLU on [x, B, C], gate by SiLU(z), optional
+RMS normalisation of the gated output) is listed point by point in the design notes.
+
+Parity status: every function below is pinned by tests (explicit sums, closed forms, textbook
+routines, the paper's printed shape / FLOP numbers) except three choices the paper leaves open and
+nothing printed can confirm -- the gated RMS norm inside each direction (both settings are
+implemented and tested), when the carried state is committed, and the stack's plain RMSNorm
+pre-norm without the MLP sublayer.  For those three: parity unpinned (by the paper); they follow
+the stated readings.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------------------------
+# Shapes and the per-token cost table (App. C)
+# --------------------------------------------------------------------------------------------
+
+def derived_dims(d_model: int, expand: int, d_state: int, n_heads: int, n_groups: int = 1) -> dict:
+    """Widths of one direction (App. C: d_inner = expand*d; conv_ch covers x, B and C; D_in adds the
+    gate and one step size per head)."""
+    d_inner = expand * d_model
+    if d_inner % n_heads or n_heads % n_groups:
+        raise ValueError("d_inner must divide into heads, heads into groups")
+    return {
+        "d_inner": d_inner,
+        "headdim": d_inner // n_heads,
+        "conv_ch": d_inner + 2 * n_groups * d_state,
+        "d_in_proj": 2 * d_inner + 2 * n_groups * d_state + n_heads,
+    }
+
+
+def flops_per_token(d_model: int, expand: int, d_state: int, d_conv: int, n_heads: int,
+                    n_groups: int = 1, d_ff: int | None = None, d_c: int = 128) -> dict:
+    """Forward FLOPs per token of one bidirectional Mamba-2 layer, with App. C's counting rules:
+    2mn per linear layer, 2*d_inner*d_state for the scan, conv_ch*d_conv for the conv, twice for the
+    two directions; MLP 4*d*d_ff; AdaLN 2*6d*d_c."""
+    dd = derived_dims(d_model, expand, d_state, n_heads, n_groups)
+    d_ff = 2 * d_model if d_ff is None else d_ff
+    one = {
+        "in_proj": 2 * d_model * dd["d_in_proj"],
+        "conv": dd["conv_ch"] * d_conv,
+        "scan": 2 * dd["d_inner"] * d_state,
+        "out_proj": 2 * dd["d_inner"] * d_model,
+    }
+    one_dir = sum(one.values())
+    out = dict(one)
+    out["one_direction"] = one_dir
+    out["mixer"] = 2 * one_dir
+    out["mlp"] = 4 * d_model * d_ff
+    out["adaln"] = 2 * 6 * d_model * d_c
+    out["layer"] = out["mixer"] + out["mlp"] + out["adaln"]
+    return out
+
+
+def param_count(d_model: int, expand: int, d_state: int, d_conv: int, n_heads: int, n_layers: int,
+                vocab: int, n_groups: int = 1, d_ff: int | None = None, d_c: int = 128) -> int:
+    """Weights of the whole denoiser with two untied directions per layer (App. A.1 "bidirectional
+    weight tie: False"), MLP and AdaLN modulation per layer, untied embedding and unembedding."""
+    dd = derived_dims(d_model, expand, d_state, n_heads, n_groups)
+    d_ff = 2 * d_model if d_ff is None else d_ff
+    one_dir = (d_model * dd["d_in_proj"] + dd["conv_ch"] * d_conv + dd["conv_ch"]
+               + 3 * n_heads + dd["d_inner"] + dd["d_inner"] * d_model)
+    mlp = 2 * d_model * d_ff + d_ff + d_model
+    adaln = 6 * d_model * d_c + 6 * d_model
+    return n_layers * (2 * one_dir + mlp + adaln) + 2 * vocab * d_model + d_model
+
+
+# --------------------------------------------------------------------------------------------
+# Scalar functions
+# --------------------------------------------------------------------------------------------
+
+def softplus(v):
+    v = np.asarray(v, dtype=F64)
+    return np.maximum(v, 0.0) + np.log1p(np.exp(-np.abs(v)))
+
+
+def silu(v):
+    v = np.asarray(v, dtype=F64)
+    with np.errstate(over="ignore"):          # exp(-v) = inf for very negative v gives the limit -0
+        return v / (1.0 + np.exp(-v))
+
+
+# --------------------------------------------------------------------------------------------
+# One direction, step by step (App. C table rows, in order)
+# --------------------------------------------------------------------------------------------
+
+def in_proj(u, w_in):
+    """Row "in_proj": zxBCdt[t] = W_in u[t], W_in [D_in, d], no bias."""
+    return np.asarray(u, F64) @ np.asarray(w_in, F64).T
+
+
+def split_zxbcdt(zxbcdt, d_inner: int, d_state: int, n_heads: int, n_groups: int = 1):
+    """Column order [ z | x | B | C | dt ]; returns z, xBC (x, B, C still joined), dt."""
+    conv_ch = d_inner + 2 * n_groups * d_state
+    z = zxbcdt[..., :d_inner]
+    xbc = zxbcdt[..., d_inner:d_inner + conv_ch]
+    dt = zxbcdt[..., d_inner + conv_ch:]
+    assert dt.shape[-1] == n_heads
+    return z, xbc, dt
+
+
+def causal_conv_silu(xbc, conv_w, conv_b=None, conv_state=None):
+    """Row "Conv1d": depthwise filter of width k over each channel, looking only at the current and
+    the k-1 previous rows, then SiLU.  Tap k-1 multiplies the current row.  Rows before the start are
+    zero, or the carried conv_state [k-1, conv_ch] (the k-1 rows that preceded this call).
+    Returns (activated [L, conv_ch], new conv_state = last k-1 pre-conv rows seen)."""
+    xbc = np.asarray(xbc, F64)
+    conv_w = np.asarray(conv_w, F64)
+    L, ch = xbc.shape
+    k = conv_w.shape[1]
+    hist = np.zeros((k - 1, ch), F64) if conv_state is None else np.asarray(conv_state, F64)
+    assert hist.shape == (k - 1, ch)
+    padded = np.concatenate([hist, xbc], axis=0)          # row i of xbc is padded[i + k - 1]
+    out = np.empty((L, ch), F64)
+    for t in range(L):
+        v = np.zeros(ch, F64) if conv_b is None else np.asarray(conv_b, F64).copy()
+        for j in range(k):
+            v += conv_w[:, j] * padded[t + j]              # padded[t + j] = xbc[t - (k-1) + j]
+        out[t] = silu(v)
+    return out, padded[L:L + k - 1].copy()
+
+
+def discretise(dt_raw, dt_bias, A_log):
+    """Step size and decay per token and head: Delta = softplus(dt + bias), A = -exp(A_log) < 0,
+    a = exp(Delta * A) in (0, 1)."""
+    delta = softplus(np.asarray(dt_raw, F64) + np.asarray(dt_bias, F64))
+    A = -np.exp(np.asarray(A_log, F64))
+    return delta, np.exp(delta * A)
+
+
+def ssm_recurrence(x, delta, a, Bm, Cm, D=None, h0=None):
+    """Row "SSM scan" (Sec. 3.2, first recurrence): for t = 0..L-1
+
+        h_t = a_t * h_{t-1} + Delta_t * x_t (outer) B_t        h: [H, P, N]
+        y_t = h_t C_t + D * x_t                                 (state after the update)
+
+    x [L,H,P]; delta, a [L,H]; Bm, Cm [L,G,N] with heads h*G//H sharing a group; D [H] or None;
+    h0 [H,P,N] or None (zeros).  Returns y [L,H,P] and the final state."""
+    x = np.asarray(x, F64)
+    L, H, P = x.shape
+    G, N = Bm.shape[1], Bm.shape[2]
+    rep = H // G
+    h = np.zeros((H, P, N), F64) if h0 is None else np.array(h0, F64)
+    y = np.empty((L, H, P), F64)
+    for t in range(L):
+        Bt = np.repeat(np.asarray(Bm[t], F64), rep, axis=0)     # [H, N]
+        Ct = np.repeat(np.asarray(Cm[t], F64), rep, axis=0)
+        h = a[t][:, None, None] * h + (delta[t][:, None] * x[t])[:, :, None] * Bt[:, None, :]
+        y[t] = np.einsum("hpn,hn->hp", h, Ct)
+        if D is not None:
+            y[t] += np.asarray(D, F64)[:, None] * x[t]
+    return y, h
+
+
+def gate(y, z, norm_w=None, eps: float = 1e-5, gated_norm: bool = True):
+    """g = y * SiLU(z); with gated_norm, g <- g / sqrt(mean_c g^2 + eps) * norm_w over the d_inner
+    channels of each token (Sec. 3.2 "normalized ... before" the output projection)."""
+    g = np.asarray(y, F64) * silu(z)
+    if gated_norm:
+        ms = np.mean(g * g, axis=-1, keepdims=True)
+        g = g / np.sqrt(ms + eps)
+        if norm_w is not None:
+            g = g * np.asarray(norm_w, F64)
+    return g
+
+
+def out_proj(g, w_out):
+    """Row "out_proj": out[t] = W_out g[t], W_out [d, d_inner], no bias."""
+    return np.asarray(g, F64) @ np.asarray(w_out, F64).T
+
+
+def mamba2_direction(u, w: dict, *, expand: int, d_state: int, n_heads: int, n_groups: int = 1,
+                     gated_norm: bool = True, conv_bias: bool = True, d_skip: bool = True,
+                     norm_eps: float = 1e-5, ssm_state=None, conv_state=None, return_parts: bool = False):
+    """One left-to-right Mamba-2 layer over u [L, d].  Returns (out [L,d], ssm_state_out [H,P,N],
+    conv_state_out [k-1, conv_ch])."""
+    u = np.asarray(u, F64)
+    L, d = u.shape
+    dd = derived_dims(d, expand, d_state, n_heads, n_groups)
+    d_inner, P = dd["d_inner"], dd["headdim"]
+    zxbcdt = in_proj(u, w["w_in"])
+    z, xbc, dt = split_zxbcdt(zxbcdt, d_inner, d_state, n_heads, n_groups)
+    xbc_act, conv_out = causal_conv_silu(xbc, w["conv_w"], w["conv_b"] if conv_bias else None, conv_state)
+    xs = xbc_act[:, :d_inner].reshape(L, n_heads, P)
+    Bm = xbc_act[:, d_inner:d_inner + n_groups * d_state].reshape(L, n_groups, d_state)
+    Cm = xbc_act[:, d_inner + n_groups * d_state:].reshape(L, n_groups, d_state)
+    delta, a = discretise(dt, w["dt_bias"], w["A_log"])
+    y, h_last = ssm_recurrence(xs, delta, a, Bm, Cm, w["D"] if d_skip else None, ssm_state)
+    g = gate(y.reshape(L, d_inner), z, w.get("norm_w"), norm_eps, gated_norm)
+    out = out_proj(g, w["w_out"])
+    if return_parts:
+        return out, h_last, conv_out, {"zxbcdt": zxbcdt, "xbc_act": xbc_act, "delta": delta, "a": a,
+                                       "y": y.reshape(L, d_inner), "g": g}
+    return out, h_last, conv_out
+
+
+# --------------------------------------------------------------------------------------------
+# The bidirectional mixer (Sec. 3.2) and its block-cache form (Sec. 4.3)
+# --------------------------------------------------------------------------------------------
+
+DIR_FWD, DIR_REV, DIR_BOTH = 1, 2, 3
+
+
+def bimamba_forward(x, w_fwd: dict, w_rev: dict, *, dir_mask: int = DIR_BOTH, **kw):
+    """Mamba(x) = h-> + h<- for x [B, L, d].  The right-to-left layer is the same operator applied
+    to the sequence in reverse order (second recurrence of Sec. 3.2: i = L..1, anti-causal conv):
+    flip, run, flip back.  dir_mask selects one direction only (for invariants)."""
+    x = np.asarray(x, F64)
+    out = np.zeros_like(x)
+    for b in range(x.shape[0]):
+        if dir_mask & DIR_FWD:
+            out[b] += mamba2_direction(x[b], w_fwd, **kw)[0]
+        if dir_mask & DIR_REV:
+            out[b] += mamba2_direction(x[b][::-1], w_rev, **kw)[0][::-1]
+    return out
+
+
+def bimamba_block_step(x_blk, w_fwd: dict, w_rev: dict, *, ssm_state_in=None, conv_state_in=None,
+                       dir_mask: int = DIR_BOTH, **kw):
+    """One pass over the active block x_blk [B, G, d] (Sec. 4.3): the left-to-right layer starts from
+    the carried (ssm, conv) state of the committed prefix; the right-to-left layer starts from zero
+    and sees the block only.  Returns (y_blk, ssm_state_out [B,H,P,N], conv_state_out [B,k-1,conv_ch]):
+    the left-to-right state after the block's last token."""
+    x_blk = np.asarray(x_blk, F64)
+    out = np.zeros_like(x_blk)
+    ssm_out, conv_out = [], []
+    for b in range(x_blk.shape[0]):
+        s_in = None if ssm_state_in is None else ssm_state_in[b]
+        c_in = None if conv_state_in is None else conv_state_in[b]
+        o, s, c = mamba2_direction(x_blk[b], w_fwd, ssm_state=s_in, conv_state=c_in, **kw)
+        ssm_out.append(s)
+        conv_out.append(c)
+        if dir_mask & DIR_FWD:
+            out[b] += o
+        if dir_mask & DIR_REV:
+            out[b] += mamba2_direction(x_blk[b][::-1], w_rev, **kw)[0][::-1]
+    return out, np.stack(ssm_out), np.stack(conv_out)
+
+
+# --------------------------------------------------------------------------------------------
+# The layer stack (App. A.1: Embed -> blocks -> OutputProj), mixer sublayer with RMSNorm pre-norm
+# --------------------------------------------------------------------------------------------
+
+def rmsnorm(r, w, eps: float = 1e-5):
+    r = np.asarray(r, F64)
+    return r / np.sqrt(np.mean(r * r, axis=-1, keepdims=True) + eps) * np.asarray(w, F64)
+
+
+def denoise_step(tokens, sw: dict, *, rms_eps: float = 1e-5, states_in=None, return_states: bool = False,
+                 return_hidden: bool = False, **kw):
+    """logits[b,t,:] = W_vocab RMSNorm(r_N[b,t]); r_0 = E[tokens]; r_{l+1} = r_l + BiMamba_l(RMSNorm(r_l)).
+    With states_in (one (ssm, conv) pair per layer, or None entries) every layer runs as a block step.
+    Returns logits [B, L, V] (and the per-layer states after the block when return_states)."""
+    tokens = np.asarray(tokens)
+    r = np.asarray(sw["embed"], F64)[tokens]                   # [B, L, d]
+    states_out = []
+    hidden = [r.copy()]
+    for i, layer in enumerate(sw["layers"]):
+        u = rmsnorm(r, layer["norm_w"], rms_eps)
+        if states_in is None and not return_states:
+            m = bimamba_forward(u, layer["fwd"], layer["rev"], **kw)
+        else:
+            s_in, c_in = (None, None) if states_in is None or states_in[i] is None else states_in[i]
+            m, s_out, c_out = bimamba_block_step(u, layer["fwd"], layer["rev"], ssm_state_in=s_in,
+                                                 conv_state_in=c_in, **kw)
+            states_out.append((s_out, c_out))
+        r = r + m
+        hidden.append(r.copy())
+    logits = rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T
+    res = (logits,)
+    if return_states:
+        res += (states_out,)
+    if return_hidden:
+        res += (hidden,)
+    return res[0] if len(res) == 1 else res
