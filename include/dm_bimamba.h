@@ -1,0 +1,171 @@
+/*
+ * dm_bimamba.h -- C ABI of the B200 (sm_100a) bidirectional Mamba-2 mixer used as the denoiser
+ * backbone of a masked-diffusion language model (DiffuMamba, Sec. 3.2 and App. A.1).
+ *
+ * General rules for every entry point
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer owned by the caller.
+ *     The structs themselves (configs, weight tables, state tables) live in HOST memory and are read
+ *     during the call only; the library keeps no pointer after the call returns.
+ *   - All tensors are dense, row-major, contiguous.  Matrices are [out_features, in_features].
+ *   - `dtype` selects the storage type of activations, matrices, conv parameters, norm weights and the
+ *     conv state (DM_F32 or DM_BF16).  Accumulation is always fp32; per-head scalars (dt_bias, A_log, D)
+ *     and the SSM state are always fp32.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the default stream)
+ *     and the call returns without synchronising.  The library allocates no device memory: scratch
+ *     comes from the caller's `workspace` (query its size first; 256-byte aligned).
+ *   - Return value: DM_OK (0) or a negative dm_status.  Arguments are checked before anything is
+ *     launched; a rejected call has no effect.  dm_last_error_message() gives a text for the last
+ *     failure on the calling thread.
+ *   - Column order of one direction's in_proj output (App. C, "D_in"):
+ *         [ z : d_inner | x : d_inner | B : n_groups*d_state | C : n_groups*d_state | dt : n_heads ].
+ *     conv_ch = d_inner + 2*n_groups*d_state channels (x, B, C) pass through the depthwise conv.
+ */
+#ifndef DM_BIMAMBA_H_
+#define DM_BIMAMBA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DM_OK = 0,
+    DM_ERR_INVALID_ARG = -1,   /* NULL pointer, non-positive size, misaligned pointer, aliasing states */
+    DM_ERR_UNSUPPORTED = -2,   /* a shape the kernels do not cover (see dm_mixer_cfg) */
+    DM_ERR_WORKSPACE = -3,     /* workspace NULL, misaligned or smaller than the queried size */
+    DM_ERR_CUDA = -4,          /* a CUDA runtime call failed (launch configuration, driver) */
+    DM_ERR_TIMEOUT = -5        /* a bounded device-side wait gave up (reported by dm_check) */
+} dm_status;
+
+enum { DM_F32 = 0, DM_BF16 = 1 };
+enum { DM_FLAG_GATED_RMSNORM = 1, DM_FLAG_CONV_BIAS = 2, DM_FLAG_D_SKIP = 4 };
+enum { DM_DIR_FWD = 1, DM_DIR_REV = 2, DM_DIR_BOTH = 3 };
+
+/* Sizes of one mixer call, in the paper's notation (Sec. 3.2: x in R^{B x L x d}; App. A.1
+ * hyper-parameter table: expansion factor, state dimension, conv dimension; App. C: heads via D_in).
+ * Supported: d_conv in [2,4]; n_groups == 1; headdim = expand*d_model/n_heads in {32, 64};
+ * d_state in {16, 32, 64, 128, 256} with headdim*d_state/16 <= 1024.  Other shapes return
+ * DM_ERR_UNSUPPORTED. */
+typedef struct {
+    int32_t batch;      /* B */
+    int32_t seqlen;     /* L; for dm_bimamba_block_step the length G of the active block */
+    int32_t d_model;    /* d */
+    int32_t expand;     /* d_inner = expand * d_model */
+    int32_t d_state;    /* N, states per channel */
+    int32_t d_conv;     /* k, width of the depthwise conv */
+    int32_t n_heads;    /* H; the decay and step size are scalars per head */
+    int32_t n_groups;   /* groups sharing B and C */
+    int32_t dtype;      /* DM_F32 | DM_BF16 */
+    int32_t flags;      /* DM_FLAG_* */
+    int32_t dir_mask;   /* DM_DIR_BOTH; one direction alone is meant for invariant tests */
+    int32_t chunk;      /* tokens per scan chunk; 0 = library default.  Results do not depend on it
+                           beyond rounding order. */
+    float   norm_eps;   /* epsilon of the gated RMS norm */
+} dm_mixer_cfg;
+
+/* One direction's parameters (the two directions are untied: App. A.1 "bidirectional weight tie: False"). */
+typedef struct {
+    const void  *w_in;     /* [d_in_proj, d_model]  dtype */
+    const void  *conv_w;   /* [conv_ch, d_conv]     dtype; tap d_conv-1 multiplies the current token */
+    const void  *conv_b;   /* [conv_ch]             dtype; ignored unless DM_FLAG_CONV_BIAS */
+    const float *dt_bias;  /* [n_heads] */
+    const float *A_log;    /* [n_heads]; A = -exp(A_log) */
+    const float *D;        /* [n_heads]; ignored unless DM_FLAG_D_SKIP */
+    const void  *norm_w;   /* [d_inner] dtype; ignored unless DM_FLAG_GATED_RMSNORM */
+    const void  *w_out;    /* [d_model, d_inner]    dtype */
+} dm_dir_weights;
+
+typedef struct {
+    const void    *norm_w;     /* [d_model] dtype: RMSNorm pre-norm weight of the layer */
+    dm_dir_weights dir[2];     /* [0] left-to-right, [1] right-to-left */
+} dm_layer_weights;
+
+typedef struct {
+    dm_mixer_cfg mixer;        /* batch/seqlen describe the token tensor of the step */
+    int32_t n_layers;
+    int32_t vocab;             /* rows of embed and w_vocab */
+    float   rms_eps;
+} dm_stack_cfg;
+
+typedef struct {
+    const void             *embed;         /* [vocab, d_model] dtype */
+    const dm_layer_weights *layers;        /* HOST array of n_layers entries */
+    const void             *final_norm_w;  /* [d_model] dtype */
+    const void             *w_vocab;       /* [vocab, d_model] dtype */
+} dm_stack_weights;
+
+/* Carried state of one layer in block mode (Sec. 4.3): only the left-to-right direction has one.
+ * *_in == NULL means zeros (no prefix yet); *_out == NULL means "do not commit".  in and out must not
+ * be the same buffer. */
+typedef struct {
+    const float *ssm_in;    /* [B, H, P, N] fp32 */
+    const void  *conv_in;   /* [B, d_conv-1, conv_ch] dtype: the d_conv-1 pre-conv rows before the block */
+    float       *ssm_out;
+    void        *conv_out;
+} dm_layer_state;
+
+/* Text for a status code (static storage, never NULL). */
+const char *dm_status_string(int status);
+
+/* Text describing the last failure on the calling thread (static thread-local storage). */
+const char *dm_last_error_message(void);
+
+/* Scratch sizes in bytes for the calls below with the same configuration. */
+int dm_bimamba_workspace_bytes(const dm_mixer_cfg *cfg, size_t *bytes);
+int dm_denoise_workspace_bytes(const dm_stack_cfg *cfg, size_t *bytes);
+
+/* Synchronises `cuda_stream` and returns the deferred device status (DM_OK, DM_ERR_TIMEOUT when a
+ * bounded wait inside a kernel expired, DM_ERR_CUDA for a sticky CUDA error).  Clears the status. */
+int dm_check(void *cuda_stream);
+
+/* The bidirectional mixer, Sec. 3.2:  y = Mamba(x) = h-> + h<-  for x [B, L, d_model].
+ * Each direction is a complete Mamba-2 layer (App. C table): in_proj, depthwise conv + SiLU over
+ * (x,B,C), Delta = softplus(dt + dt_bias), a = exp(Delta*A), the recurrence
+ * h_t = a_t h_{t-1} + Delta_t x_t (x) B_t,  y_t = h_t C_t + D x_t, gate by SiLU(z) (then the gated
+ * RMS norm when flagged), out_proj.  The right-to-left layer runs the same operator over the
+ * sequence in reverse order (anti-causal conv, recurrence from t = L-1 down to 0).
+ *   w[0], w[1]: left-to-right and right-to-left parameters.   x, y: [B, L, d_model] dtype; y != x. */
+int dm_bimamba_forward(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
+                       const void *x, void *y,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* One pass over the active block in block-autoregressive decoding, Sec. 4.3: cfg->seqlen = G.
+ * The left-to-right layer starts from the carried state of the committed prefix (ssm_state_in,
+ * conv_state_in; NULL = zeros) and, when the *_out pointers are given, writes the state after the
+ * block's last token.  The right-to-left layer starts from zero and sees the block only.
+ *   x_blk, y_blk: [B, G, d_model] dtype.  conv_state_out holds the last d_conv-1 rows of
+ *   concat(conv_state_in, pre-conv xBC of the block) -- exact copies, also when G < d_conv-1. */
+int dm_bimamba_block_step(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
+                          const void *x_blk,
+                          const float *ssm_state_in, const void *conv_state_in,
+                          float *ssm_state_out, void *conv_state_out,
+                          void *y_blk,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* One denoising step of the layer stack, App. A.1:  z = OutputProj(B_N(... B_1(E(x_t)))) with
+ * r_0 = E[tokens], r_{l+1} = r_l + Mamba_l(RMSNorm(r_l) * norm_w_l), logits = W_vocab (RMSNorm(r_N) * w_f).
+ *   tokens: [B, L] int32 ids in [0, vocab).   logits: [B, L, vocab] dtype, or NULL.
+ *   argmax_out: [B, L] int32 = index of the largest logit (lowest index on ties), or NULL.
+ *   states: HOST array of n_layers entries, or NULL for full-sequence denoising; when given, every
+ *   layer runs as dm_bimamba_block_step with that layer's state pointers. */
+int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights,
+                    const int32_t *tokens, void *logits, int32_t *argmax_out,
+                    const dm_layer_state *states,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Same as dm_bimamba_forward, but x and y are HOST buffers (pageable or pinned): the call copies x to
+ * the device, runs the mixer and copies y back, all on `cuda_stream`, then synchronises it.
+ * `workspace` must hold dm_bimamba_workspace_bytes + 2*B*L*d_model*sizeof(dtype) bytes. */
+int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
+                            const void *x_host, void *y_host,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Number of kernels this library has launched from this process since load (for benchmarks). */
+uint64_t dm_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DM_BIMAMBA_H_ */

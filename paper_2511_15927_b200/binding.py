@@ -1,0 +1,175 @@
+"""Thin ctypes binding of libdm_bimamba.so: argument marshalling only.
+
+Every function here has the name and the arguments of the C entry point it calls (see
+include/dm_bimamba.h).  Device buffers are passed as integer addresses (`tensor.data_ptr()`), host
+buffers likewise; this module never computes anything and there is no fallback: if the compiled
+library is missing, importing the module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdm_bimamba.so")
+
+DM_OK, DM_ERR_INVALID_ARG, DM_ERR_UNSUPPORTED, DM_ERR_WORKSPACE, DM_ERR_CUDA, DM_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+DM_F32, DM_BF16 = 0, 1
+DM_FLAG_GATED_RMSNORM, DM_FLAG_CONV_BIAS, DM_FLAG_D_SKIP = 1, 2, 4
+DM_DIR_FWD, DM_DIR_REV, DM_DIR_BOTH = 1, 2, 3
+DM_FLAGS_DEFAULT = DM_FLAG_GATED_RMSNORM | DM_FLAG_CONV_BIAS | DM_FLAG_D_SKIP
+
+
+class dm_mixer_cfg(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("batch", "seqlen", "d_model", "expand", "d_state", "d_conv", "n_heads",
+                                         "n_groups", "dtype", "flags", "dir_mask", "chunk")] + [("norm_eps", C.c_float)]
+
+
+class dm_dir_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_in", "conv_w", "conv_b", "dt_bias", "A_log", "D", "norm_w", "w_out")]
+
+
+class dm_layer_weights(C.Structure):
+    _fields_ = [("norm_w", C.c_void_p), ("dir", dm_dir_weights * 2)]
+
+
+class dm_stack_cfg(C.Structure):
+    _fields_ = [("mixer", dm_mixer_cfg), ("n_layers", C.c_int32), ("vocab", C.c_int32), ("rms_eps", C.c_float)]
+
+
+class dm_stack_weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("layers", C.POINTER(dm_layer_weights)), ("final_norm_w", C.c_void_p),
+                ("w_vocab", C.c_void_p)]
+
+
+class dm_layer_state(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ssm_in", "conv_in", "ssm_out", "conv_out")]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2511_15927_b200.build` "
+                      "(or __graft_entry__.build()); there is no fallback path")
+_lib = C.CDLL(LIB_PATH)
+
+_vp, _sz = C.c_void_p, C.c_size_t
+_lib.dm_status_string.restype = C.c_char_p
+_lib.dm_status_string.argtypes = [C.c_int]
+_lib.dm_last_error_message.restype = C.c_char_p
+_lib.dm_last_error_message.argtypes = []
+_lib.dm_kernel_launch_count.restype = C.c_uint64
+_lib.dm_kernel_launch_count.argtypes = []
+_lib.dm_bimamba_workspace_bytes.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(_sz)]
+_lib.dm_denoise_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(_sz)]
+_lib.dm_check.argtypes = [_vp]
+_lib.dm_bimamba_forward.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp, _sz, _vp]
+_lib.dm_bimamba_forward_host.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp, _sz, _vp]
+_lib.dm_bimamba_block_step.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp, _vp, _vp, _vp,
+                                       _vp, _sz, _vp]
+_lib.dm_denoise_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_stack_weights), _vp, _vp, _vp,
+                                 C.POINTER(dm_layer_state), _vp, _sz, _vp]
+for _f in ("dm_bimamba_workspace_bytes", "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward",
+           "dm_bimamba_forward_host", "dm_bimamba_block_step", "dm_denoise_step"):
+    getattr(_lib, _f).restype = C.c_int
+
+EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
+           "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
+           "dm_bimamba_block_step", "dm_denoise_step")
+
+
+class DmError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"{dm_status_string(status)} ({status}): {dm_last_error_message()}")
+
+
+def _ok(status: int) -> None:
+    if status != DM_OK:
+        raise DmError(status)
+
+
+def dm_status_string(status: int) -> str:
+    return _lib.dm_status_string(int(status)).decode()
+
+
+def dm_last_error_message() -> str:
+    return _lib.dm_last_error_message().decode()
+
+
+def dm_kernel_launch_count() -> int:
+    return int(_lib.dm_kernel_launch_count())
+
+
+def dm_bimamba_workspace_bytes(cfg: dm_mixer_cfg) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_bimamba_workspace_bytes(C.byref(cfg), C.byref(n)))
+    return int(n.value)
+
+
+def dm_denoise_workspace_bytes(cfg: dm_stack_cfg) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_denoise_workspace_bytes(C.byref(cfg), C.byref(n)))
+    return int(n.value)
+
+
+def dm_check(cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_check(_vp(cuda_stream)))
+
+
+def _dirs(w) -> C.Array:
+    arr = (dm_dir_weights * 2)()
+    for i in range(2):
+        arr[i] = w[i]
+    return arr
+
+
+def dm_bimamba_forward(cfg, w, x: int, y: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_bimamba_forward(C.byref(cfg), _dirs(w), _vp(x), _vp(y), _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_bimamba_forward_host(cfg, w, x_host: int, y_host: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_bimamba_forward_host(C.byref(cfg), _dirs(w), _vp(x_host), _vp(y_host), _vp(workspace), _sz(workspace_bytes),
+                                     _vp(cuda_stream)))
+
+
+def dm_bimamba_block_step(cfg, w, x_blk: int, ssm_state_in: int, conv_state_in: int, ssm_state_out: int,
+                          conv_state_out: int, y_blk: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_bimamba_block_step(C.byref(cfg), _dirs(w), _vp(x_blk), _vp(ssm_state_in or None), _vp(conv_state_in or None),
+                                   _vp(ssm_state_out or None), _vp(conv_state_out or None), _vp(y_blk), _vp(workspace),
+                                   _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_denoise_step(cfg, weights, tokens: int, logits: int, argmax_out: int, states, workspace: int,
+                    workspace_bytes: int, cuda_stream: int = 0) -> None:
+    """`states`: None, or a ctypes array (dm_layer_state * n_layers)."""
+    _ok(_lib.dm_denoise_step(C.byref(cfg), C.byref(weights), _vp(tokens), _vp(logits or None), _vp(argmax_out or None),
+                             states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+# ------------------------------------------------------------------------------------------------
+# Marshalling helpers (no arithmetic): build the C structs from shapes and from dicts of tensors.
+# ------------------------------------------------------------------------------------------------
+
+def make_mixer_cfg(batch, seqlen, d_model, expand, d_state, d_conv, n_heads, dtype, n_groups=1,
+                   flags=DM_FLAGS_DEFAULT, dir_mask=DM_DIR_BOTH, chunk=0, norm_eps=1e-5) -> dm_mixer_cfg:
+    return dm_mixer_cfg(batch, seqlen, d_model, expand, d_state, d_conv, n_heads, n_groups, dtype, flags, dir_mask,
+                        chunk, norm_eps)
+
+
+def make_dir_weights(t: dict) -> dm_dir_weights:
+    """t maps the field names of dm_dir_weights to objects with .data_ptr() (device tensors) or None."""
+    return dm_dir_weights(*[(t[n].data_ptr() if t.get(n) is not None else None)
+                            for n in ("w_in", "conv_w", "conv_b", "dt_bias", "A_log", "D", "norm_w", "w_out")])
+
+
+def make_stack_weights(t: dict):
+    """t: {"embed", "w_vocab", "final_norm_w", "layers": [{"norm_w", "fwd": {...}, "rev": {...}}]} of device tensors.
+    Returns (dm_stack_weights, keepalive) -- keep the second object alive while the first is in use."""
+    n = len(t["layers"])
+    arr = (dm_layer_weights * n)()
+    for i, l in enumerate(t["layers"]):
+        arr[i].norm_w = l["norm_w"].data_ptr()
+        arr[i].dir[0] = make_dir_weights(l["fwd"])
+        arr[i].dir[1] = make_dir_weights(l["rev"])
+    sw = dm_stack_weights(t["embed"].data_ptr(), C.cast(arr, C.POINTER(dm_layer_weights)), t["final_norm_w"].data_ptr(),
+                          t["w_vocab"].data_ptr())
+    return sw, arr

@@ -1,0 +1,388 @@
+// C-ABI entry points: argument checks, workspace layout, and the launch sequence of each call.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "dm_internal.h"
+
+namespace dm {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+__device__ int g_device_status;   // 0 = fine; kernels store a dm_status when a bounded wait gives up
+
+int *device_status_ptr() {
+    static int *cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        cached[dev] = static_cast<int *>(p);
+    }
+    return cached[dev];
+}
+
+static thread_local char g_err[512] = "";
+
+static int fail(int status, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+static int cuda_fail(cudaError_t e, const char *what) {
+    if (e == cudaErrorNotSupported) return fail(DM_ERR_UNSUPPORTED, "%s: shape not supported by the kernel", what);
+    return fail(DM_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+struct Dims {
+    int B, L, d, d_inner, H, P, N, k, G, conv_ch, d_in_proj;
+    int64_t T;
+    size_t es;
+};
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_cfg(const dm_mixer_cfg *c, Dims *o) {
+    if (!c) return fail(DM_ERR_INVALID_ARG, "cfg is NULL");
+    if (c->batch <= 0 || c->seqlen <= 0 || c->d_model <= 0 || c->expand <= 0 || c->d_state <= 0 || c->n_heads <= 0)
+        return fail(DM_ERR_INVALID_ARG, "batch, seqlen, d_model, expand, d_state and n_heads must be positive");
+    if (c->dtype != DM_F32 && c->dtype != DM_BF16) return fail(DM_ERR_INVALID_ARG, "dtype must be DM_F32 or DM_BF16");
+    if (c->dir_mask < DM_DIR_FWD || c->dir_mask > DM_DIR_BOTH) return fail(DM_ERR_INVALID_ARG, "dir_mask must be 1, 2 or 3");
+    if (c->flags & ~(DM_FLAG_GATED_RMSNORM | DM_FLAG_CONV_BIAS | DM_FLAG_D_SKIP)) return fail(DM_ERR_INVALID_ARG, "unknown flag bits");
+    if (c->chunk < 0) return fail(DM_ERR_INVALID_ARG, "chunk must be >= 0");
+    if (!(c->norm_eps >= 0.f)) return fail(DM_ERR_INVALID_ARG, "norm_eps must be >= 0");
+    if (c->n_groups != 1) return fail(DM_ERR_UNSUPPORTED, "n_groups must be 1");
+    if (c->d_conv < 2 || c->d_conv > 4) return fail(DM_ERR_UNSUPPORTED, "d_conv must be in [2,4]");
+    const int64_t d_inner = (int64_t)c->expand * c->d_model;
+    if (d_inner % c->n_heads) return fail(DM_ERR_INVALID_ARG, "expand*d_model must be divisible by n_heads");
+    const int P = (int)(d_inner / c->n_heads);
+    if (P != 32 && P != 64) return fail(DM_ERR_UNSUPPORTED, "headdim must be 32 or 64 (got %d)", P);
+    const int N = c->d_state;
+    if (N != 16 && N != 32 && N != 64 && N != 128 && N != 256) return fail(DM_ERR_UNSUPPORTED, "d_state must be 16, 32, 64, 128 or 256");
+    if ((int64_t)P * (N / 16) > 1024) return fail(DM_ERR_UNSUPPORTED, "headdim * d_state / 16 must not exceed 1024");
+    if ((int64_t)c->batch * c->seqlen > (int64_t)1 << 30) return fail(DM_ERR_UNSUPPORTED, "batch*seqlen too large");
+    o->B = c->batch; o->L = c->seqlen; o->d = c->d_model; o->d_inner = (int)d_inner; o->H = c->n_heads; o->P = P;
+    o->N = N; o->k = c->d_conv; o->G = 1;
+    o->conv_ch = o->d_inner + 2 * N;
+    o->d_in_proj = 2 * o->d_inner + 2 * N + o->H;
+    o->T = (int64_t)c->batch * c->seqlen;
+    o->es = dtype_size(c->dtype);
+    return DM_OK;
+}
+
+static int check_weights(const dm_mixer_cfg *c, const dm_dir_weights w[2]) {
+    if (!w) return fail(DM_ERR_INVALID_ARG, "weights are NULL");
+    for (int dir = 0; dir < 2; ++dir) {
+        if (!(c->dir_mask & (1 << dir))) continue;
+        const dm_dir_weights &q = w[dir];
+        if (!q.w_in || !q.conv_w || !q.dt_bias || !q.A_log || !q.w_out) return fail(DM_ERR_INVALID_ARG, "direction %d: NULL weight pointer", dir);
+        if ((c->flags & DM_FLAG_CONV_BIAS) && !q.conv_b) return fail(DM_ERR_INVALID_ARG, "direction %d: conv_b is NULL but DM_FLAG_CONV_BIAS is set", dir);
+        if ((c->flags & DM_FLAG_D_SKIP) && !q.D) return fail(DM_ERR_INVALID_ARG, "direction %d: D is NULL but DM_FLAG_D_SKIP is set", dir);
+        if ((c->flags & DM_FLAG_GATED_RMSNORM) && !q.norm_w) return fail(DM_ERR_INVALID_ARG, "direction %d: norm_w is NULL but DM_FLAG_GATED_RMSNORM is set", dir);
+        if (!aligned16(q.w_in) || !aligned16(q.w_out)) return fail(DM_ERR_INVALID_ARG, "direction %d: matrices must be 16-byte aligned", dir);
+    }
+    return DM_OK;
+}
+
+// Workspace layout of one mixer call.
+struct MixerWs {
+    size_t zx, g, ssq, rstd, ytmp, scan, total;
+};
+
+static MixerWs mixer_ws(const dm_mixer_cfg *c, const Dims &m) {
+    MixerWs w;
+    size_t off = 0;
+    w.zx = off;   off += align_up((size_t)2 * m.T * m.d_in_proj * m.es);
+    w.g = off;    off += align_up((size_t)2 * m.T * m.d_inner * m.es);
+    w.ssq = off;  off += align_up((size_t)2 * m.T * m.H * sizeof(float));
+    w.rstd = off; off += align_up((size_t)2 * m.T * sizeof(float));
+    w.ytmp = off; off += align_up((size_t)m.T * m.d * sizeof(float));
+    ScanArgs sa{};
+    sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
+    sa.d_in_proj = m.d_in_proj; sa.conv_ch = m.conv_ch; sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask;
+    w.scan = off; off += align_up(scan_ssd_workspace_bytes(sa));
+    w.total = off;
+    return w;
+}
+
+static cudaError_t gemm(const GemmArgs &a, cudaStream_t s) {
+    if (gemm_tcgen05_supports(a)) return gemm_tcgen05(a, s);
+    return gemm_simple(a, s);
+}
+
+struct MixerOut {
+    void *y; int y_dtype; const float *addend; int64_t ld_add;
+};
+
+// in_proj -> fused conv/scan/gate -> out_proj of both directions, summed (Sec. 3.2).
+static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights w[2], const void *x, const MixerOut &out,
+                     const float *ssm_in, const void *conv_in, float *ssm_out, void *conv_out,
+                     char *ws, cudaStream_t s) {
+    const MixerWs l = mixer_ws(c, m);
+    char *zx = ws + l.zx, *g = ws + l.g;
+    float *ssq = reinterpret_cast<float *>(ws + l.ssq), *rstd = reinterpret_cast<float *>(ws + l.rstd);
+    float *ytmp = reinterpret_cast<float *>(ws + l.ytmp);
+    const bool norm_on = (c->flags & DM_FLAG_GATED_RMSNORM) != 0;
+    cudaError_t e;
+
+    for (int dir = 0; dir < 2; ++dir) {
+        if (!(c->dir_mask & (1 << dir))) continue;
+        GemmArgs a{};
+        a.A = x; a.lda = m.d; a.B = w[dir].w_in; a.ldb = m.d;
+        a.C = zx + (size_t)dir * m.T * m.d_in_proj * m.es; a.ldc = m.d_in_proj;
+        a.in_dtype = c->dtype; a.c_dtype = c->dtype; a.M = (int)m.T; a.N = m.d_in_proj; a.K = m.d;
+        if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "in_proj");
+    }
+
+    ScanArgs sa{};
+    sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
+    sa.d_in_proj = m.d_in_proj; sa.conv_ch = m.conv_ch;
+    sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask; sa.chunk = c->chunk;
+    sa.zx = zx; sa.g = g; sa.ssq = norm_on ? ssq : nullptr;
+    for (int dir = 0; dir < 2; ++dir) {
+        sa.dir[dir].conv_w = w[dir].conv_w; sa.dir[dir].conv_b = w[dir].conv_b; sa.dir[dir].norm_w = w[dir].norm_w;
+        sa.dir[dir].dt_bias = w[dir].dt_bias; sa.dir[dir].A_log = w[dir].A_log; sa.dir[dir].D = w[dir].D;
+    }
+    sa.ssm_in = ssm_in; sa.conv_in = conv_in; sa.ssm_out = ssm_out;
+    if (scan_ssd_supports(sa)) e = scan_ssd(sa, ws + l.scan, s);
+    else e = scan_sequential(sa, s);
+    if (e != cudaSuccess) return cuda_fail(e, "scan");
+
+    if (conv_out && (c->dir_mask & DM_DIR_FWD)) {
+        e = conv_state_update(zx, conv_in, conv_out, c->dtype, m.B, m.L, m.k, m.d_inner, m.conv_ch, m.d_in_proj, s);
+        if (e != cudaSuccess) return cuda_fail(e, "conv_state_update");
+    }
+    if (norm_on) {
+        e = rstd_from_ssq(ssq, rstd, (int)(2 * m.T), m.H, m.d_inner, c->norm_eps, s);
+        if (e != cudaSuccess) return cuda_fail(e, "rstd");
+    }
+    // out_proj of each direction; the second one adds the first (Mamba(x) = h-> + h<-)
+    const float *carry = out.addend;
+    int64_t ld_carry = out.ld_add;
+    const int last_dir = (c->dir_mask & DM_DIR_REV) ? 1 : 0;
+    for (int dir = 0; dir < 2; ++dir) {
+        if (!(c->dir_mask & (1 << dir))) continue;
+        const bool last = dir == last_dir;
+        GemmArgs a{};
+        a.A = g + (size_t)dir * m.T * m.d_inner * m.es; a.lda = m.d_inner;
+        a.B = w[dir].w_out; a.ldb = m.d_inner;
+        a.in_dtype = c->dtype; a.M = (int)m.T; a.N = m.d; a.K = m.d_inner;
+        a.row_scale = norm_on ? rstd + (size_t)dir * m.T : nullptr;
+        a.addend = carry; a.ld_add = ld_carry;
+        if (last) { a.C = out.y; a.ldc = m.d; a.c_dtype = out.y_dtype; }
+        else { a.C = ytmp; a.ldc = m.d; a.c_dtype = DM_F32; carry = ytmp; ld_carry = m.d; }
+        if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "out_proj");
+    }
+    return DM_OK;
+}
+
+static int check_ws(const void *ws, size_t have, size_t need) {
+    if (!ws) return fail(DM_ERR_WORKSPACE, "workspace is NULL");
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(DM_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+    if (have < need) return fail(DM_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", have, need);
+    return DM_OK;
+}
+
+struct StackWs {
+    size_t r, u, logits, mixer, total;
+    int logits_rows;
+};
+
+static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m) {
+    StackWs w;
+    size_t off = 0;
+    w.r = off; off += align_up((size_t)m.T * m.d * sizeof(float));
+    w.u = off; off += align_up((size_t)m.T * m.d * m.es);
+    w.logits_rows = (int)(m.T < 2048 ? m.T : 2048);
+    w.logits = off; off += align_up((size_t)w.logits_rows * c->vocab * m.es);
+    w.mixer = off; off += mixer_ws(&c->mixer, m).total;
+    w.total = off;
+    return w;
+}
+
+}  // namespace dm
+
+using namespace dm;
+
+extern "C" {
+
+const char *dm_status_string(int status) {
+    switch (status) {
+        case DM_OK: return "ok";
+        case DM_ERR_INVALID_ARG: return "invalid argument";
+        case DM_ERR_UNSUPPORTED: return "unsupported shape or option";
+        case DM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case DM_ERR_CUDA: return "CUDA runtime error";
+        case DM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+const char *dm_last_error_message(void) { return g_err; }
+
+uint64_t dm_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int dm_bimamba_workspace_bytes(const dm_mixer_cfg *cfg, size_t *bytes) {
+    Dims m;
+    if (!bytes) return fail(DM_ERR_INVALID_ARG, "bytes is NULL");
+    int st = check_cfg(cfg, &m);
+    if (st != DM_OK) return st;
+    *bytes = mixer_ws(cfg, m).total;
+    return DM_OK;
+}
+
+int dm_denoise_workspace_bytes(const dm_stack_cfg *cfg, size_t *bytes) {
+    Dims m;
+    if (!bytes || !cfg) return fail(DM_ERR_INVALID_ARG, "NULL argument");
+    int st = check_cfg(&cfg->mixer, &m);
+    if (st != DM_OK) return st;
+    if (cfg->n_layers <= 0 || cfg->vocab <= 0) return fail(DM_ERR_INVALID_ARG, "n_layers and vocab must be positive");
+    *bytes = stack_ws(cfg, m).total;
+    return DM_OK;
+}
+
+int dm_check(void *cuda_stream) {
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e, "dm_check: synchronize");
+    int *p = device_status_ptr();
+    if (!p) return fail(DM_ERR_CUDA, "dm_check: no status word");
+    int v = 0;
+    if ((e = cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e, "dm_check: read status");
+    if (v != 0) {
+        int zero = 0;
+        cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice);
+        return fail(v, "a kernel reported status %d (%s)", v, dm_status_string(v));
+    }
+    return DM_OK;
+}
+
+int dm_bimamba_forward(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x, void *y,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    Dims m;
+    int st = check_cfg(cfg, &m);
+    if (st != DM_OK) return st;
+    if ((st = check_weights(cfg, w)) != DM_OK) return st;
+    if (!x || !y) return fail(DM_ERR_INVALID_ARG, "x or y is NULL");
+    if (x == y) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
+    if (!aligned16(x) || !aligned16(y)) return fail(DM_ERR_INVALID_ARG, "x and y must be 16-byte aligned");
+    if ((st = check_ws(workspace, workspace_bytes, mixer_ws(cfg, m).total)) != DM_OK) return st;
+    MixerOut out{y, cfg->dtype, nullptr, 0};
+    return run_mixer(cfg, m, w, x, out, nullptr, nullptr, nullptr, nullptr, static_cast<char *>(workspace),
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dm_bimamba_block_step(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x_blk,
+                          const float *ssm_state_in, const void *conv_state_in,
+                          float *ssm_state_out, void *conv_state_out, void *y_blk,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    Dims m;
+    int st = check_cfg(cfg, &m);
+    if (st != DM_OK) return st;
+    if ((st = check_weights(cfg, w)) != DM_OK) return st;
+    if (!x_blk || !y_blk) return fail(DM_ERR_INVALID_ARG, "x_blk or y_blk is NULL");
+    if (x_blk == y_blk) return fail(DM_ERR_INVALID_ARG, "y_blk must not alias x_blk");
+    if (!aligned16(x_blk) || !aligned16(y_blk) || !aligned16(ssm_state_in) || !aligned16(ssm_state_out) ||
+        !aligned16(conv_state_in) || !aligned16(conv_state_out))
+        return fail(DM_ERR_INVALID_ARG, "tensors must be 16-byte aligned");
+    if ((ssm_state_in && ssm_state_in == ssm_state_out) || (conv_state_in && conv_state_in == conv_state_out))
+        return fail(DM_ERR_INVALID_ARG, "state_in and state_out must be different buffers");
+    if ((ssm_state_out || conv_state_out) && !(cfg->dir_mask & DM_DIR_FWD))
+        return fail(DM_ERR_INVALID_ARG, "state_out needs the left-to-right direction");
+    if ((st = check_ws(workspace, workspace_bytes, mixer_ws(cfg, m).total)) != DM_OK) return st;
+    MixerOut out{y_blk, cfg->dtype, nullptr, 0};
+    return run_mixer(cfg, m, w, x_blk, out, ssm_state_in, conv_state_in, ssm_state_out, conv_state_out,
+                     static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, const int32_t *tokens, void *logits,
+                    int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
+                    void *cuda_stream) {
+    Dims m;
+    if (!cfg || !weights) return fail(DM_ERR_INVALID_ARG, "cfg or weights is NULL");
+    int st = check_cfg(&cfg->mixer, &m);
+    if (st != DM_OK) return st;
+    if (cfg->n_layers <= 0 || cfg->vocab <= 0) return fail(DM_ERR_INVALID_ARG, "n_layers and vocab must be positive");
+    if (!(cfg->rms_eps >= 0.f)) return fail(DM_ERR_INVALID_ARG, "rms_eps must be >= 0");
+    if (!tokens) return fail(DM_ERR_INVALID_ARG, "tokens is NULL");
+    if (!logits && !argmax_out) return fail(DM_ERR_INVALID_ARG, "logits and argmax_out are both NULL");
+    if (!weights->embed || !weights->layers || !weights->final_norm_w || !weights->w_vocab)
+        return fail(DM_ERR_INVALID_ARG, "NULL pointer in stack weights");
+    if (!aligned16(weights->embed) || !aligned16(weights->w_vocab) || !aligned16(logits))
+        return fail(DM_ERR_INVALID_ARG, "embed, w_vocab and logits must be 16-byte aligned");
+    if (logits && (((size_t)cfg->vocab * m.es) % 16)) return fail(DM_ERR_UNSUPPORTED, "vocab*sizeof(dtype) must be a multiple of 16");
+    for (int i = 0; i < cfg->n_layers; ++i) {
+        if (!weights->layers[i].norm_w) return fail(DM_ERR_INVALID_ARG, "layer %d: norm_w is NULL", i);
+        if ((st = check_weights(&cfg->mixer, weights->layers[i].dir)) != DM_OK) return st;
+        if (states) {
+            const dm_layer_state &q = states[i];
+            if ((q.ssm_in && q.ssm_in == q.ssm_out) || (q.conv_in && q.conv_in == q.conv_out))
+                return fail(DM_ERR_INVALID_ARG, "layer %d: state_in and state_out must be different buffers", i);
+            if (!aligned16(q.ssm_in) || !aligned16(q.ssm_out) || !aligned16(q.conv_in) || !aligned16(q.conv_out))
+                return fail(DM_ERR_INVALID_ARG, "layer %d: states must be 16-byte aligned", i);
+            if ((q.ssm_out || q.conv_out) && !(cfg->mixer.dir_mask & DM_DIR_FWD))
+                return fail(DM_ERR_INVALID_ARG, "state_out needs the left-to-right direction");
+        }
+    }
+    const StackWs l = stack_ws(cfg, m);
+    if ((st = check_ws(workspace, workspace_bytes, l.total)) != DM_OK) return st;
+    char *ws = static_cast<char *>(workspace);
+    float *r = reinterpret_cast<float *>(ws + l.r);
+    void *u = ws + l.u;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int dtype = cfg->mixer.dtype;
+    cudaError_t e;
+
+    if ((e = embed_gather(weights->embed, dtype, tokens, r, (int)m.T, m.d, cfg->vocab, s)) != cudaSuccess) return cuda_fail(e, "embed");
+    for (int i = 0; i < cfg->n_layers; ++i) {
+        const dm_layer_weights &lw = weights->layers[i];
+        if ((e = rmsnorm_rows(r, lw.norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "rmsnorm");
+        MixerOut out{r, DM_F32, r, m.d};          // r <- r + Mamba(u): the residual add rides in the out_proj epilogue
+        const dm_layer_state *q = states ? &states[i] : nullptr;
+        st = run_mixer(&cfg->mixer, m, lw.dir, u, out, q ? q->ssm_in : nullptr, q ? q->conv_in : nullptr,
+                       q ? q->ssm_out : nullptr, q ? q->conv_out : nullptr, ws + l.mixer, s);
+        if (st != DM_OK) return st;
+    }
+    if ((e = rmsnorm_rows(r, weights->final_norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "final norm");
+    const int64_t rows_per = logits ? m.T : l.logits_rows;
+    for (int64_t t0 = 0; t0 < m.T; t0 += rows_per) {
+        const int rows = (int)((m.T - t0) < rows_per ? (m.T - t0) : rows_per);
+        GemmArgs a{};
+        a.A = static_cast<char *>(u) + (size_t)t0 * m.d * m.es; a.lda = m.d;
+        a.B = weights->w_vocab; a.ldb = m.d;
+        a.C = logits ? static_cast<char *>(logits) + (size_t)t0 * cfg->vocab * m.es : ws + l.logits; a.ldc = cfg->vocab;
+        a.in_dtype = dtype; a.c_dtype = dtype; a.M = rows; a.N = cfg->vocab; a.K = m.d;
+        if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "vocab projection");
+        if (argmax_out && (e = argmax_rows(a.C, dtype, argmax_out + t0, rows, cfg->vocab, s)) != cudaSuccess) return cuda_fail(e, "argmax");
+    }
+    return DM_OK;
+}
+
+int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x_host, void *y_host,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    Dims m;
+    int st = check_cfg(cfg, &m);
+    if (st != DM_OK) return st;
+    if (!x_host || !y_host) return fail(DM_ERR_INVALID_ARG, "x_host or y_host is NULL");
+    const size_t act = align_up((size_t)m.T * m.d * m.es);
+    const size_t need = mixer_ws(cfg, m).total + 2 * act;
+    if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    void *xd = ws, *yd = ws + act;
+    cudaError_t e = cudaMemcpyAsync(xd, x_host, (size_t)m.T * m.d * m.es, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e, "copy x to the device");
+    st = dm_bimamba_forward(cfg, w, xd, yd, ws + 2 * act, workspace_bytes - 2 * act, cuda_stream);
+    if (st != DM_OK) return st;
+    if ((e = cudaMemcpyAsync(y_host, yd, (size_t)m.T * m.d * m.es, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e, "copy y to the host");
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e, "synchronize");
+    return DM_OK;
+}
+
+}  // extern "C"

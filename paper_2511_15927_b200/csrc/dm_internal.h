@@ -1,0 +1,81 @@
+// Internal declarations shared by the translation units of libdm_bimamba.so (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "dm_bimamba.h"
+
+namespace dm {
+
+// Every kernel launch goes through this counter (dm_kernel_launch_count()).
+void count_launch(int n = 1);
+
+// Device status word written by kernels whose bounded waits expire; read and cleared by dm_check().
+int *device_status_ptr();
+
+inline size_t dtype_size(int dtype) { return dtype == DM_BF16 ? 2 : 4; }
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------------
+// GEMM:  C[m, n] = row_scale[m] * sum_k A[m, k] * B[n, k]  +  addend[m, n]
+// A [M, K] (lda), B [N, K] (ldb): in_dtype.  C [M, N] (ldc): c_dtype.  row_scale [M] fp32 or NULL.
+// addend [M, N] (ld_add) fp32 or NULL; it may alias C when c_dtype is DM_F32 and ldc == ld_add.
+// ---------------------------------------------------------------------------------------------
+struct GemmArgs {
+    const void *A; int64_t lda;
+    const void *B; int64_t ldb;
+    void *C; int64_t ldc;
+    int in_dtype, c_dtype;
+    int M, N, K;
+    const float *row_scale;
+    const float *addend; int64_t ld_add;
+};
+cudaError_t gemm_simple(const GemmArgs &a, cudaStream_t s);
+// Tensor-core path (tcgen05 + TMEM + TMA).  Returns cudaErrorNotSupported for shapes it does not take.
+cudaError_t gemm_tcgen05(const GemmArgs &a, cudaStream_t s);
+bool gemm_tcgen05_supports(const GemmArgs &a);
+
+// ---------------------------------------------------------------------------------------------
+// Fused conv + SiLU + discretisation + selective scan + gate, both directions in one launch.
+// ---------------------------------------------------------------------------------------------
+struct ScanDir {
+    const void *conv_w, *conv_b, *norm_w;
+    const float *dt_bias, *A_log, *D;
+};
+struct ScanArgs {
+    int B, L, d_inner, H, P, N, k, d_in_proj, conv_ch;
+    int dtype, flags, dir_mask, chunk;
+    const void *zx;          // [2][B*L][d_in_proj] dtype: in_proj output of each direction
+    void *g;                 // [2][B*L][d_inner]   dtype: gated output (times norm_w when the norm is on)
+    float *ssq;              // [2][B*L][H] per-head sum of squares of the gated output (norm on), or NULL
+    ScanDir dir[2];
+    const float *ssm_in;     // [B,H,P,N] or NULL   (left-to-right direction only)
+    const void *conv_in;     // [B,k-1,conv_ch] or NULL
+    float *ssm_out;          // [B,H,P,N] or NULL
+};
+cudaError_t scan_sequential(const ScanArgs &a, cudaStream_t s);
+bool scan_ssd_supports(const ScanArgs &a);
+size_t scan_ssd_workspace_bytes(const ScanArgs &a);
+cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s);
+
+// ---------------------------------------------------------------------------------------------
+// Small row-wise kernels
+// ---------------------------------------------------------------------------------------------
+// rstd[dir][t] = rsqrt(sum_h ssq[dir][t][h] / d_inner + eps)
+cudaError_t rstd_from_ssq(const float *ssq, float *rstd, int rows, int H, int d_inner, float eps, cudaStream_t s);
+// r[t, :] = embed[tokens[t], :]  (fp32 residual stream)
+cudaError_t embed_gather(const void *embed, int dtype, const int32_t *tokens, float *r, int T, int d, int vocab, cudaStream_t s);
+// u[t, :] = r[t, :] * rsqrt(mean(r[t]^2) + eps) * w
+cudaError_t rmsnorm_rows(const float *r, const void *w, void *u, int dtype, int T, int d, float eps, cudaStream_t s);
+// out[t] = argmax_v logits[t, v], lowest index on ties
+cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s);
+// conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])
+cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *conv_out, int dtype, int B, int L,
+                              int k, int d_inner, int conv_ch, int d_in_proj, cudaStream_t s);
+// y[i] = (dtype) src[i]
+cudaError_t cast_f32_rows(const float *src, void *dst, int dtype, size_t n, cudaStream_t s);
+
+}  // namespace dm

@@ -1,0 +1,149 @@
+// Small row-wise kernels around the mixer: embedding gather, RMSNorm, the gated norm's rstd, arg-max
+// over the vocabulary, the carried conv state.  All are bandwidth-trivial next to the GEMMs and the scan.
+#include "dm_internal.h"
+
+namespace dm {
+namespace {
+
+template <typename T> __device__ __forceinline__ float ldf(const T *p);
+template <> __device__ __forceinline__ float ldf<float>(const float *p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T *p, float v);
+template <> __device__ __forceinline__ void stf<float>(float *p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float block_sum(float v, float *red) {
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int i = 0; i < nwarp; ++i) t += red[i];      // same order in every thread: deterministic
+    return t;
+}
+
+__global__ void rstd_kernel(const float *__restrict__ ssq, float *__restrict__ rstd, int rows, int H, float inv_n, float eps) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    float s = 0.f;
+    for (int h = 0; h < H; ++h) s += ssq[(int64_t)r * H + h];
+    rstd[r] = rsqrtf(s * inv_n + eps);
+}
+
+template <typename T>
+__global__ void embed_kernel(const T *__restrict__ embed, const int32_t *__restrict__ tokens, float *__restrict__ r, int d, int vocab) {
+    const int64_t t = blockIdx.x;
+    int id = tokens[t];
+    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);      // ids are validated on the host side of the tests; clamp keeps reads in bounds
+    for (int c = threadIdx.x; c < d; c += blockDim.x) r[t * d + c] = ldf(embed + (int64_t)id * d + c);
+}
+
+template <typename T>
+__global__ void rmsnorm_kernel(const float *__restrict__ r, const T *__restrict__ w, T *__restrict__ u, int d, float eps) {
+    __shared__ float red[32];
+    const int64_t t = blockIdx.x;
+    float s = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = r[t * d + c]; s = fmaf(v, v, s); }
+    s = block_sum(s, red);
+    const float rs = rsqrtf(s / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) stf(u + t * d + c, r[t * d + c] * rs * ldf(w + c));
+}
+
+template <typename T>
+__global__ void argmax_kernel(const T *__restrict__ logits, int32_t *__restrict__ out, int V) {
+    __shared__ float bv[32];
+    __shared__ int bi[32];
+    const int64_t t = blockIdx.x;
+    float best = -INFINITY; int idx = 0x7fffffff;
+    for (int v = threadIdx.x; v < V; v += blockDim.x) {
+        const float x = ldf(logits + t * V + v);
+        if (x > best || (x == best && v < idx)) { best = x; idx = v; }
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+        if (ob > best || (ob == best && oi < idx)) { best = ob; idx = oi; }
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+    if (lane == 0) { bv[warp] = best; bi[warp] = idx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < nwarp; ++i)
+            if (bv[i] > best || (bv[i] == best && bi[i] < idx)) { best = bv[i]; idx = bi[i]; }
+        out[t] = idx == 0x7fffffff ? 0 : idx;
+    }
+}
+
+// Row r (0..k-2) of the new conv state of batch row b is row L + r - (k-1) of the block when that is
+// >= 0, otherwise row (k-1) + (L + r - (k-1)) of the old state (or zero).
+template <typename T>
+__global__ void conv_state_kernel(const T *__restrict__ zx, const T *__restrict__ conv_in, T *__restrict__ conv_out,
+                                  int L, int k, int d_inner, int conv_ch, int d_in_proj) {
+    const int b = blockIdx.y, r = blockIdx.z;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= conv_ch) return;
+    const int src = L + r - (k - 1);
+    T v;
+    if (src >= 0) v = zx[((int64_t)b * L + src) * d_in_proj + d_inner + c];
+    else if (conv_in) v = conv_in[((int64_t)b * (k - 1) + (k - 1 + src)) * conv_ch + c];
+    else { stf(&v, 0.f); }
+    conv_out[((int64_t)b * (k - 1) + r) * conv_ch + c] = v;
+}
+
+template <typename T>
+__global__ void cast_kernel(const float *__restrict__ src, T *__restrict__ dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) stf(dst + i, src[i]);
+}
+
+}  // namespace
+
+cudaError_t rstd_from_ssq(const float *ssq, float *rstd, int rows, int H, int d_inner, float eps, cudaStream_t s) {
+    rstd_kernel<<<(rows + 255) / 256, 256, 0, s>>>(ssq, rstd, rows, H, 1.f / (float)d_inner, eps);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t embed_gather(const void *embed, int dtype, const int32_t *tokens, float *r, int T, int d, int vocab, cudaStream_t s) {
+    if (dtype == DM_BF16) embed_kernel<<<T, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(embed), tokens, r, d, vocab);
+    else embed_kernel<<<T, 256, 0, s>>>(static_cast<const float *>(embed), tokens, r, d, vocab);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t rmsnorm_rows(const float *r, const void *w, void *u, int dtype, int T, int d, float eps, cudaStream_t s) {
+    if (dtype == DM_BF16) rmsnorm_kernel<<<T, 256, 0, s>>>(r, static_cast<const __nv_bfloat16 *>(w), static_cast<__nv_bfloat16 *>(u), d, eps);
+    else rmsnorm_kernel<<<T, 256, 0, s>>>(r, static_cast<const float *>(w), static_cast<float *>(u), d, eps);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s) {
+    if (dtype == DM_BF16) argmax_kernel<<<T, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(logits), out, V);
+    else argmax_kernel<<<T, 256, 0, s>>>(static_cast<const float *>(logits), out, V);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *conv_out, int dtype, int B, int L,
+                              int k, int d_inner, int conv_ch, int d_in_proj, cudaStream_t s) {
+    dim3 grid((conv_ch + 255) / 256, B, k - 1);
+    if (dtype == DM_BF16)
+        conv_state_kernel<<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(zx_fwd), static_cast<const __nv_bfloat16 *>(conv_in),
+                                               static_cast<__nv_bfloat16 *>(conv_out), L, k, d_inner, conv_ch, d_in_proj);
+    else
+        conv_state_kernel<<<grid, 256, 0, s>>>(static_cast<const float *>(zx_fwd), static_cast<const float *>(conv_in),
+                                               static_cast<float *>(conv_out), L, k, d_inner, conv_ch, d_in_proj);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t cast_f32_rows(const float *src, void *dst, int dtype, size_t n, cudaStream_t s) {
+    const int blocks = (int)((n + 255) / 256 > 148 * 16 ? 148 * 16 : (n + 255) / 256);
+    if (dtype == DM_BF16) cast_kernel<<<blocks, 256, 0, s>>>(src, static_cast<__nv_bfloat16 *>(dst), n);
+    else cast_kernel<<<blocks, 256, 0, s>>>(src, static_cast<float *>(dst), n);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace dm

@@ -1,0 +1,129 @@
+"""Helpers for the GPU parity tests: move the seeded host inputs to the device, call the library through
+its C ABI (via the ctypes binding) and bring results back as float64 numpy arrays."""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+import torch
+
+from paper_2511_15927_b200 import binding as dm
+from paper_2511_15927_b200 import inputs as I
+
+TYPED = ("w_in", "conv_w", "conv_b", "norm_w", "w_out")
+
+
+def tdtype(dtype):
+    return torch.bfloat16 if dtype == I.BF16 else torch.float32
+
+
+def dm_dtype(dtype):
+    return dm.DM_BF16 if dtype == I.BF16 else dm.DM_F32
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.to(tdtype(dtype)) if dtype is not None else t
+
+
+def dev_dir_weights(w: dict, dtype) -> dict:
+    return {k: dev(v, dtype if k in TYPED else None) for k, v in w.items()}
+
+
+def cfg_of(shape: I.MixerShape, dtype, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, chunk=0, eps=1e-5):
+    return dm.make_mixer_cfg(shape.batch, shape.seqlen, shape.d_model, shape.expand, shape.d_state, shape.d_conv,
+                             shape.n_heads, dm_dtype(dtype), shape.n_groups, flags, dir_mask, chunk, eps)
+
+
+def workspace(nbytes: int) -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+
+
+def run_forward(shape, dtype, wf, wr, x, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, chunk=0):
+    cfg = cfg_of(shape, dtype, flags, dir_mask, chunk)
+    dwf, dwr = dev_dir_weights(wf, dtype), dev_dir_weights(wr, dtype)
+    xd = dev(x, dtype)
+    yd = torch.empty_like(xd)
+    nb = dm.dm_bimamba_workspace_bytes(cfg)
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_bimamba_forward(cfg, (dm.make_dir_weights(dwf), dm.make_dir_weights(dwr)), xd.data_ptr(), yd.data_ptr(),
+                          ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    return yd.float().cpu().numpy().astype(np.float64)
+
+
+def run_block_step(shape, dtype, wf, wr, x_blk, ssm_in=None, conv_in=None, want_state=True, flags=dm.DM_FLAGS_DEFAULT,
+                   dir_mask=dm.DM_DIR_BOTH, chunk=0):
+    cfg = cfg_of(shape, dtype, flags, dir_mask, chunk)
+    dwf, dwr = dev_dir_weights(wf, dtype), dev_dir_weights(wr, dtype)
+    xd = dev(x_blk, dtype)
+    yd = torch.empty_like(xd)
+    s_in = dev(ssm_in.astype(np.float32)) if ssm_in is not None else None
+    c_in = dev(conv_in.astype(np.float32), dtype) if conv_in is not None else None
+    s_out = torch.full((shape.batch, shape.n_heads, shape.headdim, shape.d_state), float("nan"), device="cuda") if want_state else None
+    c_out = torch.full((shape.batch, shape.d_conv - 1, shape.conv_ch), float("nan"), device="cuda", dtype=tdtype(dtype)) if want_state else None
+    nb = dm.dm_bimamba_workspace_bytes(cfg)
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    p = lambda t: t.data_ptr() if t is not None else 0
+    dm.dm_bimamba_block_step(cfg, (dm.make_dir_weights(dwf), dm.make_dir_weights(dwr)), xd.data_ptr(), p(s_in), p(c_in),
+                             p(s_out), p(c_out), yd.data_ptr(), ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    f = lambda t: None if t is None else t.float().cpu().numpy().astype(np.float64)
+    return f(yd), f(s_out), f(c_out)
+
+
+def dev_stack_weights(sw: dict, dtype) -> dict:
+    return {"embed": dev(sw["embed"], dtype), "w_vocab": dev(sw["w_vocab"], dtype),
+            "final_norm_w": dev(sw["final_norm_w"], dtype),
+            "layers": [{"norm_w": dev(l["norm_w"], dtype), "fwd": dev_dir_weights(l["fwd"], dtype),
+                        "rev": dev_dir_weights(l["rev"], dtype)} for l in sw["layers"]]}
+
+
+def run_denoise(shape, dtype, sw, tokens, vocab, want_logits=True, want_argmax=True, states_in=None, want_states=False,
+                flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, rms_eps=1e-5):
+    n_layers = len(sw["layers"])
+    scfg = dm.dm_stack_cfg(cfg_of(shape, dtype, flags, dir_mask), n_layers, vocab, rms_eps)
+    dsw = dev_stack_weights(sw, dtype)
+    csw, keep = dm.make_stack_weights(dsw)
+    tok = dev(tokens.astype(np.int32))
+    T = shape.batch * shape.seqlen
+    logits = torch.empty((shape.batch, shape.seqlen, vocab), device="cuda", dtype=tdtype(dtype)) if want_logits else None
+    amax = torch.full((shape.batch, shape.seqlen), -1, device="cuda", dtype=torch.int32) if want_argmax else None
+    states = None
+    bufs = []
+    if states_in is not None or want_states:
+        states = (dm.dm_layer_state * n_layers)()
+        for i in range(n_layers):
+            s_in = c_in = None
+            if states_in is not None and states_in[i] is not None:
+                s_in = dev(states_in[i][0].astype(np.float32)); c_in = dev(states_in[i][1].astype(np.float32), dtype)
+            s_out = torch.empty((shape.batch, shape.n_heads, shape.headdim, shape.d_state), device="cuda") if want_states else None
+            c_out = torch.empty((shape.batch, shape.d_conv - 1, shape.conv_ch), device="cuda", dtype=tdtype(dtype)) if want_states else None
+            bufs.append((s_in, c_in, s_out, c_out))
+            p = lambda t: t.data_ptr() if t is not None else None
+            states[i] = dm.dm_layer_state(p(s_in), p(c_in), p(s_out), p(c_out))
+    nb = dm.dm_denoise_workspace_bytes(scfg)
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_denoise_step(scfg, csw, tok.data_ptr(), logits.data_ptr() if want_logits else 0,
+                       amax.data_ptr() if want_argmax else 0, states, ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    f = lambda t: None if t is None else t.float().cpu().numpy().astype(np.float64)
+    out_states = [(f(b[2]), f(b[3])) for b in bufs] if want_states else None
+    return f(logits), (amax.cpu().numpy() if want_argmax else None), out_states
+
+
+def rel_l2(a, b):
+    return float(np.linalg.norm(np.asarray(a, np.float64) - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def max_abs(a, b):
+    return float(np.max(np.abs(np.asarray(a, np.float64) - b)))
+
+
+def oracle_kwargs(shape, flags=dm.DM_FLAGS_DEFAULT, eps=1e-5):
+    return dict(expand=shape.expand, d_state=shape.d_state, n_heads=shape.n_heads, n_groups=shape.n_groups,
+                gated_norm=bool(flags & dm.DM_FLAG_GATED_RMSNORM), conv_bias=bool(flags & dm.DM_FLAG_CONV_BIAS),
+                d_skip=bool(flags & dm.DM_FLAG_D_SKIP), norm_eps=eps)
