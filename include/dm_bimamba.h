@@ -165,6 +165,15 @@ int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
 /* Number of kernels this library has launched from this process since load (for benchmarks). */
 uint64_t dm_kernel_launch_count(void);
 
+/* Measurement aid (no counterpart in the paper).  While enabled, every mixer call records CUDA event
+ * pairs on its stream around its three stages: in_proj (one span per direction), the fused
+ * conv+scan+gate launch, out_proj (one span per direction).  dm_profile_read waits for the recorded
+ * events, writes the summed device time in milliseconds and the number of spans per stage into the HOST
+ * arrays ms[DM_STAGE_COUNT], spans[DM_STAGE_COUNT], and forgets them.  Not for use during stream capture. */
+enum { DM_STAGE_IN_PROJ = 0, DM_STAGE_SCAN = 1, DM_STAGE_OUT_PROJ = 2, DM_STAGE_COUNT = 3 };
+int dm_profile_enable(int on);
+int dm_profile_read(float *ms, uint64_t *spans);
+
 #ifdef __cplusplus
 }
 #endif

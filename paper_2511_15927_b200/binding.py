@@ -67,13 +67,16 @@ _lib.dm_bimamba_block_step.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir
                                        _vp, _sz, _vp]
 _lib.dm_denoise_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_stack_weights), _vp, _vp, _vp,
                                  C.POINTER(dm_layer_state), _vp, _sz, _vp]
-for _f in ("dm_bimamba_workspace_bytes", "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward",
+_lib.dm_profile_enable.argtypes = [C.c_int]
+_lib.dm_profile_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_uint64)]
+for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes", "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward",
            "dm_bimamba_forward_host", "dm_bimamba_block_step", "dm_denoise_step"):
     getattr(_lib, _f).restype = C.c_int
 
 EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
-           "dm_bimamba_block_step", "dm_denoise_step")
+           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read")
+DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
 
 class DmError(RuntimeError):
@@ -97,6 +100,18 @@ def dm_last_error_message() -> str:
 
 def dm_kernel_launch_count() -> int:
     return int(_lib.dm_kernel_launch_count())
+
+
+def dm_profile_enable(on: bool) -> None:
+    _ok(_lib.dm_profile_enable(1 if on else 0))
+
+
+def dm_profile_read():
+    """Returns (ms, spans): two lists indexed by DM_STAGE_*."""
+    ms = (C.c_float * DM_STAGE_COUNT)()
+    n = (C.c_uint64 * DM_STAGE_COUNT)()
+    _ok(_lib.dm_profile_read(ms, n))
+    return list(ms), [int(v) for v in n]
 
 
 def dm_bimamba_workspace_bytes(cfg: dm_mixer_cfg) -> int:

@@ -3,6 +3,8 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "dm_internal.h"
 
@@ -26,6 +28,28 @@ int *device_status_ptr() {
 }
 
 static thread_local char g_err[512] = "";
+
+// Optional per-stage timing: CUDA event pairs recorded on the caller's stream around in_proj, the fused
+// scan and out_proj of every mixer call; summed and released by dm_profile_read().
+struct StageSpan { int stage; cudaEvent_t a, b; };
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<StageSpan> g_spans;
+
+struct StageTimer {
+    bool on; int stage; cudaStream_t s; cudaEvent_t a = nullptr;
+    StageTimer(int stage_, cudaStream_t s_) : on(g_prof_on), stage(stage_), s(s_) {
+        if (on && (cudaEventCreate(&a) != cudaSuccess || cudaEventRecord(a, s) != cudaSuccess)) on = false;
+    }
+    ~StageTimer() {
+        if (!on) return;
+        cudaEvent_t b = nullptr;
+        if (cudaEventCreate(&b) == cudaSuccess && cudaEventRecord(b, s) == cudaSuccess) {
+            std::lock_guard<std::mutex> lk(g_prof_mu);
+            g_spans.push_back({stage, a, b});
+        }
+    }
+};
 
 static int fail(int status, const char *fmt, ...) {
     va_list ap;
@@ -133,6 +157,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
 
     for (int dir = 0; dir < 2; ++dir) {
         if (!(c->dir_mask & (1 << dir))) continue;
+        StageTimer tm(DM_STAGE_IN_PROJ, s);
         GemmArgs a{};
         a.A = x; a.lda = m.d; a.B = w[dir].w_in; a.ldb = m.d;
         a.C = zx + (size_t)dir * m.T * m.d_in_proj * m.es; a.ldc = m.d_in_proj;
@@ -150,8 +175,11 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         sa.dir[dir].dt_bias = w[dir].dt_bias; sa.dir[dir].A_log = w[dir].A_log; sa.dir[dir].D = w[dir].D;
     }
     sa.ssm_in = ssm_in; sa.conv_in = conv_in; sa.ssm_out = ssm_out;
-    if (scan_ssd_supports(sa)) e = scan_ssd(sa, ws + l.scan, s);
-    else e = scan_sequential(sa, s);
+    {
+        StageTimer tm(DM_STAGE_SCAN, s);
+        if (scan_ssd_supports(sa)) e = scan_ssd(sa, ws + l.scan, s);
+        else e = scan_sequential(sa, s);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "scan");
 
     if (conv_out && (c->dir_mask & DM_DIR_FWD)) {
@@ -169,6 +197,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
     for (int dir = 0; dir < 2; ++dir) {
         if (!(c->dir_mask & (1 << dir))) continue;
         const bool last = dir == last_dir;
+        StageTimer tm(DM_STAGE_OUT_PROJ, s);
         GemmArgs a{};
         a.A = g + (size_t)dir * m.T * m.d_inner * m.es; a.lda = m.d_inner;
         a.B = w[dir].w_out; a.ldb = m.d_inner;
@@ -227,6 +256,33 @@ const char *dm_status_string(int status) {
 const char *dm_last_error_message(void) { return g_err; }
 
 uint64_t dm_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int dm_profile_enable(int on) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = on != 0;
+    return DM_OK;
+}
+
+int dm_profile_read(float *ms, uint64_t *spans) {
+    if (!ms || !spans) return fail(DM_ERR_INVALID_ARG, "ms or spans is NULL");
+    std::vector<StageSpan> v;
+    {
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        v.swap(g_spans);
+    }
+    for (int i = 0; i < DM_STAGE_COUNT; ++i) { ms[i] = 0.f; spans[i] = 0; }
+    int st = DM_OK;
+    for (const StageSpan &sp : v) {
+        float t = 0.f;
+        cudaError_t e = cudaEventSynchronize(sp.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t, sp.a, sp.b);
+        if (e == cudaSuccess && sp.stage >= 0 && sp.stage < DM_STAGE_COUNT) { ms[sp.stage] += t; spans[sp.stage] += 1; }
+        else if (e != cudaSuccess) st = cuda_fail(e, "dm_profile_read");
+        cudaEventDestroy(sp.a);
+        cudaEventDestroy(sp.b);
+    }
+    return st;
+}
 
 int dm_bimamba_workspace_bytes(const dm_mixer_cfg *cfg, size_t *bytes) {
     Dims m;

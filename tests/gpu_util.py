@@ -2,41 +2,13 @@
 its C ABI (via the ctypes binding) and bring results back as float64 numpy arrays."""
 from __future__ import annotations
 
-import ctypes as C
-
 import numpy as np
 import torch
 
 from paper_2511_15927_b200 import binding as dm
 from paper_2511_15927_b200 import inputs as I
-
-TYPED = ("w_in", "conv_w", "conv_b", "norm_w", "w_out")
-
-
-def tdtype(dtype):
-    return torch.bfloat16 if dtype == I.BF16 else torch.float32
-
-
-def dm_dtype(dtype):
-    return dm.DM_BF16 if dtype == I.BF16 else dm.DM_F32
-
-
-def dev(a, dtype=None):
-    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
-    return t.to(tdtype(dtype)) if dtype is not None else t
-
-
-def dev_dir_weights(w: dict, dtype) -> dict:
-    return {k: dev(v, dtype if k in TYPED else None) for k, v in w.items()}
-
-
-def cfg_of(shape: I.MixerShape, dtype, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, chunk=0, eps=1e-5):
-    return dm.make_mixer_cfg(shape.batch, shape.seqlen, shape.d_model, shape.expand, shape.d_state, shape.d_conv,
-                             shape.n_heads, dm_dtype(dtype), shape.n_groups, flags, dir_mask, chunk, eps)
-
-
-def workspace(nbytes: int) -> torch.Tensor:
-    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+from paper_2511_15927_b200.torch_io import (cfg_of, dev, dev_dir_weights, dev_stack_weights, dm_dtype, tdtype,  # noqa: F401
+                                            workspace)
 
 
 def run_forward(shape, dtype, wf, wr, x, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, chunk=0):
@@ -72,13 +44,6 @@ def run_block_step(shape, dtype, wf, wr, x_blk, ssm_in=None, conv_in=None, want_
     dm.dm_check(st)
     f = lambda t: None if t is None else t.float().cpu().numpy().astype(np.float64)
     return f(yd), f(s_out), f(c_out)
-
-
-def dev_stack_weights(sw: dict, dtype) -> dict:
-    return {"embed": dev(sw["embed"], dtype), "w_vocab": dev(sw["w_vocab"], dtype),
-            "final_norm_w": dev(sw["final_norm_w"], dtype),
-            "layers": [{"norm_w": dev(l["norm_w"], dtype), "fwd": dev_dir_weights(l["fwd"], dtype),
-                        "rev": dev_dir_weights(l["rev"], dtype)} for l in sw["layers"]]}
 
 
 def run_denoise(shape, dtype, sw, tokens, vocab, want_logits=True, want_argmax=True, states_in=None, want_states=False,
