@@ -148,7 +148,7 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference arm's sample")
-    ap.add_argument("--cpu-baseline-tokens", type=int, default=512)
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()

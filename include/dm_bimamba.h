@@ -155,6 +155,16 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights,
                     const dm_layer_state *states,
                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* One dense projection as the mixer uses it (App. C counts 2mn FLOPs per token for a weight W in R^{m x n}):
+ *     y[r, :] = row_scale[r] * (W x[r, :]) + addend[r, :]
+ * x [rows, in_features] dtype; w [out_features, in_features] dtype; y [rows, out_features] of y_dtype
+ * (DM_F32 or DM_BF16); row_scale [rows] fp32 or NULL (= 1); addend [rows, out_features] fp32 or NULL (= 0),
+ * which may be y itself when y_dtype is DM_F32.  bf16 inputs run on the tensor cores when in_features is a
+ * multiple of 8 and the pointers are 16-byte aligned, otherwise (and for fp32) on the CUDA cores. */
+int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype,
+              int64_t rows, int32_t in_features, int32_t out_features,
+              const float *row_scale, const float *addend, void *cuda_stream);
+
 /* Same as dm_bimamba_forward, but x and y are HOST buffers (pageable or pinned): the call copies x to
  * the device, runs the mixer and copies y back, all on `cuda_stream`, then synchronises it.
  * `workspace` must hold dm_bimamba_workspace_bytes + 2*B*L*d_model*sizeof(dtype) bytes. */

@@ -67,6 +67,8 @@ _lib.dm_bimamba_block_step.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir
                                        _vp, _sz, _vp]
 _lib.dm_denoise_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_stack_weights), _vp, _vp, _vp,
                                  C.POINTER(dm_layer_state), _vp, _sz, _vp]
+_lib.dm_linear.argtypes = [C.c_int, _vp, _vp, _vp, C.c_int, C.c_int64, C.c_int32, C.c_int32, _vp, _vp, _vp]
+_lib.dm_linear.restype = C.c_int
 _lib.dm_profile_enable.argtypes = [C.c_int]
 _lib.dm_profile_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_uint64)]
 for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes", "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward",
@@ -75,7 +77,7 @@ for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes",
 
 EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
-           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read")
+           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear")
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
 
@@ -144,6 +146,12 @@ def dm_bimamba_forward(cfg, w, x: int, y: int, workspace: int, workspace_bytes: 
 def dm_bimamba_forward_host(cfg, w, x_host: int, y_host: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
     _ok(_lib.dm_bimamba_forward_host(C.byref(cfg), _dirs(w), _vp(x_host), _vp(y_host), _vp(workspace), _sz(workspace_bytes),
                                      _vp(cuda_stream)))
+
+
+def dm_linear(dtype: int, x: int, w: int, y: int, y_dtype: int, rows: int, in_features: int, out_features: int,
+              row_scale: int = 0, addend: int = 0, cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_linear(dtype, _vp(x), _vp(w), _vp(y), y_dtype, rows, in_features, out_features, _vp(row_scale or None),
+                       _vp(addend or None), _vp(cuda_stream)))
 
 
 def dm_bimamba_block_step(cfg, w, x_blk: int, ssm_state_in: int, conv_state_in: int, ssm_state_out: int,

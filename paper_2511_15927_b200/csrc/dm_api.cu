@@ -420,6 +420,22 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, co
     return DM_OK;
 }
 
+int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype, int64_t rows, int32_t in_features,
+              int32_t out_features, const float *row_scale, const float *addend, void *cuda_stream) {
+    if ((dtype != DM_F32 && dtype != DM_BF16) || (y_dtype != DM_F32 && y_dtype != DM_BF16)) return fail(DM_ERR_INVALID_ARG, "bad dtype");
+    if (!x || !w || !y) return fail(DM_ERR_INVALID_ARG, "x, w or y is NULL");
+    if (rows <= 0 || rows > (int64_t)1 << 30 || in_features <= 0 || out_features <= 0) return fail(DM_ERR_INVALID_ARG, "sizes must be positive");
+    if (x == y) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
+    if (addend && static_cast<const void *>(addend) == y && y_dtype != DM_F32) return fail(DM_ERR_INVALID_ARG, "addend may alias y only for fp32 y");
+    GemmArgs a{};
+    a.A = x; a.lda = in_features; a.B = w; a.ldb = in_features; a.C = y; a.ldc = out_features;
+    a.in_dtype = dtype; a.c_dtype = y_dtype; a.M = (int)rows; a.N = out_features; a.K = in_features;
+    a.row_scale = row_scale; a.addend = addend; a.ld_add = out_features;
+    cudaError_t e = gemm(a, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "dm_linear");
+    return DM_OK;
+}
+
 int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x_host, void *y_host,
                             void *workspace, size_t workspace_bytes, void *cuda_stream) {
     Dims m;
