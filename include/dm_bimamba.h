@@ -172,6 +172,24 @@ int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
                             const void *x_host, void *y_host,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The mixer without a caller workspace (the paper has no counterpart: this is a deployment aid).
+ * For callers that cannot hand the library device memory of their own: code running where cudaMalloc is
+ * not allowed or would stall the device (a serving loop that has given all free memory to its own pool, a
+ * plug-in host that forbids allocation, a latency-critical path, since cudaMalloc synchronises the
+ * device).  Same computation and arguments as dm_bimamba_forward, but every intermediate lives in a fixed
+ * array of DM_STATIC_WORKSPACE_BYTES that is part of the library image: each GPU that loads the library
+ * holds that much memory until the process exits.  The call allocates and frees nothing.
+ *   - A configuration whose dm_bimamba_workspace_bytes exceeds DM_STATIC_WORKSPACE_BYTES is rejected
+ *     with DM_ERR_WORKSPACE before anything is launched (use dm_bimamba_forward with your own buffer).
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  Every call
+ *     overwrites each region before reading it, so nothing needs clearing, but two calls whose kernels
+ *     can overlap on the GPU (different streams, no dependency between them) race on it: serialise them. */
+#define DM_STATIC_WORKSPACE_BYTES ((size_t)32 << 20)
+int dm_bimamba_forward_static(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
+                              const void *x, void *y, void *cuda_stream);
+
 /* Number of kernels this library has launched from this process since load (for benchmarks). */
 uint64_t dm_kernel_launch_count(void);
 

@@ -63,6 +63,8 @@ _lib.dm_denoise_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(_
 _lib.dm_check.argtypes = [_vp]
 _lib.dm_bimamba_forward.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp, _sz, _vp]
 _lib.dm_bimamba_forward_host.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp, _sz, _vp]
+_lib.dm_bimamba_forward_static.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp]
+_lib.dm_bimamba_forward_static.restype = C.c_int
 _lib.dm_bimamba_block_step.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir_weights), _vp, _vp, _vp, _vp, _vp, _vp,
                                        _vp, _sz, _vp]
 _lib.dm_denoise_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_stack_weights), _vp, _vp, _vp,
@@ -77,7 +79,8 @@ for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes",
 
 EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
-           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear")
+           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static")
+DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
 
@@ -146,6 +149,11 @@ def dm_bimamba_forward(cfg, w, x: int, y: int, workspace: int, workspace_bytes: 
 def dm_bimamba_forward_host(cfg, w, x_host: int, y_host: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
     _ok(_lib.dm_bimamba_forward_host(C.byref(cfg), _dirs(w), _vp(x_host), _vp(y_host), _vp(workspace), _sz(workspace_bytes),
                                      _vp(cuda_stream)))
+
+
+def dm_bimamba_forward_static(cfg, w, x: int, y: int, cuda_stream: int = 0) -> None:
+    """dm_bimamba_forward on the library's built-in scratch array (no workspace argument, nothing allocated)."""
+    _ok(_lib.dm_bimamba_forward_static(C.byref(cfg), _dirs(w), _vp(x), _vp(y), _vp(cuda_stream)))
 
 
 def dm_linear(dtype: int, x: int, w: int, y: int, y_dtype: int, rows: int, in_features: int, out_features: int,

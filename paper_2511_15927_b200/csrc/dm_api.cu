@@ -235,6 +235,28 @@ static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m) {
     return w;
 }
 
+// Fixed scratch for dm_bimamba_forward_static.  In host code the symbol below is only a handle: the device
+// address has to be asked for, once per device, with that device current.
+static __device__ __align__(256) unsigned char g_static_ws[DM_STATIC_WORKSPACE_BYTES];
+
+static int static_ws_ptr(char **out) {
+    static char *cached[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "dm_bimamba_forward_static: cudaGetDevice");
+    if (dev < 0 || dev >= 64) return fail(DM_ERR_UNSUPPORTED, "dm_bimamba_forward_static: device index %d out of range", dev);
+    std::lock_guard<std::mutex> lk(mu);
+    if (!cached[dev]) {
+        void *p = nullptr;
+        if ((e = cudaGetSymbolAddress(&p, g_static_ws)) != cudaSuccess)
+            return cuda_fail(e, "dm_bimamba_forward_static: cudaGetSymbolAddress");
+        cached[dev] = static_cast<char *>(p);
+    }
+    *out = cached[dev];
+    return DM_OK;
+}
+
 }  // namespace dm
 
 using namespace dm;
@@ -332,6 +354,24 @@ int dm_bimamba_forward(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const
     MixerOut out{y, cfg->dtype, nullptr, 0};
     return run_mixer(cfg, m, w, x, out, nullptr, nullptr, nullptr, nullptr, static_cast<char *>(workspace),
                      static_cast<cudaStream_t>(cuda_stream));
+}
+
+int dm_bimamba_forward_static(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x, void *y, void *cuda_stream) {
+    Dims m;
+    int st = check_cfg(cfg, &m);
+    if (st != DM_OK) return st;
+    if ((st = check_weights(cfg, w)) != DM_OK) return st;
+    if (!x || !y) return fail(DM_ERR_INVALID_ARG, "x or y is NULL");
+    if (x == y) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
+    if (!aligned16(x) || !aligned16(y)) return fail(DM_ERR_INVALID_ARG, "x and y must be 16-byte aligned");
+    const size_t need = mixer_ws(cfg, m).total;
+    if (need > DM_STATIC_WORKSPACE_BYTES)
+        return fail(DM_ERR_WORKSPACE, "this configuration needs %zu bytes of scratch, the built-in array holds %zu: "
+                    "call dm_bimamba_forward with a workspace of your own", need, (size_t)DM_STATIC_WORKSPACE_BYTES);
+    char *ws = nullptr;
+    if ((st = static_ws_ptr(&ws)) != DM_OK) return st;
+    MixerOut out{y, cfg->dtype, nullptr, 0};
+    return run_mixer(cfg, m, w, x, out, nullptr, nullptr, nullptr, nullptr, ws, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int dm_bimamba_block_step(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x_blk,
