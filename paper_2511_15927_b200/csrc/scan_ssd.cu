@@ -5,19 +5,28 @@
 // Lambda_i = sum_{r <= i} Delta_r A (inclusive, in the direction's own time order) gives
 //     y_i   = sum_{j <= i} exp(Lambda_i - Lambda_j) (C_i . B_j) Delta_j x_j  +  exp(Lambda_i) C_i . h_in  +  D x_i
 //     h_out = exp(Lambda_last) h_in + sum_j exp(Lambda_last - Lambda_j) Delta_j x_j (x) B_j
-// Only differences of Lambda with non-positive sign are exponentiated; nothing is divided by a decay.
+// Only differences of Lambda with non-positive sign are kept; nothing is divided by a decay.  Delta_j is
+// folded into the exponent (Lambda'_j = Lambda_j - log Delta_j), and D x_i into the diagonal of the masked
+// product, so that  y_i = sum_j W_ij x_j + exp(Lambda_i) C_i . h_in  with  W_ij = S_ij exp(Lambda_i - Lambda'_j) [+ D].
 //
 // Launch 1 (ssd_prep): per (direction, batch row, chunk): conv + SiLU of the B and C columns (shared by
-// all heads) to bf16, and Delta, Lambda of every head, into scratch.
+// all heads) to bf16, and Lambda, Lambda' of every head (in log2 units), into scratch.
 // Launch 2 (ssd_scan): one CTA per (batch row, direction, head) walks the chunks in the direction's time
 // order.  Both directions use the same physical chunk grid [c*Q, (c+1)*Q); the reverse direction visits
 // the chunks in descending order and uses the transposed causal mask, so nothing is ever flipped in memory.
-// Per chunk:  S = C B^T,  W = S o mask  (bf16, shared memory),  Y = W x' + diag(exp Lambda) C h_in,
-// state accumulator = B^T (w o x'), all four products as tcgen05 MMAs with fp32 accumulators in TMEM.
-// The running state h [d_state x headdim] stays in fp32 registers (one state row per thread of warps 4-7).
-//
-// Every mbarrier wait is bounded; on expiry the CTA stores DM_ERR_TIMEOUT in the device status word,
-// lets its outstanding TMA loads land (bounded), frees TMEM and returns.
+// The CTA is a pipeline of specialised warps that work on different chunks at the same time:
+//     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
+//     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  St = B^T (w o x'),  Ya = W x'
+//     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
+//     warps 4-7   copy C' into TMEM (it is the A operand of S and Yb); depthwise conv + SiLU of the x tile in place,
+//                 and the decay-weighted copy w o x'
+//     warps 8-11  mask: S (TMEM, fp32) -> W (TMEM, bf16);  state: h <- exp(Lambda_last) h + St (fp32, kept in TMEM),
+//                 bf16 copy of h for the next chunk's Yb
+//     warps 12-15 epilogue: y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w], per-head sum of squares,
+//                 written over the z tile and stored with TMA
+// Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
+// device status word, all roles leave their loops, outstanding TMA traffic is waited for (bounded), TMEM is
+// freed and the CTA returns.
 #include "dm_internal.h"
 #include "tc_ptx.cuh"
 
@@ -33,91 +42,146 @@ constexpr int HALO = 8;           // conv look-back rows kept with the x tile (8
 constexpr int XROWS = Q + HALO;
 constexpr uint32_t T16 = Q * 128;           // bytes of a [128 rows][64 bf16] tile
 constexpr uint32_t XTILE = XROWS * 128;     // 17408
-constexpr int NTHREADS = 256;
+constexpr int NX = 3, NZ = 2, NB = 2, NDL = 4;      // pipeline depths: x tile, z tile, B' tile, (Lambda, Lambda')
+constexpr int NTHREADS = 512;
+constexpr int WG = 128;                     // threads of one worker group
 
-// shared-memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t OFF_X = 0;                       // 2 stages of the x tile (raw, then conv'd in place)
-constexpr uint32_t OFF_B = OFF_X + 2 * XTILE;       // B' as two [Q][64] tiles (d_state halves)
-constexpr uint32_t OFF_C = OFF_B + 2 * T16;
-constexpr uint32_t OFF_W = OFF_C + 2 * T16;         // masked S, two [Q][64] tiles (halves of the j axis)
-constexpr uint32_t OFF_XS = OFF_W + 2 * T16;        // w_j x'_j
-constexpr uint32_t OFF_H = OFF_XS + T16;            // bf16 copy of the incoming state [d_state rows][headdim]
-constexpr uint32_t OFF_DL = OFF_H + T16;            // 2 stages x (Delta[Q], Lambda[Q]) fp32
-constexpr uint32_t OFF_MISC = OFF_DL + 2 * 2 * Q * 4;
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 1024 + 1024;   // + barriers/scalars + alignment slack
+// shared-memory map (offsets from a 1024-byte aligned base; every tile starts on a 1024-byte boundary)
+constexpr uint32_t OFF_X = 0;                           // NX stages of the x tile (raw, then conv'd in place)
+constexpr uint32_t OFF_Z = OFF_X + NX * XTILE;          // NZ stages of the z tile, overwritten by the gated output
+constexpr uint32_t OFF_B = OFF_Z + NZ * T16;            // NB stages of B' as two [Q][64] tiles (d_state halves)
+constexpr uint32_t OFF_C = OFF_B + NB * 2 * T16;        // C' in transit to TMEM, two [Q][64] tiles
+constexpr uint32_t OFF_XS = OFF_C + 2 * T16;            // w_j x'_j
+constexpr uint32_t OFF_H = OFF_XS + T16;                // bf16 copy of the incoming state [d_state rows][headdim]
+constexpr uint32_t OFF_DL = OFF_H + T16;                // NDL stages x (Lambda[Q], Lambda'[Q]) fp32
+constexpr uint32_t OFF_MISC = OFF_DL + NDL * 2 * Q * 4;
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 2048 + 1024;  // + barriers/scalars + alignment slack
+static_assert(OFF_Z % 1024 == 0 && OFF_B % 1024 == 0 && OFF_C % 1024 == 0 && OFF_XS % 1024 == 0 && OFF_H % 1024 == 0, "tile alignment");
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
-// TMEM columns
-constexpr uint32_t TM_S = 0, TM_YA = 128, TM_YB = 192, TM_ST = 256, TM_COLS = 512;
+// TMEM columns (all 512 are allocated)
+constexpr uint32_t TM_S = 0, TM_W = 128, TM_CT = 192, TM_YA = 256, TM_YB = 320, TM_ST = 384, TM_HS = 448, TM_COLS = 512;
 
 struct Misc {
-    uint64_t in_full[2], bc_full, mma_done;
+    uint64_t full_x[NX], empty_x[NX], full_z[NZ], empty_z[NZ], full_b[NB], empty_b[NB], full_c, empty_c, full_dl[NDL], empty_dl[NDL];
+    uint64_t xs_full, xs_empty, ct_full, ct_empty, s_full, s_empty, w_full, w_empty, st_full, st_empty, h_full, h_empty, y_full, y_empty;
     uint32_t tmem_base;
     int abort;
     float norm_w[P];
+    float wbuf[Q];
 };
+static_assert(sizeof(Misc) <= 2048, "Misc must fit its slot");
 
 struct SsdArgs {
     int B, L, H, d_inner, d_in_proj, conv_ch, k, flags, nch, Lp;
     const __nv_bfloat16 *zx;
-    __nv_bfloat16 *g;
     float *ssq;
-    const float *dA;             // [2][B][H][2][Lp]
+    const float *dA;             // [2][B][H][2][Lp]: Lambda, Lambda' (log2 units)
     const float *ssm_in; float *ssm_out;
     ScanDir dir[2];
 };
 
 __device__ __forceinline__ float silu_fast(float v) { return v / (1.f + __expf(-v)); }
+// SiLU through one tanh: v sigmoid(v) = h + h tanh(h), h = v/2
+__device__ __forceinline__ float silu_tanh(float v) {
+    const float h = 0.5f * v;
+    return fmaf(h, tanh_fast(h), h);
+}
 
 // --------------------------------------------------------------------------------------------------
-// Launch 1: B', C' (bf16) and Delta, Lambda (fp32) for one physical chunk of one (direction, batch row).
+// Launch 1: B', C' (bf16) and Lambda, Lambda' (fp32, log2 units) for one physical chunk of one (direction, batch row).
 // --------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, int dir0) {
+    __shared__ float dsm[Q][65];
     const int pc = blockIdx.x, b = blockIdx.y, dir = dir0 + blockIdx.z;
     const bool rev = dir == 1;
-    const int L = a.L, k = a.k;
+    const int L = a.L, k = a.k, tid = threadIdx.x;
     const ScanDir &w = a.dir[dir];
     const int64_t seq = (int64_t)dir * a.B + b;
     const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
     const int r0 = pc * Q;
     const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
-    // B and C channels
-    for (int c = threadIdx.x; c < 2 * N; c += blockDim.x) {
-        const int cc = a.d_inner + c;                                  // conv channel
+
+    // ---- B and C channels: thread = (channel pair, block of 32 rows); the 35-row window is loaded up front
+    {
+        const int cp = tid & 127, rg = tid >> 7;
+        const int cc = a.d_inner + 2 * cp;                               // conv channel of the pair's first member
         const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)cc * k;
-        float wl[4] = {0.f, 0.f, 0.f, 0.f};                            // wl[m]: weight of the row m steps back in time
-        for (int m = 0; m < k; ++m) wl[m] = __bfloat162float(cw[k - 1 - m]);
-        const float bias = has_bias ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc]) : 0.f;
-        const __nv_bfloat16 *col = zx + a.d_inner + cc;
-        auto raw = [&](int t) -> float { return (t >= 0 && t < L) ? __bfloat162float(col[(int64_t)t * a.d_in_proj]) : 0.f; };
-        __nv_bfloat16 *dst = (c < N ? Bp + c : Cp + (c - N)) + seq * L * N;
-        const int step = rev ? -1 : 1;                                 // direction of time in physical rows
-        int t = rev ? min(r0 + Q, L) - 1 : r0;
-        float h1 = raw(t - step), h2 = raw(t - 2 * step), h3 = raw(t - 3 * step);
-        const int rows = min(r0 + Q, L) - r0;
-        for (int i = 0; i < rows; ++i, t += step) {
-            const float cur = raw(t);
-            float v = bias;
-            v = fmaf(wl[3], h3, v); v = fmaf(wl[2], h2, v); v = fmaf(wl[1], h1, v); v = fmaf(wl[0], cur, v);
-            dst[(int64_t)t * N] = __float2bfloat16_rn(silu_fast(v));
-            h3 = h2; h2 = h1; h1 = cur;
+        float wl[2][4];                                                  // wl[e][m]: weight of the row m steps back in time
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+            for (int m = 0; m < 4; ++m) wl[e][m] = m < k ? __bfloat162float(cw[e * k + k - 1 - m]) : 0.f;
+        float bias[2] = {0.f, 0.f};
+        if (has_bias) {
+            bias[0] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc]);
+            bias[1] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc + 1]);
+        }
+        const uint32_t *col = reinterpret_cast<const uint32_t *>(zx + a.d_inner + cc);      // 4-byte aligned: all widths are even
+        const int64_t ld32 = a.d_in_proj / 2;
+        const int first = rev ? r0 + rg * 32 + 31 : r0 + rg * 32, step = rev ? -1 : 1;        // first-in-time row of the block
+        uint32_t raw[35];
+#pragma unroll
+        for (int i = 0; i < 35; ++i) {
+            const int t = first + (i - 3) * step;
+            raw[i] = (t >= 0 && t < L) ? __ldg(col + (int64_t)t * ld32) : 0u;
+        }
+        __nv_bfloat16 *dst = (cp < 64 ? Bp + 2 * cp : Cp + 2 * (cp - 64)) + seq * L * N;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int t = first + i * step;
+            float v0 = bias[0], v1 = bias[1];
+#pragma unroll
+            for (int m = 3; m >= 0; --m) {
+                v0 = fmaf(wl[0][m], bf16_lo(raw[i + 3 - m]), v0);
+                v1 = fmaf(wl[1][m], bf16_hi(raw[i + 3 - m]), v1);
+            }
+            if (t < L) *reinterpret_cast<uint32_t *>(dst + (int64_t)t * N) = pack_bf16(silu_fast(v0), silu_fast(v1));
         }
     }
-    // Delta and the inclusive cumulative log-decay of every head, in the direction's time order
-    for (int h = threadIdx.x; h < a.H; h += blockDim.x) {
-        const float Ah = -expf(w.A_log[h]), dtb = w.dt_bias[h];
-        float *dl = dA + ((seq * a.H + h) * 2) * a.Lp + r0, *lam = dl + a.Lp;
-        float cum = 0.f;
-        for (int i = 0; i < Q; ++i) {
-            const int r = rev ? Q - 1 - i : i, t = r0 + r;
+    // ---- Delta, then the inclusive cumulative log-decay of every head in the direction's time order
+    const float LOG2E = 1.4426950408889634f;
+    for (int h0 = 0; h0 < a.H; h0 += 64) {
+        __syncthreads();
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+            const int idx = tid + 512 * i, hh = idx & 63, r = idx >> 6, t = r0 + r, h = h0 + hh;
             float d = 0.f;
-            if (t < L) {
-                const float v = __bfloat162float(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h]) + dtb;
+            if (t < L && h < a.H) {
+                const float v = __bfloat162float(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h]) + w.dt_bias[h];
                 d = fmaxf(v, 0.f) + log1pf(expf(-fabsf(v)));
             }
-            cum = fmaf(d, Ah, cum);
-            dl[r] = d;
-            lam[r] = cum;
+            dsm[r][hh] = d;
+        }
+        __syncthreads();
+        const int warp = tid >> 5, lane = tid & 31;
+        for (int hh = warp; hh < 64 && h0 + hh < a.H; hh += 16) {
+            const int h = h0 + hh;
+            const float Ah = -expf(w.A_log[h]) * LOG2E;
+            float d[4], cum[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int tau = 4 * lane + e, r = rev ? Q - 1 - tau : tau;
+                d[e] = dsm[r][hh];
+            }
+            cum[0] = d[0] * Ah; cum[1] = fmaf(d[1], Ah, cum[0]); cum[2] = fmaf(d[2], Ah, cum[1]); cum[3] = fmaf(d[3], Ah, cum[2]);
+            float run = cum[3];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float up = __shfl_up_sync(0xffffffffu, run, off);
+                if (lane >= off) run += up;
+            }
+            const float base = run - cum[3];                             // sum over the lanes before this one
+            float lam[4], lamp[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { lam[e] = base + cum[e]; lamp[e] = lam[e] - log2f(d[e]); }    // Delta = 0 (padding): Lambda' = +inf
+            float *dl = dA + ((seq * a.H + h) * 2) * a.Lp + r0;
+            const int rlo = rev ? Q - 4 - 4 * lane : 4 * lane;           // lowest physical row of this lane's four
+            const float4 v0 = rev ? make_float4(lam[3], lam[2], lam[1], lam[0]) : make_float4(lam[0], lam[1], lam[2], lam[3]);
+            const float4 v1 = rev ? make_float4(lamp[3], lamp[2], lamp[1], lamp[0]) : make_float4(lamp[0], lamp[1], lamp[2], lamp[3]);
+            *reinterpret_cast<float4 *>(dl + rlo) = v0;
+            *reinterpret_cast<float4 *>(dl + a.Lp + rlo) = v1;
         }
     }
 }
@@ -126,8 +190,9 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
 // Launch 2: the chunked scan.
 // --------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(NTHREADS, 1)
-ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_c, const SsdArgs a, int dir0, int *status) {
+ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_z,
+                const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_c,
+                const __grid_constant__ CUtensorMap map_g, const SsdArgs a, int dir0, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Misc *misc = reinterpret_cast<Misc *>(smem + OFF_MISC);
@@ -140,261 +205,387 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const int seq = dir * a.B + b;
     const ScanDir &w = a.dir[dir];
     const bool norm_on = (a.flags & DM_FLAG_GATED_RMSNORM) != 0;
-    const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
-    const bool group_a = warp < 4;                  // conv, mask, epilogue: thread <-> token row
-    const int row = tid & 127;                      // token row (group A) or state row n (group B)
-    const int quarter = warp & 3;                   // TMEM lane quarter this warp may read
 
     if (tid == 0) {
-        mbar_init(&misc->in_full[0], 1); mbar_init(&misc->in_full[1], 1);
-        mbar_init(&misc->bc_full, 1); mbar_init(&misc->mma_done, 1);
+        for (int i = 0; i < NX; ++i) { mbar_init(&misc->full_x[i], 1); mbar_init(&misc->empty_x[i], 1); }
+        for (int i = 0; i < NZ; ++i) { mbar_init(&misc->full_z[i], 1); mbar_init(&misc->empty_z[i], 1); }
+        for (int i = 0; i < NB; ++i) { mbar_init(&misc->full_b[i], 1); mbar_init(&misc->empty_b[i], 1); }
+        for (int i = 0; i < NDL; ++i) { mbar_init(&misc->full_dl[i], 1); mbar_init(&misc->empty_dl[i], 3 * WG); }
+        mbar_init(&misc->full_c, 1);   mbar_init(&misc->empty_c, WG);
+        mbar_init(&misc->xs_full, WG); mbar_init(&misc->xs_empty, 1);
+        mbar_init(&misc->ct_full, WG); mbar_init(&misc->ct_empty, 1);
+        mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, WG);
+        mbar_init(&misc->w_full, WG);  mbar_init(&misc->w_empty, 1);
+        mbar_init(&misc->st_full, 1);  mbar_init(&misc->st_empty, WG);
+        mbar_init(&misc->h_full, WG);  mbar_init(&misc->h_empty, 1);
+        mbar_init(&misc->y_full, 1);   mbar_init(&misc->y_empty, WG);
         misc->abort = 0;
         mbar_fence_init();
     }
     if (tid < P) misc->norm_w[tid] = (norm_on && w.norm_w) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * P + tid]) : 1.f;
-    if (warp == 0) tmem_alloc(&misc->tmem_base, TM_COLS);
+    if (warp == 1) tmem_alloc(&misc->tmem_base, TM_COLS);
     fence_before();
     __syncthreads();
     fence_after();
     const uint32_t tmem = misc->tmem_base;
-
-    // conv parameters of this thread's 8 channels (group A): wl[e][m] multiplies the row m steps back in time
-    const int cc8 = row & 7, rb = row >> 3;
-    float wl[8][4], cbias[8];
-    if (group_a) {
-        const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int ch = h * P + cc8 * 8 + e;
-            const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)ch * a.k;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) wl[e][m] = m < a.k ? __bfloat162float(cw[a.k - 1 - m]) : 0.f;
-            cbias[e] = has_bias ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[ch]) : 0.f;
-        }
-    }
-    // running state of state row n = row (group B): hreg[p], fp32
-    float hreg[P];
-    if (!group_a) {
-        if (!rev && a.ssm_in) {
-            const float *h0 = a.ssm_in + (((int64_t)b * a.H + h) * P) * N + row;
-#pragma unroll
-            for (int p = 0; p < P; ++p) hreg[p] = h0[(int64_t)p * N];
-        } else {
-#pragma unroll
-            for (int p = 0; p < P; ++p) hreg[p] = 0.f;
-        }
-    }
-
+    const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's TMEM lane quarter
     const float *dA_head = a.dA + (((int64_t)seq * a.H + h) * 2) * a.Lp;
-    auto issue_in = [&](int c, int s) {             // x tile (+halo) and Delta/Lambda of chunk index c into stage s
-        const int pc = rev ? nch - 1 - c : c;
-        mbar_expect_tx(&misc->in_full[s], XTILE + 2 * Q * 4);
-        tma_load_3d(smem + OFF_X + s * XTILE, &map_x, a.d_inner + h * P, rev ? pc * Q : pc * Q - HALO, seq, &misc->in_full[s]);
-        bulk_load(smem + OFF_DL + s * 2 * Q * 4, dA_head + pc * Q, Q * 4, &misc->in_full[s]);
-        bulk_load(smem + OFF_DL + s * 2 * Q * 4 + Q * 4, dA_head + a.Lp + pc * Q, Q * 4, &misc->in_full[s]);
-    };
-    auto issue_bc = [&](int c) {
-        const int pc = rev ? nch - 1 - c : c;
-        mbar_expect_tx(&misc->bc_full, 4 * T16);
-        tma_load_3d(smem + OFF_B, &map_b, 0, pc * Q, seq, &misc->bc_full);
-        tma_load_3d(smem + OFF_B + T16, &map_b, 64, pc * Q, seq, &misc->bc_full);
-        tma_load_3d(smem + OFF_C, &map_c, 0, pc * Q, seq, &misc->bc_full);
-        tma_load_3d(smem + OFF_C + T16, &map_c, 64, pc * Q, seq, &misc->bc_full);
-    };
-    if (tid == 0) { issue_in(0, 0); issue_bc(0); }
+    auto WAIT = [&](uint64_t *bar, uint32_t parity) { return mbar_wait(bar, parity, abort_flag, status); };
 
-    uint32_t mma_phase = 0;
-    int in_issued = 1, bc_issued = 1;               // chunks whose loads have been issued (thread 0 bookkeeping)
-    bool ok = true;
-    for (int c = 0; c < nch; ++c) {
-        const int s = c & 1;
-        const int pc = rev ? nch - 1 - c : c;
-        uint8_t *xt = smem + OFF_X + s * XTILE;
-        const float *dl = reinterpret_cast<const float *>(smem + OFF_DL + s * 2 * Q * 4), *lam = dl + Q;
-        if (tid == 0 && c + 1 < nch) { issue_in(c + 1, s ^ 1); in_issued = c + 2; }
-
-        ok = mbar_wait(&misc->in_full[s], (c >> 1) & 1, abort_flag, status);
-        if (!__syncthreads_and(ok)) { ok = false; break; }
-
-        const float lam_last = lam[rev ? 0 : Q - 1];
-        // ---------------- phase A: conv + SiLU in place (group A) | bf16 copy of the incoming state (group B)
-        if (group_a) {
-            uint4 win[11];
-            const int base_row = rev ? rb * 8 : rb * 8 + HALO - 3;
-#pragma unroll
-            for (int i = 0; i < 11; ++i) {
-                const int r = base_row + i;
-                win[i] = *reinterpret_cast<const uint4 *>(xt + r * 128 + ((cc8 ^ (r & 7)) << 4));
+    if (warp == 0) {
+        // ============================================================ TMA: x tile (+halo) and Lambda, Lambda'
+        if (lane == 0) {
+            int issued = 0;
+            for (int c = 0; c < nch; ++c) {
+                const int sx = c % NX, sd = c % NDL, pc = rev ? nch - 1 - c : c;
+                if (!WAIT(&misc->empty_x[sx], ((c / NX) & 1) ^ 1) || !WAIT(&misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
+                mbar_expect_tx(&misc->full_x[sx], XTILE);
+                tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * P, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
+                mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
+                bulk_load(smem + OFF_DL + sd * 2 * Q * 4, dA_head + pc * Q, Q * 4, &misc->full_dl[sd]);
+                bulk_load(smem + OFF_DL + sd * 2 * Q * 4 + Q * 4, dA_head + a.Lp + pc * Q, Q * 4, &misc->full_dl[sd]);
+                issued = c + 1;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");          // all raw rows are read before anyone overwrites
+            if (*abort_flag)            // aborting: bounded wait for the loads still in flight
+                for (int c = max(0, issued - NDL); c < issued; ++c) {
+                    if (c >= issued - NX) mbar_wait_quiet(&misc->full_x[c % NX], (c / NX) & 1, 100000000ull);
+                    mbar_wait_quiet(&misc->full_dl[c % NDL], (c / NDL) & 1, 100000000ull);
+                }
+        }
+    } else if (warp == 2) {
+        // ============================================================ TMA: z tile
+        if (lane == 0) {
+            int issued = 0;
+            for (int c = 0; c < nch; ++c) {
+                const int sz = c % NZ, pc = rev ? nch - 1 - c : c;
+                if (!WAIT(&misc->empty_z[sz], ((c / NZ) & 1) ^ 1)) break;
+                mbar_expect_tx(&misc->full_z[sz], T16);
+                tma_load_3d(smem + OFF_Z + sz * T16, &map_z, h * P, pc * Q, seq, &misc->full_z[sz]);
+                issued = c + 1;
+            }
+            if (*abort_flag)
+                for (int c = max(0, issued - NZ); c < issued; ++c) mbar_wait_quiet(&misc->full_z[c % NZ], (c / NZ) & 1, 100000000ull);
+        }
+    } else if (warp == 3) {
+        // ============================================================ TMA: B' and C' tiles
+        if (lane == 0) {
+            int issued_b = 0, issued_c = 0;
+            for (int c = 0; c < nch; ++c) {
+                const int sb = c % NB, pc = rev ? nch - 1 - c : c;
+                if (!WAIT(&misc->empty_b[sb], ((c / NB) & 1) ^ 1)) break;
+                mbar_expect_tx(&misc->full_b[sb], 2 * T16);
+                tma_load_3d(smem + OFF_B + sb * 2 * T16, &map_b, 0, pc * Q, seq, &misc->full_b[sb]);
+                tma_load_3d(smem + OFF_B + sb * 2 * T16 + T16, &map_b, 64, pc * Q, seq, &misc->full_b[sb]);
+                issued_b = c + 1;
+                if (!WAIT(&misc->empty_c, (c & 1) ^ 1)) break;
+                mbar_expect_tx(&misc->full_c, 2 * T16);
+                tma_load_3d(smem + OFF_C, &map_c, 0, pc * Q, seq, &misc->full_c);
+                tma_load_3d(smem + OFF_C + T16, &map_c, 64, pc * Q, seq, &misc->full_c);
+                issued_c = c + 1;
+            }
+            if (*abort_flag) {
+                for (int c = max(0, issued_b - NB); c < issued_b; ++c) mbar_wait_quiet(&misc->full_b[c % NB], (c / NB) & 1, 100000000ull);
+                if (issued_c > 0) mbar_wait_quiet(&misc->full_c, (issued_c - 1) & 1, 100000000ull);
+            }
+        }
+    } else if (warp == 1) {
+        // ============================================================ MMA issuer
+        if (lane == 0) {
+            const uint32_t sH = smem_u32(smem + OFF_H), sXs = smem_u32(smem + OFF_XS);
+            for (int c = 0; c < nch; ++c) {
+                const int sb = c % NB, sx = c % NX;
+                const uint32_t par = c & 1;
+                const uint32_t sB = smem_u32(smem + OFF_B + sb * 2 * T16);
+                // S = C' B'^T  (A = C' from TMEM, B = B' K-major)
+                if (!WAIT(&misc->ct_full, par) || !WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
+                fence_after();
 #pragma unroll
-            for (int e8 = 0; e8 < 8; ++e8) {
-                const int j = rb * 8 + e8;                          // chunk row
-                const float wj = __expf(lam_last - lam[j]) * dl[j];
-                float o[8];
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_bf16_ta(tmem + TM_S, tmem + TM_CT + 8 * kk, desc_k_sw128(sB + (kk >> 2) * T16) + 2 * (kk & 3),
+                                 idesc_bf16(128, 128, 0, 0), kk != 0);
+                umma_commit(&misc->s_full);
+                // Yb = C' h_in  (B = bf16 state [n][p], MN-major)
+                if (!WAIT(&misc->h_full, par) || !WAIT(&misc->y_empty, par ^ 1)) break;
+                fence_after();
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_bf16_ta(tmem + TM_YB, tmem + TM_CT + 8 * kk, desc_mn_sw128(sH + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
+                umma_commit(&misc->ct_empty);
+                umma_commit(&misc->h_empty);
+                // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
+                if (!WAIT(&misc->xs_full, par) || !WAIT(&misc->st_empty, par ^ 1)) break;
+                fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_bf16(tmem + TM_ST, desc_mn_sw128(sB + kk * 2048, T16, 1024), desc_mn_sw128(sXs + kk * 2048, T16, 1024),
+                              idesc_bf16(128, 64, 1, 1), kk != 0);
+                umma_commit(&misc->st_full);
+                umma_commit(&misc->xs_empty);
+                umma_commit(&misc->empty_b[sb]);
+                // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
+                if (!WAIT(&misc->w_full, par)) break;
+                fence_after();
+                const uint32_t sX = smem_u32(smem + OFF_X + sx * XTILE) + (rev ? 0 : HALO * 128);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_bf16_ta(tmem + TM_YA, tmem + TM_W + 8 * kk, desc_mn_sw128(sX + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
+                umma_commit(&misc->y_full);
+                umma_commit(&misc->w_empty);
+                umma_commit(&misc->empty_x[sx]);
+            }
+        }
+    } else if (warp < 8) {
+        // ============================================================ C' -> TMEM; conv + SiLU of the x tile; w o x'
+        const int t = tid - 4 * 32;                     // 0..127; also this thread's row of C'
+        const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of 16 rows
+        float wl[4][4], cbias[4];                       // wl[e][m] multiplies the row m steps back in time
+        {
+            const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int ch = h * P + cg * 4 + e;
+                const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)ch * a.k;
+#pragma unroll
+                for (int m = 0; m < 4; ++m) wl[e][m] = m < a.k ? __bfloat162float(cw[a.k - 1 - m]) : 0.f;
+                cbias[e] = has_bias ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[ch]) : 0.f;
+            }
+        }
+        bool ok = true;
+        for (int c = 0; c < nch; ++c) {
+            const int sx = c % NX, sd = c % NDL;
+            const uint32_t par = c & 1;
+            if (ok) ok = WAIT(&misc->full_c, par) && WAIT(&misc->ct_empty, par ^ 1) && WAIT(&misc->full_x[sx], (c / NX) & 1) &&
+                         WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->xs_empty, par ^ 1);
+            if (!named_all(1, WG, ok)) { ok = false; break; }
+            fence_after();
+            // ---- C' row t -> TMEM lanes (A operand layout: lane = row, 32-bit column = two consecutive d_state entries)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t r[32];
+                const uint8_t *src = smem + OFF_C + half * T16 + t * 128;
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(src + ((c8 ^ (t & 7)) << 4));
+                    r[c8 * 4] = v.x; r[c8 * 4 + 1] = v.y; r[c8 * 4 + 2] = v.z; r[c8 * 4 + 3] = v.w;
+                }
+                tmem_st_x32(tlane + TM_CT + half * 32, r);
+            }
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(&misc->ct_full);
+            mbar_arrive(&misc->empty_c);
+            // ---- conv: raw window in time order (3 history rows, then the 16 rows of the block)
+            uint8_t *xt = smem + OFF_X + sx * XTILE;
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
+            uint2 raw[19];
+#pragma unroll
+            for (int i = 0; i < 19; ++i) {
+                const int r = rev ? rb * 16 + 18 - i : rb * 16 + i - 3 + HALO;          // tile row
+                raw[i] = *reinterpret_cast<const uint2 *>(xt + r * 128 + (((cg >> 1) ^ (r & 7)) << 4) + (cg & 1) * 8);
+            }
+            misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
+            mbar_arrive(&misc->empty_dl[sd]);
+            named_sync(1, WG);                           // every raw row is in registers before anyone overwrites; wbuf is visible
+            float h3[4] = {bf16_lo(raw[0].x), bf16_hi(raw[0].x), bf16_lo(raw[0].y), bf16_hi(raw[0].y)};
+            float h2[4] = {bf16_lo(raw[1].x), bf16_hi(raw[1].x), bf16_lo(raw[1].y), bf16_hi(raw[1].y)};
+            float h1[4] = {bf16_lo(raw[2].x), bf16_hi(raw[2].x), bf16_lo(raw[2].y), bf16_hi(raw[2].y)};
+#pragma unroll
+            for (int tau = 0; tau < 16; ++tau) {
+                const float cur[4] = {bf16_lo(raw[3 + tau].x), bf16_hi(raw[3 + tau].x), bf16_lo(raw[3 + tau].y), bf16_hi(raw[3 + tau].y)};
+                const int j = rev ? rb * 16 + 15 - tau : rb * 16 + tau;                 // chunk row
+                const float wj = misc->wbuf[j];
+                float o[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
                     float v = cbias[e];
-#pragma unroll
-                    for (int m = 3; m >= 0; --m) {
-                        const int wi = rev ? e8 + m : e8 + 3 - m;
-                        const uint32_t word = reinterpret_cast<const uint32_t *>(&win[wi])[e >> 1];
-                        v = fmaf(wl[e][m], (e & 1) ? bf16_hi(word) : bf16_lo(word), v);
-                    }
-                    o[e] = silu_fast(v);
+                    v = fmaf(wl[e][3], h3[e], v); v = fmaf(wl[e][2], h2[e], v); v = fmaf(wl[e][1], h1[e], v); v = fmaf(wl[e][0], cur[e], v);
+                    o[e] = silu_tanh(v);
+                    h3[e] = h2[e]; h2[e] = h1[e]; h1[e] = cur[e];
                 }
                 const int xr = rev ? j : j + HALO;
-                *reinterpret_cast<uint4 *>(xt + xr * 128 + ((cc8 ^ (xr & 7)) << 4)) =
-                    make_uint4(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]), pack_bf16(o[4], o[5]), pack_bf16(o[6], o[7]));
-                *reinterpret_cast<uint4 *>(smem + OFF_XS + j * 128 + ((cc8 ^ (j & 7)) << 4)) =
-                    make_uint4(pack_bf16(wj * o[0], wj * o[1]), pack_bf16(wj * o[2], wj * o[3]), pack_bf16(wj * o[4], wj * o[5]),
-                               pack_bf16(wj * o[6], wj * o[7]));
+                *reinterpret_cast<uint2 *>(xt + xr * 128 + (((cg >> 1) ^ (xr & 7)) << 4) + (cg & 1) * 8) =
+                    make_uint2(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]));
+                *reinterpret_cast<uint2 *>(smem + OFF_XS + j * 128 + (((cg >> 1) ^ (j & 7)) << 4) + (cg & 1) * 8) =
+                    make_uint2(pack_bf16(wj * o[0], wj * o[1]), pack_bf16(wj * o[2], wj * o[3]));
             }
-        } else {
-#pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8)
-                *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + ((c8 ^ (row & 7)) << 4)) =
-                    make_uint4(pack_bf16(hreg[c8 * 8], hreg[c8 * 8 + 1]), pack_bf16(hreg[c8 * 8 + 2], hreg[c8 * 8 + 3]),
-                               pack_bf16(hreg[c8 * 8 + 4], hreg[c8 * 8 + 5]), pack_bf16(hreg[c8 * 8 + 6], hreg[c8 * 8 + 7]));
+            fence_proxy_async();
+            mbar_arrive(&misc->xs_full);
         }
-        fence_proxy_async();
-        ok = mbar_wait(&misc->bc_full, c & 1, abort_flag, status);
-        fence_before();
-        if (!__syncthreads_and(ok)) { ok = false; break; }
-        // ---------------- MMAs: S = C B^T;  Y_b = C h_in;  state accumulator = B^T (w o x')
-        if (tid == 0) {
+    } else if (warp < 12) {
+        // ============================================================ mask S -> W; state update
+        const int row = tid - 8 * 32;                   // token row i (mask) / state row n (state)
+        const int q = warp & 3;
+        const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
+        // incoming state -> TMEM (fp32) and shared memory (bf16)
+        {
+            const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * N + row : nullptr;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t hs[32];
+#pragma unroll
+                for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * N]) : 0u;
+                tmem_st_x32(tlane + TM_HS + half * 32, hs);
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4)
+                    *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + (((half * 4 + c4) ^ (row & 7)) << 4)) =
+                        make_uint4(pack_bf16(__uint_as_float(hs[c4 * 8]), __uint_as_float(hs[c4 * 8 + 1])),
+                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 2]), __uint_as_float(hs[c4 * 8 + 3])),
+                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 4]), __uint_as_float(hs[c4 * 8 + 5])),
+                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 6]), __uint_as_float(hs[c4 * 8 + 7])));
+            }
+            fence_proxy_async();
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(&misc->h_full);
+        }
+        bool ok = true;
+        for (int c = 0; c < nch; ++c) {
+            const int sd = c % NDL;
+            const uint32_t par = c & 1;
+            if (ok) ok = WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->s_full, par) && WAIT(&misc->w_empty, par ^ 1);
+            if (!named_all(3, WG, ok)) { ok = false; break; }
             fence_after();
-            const uint32_t sB = smem_u32(smem + OFF_B), sC = smem_u32(smem + OFF_C), sH = smem_u32(smem + OFF_H), sXs = smem_u32(smem + OFF_XS);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint64_t dc = desc_k_sw128(sC + (kk >> 2) * T16) + 2 * (kk & 3);
-                umma_bf16(tmem + TM_S, dc, desc_k_sw128(sB + (kk >> 2) * T16) + 2 * (kk & 3), idesc_bf16(128, 128, 0, 0), kk != 0);
-                umma_bf16(tmem + TM_YB, dc, desc_mn_sw128(sH + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
-            }
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                umma_bf16(tmem + TM_ST, desc_mn_sw128(sB + kk * 2048, T16, 1024), desc_mn_sw128(sXs + kk * 2048, T16, 1024),
-                          idesc_bf16(128, 64, 1, 1), kk != 0);
-            umma_commit(&misc->mma_done);
-        }
-        ok = mbar_wait(&misc->mma_done, mma_phase, abort_flag, status);
-        mma_phase ^= 1;
-        if (!__syncthreads_and(ok)) { ok = false; break; }
-        fence_after();
-        if (tid == 0 && c + 1 < nch) { issue_bc(c + 1); bc_issued = c + 2; }     // B', C' tiles are free again
-        // ---------------- phase B: W = S o mask (group A) | state update (group B)
-        if (group_a) {
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
             const float li = lam[row];
+            const float dec = ex2f(lam[rev ? 0 : Q - 1]);
+            // ---- W_ij = S_ij 2^(Lambda_i - Lambda'_j) for j not after i in time, + D on the diagonal; 0 elsewhere
 #pragma unroll 1
             for (int jb = 0; jb < 4; ++jb) {
-                const bool needed = rev ? jb >= quarter : jb <= quarter;
+                const bool needed = rev ? jb >= q : jb <= q;
                 uint32_t out[16];
                 if (needed) {
                     uint32_t r[32];
-                    tmem_ld_x32(tmem + ((uint32_t)(quarter * 32) << 16) + TM_S + jb * 32, r);
+                    tmem_ld_x32(tlane + TM_S + jb * 32, r);
                     tmem_wait_ld();
+                    const bool diag = jb == q;
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2) {
+                    for (int jj = 0; jj < 32; jj += 4) {
                         const int j0 = jb * 32 + jj;
-                        const bool v0 = rev ? j0 >= row : j0 <= row, v1 = rev ? j0 + 1 >= row : j0 + 1 <= row;
-                        const float m0 = v0 ? __expf(li - lam[j0]) * dl[j0] : 0.f;
-                        const float m1 = v1 ? __expf(li - lam[j0 + 1]) * dl[j0 + 1] : 0.f;
-                        out[jj >> 1] = pack_bf16(__uint_as_float(r[jj]) * m0, __uint_as_float(r[jj + 1]) * m1);
+                        const float4 lp = *reinterpret_cast<const float4 *>(lamp + j0);
+                        float m[4] = {ex2f(li - lp.x), ex2f(li - lp.y), ex2f(li - lp.z), ex2f(li - lp.w)};
+                        float v[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int j = j0 + e;
+                            if (diag && (rev ? j < row : j > row)) m[e] = 0.f;
+                            v[e] = __uint_as_float(r[jj + e]) * m[e];
+                            if (diag && j == row) v[e] += Dh;
+                        }
+                        out[jj >> 1] = pack_bf16(v[0], v[1]);
+                        out[(jj >> 1) + 1] = pack_bf16(v[2], v[3]);
                     }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) out[i] = 0u;
                 }
-                uint8_t *wt = smem + OFF_W + (jb >> 1) * T16 + row * 128;
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    const int cidx = (jb & 1) * 4 + c4;
-                    *reinterpret_cast<uint4 *>(wt + ((cidx ^ (row & 7)) << 4)) = make_uint4(out[c4 * 4], out[c4 * 4 + 1], out[c4 * 4 + 2], out[c4 * 4 + 3]);
-                }
+                tmem_st_x16(tlane + TM_W + jb * 16, out);
             }
-        } else {
-            const float dec = __expf(lam_last);
+            fence_before();
+            mbar_arrive(&misc->s_empty);                 // every read of S has completed (wait::ld above)
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(&misc->w_full);
+            // ---- state: h <- 2^(Lambda_last) h + St; bf16 copy for the next chunk's Yb
+            if (!(WAIT(&misc->st_full, par) && WAIT(&misc->h_empty, par))) { ok = false; continue; }
+            fence_after();
+            const bool more = c + 1 < nch;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                uint32_t r[32];
-                tmem_ld_x32(tmem + ((uint32_t)(quarter * 32) << 16) + TM_ST + half * 32, r);
+                uint32_t st[32], hs[32];
+                tmem_ld_x32(tlane + TM_ST + half * 32, st);
+                tmem_ld_x32(tlane + TM_HS + half * 32, hs);
                 tmem_wait_ld();
 #pragma unroll
-                for (int p = 0; p < 32; ++p) hreg[half * 32 + p] = fmaf(dec, hreg[half * 32 + p], __uint_as_float(r[p]));
+                for (int p = 0; p < 32; ++p) hs[p] = __float_as_uint(fmaf(dec, __uint_as_float(hs[p]), __uint_as_float(st[p])));
+                tmem_st_x32(tlane + TM_HS + half * 32, hs);
+                if (more) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4)
+                        *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + (((half * 4 + c4) ^ (row & 7)) << 4)) =
+                            make_uint4(pack_bf16(__uint_as_float(hs[c4 * 8]), __uint_as_float(hs[c4 * 8 + 1])),
+                                       pack_bf16(__uint_as_float(hs[c4 * 8 + 2]), __uint_as_float(hs[c4 * 8 + 3])),
+                                       pack_bf16(__uint_as_float(hs[c4 * 8 + 4]), __uint_as_float(hs[c4 * 8 + 5])),
+                                       pack_bf16(__uint_as_float(hs[c4 * 8 + 6]), __uint_as_float(hs[c4 * 8 + 7])));
+                }
+            }
+            mbar_arrive(&misc->empty_dl[sd]);
+            fence_before();
+            mbar_arrive(&misc->st_empty);
+            fence_proxy_async();
+            tmem_wait_st();
+            fence_before();
+            if (more) mbar_arrive(&misc->h_full);
+        }
+        if (ok && !rev && a.ssm_out) {
+            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * N + row;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t hs[32];
+                tmem_ld_x32(tlane + TM_HS + half * 32, hs);
+                tmem_wait_ld();
+#pragma unroll
+                for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * N] = __uint_as_float(hs[p]);
             }
         }
-        fence_proxy_async();
-        fence_before();
-        __syncthreads();
-        // ---------------- MMA: Y_a = W x'
-        if (tid == 0) {
+    } else {
+        // ============================================================ epilogue
+        const int row = tid - 12 * 32;
+        bool ok = true;
+        for (int c = 0; c < nch; ++c) {
+            const int sz = c % NZ, sd = c % NDL, pc = rev ? nch - 1 - c : c;
+            const uint32_t par = c & 1;
+            if (ok) ok = WAIT(&misc->full_z[sz], (c / NZ) & 1) && WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->y_full, par);
+            if (!named_all(2, WG, ok)) { ok = false; break; }
             fence_after();
-            const uint32_t sW = smem_u32(smem + OFF_W), sX = smem_u32(xt) + (rev ? 0 : HALO * 128);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                umma_bf16(tmem + TM_YA, desc_k_sw128(sW + (kk >> 2) * T16) + 2 * (kk & 3), desc_mn_sw128(sX + kk * 2048, T16, 1024),
-                          idesc_bf16(128, 64, 0, 1), kk != 0);
-            umma_commit(&misc->mma_done);
-        }
-        ok = mbar_wait(&misc->mma_done, mma_phase, abort_flag, status);
-        mma_phase ^= 1;
-        if (!__syncthreads_and(ok)) { ok = false; break; }
-        fence_after();
-        // ---------------- phase C: y = Y_a + exp(Lambda_i) Y_b + D x';  g = y SiLU(z);  store
-        if (group_a) {
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4);
+            const float ei = ex2f(lam[row]);
+            mbar_arrive(&misc->empty_dl[sd]);
             const int t = pc * Q + row;
-            const bool valid = t < L;
-            const float ei = __expf(lam[row]);
-            const int xr = rev ? row : row + HALO;
-            const __nv_bfloat16 *zrow = a.zx + ((int64_t)seq * L + (valid ? t : 0)) * a.d_in_proj + h * P;
-            __nv_bfloat16 *grow = a.g + ((int64_t)seq * L + (valid ? t : 0)) * a.d_inner + h * P;
+            uint8_t *zt = smem + OFF_Z + sz * T16;
             float ss = 0.f;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t ya[32], yb[32];
-                tmem_ld_x32(tmem + ((uint32_t)(quarter * 32) << 16) + TM_YA + half * 32, ya);
-                tmem_ld_x32(tmem + ((uint32_t)(quarter * 32) << 16) + TM_YB + half * 32, yb);
+                tmem_ld_x32(tlane + TM_YA + half * 32, ya);
+                tmem_ld_x32(tlane + TM_YB + half * 32, yb);
                 tmem_wait_ld();
-                if (valid) {
+                if (half == 1) { fence_before(); mbar_arrive(&misc->y_empty); }
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {                 // 8 channels per 16-byte chunk
-                        const int c8 = half * 4 + c4;
-                        const uint4 xv = *reinterpret_cast<const uint4 *>(xt + xr * 128 + ((c8 ^ (xr & 7)) << 4));
-                        const uint4 zv = *reinterpret_cast<const uint4 *>(zrow + c8 * 8);
-                        const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w}, zw[4] = {zv.x, zv.y, zv.z, zv.w};
-                        uint32_t ow[4];
+                for (int c4 = 0; c4 < 4; ++c4) {                 // 8 channels per 16-byte chunk
+                    const int c8 = half * 4 + c4;
+                    uint4 *zp = reinterpret_cast<uint4 *>(zt + row * 128 + ((c8 ^ (row & 7)) << 4));
+                    const uint4 zv = *zp;
+                    const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
+                    uint32_t ow[4];
 #pragma unroll
-                        for (int e2 = 0; e2 < 4; ++e2) {
-                            const int p = c4 * 8 + e2 * 2;           // within this half
-                            const float y0 = fmaf(ei, __uint_as_float(yb[p]), __uint_as_float(ya[p])) + Dh * bf16_lo(xw[e2]);
-                            const float y1 = fmaf(ei, __uint_as_float(yb[p + 1]), __uint_as_float(ya[p + 1])) + Dh * bf16_hi(xw[e2]);
-                            const float g0 = y0 * silu_fast(bf16_lo(zw[e2])), g1 = y1 * silu_fast(bf16_hi(zw[e2]));
-                            ss = fmaf(g0, g0, ss); ss = fmaf(g1, g1, ss);
-                            ow[e2] = pack_bf16(g0 * misc->norm_w[half * 32 + p], g1 * misc->norm_w[half * 32 + p + 1]);
-                        }
-                        *reinterpret_cast<uint4 *>(grow + c8 * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                    for (int e2 = 0; e2 < 4; ++e2) {
+                        const int p = c4 * 8 + e2 * 2;           // within this half
+                        const float y0 = fmaf(ei, __uint_as_float(yb[p]), __uint_as_float(ya[p]));
+                        const float y1 = fmaf(ei, __uint_as_float(yb[p + 1]), __uint_as_float(ya[p + 1]));
+                        const float g0 = y0 * silu_tanh(bf16_lo(zw[e2])), g1 = y1 * silu_tanh(bf16_hi(zw[e2]));
+                        ss = fmaf(g0, g0, ss); ss = fmaf(g1, g1, ss);
+                        ow[e2] = pack_bf16(g0 * misc->norm_w[half * 32 + p], g1 * misc->norm_w[half * 32 + p + 1]);
                     }
+                    *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                 }
             }
-            if (valid && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss;
+            if (t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss;
+            fence_proxy_async();
+            named_sync(2, WG);
+            if (row == 0) {
+                tma_store_3d(&map_g, zt, h * P, pc * Q, seq);    // rows past the end of the sequence are clipped
+                bulk_commit();
+                bulk_wait_read0();
+                mbar_arrive(&misc->empty_z[sz]);
+            }
         }
-        fence_before();
-        __syncthreads();
+        if (row == 0) bulk_wait0();
     }
 
     // ---------------------------------------------------------------- teardown
-    if (!ok && tid == 0) {          // aborting: bounded wait for the loads still in flight
-        for (int c = max(0, in_issued - 2); c < in_issued; ++c) mbar_wait_quiet(&misc->in_full[c & 1], (c >> 1) & 1, 100000000ull);
-        if (bc_issued > 0) mbar_wait_quiet(&misc->bc_full, (bc_issued - 1) & 1, 100000000ull);
-    }
-    if (ok && !group_a && !rev && a.ssm_out) {
-        float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * N + row;
-#pragma unroll
-        for (int p = 0; p < P; ++p) ho[(int64_t)p * N] = hreg[p];
-    }
     fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 1) {
         fence_after();
         tmem_dealloc(tmem, TM_COLS);
     }
@@ -441,17 +632,17 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     SsdArgs k{};
     k.B = a.B; k.L = a.L; k.H = a.H; k.d_inner = a.d_inner; k.d_in_proj = a.d_in_proj; k.conv_ch = a.conv_ch; k.k = a.k;
     k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp;
-    k.zx = static_cast<const __nv_bfloat16 *>(a.zx); k.g = static_cast<__nv_bfloat16 *>(a.g); k.ssq = a.ssq; k.dA = dA;
+    k.zx = static_cast<const __nv_bfloat16 *>(a.zx); k.ssq = a.ssq; k.dA = dA;
     k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out;
     k.dir[0] = a.dir[0]; k.dir[1] = a.dir[1];
     const int ndir = a.dir_mask == DM_DIR_BOTH ? 2 : 1, dir0 = a.dir_mask == DM_DIR_REV ? 1 : 0;
 
-    CUtensorMap mx, mb, mc;
+    CUtensorMap mx, mz, mb, mc, mg;
     {
         const uint64_t dims[3] = {(uint64_t)a.d_in_proj, (uint64_t)a.L, (uint64_t)2 * a.B};
         const uint64_t str[2] = {(uint64_t)a.d_in_proj, (uint64_t)a.L * a.d_in_proj};
-        const uint32_t box[3] = {64, (uint32_t)XROWS, 1};
-        if (!make_map_bf16(&mx, a.zx, 3, dims, str, box)) return cudaErrorInvalidValue;
+        const uint32_t box_x[3] = {64, (uint32_t)XROWS, 1}, box_z[3] = {64, (uint32_t)Q, 1};
+        if (!make_map_bf16(&mx, a.zx, 3, dims, str, box_x) || !make_map_bf16(&mz, a.zx, 3, dims, str, box_z)) return cudaErrorInvalidValue;
     }
     {
         const uint64_t dims[3] = {(uint64_t)N, (uint64_t)a.L, (uint64_t)2 * a.B};
@@ -459,16 +650,22 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
         const uint32_t box[3] = {64, (uint32_t)Q, 1};
         if (!make_map_bf16(&mb, Bp, 3, dims, str, box) || !make_map_bf16(&mc, Cp, 3, dims, str, box)) return cudaErrorInvalidValue;
     }
+    {
+        const uint64_t dims[3] = {(uint64_t)a.d_inner, (uint64_t)a.L, (uint64_t)2 * a.B};
+        const uint64_t str[2] = {(uint64_t)a.d_inner, (uint64_t)a.L * a.d_inner};
+        const uint32_t box[3] = {64, (uint32_t)Q, 1};
+        if (!make_map_bf16(&mg, a.g, 3, dims, str, box)) return cudaErrorInvalidValue;
+    }
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
 
-    ssd_prep_kernel<<<dim3(l.nch, a.B, ndir), 256, 0, s>>>(k, Bp, Cp, dA, dir0);
+    ssd_prep_kernel<<<dim3(l.nch, a.B, ndir), 512, 0, s>>>(k, Bp, Cp, dA, dir0);
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(ssd_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    ssd_scan_kernel<<<dim3(a.H, ndir, a.B), NTHREADS, SMEM_BYTES, s>>>(mx, mb, mc, k, dir0, status);
+    ssd_scan_kernel<<<dim3(a.H, ndir, a.B), NTHREADS, SMEM_BYTES, s>>>(mx, mz, mb, mc, mg, k, dir0, status);
     count_launch();
     return cudaGetLastError();
 }
