@@ -11,7 +11,8 @@ import ctypes as C
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdm_bimamba.so")
+# DM_BIMAMBA_LIB selects another build of the same library (e.g. one compiled with different flags).
+LIB_PATH = os.environ.get("DM_BIMAMBA_LIB") or os.path.join(_HERE, "libdm_bimamba.so")
 
 DM_OK, DM_ERR_INVALID_ARG, DM_ERR_UNSUPPORTED, DM_ERR_WORKSPACE, DM_ERR_CUDA, DM_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 DM_F32, DM_BF16 = 0, 1

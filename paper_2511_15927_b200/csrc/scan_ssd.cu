@@ -16,7 +16,7 @@
 // the chunks in descending order and uses the transposed causal mask, so nothing is ever flipped in memory.
 // The CTA is a pipeline of specialised warps that work on different chunks at the same time:
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
-//     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  St = B^T (w o x'),  Ya = W x'
+//     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  St = B^T (w o x'),  Yb = C h_in,  Ya = W x'
 //     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
 //     warps 4-7   copy C' into TMEM (it is the A operand of S and Yb); depthwise conv + SiLU of the x tile in place,
 //                 and the decay-weighted copy w o x'
@@ -27,6 +27,8 @@
 // Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
 // device status word, all roles leave their loops, outstanding TMA traffic is waited for (bounded), TMEM is
 // freed and the CTA returns.
+#include <cstddef>
+
 #include "dm_internal.h"
 #include "tc_ptx.cuh"
 
@@ -55,7 +57,7 @@ constexpr uint32_t OFF_XS = OFF_C + 2 * T16;            // w_j x'_j
 constexpr uint32_t OFF_H = OFF_XS + T16;                // bf16 copy of the incoming state [d_state rows][headdim]
 constexpr uint32_t OFF_DL = OFF_H + T16;                // NDL stages x (Lambda[Q], Lambda'[Q]) fp32
 constexpr uint32_t OFF_MISC = OFF_DL + NDL * 2 * Q * 4;
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 2048 + 1024;  // + barriers/scalars + alignment slack
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 4096 + 1024;  // + barriers/scalars + alignment slack
 static_assert(OFF_Z % 1024 == 0 && OFF_B % 1024 == 0 && OFF_C % 1024 == 0 && OFF_XS % 1024 == 0 && OFF_H % 1024 == 0, "tile alignment");
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
@@ -67,10 +69,12 @@ struct Misc {
     uint64_t xs_full, xs_empty, ct_full, ct_empty, s_full, s_empty, w_full, w_empty, st_full, st_empty, h_full, h_empty, y_full, y_empty;
     uint32_t tmem_base;
     int abort;
-    float norm_w[P];
-    float wbuf[Q];
+    alignas(16) float norm_w[P];  // the three arrays below are read as float4
+    alignas(16) float wbuf[Q];
+    alignas(16) float cbuf[4][Q]; // per mask warp: column factors of the off-diagonal blocks
 };
-static_assert(sizeof(Misc) <= 2048, "Misc must fit its slot");
+static_assert(sizeof(Misc) <= 4096, "Misc must fit its slot");
+static_assert(offsetof(Misc, norm_w) % 16 == 0 && offsetof(Misc, wbuf) % 16 == 0 && offsetof(Misc, cbuf) % 16 == 0, "float4 access");
 
 struct SsdArgs {
     int B, L, H, d_inner, d_in_proj, conv_ch, k, flags, nch, Lp;
@@ -82,12 +86,6 @@ struct SsdArgs {
 };
 
 __device__ __forceinline__ float silu_fast(float v) { return v / (1.f + __expf(-v)); }
-// SiLU through one tanh: v sigmoid(v) = h + h tanh(h), h = v/2
-__device__ __forceinline__ float silu_tanh(float v) {
-    const float h = 0.5f * v;
-    return fmaf(h, tanh_fast(h), h);
-}
-
 // --------------------------------------------------------------------------------------------------
 // Launch 1: B', C' (bf16) and Lambda, Lambda' (fp32, log2 units) for one physical chunk of one (direction, batch row).
 // --------------------------------------------------------------------------------------------------
@@ -290,10 +288,26 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     } else if (warp == 1) {
         // ============================================================ MMA issuer
+        // Order per iteration: S(c), Ya(c-1), St(c), Yb(c): S(c) goes out as soon as the mask of chunk c-1 has
+        // read S(c-1), so the mask group is never waiting for more than one product.
         if (lane == 0) {
             const uint32_t sH = smem_u32(smem + OFF_H), sXs = smem_u32(smem + OFF_XS);
-            for (int c = 0; c < nch; ++c) {
-                const int sb = c % NB, sx = c % NX;
+            auto issue_ya = [&](int c) -> bool {       // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
+                const int sx = c % NX;
+                if (!WAIT(&misc->w_full, c & 1)) return false;
+                fence_after();
+                const uint32_t sX = smem_u32(smem + OFF_X + sx * XTILE) + (rev ? 0 : HALO * 128);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_bf16_ta(tmem + TM_YA, tmem + TM_W + 8 * kk, desc_mn_sw128(sX + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
+                umma_commit(&misc->y_full);
+                umma_commit(&misc->w_empty);
+                umma_commit(&misc->empty_x[sx]);
+                return true;
+            };
+            bool ok = true;
+            for (int c = 0; c < nch && ok; ++c) {
+                const int sb = c % NB;
                 const uint32_t par = c & 1;
                 const uint32_t sB = smem_u32(smem + OFF_B + sb * 2 * T16);
                 // S = C' B'^T  (A = C' from TMEM, B = B' K-major)
@@ -304,14 +318,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     umma_bf16_ta(tmem + TM_S, tmem + TM_CT + 8 * kk, desc_k_sw128(sB + (kk >> 2) * T16) + 2 * (kk & 3),
                                  idesc_bf16(128, 128, 0, 0), kk != 0);
                 umma_commit(&misc->s_full);
-                // Yb = C' h_in  (B = bf16 state [n][p], MN-major)
-                if (!WAIT(&misc->h_full, par) || !WAIT(&misc->y_empty, par ^ 1)) break;
-                fence_after();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_bf16_ta(tmem + TM_YB, tmem + TM_CT + 8 * kk, desc_mn_sw128(sH + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
-                umma_commit(&misc->ct_empty);
-                umma_commit(&misc->h_empty);
+                if (c > 0 && !issue_ya(c - 1)) break;
                 // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
                 if (!WAIT(&misc->xs_full, par) || !WAIT(&misc->st_empty, par ^ 1)) break;
                 fence_after();
@@ -322,25 +329,26 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&misc->st_full);
                 umma_commit(&misc->xs_empty);
                 umma_commit(&misc->empty_b[sb]);
-                // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
-                if (!WAIT(&misc->w_full, par)) break;
+                // Yb = C' h_in  (B = bf16 state [n][p], MN-major)
+                if (!WAIT(&misc->h_full, par) || !WAIT(&misc->y_empty, par ^ 1)) break;
                 fence_after();
-                const uint32_t sX = smem_u32(smem + OFF_X + sx * XTILE) + (rev ? 0 : HALO * 128);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    umma_bf16_ta(tmem + TM_YA, tmem + TM_W + 8 * kk, desc_mn_sw128(sX + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
-                umma_commit(&misc->y_full);
-                umma_commit(&misc->w_empty);
-                umma_commit(&misc->empty_x[sx]);
+                    umma_bf16_ta(tmem + TM_YB, tmem + TM_CT + 8 * kk, desc_mn_sw128(sH + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
+                umma_commit(&misc->ct_empty);
+                umma_commit(&misc->h_empty);
+                if (c == nch - 1) ok = issue_ya(c);
             }
         }
     } else if (warp < 8) {
         // ============================================================ C' -> TMEM; conv + SiLU of the x tile; w o x'
         const int t = tid - 4 * 32;                     // 0..127; also this thread's row of C'
         const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of 16 rows
-        float wl[4][4], cbias[4];                       // wl[e][m] multiplies the row m steps back in time
+        const uint32_t colx = cg >> 1, sub = (cg & 1) * 8;
+        f32x2 wl2[2][4], cb2[2];                        // per channel pair; wl2[.][m] multiplies the row m steps back in time
         {
             const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
+            float wl[4][4], cbias[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int ch = h * P + cg * 4 + e;
@@ -349,7 +357,16 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 for (int m = 0; m < 4; ++m) wl[e][m] = m < a.k ? __bfloat162float(cw[a.k - 1 - m]) : 0.f;
                 cbias[e] = has_bias ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[ch]) : 0.f;
             }
+#pragma unroll
+            for (int e2 = 0; e2 < 2; ++e2) {
+                cb2[e2] = pk2(cbias[2 * e2], cbias[2 * e2 + 1]);
+#pragma unroll
+                for (int m = 0; m < 4; ++m) wl2[e2][m] = pk2(wl[2 * e2][m], wl[2 * e2 + 1][m]);
+            }
         }
+        const f32x2 half2 = pk2(0.5f, 0.5f);
+        const int first = rev ? rb * 16 + 15 : rb * 16, step = rev ? -1 : 1;     // first-in-time chunk row of the block
+        const int toff = rev ? 0 : HALO;                                          // tile row = chunk row + toff
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
@@ -374,39 +391,48 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_before();
             mbar_arrive(&misc->ct_full);
             mbar_arrive(&misc->empty_c);
-            // ---- conv: raw window in time order (3 history rows, then the 16 rows of the block)
+            // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
+            // place: they are read before the group barrier; the block's own rows are read just before being replaced.
             uint8_t *xt = smem + OFF_X + sx * XTILE;
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
-            uint2 raw[19];
+            f32x2 h1[2], h2[2], h3[2];
+            {
+                uint2 hr[3];
 #pragma unroll
-            for (int i = 0; i < 19; ++i) {
-                const int r = rev ? rb * 16 + 18 - i : rb * 16 + i - 3 + HALO;          // tile row
-                raw[i] = *reinterpret_cast<const uint2 *>(xt + r * 128 + (((cg >> 1) ^ (r & 7)) << 4) + (cg & 1) * 8);
+                for (int m = 1; m <= 3; ++m) {
+                    const int r = first - m * step + toff;
+                    hr[m - 1] = *reinterpret_cast<const uint2 *>(xt + r * 128 + ((colx ^ (r & 7)) << 4) + sub);
+                }
+                h1[0] = bf2_to_f2(hr[0].x); h1[1] = bf2_to_f2(hr[0].y);
+                h2[0] = bf2_to_f2(hr[1].x); h2[1] = bf2_to_f2(hr[1].y);
+                h3[0] = bf2_to_f2(hr[2].x); h3[1] = bf2_to_f2(hr[2].y);
             }
             misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
             mbar_arrive(&misc->empty_dl[sd]);
-            named_sync(1, WG);                           // every raw row is in registers before anyone overwrites; wbuf is visible
-            float h3[4] = {bf16_lo(raw[0].x), bf16_hi(raw[0].x), bf16_lo(raw[0].y), bf16_hi(raw[0].y)};
-            float h2[4] = {bf16_lo(raw[1].x), bf16_hi(raw[1].x), bf16_lo(raw[1].y), bf16_hi(raw[1].y)};
-            float h1[4] = {bf16_lo(raw[2].x), bf16_hi(raw[2].x), bf16_lo(raw[2].y), bf16_hi(raw[2].y)};
-#pragma unroll
+            named_sync(1, WG);                           // halo rows are in registers; wbuf is visible
+#pragma unroll 4
             for (int tau = 0; tau < 16; ++tau) {
-                const float cur[4] = {bf16_lo(raw[3 + tau].x), bf16_hi(raw[3 + tau].x), bf16_lo(raw[3 + tau].y), bf16_hi(raw[3 + tau].y)};
-                const int j = rev ? rb * 16 + 15 - tau : rb * 16 + tau;                 // chunk row
+                const int j = first + tau * step, xr = j + toff;
+                uint2 *xp = reinterpret_cast<uint2 *>(xt + xr * 128 + ((colx ^ (xr & 7)) << 4) + sub);
+                const uint2 rw = *xp;
+                const f32x2 cur[2] = {bf2_to_f2(rw.x), bf2_to_f2(rw.y)};
                 const float wj = misc->wbuf[j];
-                float o[4];
+                const f32x2 w2 = pk2(wj, wj);
+                uint32_t ox[2], os[2];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = cbias[e];
-                    v = fmaf(wl[e][3], h3[e], v); v = fmaf(wl[e][2], h2[e], v); v = fmaf(wl[e][1], h1[e], v); v = fmaf(wl[e][0], cur[e], v);
-                    o[e] = silu_tanh(v);
-                    h3[e] = h2[e]; h2[e] = h1[e]; h1[e] = cur[e];
+                for (int e2 = 0; e2 < 2; ++e2) {
+                    f32x2 v = fma2(wl2[e2][3], h3[e2], cb2[e2]);
+                    v = fma2(wl2[e2][2], h2[e2], v); v = fma2(wl2[e2][1], h1[e2], v); v = fma2(wl2[e2][0], cur[e2], v);
+                    const f32x2 hh = mul2(v, half2);             // SiLU(v) = v/2 + v/2 tanh(v/2)
+                    float ha, hb;
+                    upk2(hh, ha, hb);
+                    const f32x2 o = fma2(hh, pk2(tanh_fast(ha), tanh_fast(hb)), hh);
+                    ox[e2] = f2_to_bf2(o);
+                    os[e2] = f2_to_bf2(mul2(o, w2));
+                    h3[e2] = h2[e2]; h2[e2] = h1[e2]; h1[e2] = cur[e2];
                 }
-                const int xr = rev ? j : j + HALO;
-                *reinterpret_cast<uint2 *>(xt + xr * 128 + (((cg >> 1) ^ (xr & 7)) << 4) + (cg & 1) * 8) =
-                    make_uint2(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]));
-                *reinterpret_cast<uint2 *>(smem + OFF_XS + j * 128 + (((cg >> 1) ^ (j & 7)) << 4) + (cg & 1) * 8) =
-                    make_uint2(pack_bf16(wj * o[0], wj * o[1]), pack_bf16(wj * o[2], wj * o[3]));
+                *xp = make_uint2(ox[0], ox[1]);
+                *reinterpret_cast<uint2 *>(smem + OFF_XS + j * 128 + ((colx ^ (j & 7)) << 4) + sub) = make_uint2(os[0], os[1]);
             }
             fence_proxy_async();
             mbar_arrive(&misc->xs_full);
@@ -416,6 +442,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int row = tid - 8 * 32;                   // token row i (mask) / state row n (state)
         const int q = warp & 3;
         const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
+        float *cbuf = misc->cbuf[q];
         // incoming state -> TMEM (fp32) and shared memory (bf16)
         {
             const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * N + row : nullptr;
@@ -448,37 +475,62 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
             const float li = lam[row];
             const float dec = ex2f(lam[rev ? 0 : Q - 1]);
-            // ---- W_ij = S_ij 2^(Lambda_i - Lambda'_j) for j not after i in time, + D on the diagonal; 0 elsewhere
+            // ---- W_ij = S_ij 2^(Lambda_i - Lambda'_j) for j not after i in time, + D on the diagonal; 0 elsewhere.
+            // Blocks of 32 x 32: the block on the diagonal takes one exponential per entry; a block before it (in
+            // time) uses 2^(Lambda_i - Lambda_ref) * 2^(Lambda_ref - Lambda'_j) with Lambda_ref the last row before this
+            // warp's rows -- both exponents are non-positive -- so it costs one exponential per row and per column.
+            const int n_off = rev ? 3 - q : q;
+            float ri = 1.f;
+            if (n_off > 0) {
+                const float ref = lam[rev ? 32 * (q + 1) : 32 * q - 1];
+                ri = ex2f(li - ref);
+                for (int i = 0; i < n_off; ++i) {
+                    const int j = (rev ? 32 * (q + 1) : 0) + 32 * i + lane;
+                    cbuf[j] = ex2f(ref - lamp[j]);
+                }
+                __syncwarp();
+            }
+            const f32x2 ri2 = pk2(ri, ri);
 #pragma unroll 1
-            for (int jb = 0; jb < 4; ++jb) {
-                const bool needed = rev ? jb >= q : jb <= q;
-                uint32_t out[16];
-                if (needed) {
-                    uint32_t r[32];
-                    tmem_ld_x32(tlane + TM_S + jb * 32, r);
+            for (int gi = 0; gi < 8; ++gi) {             // groups of 16 columns
+                const int jb = gi >> 1, j0 = gi * 16;
+                uint32_t out[8];
+                if (rev ? jb > q : jb < q) {
+                    uint32_t r[16];
+                    tmem_ld_x16(tlane + TM_S + j0, r);
                     tmem_wait_ld();
-                    const bool diag = jb == q;
+                    const float4 *cp = reinterpret_cast<const float4 *>(cbuf + j0);
 #pragma unroll
-                    for (int jj = 0; jj < 32; jj += 4) {
-                        const int j0 = jb * 32 + jj;
-                        const float4 lp = *reinterpret_cast<const float4 *>(lamp + j0);
-                        float m[4] = {ex2f(li - lp.x), ex2f(li - lp.y), ex2f(li - lp.z), ex2f(li - lp.w)};
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        const float4 cv = cp[v4];
+                        out[2 * v4] = f2_to_bf2(mul2(mul2(pk2(__uint_as_float(r[4 * v4]), __uint_as_float(r[4 * v4 + 1])), pk2(cv.x, cv.y)), ri2));
+                        out[2 * v4 + 1] = f2_to_bf2(mul2(mul2(pk2(__uint_as_float(r[4 * v4 + 2]), __uint_as_float(r[4 * v4 + 3])), pk2(cv.z, cv.w)), ri2));
+                    }
+                } else if (jb == q) {
+                    uint32_t r[16];
+                    tmem_ld_x16(tlane + TM_S + j0, r);
+                    tmem_wait_ld();
+                    const float4 *lp4 = reinterpret_cast<const float4 *>(lamp + j0);
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        const float4 lp = lp4[v4];
+                        const float lpv[4] = {lp.x, lp.y, lp.z, lp.w};
                         float v[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const int j = j0 + e;
-                            if (diag && (rev ? j < row : j > row)) m[e] = 0.f;
-                            v[e] = __uint_as_float(r[jj + e]) * m[e];
-                            if (diag && j == row) v[e] += Dh;
+                            const int j = j0 + 4 * v4 + e;
+                            float m = ex2f(li - lpv[e]);
+                            if (rev ? j < row : j > row) m = 0.f;
+                            v[e] = fmaf(__uint_as_float(r[4 * v4 + e]), m, j == row ? Dh : 0.f);
                         }
-                        out[jj >> 1] = pack_bf16(v[0], v[1]);
-                        out[(jj >> 1) + 1] = pack_bf16(v[2], v[3]);
+                        out[2 * v4] = pack_bf16(v[0], v[1]);
+                        out[2 * v4 + 1] = pack_bf16(v[2], v[3]);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) out[i] = 0u;
+                    for (int i = 0; i < 8; ++i) out[i] = 0u;
                 }
-                tmem_st_x16(tlane + TM_W + jb * 16, out);
+                tmem_st_x8(tlane + TM_W + gi * 8, out);
             }
             fence_before();
             mbar_arrive(&misc->s_empty);                 // every read of S has completed (wait::ld above)
@@ -489,24 +541,25 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (!(WAIT(&misc->st_full, par) && WAIT(&misc->h_empty, par))) { ok = false; continue; }
             fence_after();
             const bool more = c + 1 < nch;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t st[32], hs[32];
-                tmem_ld_x32(tlane + TM_ST + half * 32, st);
-                tmem_ld_x32(tlane + TM_HS + half * 32, hs);
+            const f32x2 dec2 = pk2(dec, dec);
+#pragma unroll 2
+            for (int c8 = 0; c8 < 8; ++c8) {             // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
+                uint32_t st[8], hs[8];
+                tmem_ld_x8(tlane + TM_ST + c8 * 8, st);
+                tmem_ld_x8(tlane + TM_HS + c8 * 8, hs);
                 tmem_wait_ld();
+                uint32_t hb[4];
 #pragma unroll
-                for (int p = 0; p < 32; ++p) hs[p] = __float_as_uint(fmaf(dec, __uint_as_float(hs[p]), __uint_as_float(st[p])));
-                tmem_st_x32(tlane + TM_HS + half * 32, hs);
-                if (more) {
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4)
-                        *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + (((half * 4 + c4) ^ (row & 7)) << 4)) =
-                            make_uint4(pack_bf16(__uint_as_float(hs[c4 * 8]), __uint_as_float(hs[c4 * 8 + 1])),
-                                       pack_bf16(__uint_as_float(hs[c4 * 8 + 2]), __uint_as_float(hs[c4 * 8 + 3])),
-                                       pack_bf16(__uint_as_float(hs[c4 * 8 + 4]), __uint_as_float(hs[c4 * 8 + 5])),
-                                       pack_bf16(__uint_as_float(hs[c4 * 8 + 6]), __uint_as_float(hs[c4 * 8 + 7])));
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    const f32x2 hn = fma2(dec2, pk2(__uint_as_float(hs[2 * e2]), __uint_as_float(hs[2 * e2 + 1])),
+                                          pk2(__uint_as_float(st[2 * e2]), __uint_as_float(st[2 * e2 + 1])));
+                    float lo, hi;
+                    upk2(hn, lo, hi);
+                    hs[2 * e2] = __float_as_uint(lo); hs[2 * e2 + 1] = __float_as_uint(hi);
+                    hb[e2] = pack_bf16(lo, hi);
                 }
+                tmem_st_x8(tlane + TM_HS + c8 * 8, hs);
+                if (more) *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + ((c8 ^ (row & 7)) << 4)) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
             }
             mbar_arrive(&misc->empty_dl[sd]);
             fence_before();
@@ -542,33 +595,37 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             mbar_arrive(&misc->empty_dl[sd]);
             const int t = pc * Q + row;
             uint8_t *zt = smem + OFF_Z + sz * T16;
-            float ss = 0.f;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t ya[32], yb[32];
-                tmem_ld_x32(tlane + TM_YA + half * 32, ya);
-                tmem_ld_x32(tlane + TM_YB + half * 32, yb);
+            const f32x2 ei2 = pk2(ei, ei), half2 = pk2(0.5f, 0.5f);
+            f32x2 ss2 = pk2(0.f, 0.f);
+#pragma unroll 2
+            for (int c8 = 0; c8 < 8; ++c8) {             // 8 channels (one 16-byte chunk of z) at a time
+                uint32_t ya[8], yb[8];
+                tmem_ld_x8(tlane + TM_YA + c8 * 8, ya);
+                tmem_ld_x8(tlane + TM_YB + c8 * 8, yb);
                 tmem_wait_ld();
-                if (half == 1) { fence_before(); mbar_arrive(&misc->y_empty); }
+                if (c8 == 7) { fence_before(); mbar_arrive(&misc->y_empty); }
+                uint4 *zp = reinterpret_cast<uint4 *>(zt + row * 128 + ((c8 ^ (row & 7)) << 4));
+                const uint4 zv = *zp;
+                const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
+                const float4 n0 = *reinterpret_cast<const float4 *>(misc->norm_w + c8 * 8), n1 = *reinterpret_cast<const float4 *>(misc->norm_w + c8 * 8 + 4);
+                const f32x2 nw[4] = {pk2(n0.x, n0.y), pk2(n0.z, n0.w), pk2(n1.x, n1.y), pk2(n1.z, n1.w)};
+                uint32_t ow[4];
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {                 // 8 channels per 16-byte chunk
-                    const int c8 = half * 4 + c4;
-                    uint4 *zp = reinterpret_cast<uint4 *>(zt + row * 128 + ((c8 ^ (row & 7)) << 4));
-                    const uint4 zv = *zp;
-                    const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
-                    uint32_t ow[4];
-#pragma unroll
-                    for (int e2 = 0; e2 < 4; ++e2) {
-                        const int p = c4 * 8 + e2 * 2;           // within this half
-                        const float y0 = fmaf(ei, __uint_as_float(yb[p]), __uint_as_float(ya[p]));
-                        const float y1 = fmaf(ei, __uint_as_float(yb[p + 1]), __uint_as_float(ya[p + 1]));
-                        const float g0 = y0 * silu_tanh(bf16_lo(zw[e2])), g1 = y1 * silu_tanh(bf16_hi(zw[e2]));
-                        ss = fmaf(g0, g0, ss); ss = fmaf(g1, g1, ss);
-                        ow[e2] = pack_bf16(g0 * misc->norm_w[half * 32 + p], g1 * misc->norm_w[half * 32 + p + 1]);
-                    }
-                    *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    const f32x2 y = fma2(ei2, pk2(__uint_as_float(yb[2 * e2]), __uint_as_float(yb[2 * e2 + 1])),
+                                         pk2(__uint_as_float(ya[2 * e2]), __uint_as_float(ya[2 * e2 + 1])));
+                    const f32x2 hh = mul2(bf2_to_f2(zw[e2]), half2);     // SiLU(z) = z/2 + z/2 tanh(z/2)
+                    float ha, hb;
+                    upk2(hh, ha, hb);
+                    const f32x2 g = mul2(y, fma2(hh, pk2(tanh_fast(ha), tanh_fast(hb)), hh));
+                    ss2 = fma2(g, g, ss2);
+                    ow[e2] = f2_to_bf2(mul2(g, nw[e2]));
                 }
+                *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
             }
+            float ss, ss_hi;
+            upk2(ss2, ss, ss_hi);
+            ss += ss_hi;
             if (t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss;
             fence_proxy_async();
             named_sync(2, WG);
