@@ -16,10 +16,9 @@
 // the chunks in descending order and uses the transposed causal mask, so nothing is ever flipped in memory.
 // The CTA is a pipeline of specialised warps that work on different chunks at the same time:
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
-//     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  St = B^T (w o x'),  Yb = C h_in,  Ya = W x'
+//     warp 1      copies C' into TMEM (tcgen05.cp; it is the A operand of S and Yb) and issues the four tcgen05 products of a chunk:  S = C B^T,  St = B^T (w o x'),  Yb = C h_in,  Ya = W x'
 //     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
-//     warps 4-7   copy C' into TMEM (it is the A operand of S and Yb); depthwise conv + SiLU of the x tile in place,
-//                 and the decay-weighted copy w o x'
+//     warps 4-7   depthwise conv + SiLU of the x tile in place, and the decay-weighted copy w o x'
 //     warps 8-11  mask: S (TMEM, fp32) -> W (TMEM, bf16);  state: h <- exp(Lambda_last) h + St (fp32, kept in TMEM),
 //                 bf16 copy of h for the next chunk's Yb
 //     warps 12-15 epilogue: y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w], per-head sum of squares,
@@ -209,7 +208,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int i = 0; i < NZ; ++i) { mbar_init(&misc->full_z[i], 1); mbar_init(&misc->empty_z[i], 1); }
         for (int i = 0; i < NB; ++i) { mbar_init(&misc->full_b[i], 1); mbar_init(&misc->empty_b[i], 1); }
         for (int i = 0; i < NDL; ++i) { mbar_init(&misc->full_dl[i], 1); mbar_init(&misc->empty_dl[i], 3 * WG); }
-        mbar_init(&misc->full_c, 1);   mbar_init(&misc->empty_c, WG);
+        mbar_init(&misc->full_c, 1);   mbar_init(&misc->empty_c, 1);
         mbar_init(&misc->xs_full, WG); mbar_init(&misc->xs_empty, 1);
         mbar_init(&misc->ct_full, WG); mbar_init(&misc->ct_empty, 1);
         mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, WG);
@@ -305,13 +304,25 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&misc->empty_x[sx]);
                 return true;
             };
-            bool ok = true;
+            // C' of chunk c: shared memory -> TMEM (A operand of S and Yb), by tcgen05.cp from this thread, so that it is
+            // ordered before the products that follow; the transit buffer is released when the copies have completed
+            auto copy_c = [&](int c) -> bool {
+                if (!WAIT(&misc->full_c, c & 1) || !WAIT(&misc->ct_empty, (c & 1) ^ 1)) return false;
+                fence_after();
+                const uint32_t sC = smem_u32(smem + OFF_C);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    tmem_cp_128x256b(tmem + TM_CT + 8 * kk, desc_k_sw128(sC + (kk >> 2) * T16) + 2 * (kk & 3));
+                umma_commit(&misc->empty_c);
+                return true;
+            };
+            bool ok = copy_c(0);
             for (int c = 0; c < nch && ok; ++c) {
                 const int sb = c % NB;
                 const uint32_t par = c & 1;
                 const uint32_t sB = smem_u32(smem + OFF_B + sb * 2 * T16);
                 // S = C' B'^T  (A = C' from TMEM, B = B' K-major)
-                if (!WAIT(&misc->ct_full, par) || !WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
+                if (!WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
                 fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
@@ -338,10 +349,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&misc->ct_empty);
                 umma_commit(&misc->h_empty);
                 if (c == nch - 1) ok = issue_ya(c);
+                else ok = copy_c(c + 1);
             }
         }
     } else if (warp < 8) {
-        // ============================================================ C' -> TMEM; conv + SiLU of the x tile; w o x'
+        // ============================================================ conv + SiLU of the x tile; w o x'
         const int t = tid - 4 * 32;                     // 0..127; also this thread's row of C'
         const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of 16 rows
         const uint32_t colx = cg >> 1, sub = (cg & 1) * 8;
@@ -371,26 +383,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
             const uint32_t par = c & 1;
-            if (ok) ok = WAIT(&misc->full_c, par) && WAIT(&misc->ct_empty, par ^ 1) && WAIT(&misc->full_x[sx], (c / NX) & 1) &&
-                         WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->xs_empty, par ^ 1);
+            if (ok) ok = WAIT(&misc->full_x[sx], (c / NX) & 1) && WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->xs_empty, par ^ 1);
             if (!named_all(1, WG, ok)) { ok = false; break; }
-            fence_after();
-            // ---- C' row t -> TMEM lanes (A operand layout: lane = row, 32-bit column = two consecutive d_state entries)
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t r[32];
-                const uint8_t *src = smem + OFF_C + half * T16 + t * 128;
-#pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(src + ((c8 ^ (t & 7)) << 4));
-                    r[c8 * 4] = v.x; r[c8 * 4 + 1] = v.y; r[c8 * 4 + 2] = v.z; r[c8 * 4 + 3] = v.w;
-                }
-                tmem_st_x32(tlane + TM_CT + half * 32, r);
-            }
-            tmem_wait_st();
-            fence_before();
-            mbar_arrive(&misc->ct_full);
-            mbar_arrive(&misc->empty_c);
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
             // place: they are read before the group barrier; the block's own rows are read just before being replaced.
             uint8_t *xt = smem + OFF_X + sx * XTILE;

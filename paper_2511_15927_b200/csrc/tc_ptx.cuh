@@ -150,6 +150,11 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, u
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Copy of one K = 16 slice (128 rows x 32 bytes) of a K-major shared-memory operand into TMEM, in the layout the
+// MMA expects for an A operand held in TMEM (row m in lane m, 8 columns of bf16 pairs).
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t s_desc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
+}
 // TMA store of a shared-memory tile (bulk async-group completion).
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, const void *smem_src, int x, int y, int z) {
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
@@ -210,6 +215,15 @@ __device__ __forceinline__ uint32_t f2_to_bf2(f32x2 v) {
     upk2(v, lo, hi);
     __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&b);
+}
+
+// Compiler-level ordering for pipelined TMEM loads: placed after tmem_wait_ld(), it makes every later use of the
+// loaded registers depend on a point after the wait (volatile asm statements keep their order).
+__device__ __forceinline__ void reg_fence8(uint32_t *r) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]));
+}
+__device__ __forceinline__ void reg_fence32(uint32_t *r) {
+    reg_fence8(r); reg_fence8(r + 8); reg_fence8(r + 16); reg_fence8(r + 24);
 }
 
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
