@@ -290,15 +290,21 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // Order per iteration: S(c), Ya(c-1), St(c), Yb(c): S(c) goes out as soon as the mask of chunk c-1 has
         // read S(c-1), so the mask group is never waiting for more than one product.
         if (lane == 0) {
-            const uint32_t sH = smem_u32(smem + OFF_H), sXs = smem_u32(smem + OFF_XS);
+            // low halves of the operand descriptors; a K step of 16 advances a K-major operand by 32 bytes inside its
+            // 64-wide tile (+2) or to the next tile (+T16/16), an MN-major operand by 16 rows (+2048/16)
+            const uint32_t dH = desc_lo_mn(smem_u32(smem + OFF_H), T16), dXs = desc_lo_mn(smem_u32(smem + OFF_XS), T16);
+            const uint32_t dC = desc_lo_k(smem_u32(smem + OFF_C));
+            const uint32_t dBk0 = desc_lo_k(smem_u32(smem + OFF_B)), dBm0 = desc_lo_mn(smem_u32(smem + OFF_B), T16);
+            const uint32_t dX0 = desc_lo_mn(smem_u32(smem + OFF_X) + (rev ? 0 : HALO * 128), T16);
+            constexpr uint32_t I128 = idesc_bf16(128, 128, 0, 0), I64 = idesc_bf16(128, 64, 0, 1), I64T = idesc_bf16(128, 64, 1, 1);
             auto issue_ya = [&](int c) -> bool {       // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
                 const int sx = c % NX;
                 if (!WAIT(&misc->w_full, c & 1)) return false;
                 fence_after();
-                const uint32_t sX = smem_u32(smem + OFF_X + sx * XTILE) + (rev ? 0 : HALO * 128);
+                const uint32_t dX = dX0 + (uint32_t)sx * (XTILE >> 4);
+                umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_bf16_ta(tmem + TM_YA, tmem + TM_W + 8 * kk, desc_mn_sw128(sX + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
+                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
                 umma_commit(&misc->y_full);
                 umma_commit(&misc->w_empty);
                 umma_commit(&misc->empty_x[sx]);
@@ -309,10 +315,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             auto copy_c = [&](int c) -> bool {
                 if (!WAIT(&misc->full_c, c & 1) || !WAIT(&misc->ct_empty, (c & 1) ^ 1)) return false;
                 fence_after();
-                const uint32_t sC = smem_u32(smem + OFF_C);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    tmem_cp_128x256b(tmem + TM_CT + 8 * kk, desc_k_sw128(sC + (kk >> 2) * T16) + 2 * (kk & 3));
+                for (int kk = 0; kk < 8; ++kk) tmem_cp_128x256b_lo(tmem + TM_CT + 8 * kk, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3));
                 umma_commit(&misc->empty_c);
                 return true;
             };
@@ -320,32 +324,30 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int c = 0; c < nch && ok; ++c) {
                 const int sb = c % NB;
                 const uint32_t par = c & 1;
-                const uint32_t sB = smem_u32(smem + OFF_B + sb * 2 * T16);
+                const uint32_t dBk = dBk0 + (uint32_t)sb * (2 * T16 >> 4), dBm = dBm0 + (uint32_t)sb * (2 * T16 >> 4);
                 // S = C' B'^T  (A = C' from TMEM, B = B' K-major)
                 if (!WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
                 fence_after();
+                umma_ts<0>(tmem + TM_S, tmem + TM_CT, dBk, I128);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_bf16_ta(tmem + TM_S, tmem + TM_CT + 8 * kk, desc_k_sw128(sB + (kk >> 2) * T16) + 2 * (kk & 3),
-                                 idesc_bf16(128, 128, 0, 0), kk != 0);
+                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_S, tmem + TM_CT + 8 * kk, dBk + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), I128);
                 umma_commit(&misc->s_full);
                 if (c > 0 && !issue_ya(c - 1)) break;
                 // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
                 if (!WAIT(&misc->xs_full, par) || !WAIT(&misc->st_empty, par ^ 1)) break;
                 fence_after();
+                umma_ss<0>(tmem + TM_ST, dBm, dXs, I64T);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_bf16(tmem + TM_ST, desc_mn_sw128(sB + kk * 2048, T16, 1024), desc_mn_sw128(sXs + kk * 2048, T16, 1024),
-                              idesc_bf16(128, 64, 1, 1), kk != 0);
+                for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tmem + TM_ST, dBm + kk * 128, dXs + kk * 128, I64T);
                 umma_commit(&misc->st_full);
                 umma_commit(&misc->xs_empty);
                 umma_commit(&misc->empty_b[sb]);
                 // Yb = C' h_in  (B = bf16 state [n][p], MN-major)
                 if (!WAIT(&misc->h_full, par) || !WAIT(&misc->y_empty, par ^ 1)) break;
                 fence_after();
+                umma_ts<0>(tmem + TM_YB, tmem + TM_CT, dH, I64);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_bf16_ta(tmem + TM_YB, tmem + TM_CT + 8 * kk, desc_mn_sw128(sH + kk * 2048, T16, 1024), idesc_bf16(128, 64, 0, 1), kk != 0);
+                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_YB, tmem + TM_CT + 8 * kk, dH + kk * 128, I64);
                 umma_commit(&misc->ct_empty);
                 umma_commit(&misc->h_empty);
                 if (c == nch - 1) ok = issue_ya(c);
