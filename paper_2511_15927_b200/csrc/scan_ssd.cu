@@ -44,8 +44,10 @@ constexpr int XROWS = Q + HALO;
 constexpr uint32_t T16 = Q * 128;           // bytes of a [128 rows][64 bf16] tile
 constexpr uint32_t XTILE = XROWS * 128;     // 17408
 constexpr int NX = 3, NZ = 2, NB = 2, NDL = 4;      // pipeline depths: x tile, z tile, B' tile, (Lambda, Lambda')
-constexpr int NTHREADS = 512;
-constexpr int WG = 128;                     // threads of one worker group
+constexpr int WG = 128;                     // threads of one worker group (four warps = the four TMEM lane quarters)
+constexpr int NWG = 2;                      // worker groups per role: conv, mask + state, epilogue (the column splits below assume 2)
+constexpr int ROLE = NWG * WG;              // threads of one role
+constexpr int NTHREADS = 128 + 3 * ROLE;    // warps 0-3: TMA producers and the MMA issuer
 
 // shared-memory map (offsets from a 1024-byte aligned base; every tile starts on a 1024-byte boundary)
 constexpr uint32_t OFF_X = 0;                           // NX stages of the x tile (raw, then conv'd in place)
@@ -56,7 +58,7 @@ constexpr uint32_t OFF_XS = OFF_C + 2 * T16;            // w_j x'_j
 constexpr uint32_t OFF_H = OFF_XS + T16;                // bf16 copy of the incoming state [d_state rows][headdim]
 constexpr uint32_t OFF_DL = OFF_H + T16;                // NDL stages x (Lambda[Q], Lambda'[Q]) fp32
 constexpr uint32_t OFF_MISC = OFF_DL + NDL * 2 * Q * 4;
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 4096 + 1024;  // + barriers/scalars + alignment slack
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 7168 + 1024;  // + barriers/scalars + alignment slack
 static_assert(OFF_Z % 1024 == 0 && OFF_B % 1024 == 0 && OFF_C % 1024 == 0 && OFF_XS % 1024 == 0 && OFF_H % 1024 == 0, "tile alignment");
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
@@ -70,9 +72,10 @@ struct Misc {
     int abort;
     alignas(16) float norm_w[P];  // the three arrays below are read as float4
     alignas(16) float wbuf[Q];
-    alignas(16) float cbuf[4][Q]; // per mask warp: column factors of the off-diagonal blocks
+    alignas(16) float cbuf[NWG][4][Q]; // per mask warp: column factors of the off-diagonal blocks
+    float ssq_part[Q];            // sum of squares of the second epilogue group's channels
 };
-static_assert(sizeof(Misc) <= 4096, "Misc must fit its slot");
+static_assert(sizeof(Misc) <= 7168, "Misc must fit its slot");
 static_assert(offsetof(Misc, norm_w) % 16 == 0 && offsetof(Misc, wbuf) % 16 == 0 && offsetof(Misc, cbuf) % 16 == 0, "float4 access");
 
 struct SsdArgs {
@@ -207,15 +210,15 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int i = 0; i < NX; ++i) { mbar_init(&misc->full_x[i], 1); mbar_init(&misc->empty_x[i], 1); }
         for (int i = 0; i < NZ; ++i) { mbar_init(&misc->full_z[i], 1); mbar_init(&misc->empty_z[i], 1); }
         for (int i = 0; i < NB; ++i) { mbar_init(&misc->full_b[i], 1); mbar_init(&misc->empty_b[i], 1); }
-        for (int i = 0; i < NDL; ++i) { mbar_init(&misc->full_dl[i], 1); mbar_init(&misc->empty_dl[i], 3 * WG); }
+        for (int i = 0; i < NDL; ++i) { mbar_init(&misc->full_dl[i], 1); mbar_init(&misc->empty_dl[i], 3 * ROLE); }
         mbar_init(&misc->full_c, 1);   mbar_init(&misc->empty_c, 1);
-        mbar_init(&misc->xs_full, WG); mbar_init(&misc->xs_empty, 1);
+        mbar_init(&misc->xs_full, ROLE); mbar_init(&misc->xs_empty, 1);
         mbar_init(&misc->ct_full, WG); mbar_init(&misc->ct_empty, 1);
-        mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, WG);
-        mbar_init(&misc->w_full, WG);  mbar_init(&misc->w_empty, 1);
-        mbar_init(&misc->st_full, 1);  mbar_init(&misc->st_empty, WG);
-        mbar_init(&misc->h_full, WG);  mbar_init(&misc->h_empty, 1);
-        mbar_init(&misc->y_full, 1);   mbar_init(&misc->y_empty, WG);
+        mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, ROLE);
+        mbar_init(&misc->w_full, ROLE);  mbar_init(&misc->w_empty, 1);
+        mbar_init(&misc->st_full, 1);  mbar_init(&misc->st_empty, ROLE);
+        mbar_init(&misc->h_full, ROLE);  mbar_init(&misc->h_empty, 1);
+        mbar_init(&misc->y_full, 1);   mbar_init(&misc->y_empty, ROLE);
         misc->abort = 0;
         mbar_fence_init();
     }
@@ -354,10 +357,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 else ok = copy_c(c + 1);
             }
         }
-    } else if (warp < 8) {
+    } else if (warp < 4 + 4 * NWG) {
         // ============================================================ conv + SiLU of the x tile; w o x'
-        const int t = tid - 4 * 32;                     // 0..127; also this thread's row of C'
-        const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of 16 rows
+        constexpr int RB = Q * 16 / ROLE;               // rows per thread
+        const int t = tid - 4 * 32;                     // 0..ROLE-1
+        const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of RB rows
         const uint32_t colx = cg >> 1, sub = (cg & 1) * 8;
         f32x2 wl2[2][4], cb2[2];                        // per channel pair; wl2[.][m] multiplies the row m steps back in time
         {
@@ -379,14 +383,14 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
         }
         const f32x2 half2 = pk2(0.5f, 0.5f);
-        const int first = rev ? rb * 16 + 15 : rb * 16, step = rev ? -1 : 1;     // first-in-time chunk row of the block
+        const int first = rev ? rb * RB + RB - 1 : rb * RB, step = rev ? -1 : 1;   // first-in-time chunk row of the block
         const int toff = rev ? 0 : HALO;                                          // tile row = chunk row + toff
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
             const uint32_t par = c & 1;
             if (ok) ok = WAIT(&misc->full_x[sx], (c / NX) & 1) && WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->xs_empty, par ^ 1);
-            if (!named_all(1, WG, ok)) { ok = false; break; }
+            if (!named_all(1, ROLE, ok)) { ok = false; break; }
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
             // place: they are read before the group barrier; the block's own rows are read just before being replaced.
             uint8_t *xt = smem + OFF_X + sx * XTILE;
@@ -403,11 +407,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 h2[0] = bf2_to_f2(hr[1].x); h2[1] = bf2_to_f2(hr[1].y);
                 h3[0] = bf2_to_f2(hr[2].x); h3[1] = bf2_to_f2(hr[2].y);
             }
-            misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
+            if (t < Q) misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
             mbar_arrive(&misc->empty_dl[sd]);
-            named_sync(1, WG);                           // halo rows are in registers; wbuf is visible
-#pragma unroll 4
-            for (int tau = 0; tau < 16; ++tau) {
+            named_sync(1, ROLE);                           // halo rows are in registers; wbuf is visible
+#pragma unroll 2
+            for (int tau = 0; tau < RB; ++tau) {
                 const int j = first + tau * step, xr = j + toff;
                 uint2 *xp = reinterpret_cast<uint2 *>(xt + xr * 128 + ((colx ^ (xr & 7)) << 4) + sub);
                 const uint2 rw = *xp;
@@ -433,17 +437,20 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_proxy_async();
             mbar_arrive(&misc->xs_full);
         }
-    } else if (warp < 12) {
+    } else if (warp < 4 + 8 * NWG) {
         // ============================================================ mask S -> W; state update
-        const int row = tid - 8 * 32;                   // token row i (mask) / state row n (state)
+        // The NWG groups share every row: group g takes the 16-column groups gi = g, g + NWG, ... of the mask and the
+        // state columns [g, g+1) * P / NWG, so the triangular mask is split evenly between them.
+        const int mg = (warp - 4 - 4 * NWG) >> 2;       // group index
+        const int row = (tid - (4 + 4 * NWG) * 32) & (WG - 1);      // token row i (mask) / state row n (state)
         const int q = warp & 3;
         const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
-        float *cbuf = misc->cbuf[q];
+        float *cbuf = misc->cbuf[mg][q];
         // incoming state -> TMEM (fp32) and shared memory (bf16)
         {
             const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * N + row : nullptr;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            {
+                const int half = mg;                     // this group's half of the state columns
                 uint32_t hs[32];
 #pragma unroll
                 for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * N]) : 0u;
@@ -466,7 +473,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const int sd = c % NDL;
             const uint32_t par = c & 1;
             if (ok) ok = WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->s_full, par) && WAIT(&misc->w_empty, par ^ 1);
-            if (!named_all(3, WG, ok)) { ok = false; break; }
+            if (!named_all(3 + mg, WG, ok)) { ok = false; break; }
             fence_after();
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
             const float li = lam[row];
@@ -488,7 +495,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
             const f32x2 ri2 = pk2(ri, ri);
 #pragma unroll 1
-            for (int gi = 0; gi < 8; ++gi) {             // groups of 16 columns
+            for (int gi = mg; gi < 8; gi += NWG) {        // this group's share of the 8 groups of 16 columns
                 const int jb = gi >> 1, j0 = gi * 16;
                 uint32_t out[8];
                 if (rev ? jb > q : jb < q) {
@@ -538,8 +545,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_after();
             const bool more = c + 1 < nch;
             const f32x2 dec2 = pk2(dec, dec);
-#pragma unroll 2
-            for (int c8 = 0; c8 < 8; ++c8) {             // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
+#pragma unroll 1
+            for (int c8 = mg * 4; c8 < mg * 4 + 4; ++c8) {   // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
                 uint32_t st[8], hs[8];
                 tmem_ld_x8(tlane + TM_ST + c8 * 8, st);
                 tmem_ld_x8(tlane + TM_HS + c8 * 8, hs);
@@ -567,8 +574,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
         if (ok && !rev && a.ssm_out) {
             float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * N + row;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            {
+                const int half = mg;
                 uint32_t hs[32];
                 tmem_ld_x32(tlane + TM_HS + half * 32, hs);
                 tmem_wait_ld();
@@ -578,13 +585,14 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     } else {
         // ============================================================ epilogue
-        const int row = tid - 12 * 32;
+        const int eg = (warp - 4 - 8 * NWG) >> 2;       // group index: channels [eg, eg+1) * P / NWG
+        const int row = (tid - (4 + 8 * NWG) * 32) & (WG - 1);
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sz = c % NZ, sd = c % NDL, pc = rev ? nch - 1 - c : c;
             const uint32_t par = c & 1;
             if (ok) ok = WAIT(&misc->full_z[sz], (c / NZ) & 1) && WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->y_full, par);
-            if (!named_all(2, WG, ok)) { ok = false; break; }
+            if (!named_all(2, ROLE, ok)) { ok = false; break; }
             fence_after();
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4);
             const float ei = ex2f(lam[row]);
@@ -593,13 +601,13 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             uint8_t *zt = smem + OFF_Z + sz * T16;
             const f32x2 ei2 = pk2(ei, ei), half2 = pk2(0.5f, 0.5f);
             f32x2 ss2 = pk2(0.f, 0.f);
-#pragma unroll 2
-            for (int c8 = 0; c8 < 8; ++c8) {             // 8 channels (one 16-byte chunk of z) at a time
+#pragma unroll 1
+            for (int c8 = eg * 4; c8 < eg * 4 + 4; ++c8) {   // 8 channels (one 16-byte chunk of z) at a time
                 uint32_t ya[8], yb[8];
                 tmem_ld_x8(tlane + TM_YA + c8 * 8, ya);
                 tmem_ld_x8(tlane + TM_YB + c8 * 8, yb);
                 tmem_wait_ld();
-                if (c8 == 7) { fence_before(); mbar_arrive(&misc->y_empty); }
+                if (c8 == eg * 4 + 3) { fence_before(); mbar_arrive(&misc->y_empty); }
                 uint4 *zp = reinterpret_cast<uint4 *>(zt + row * 128 + ((c8 ^ (row & 7)) << 4));
                 const uint4 zv = *zp;
                 const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
@@ -622,17 +630,18 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             float ss, ss_hi;
             upk2(ss2, ss, ss_hi);
             ss += ss_hi;
-            if (t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss;
+            if (eg == 1) misc->ssq_part[row] = ss;
             fence_proxy_async();
-            named_sync(2, WG);
-            if (row == 0) {
+            named_sync(2, ROLE);
+            if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + misc->ssq_part[row];
+            if (eg == 0 && row == 0) {
                 tma_store_3d(&map_g, zt, h * P, pc * Q, seq);    // rows past the end of the sequence are clipped
                 bulk_commit();
                 bulk_wait_read0();
                 mbar_arrive(&misc->empty_z[sz]);
             }
         }
-        if (row == 0) bulk_wait0();
+        if (eg == 0 && row == 0) bulk_wait0();
     }
 
     // ---------------------------------------------------------------- teardown
