@@ -130,7 +130,10 @@ static MixerWs mixer_ws(const dm_mixer_cfg *c, const Dims &m) {
     ScanArgs sa{};
     sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
     sa.d_in_proj = m.d_in_proj; sa.conv_ch = m.conv_ch; sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask;
-    w.scan = off; off += align_up(scan_ssd_workspace_bytes(sa));
+    {
+        const size_t a_ssd = scan_ssd_workspace_bytes(sa), a_seq = scan_seq_workspace_bytes(sa);
+        w.scan = off; off += align_up(a_ssd > a_seq ? a_ssd : a_seq);
+    }
     w.total = off;
     return w;
 }
@@ -178,7 +181,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
     {
         StageTimer tm(DM_STAGE_SCAN, s);
         if (scan_ssd_supports(sa)) e = scan_ssd(sa, ws + l.scan, s);
-        else e = scan_sequential(sa, s);
+        else e = scan_sequential(sa, ws + l.scan, s);
     }
     if (e != cudaSuccess) return cuda_fail(e, "scan");
 

@@ -56,7 +56,8 @@ struct ScanArgs {
     const void *conv_in;     // [B,k-1,conv_ch] or NULL
     float *ssm_out;          // [B,H,P,N] or NULL
 };
-cudaError_t scan_sequential(const ScanArgs &a, cudaStream_t s);
+size_t scan_seq_workspace_bytes(const ScanArgs &a);
+cudaError_t scan_sequential(const ScanArgs &a, void *ws, cudaStream_t s);
 bool scan_ssd_supports(const ScanArgs &a);
 size_t scan_ssd_workspace_bytes(const ScanArgs &a);
 cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s);
