@@ -151,12 +151,206 @@ def run_reference(args, shape, dtype, rank):
     print(json.dumps(line), flush=True)
 
 
+# Stack workloads (dm_denoise_step): shape of one step's token tensor, layers, vocabulary; "prefix" marks block decoding.
+STACKS = {
+    "cfg2_stack": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304),
+    "cfg2_stack_n128": dict(shape=I.MixerShape(4, 4096, 1024, 2, 128, 4, 32), layers=24, vocab=50304),
+    "cfg4_decode": dict(shape=I.MixerShape(16, 32, 2048, 2, 128, 4, 64), layers=24, vocab=50304, prefix=2048),
+}
+
+
+def device_stack_weights(torch, shape, layers, vocab, seed=0):
+    """Random-init bf16 weights of a stack, drawn on the device with the distributions of inputs.py (the host
+    generator would take minutes at these sizes).  Returns the dict layout make_stack_weights() of the binding takes."""
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    s, bf = shape, torch.bfloat16
+    k = s.d_conv
+
+    def normal(*sz):
+        return (0.02 * torch.randn(*sz, generator=g, device="cuda", dtype=torch.float32)).to(bf)
+
+    def uniform(lo, hi, *sz):
+        return lo + (hi - lo) * torch.rand(*sz, generator=g, device="cuda", dtype=torch.float32)
+
+    def direction():
+        dt = torch.exp(uniform(float(np.log(1e-3)), float(np.log(1e-1)), s.n_heads))
+        return {"w_in": normal(s.d_in_proj, s.d_model), "conv_w": uniform(-k ** -0.5, k ** -0.5, s.conv_ch, k).to(bf),
+                "conv_b": uniform(-k ** -0.5, k ** -0.5, s.conv_ch).to(bf), "A_log": torch.log(uniform(1.0, 16.0, s.n_heads)),
+                "dt_bias": dt + torch.log(-torch.expm1(-dt)), "D": torch.ones(s.n_heads, device="cuda"),
+                "norm_w": torch.ones(s.d_inner, device="cuda", dtype=bf), "w_out": normal(s.d_model, s.d_inner)}
+
+    return {"embed": normal(vocab, s.d_model), "w_vocab": normal(vocab, s.d_model),
+            "final_norm_w": torch.ones(s.d_model, device="cuda", dtype=bf),
+            "layers": [{"norm_w": torch.ones(s.d_model, device="cuda", dtype=bf), "fwd": direction(), "rev": direction()}
+                       for _ in range(layers)]}
+
+
+def run_stack(args, rank, local_rank, world):
+    """One step = one dm_denoise_step (embedding, 24 x (RMSNorm, mixer, residual), final norm, vocabulary projection,
+    arg-max).  cfg4_decode: the step covers the 32-token active block of every sequence, starting from the carried
+    state of a committed 2048-token prefix; the same stack's full re-encode of prefix + block is timed beside it."""
+    import torch
+    import torch.distributed as dist
+    from paper_2511_15927_b200 import build
+    if rank == 0 or world == 1:
+        build.build()
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    from paper_2511_15927_b200 import binding as dm
+    torch.cuda.set_device(local_rank)
+    from paper_2511_15927_b200 import torch_io as G
+    spec = STACKS[args.workload]
+    shape, layers, vocab, prefix = spec["shape"], spec["layers"], spec["vocab"], spec.get("prefix")
+    B, Lb = shape.batch, shape.seqlen
+    w = device_stack_weights(torch, shape, layers, vocab)
+    csw, keep = dm.make_stack_weights(w)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def stack_cfg(L):
+        sh = I.MixerShape(B, L, shape.d_model, shape.expand, shape.d_state, shape.d_conv, shape.n_heads)
+        return dm.dm_stack_cfg(G.cfg_of(sh, I.BF16), layers, vocab, 1e-5)
+
+    def tokens(L, n):
+        return [torch.from_numpy(I.make_tokens(B, L, 50257, 50257, seed=i)).cuda() for i in range(n)]
+
+    scfg = stack_cfg(Lb)
+    nb = dm.dm_denoise_workspace_bytes(scfg)
+    states = None
+    extra = {}
+    if prefix:
+        # commit the prefix once (block step over the prefix, NULL state in), then time steps over the active block
+        pcfg = stack_cfg(prefix)
+        nbp = dm.dm_denoise_workspace_bytes(pcfg)
+        ws = G.workspace(max(nb, nbp, dm.dm_denoise_workspace_bytes(stack_cfg(prefix + Lb))))
+        st_bufs = [(torch.empty((B, shape.n_heads, shape.headdim, shape.d_state), device="cuda"),
+                    torch.empty((B, shape.d_conv - 1, shape.conv_ch), device="cuda", dtype=torch.bfloat16)) for _ in range(layers)]
+        pst = (dm.dm_layer_state * layers)()
+        for i, (sb, cb) in enumerate(st_bufs):
+            pst[i] = dm.dm_layer_state(None, None, sb.data_ptr(), cb.data_ptr())
+        ptok = tokens(prefix, 1)[0]
+        amax_p = torch.empty((B, prefix), device="cuda", dtype=torch.int32)
+        dm.dm_denoise_step(pcfg, csw, ptok.data_ptr(), 0, amax_p.data_ptr(), pst, ws.data_ptr(), ws.numel(), stream)
+        dm.dm_check(stream)
+        states = (dm.dm_layer_state * layers)()
+        for i, (sb, cb) in enumerate(st_bufs):
+            states[i] = dm.dm_layer_state(sb.data_ptr(), cb.data_ptr(), None, None)
+    else:
+        ws = G.workspace(nb)
+    toks = tokens(Lb, 4)
+    amax = torch.empty((B, Lb), device="cuda", dtype=torch.int32)
+
+    def step(i):
+        dm.dm_denoise_step(scfg, csw, toks[i % 4].data_ptr(), 0, amax.data_ptr(), states, ws.data_ptr(), ws.numel(), stream)
+
+    def timed(fn, n):
+        for i in range(args.warmup):
+            fn(i)
+        dm.dm_check(stream)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            fn(i)
+        e1.record()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    dm.dm_profile_enable(True)
+    dm.dm_profile_read()
+    launches0 = dm.dm_kernel_launch_count()
+    ms_total = timed(step, args.steps)
+    launches = dm.dm_kernel_launch_count() - launches0
+    stage_ms, stage_n = dm.dm_profile_read()          # includes the warm-up steps
+    dm.dm_profile_enable(False)
+    clocks = sampler.stop() if sampler else None
+    dm.dm_check(stream)
+    T = B * Lb
+    ms_step = ms_total / args.steps
+    if prefix:
+        # the alternative without a cache: re-encode prefix + block
+        fcfg = stack_cfg(prefix + Lb)
+        ftok = tokens(prefix + Lb, 2)
+        famax = torch.empty((B, prefix + Lb), device="cuda", dtype=torch.int32)
+        ms_full = timed(lambda i: dm.dm_denoise_step(fcfg, csw, ftok[i % 2].data_ptr(), 0, famax.data_ptr(), None, ws.data_ptr(),
+                                                      ws.numel(), stream), max(2, args.steps // 4)) / max(2, args.steps // 4)
+        extra = {"prefix": prefix, "full_reencode_ms_per_step": ms_full, "state_carry_speedup": ms_full / ms_step}
+    # end to end: token ids from pinned host memory in, arg-max ids back, inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        th = torch.from_numpy(I.make_tokens(B, Lb, 50257, 50257, seed=9)).pin_memory()
+        ah = torch.empty((B, Lb), dtype=torch.int32).pin_memory()
+        td = torch.empty((B, Lb), device="cuda", dtype=torch.int32)
+
+        def host_step(i):
+            td.copy_(th, non_blocking=True)
+            dm.dm_denoise_step(scfg, csw, td.data_ptr(), 0, amax.data_ptr(), states, ws.data_ptr(), ws.numel(), stream)
+            ah.copy_(amax, non_blocking=True)
+            torch.cuda.synchronize()
+        for i in range(2):
+            host_step(i)
+        t0 = time.perf_counter()
+        for i in range(args.steps):
+            host_step(i)
+        sec = time.perf_counter() - t0
+        e2e = {"value": world * T * layers * args.steps / sec, "unit": UNIT, "h2d_bytes_per_step": T * 4, "d2h_bytes_per_step": T * 4}
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = load_peaks()
+    n_calls = max(stage_n[dm.DM_STAGE_SCAN], 1)       # mixer calls profiled (warm-up included)
+    inp = stage_ms[dm.DM_STAGE_IN_PROJ] / n_calls
+    scn = stage_ms[dm.DM_STAGE_SCAN] / n_calls
+    outp = stage_ms[dm.DM_STAGE_OUT_PROJ] / n_calls
+    f_in, f_out = gemm_flops_per_token(shape)
+    in_tf, out_tf = f_in * T / (inp * 1e-3) / 1e12, f_out * T / (outp * 1e-3) / 1e12
+    scan_bytes = scan_bytes_per_token(shape, 2) * T
+    if prefix:
+        scan_bytes += B * shape.n_heads * shape.headdim * shape.d_state * 4        # one read of the carried state
+    scan_gbs = scan_bytes / (scn * 1e-3) / 1e9
+    kernels = {"in_proj_per_layer": {"ms": inp, "tflops": in_tf}, "scan_per_layer": {"ms": scn, "gbs": scan_gbs},
+               "out_proj_per_layer": {"ms": outp, "tflops": out_tf},
+               "rest_of_step_ms": ms_step - layers * (inp + scn + outp)}
+    if scn >= max(inp, outp):
+        roofline = {"kernel": "fused conv+scan+gate (per layer)", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": scan_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+    else:
+        tf = in_tf if inp >= outp else out_tf
+        roofline = {"kernel": ("in_proj" if inp >= outp else "out_proj") + " GEMM (per layer)", "bound": "tensor", "achieved": tf,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops_sustained"],
+                    "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)"}
+    line = {"metric": METRIC, "value": world * T * layers / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": dict({"workload": args.workload, "batch": B, "seq_len": Lb, "d_model": shape.d_model, "d_state": shape.d_state,
+                            "heads": shape.n_heads, "layers": layers, "vocab": vocab, "tokens_per_s_whole_stack": world * T / (ms_step * 1e-3),
+                            "parallelism": "replicas only" if world > 1 else "1 GPU",
+                            "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
+                           **extra),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels, "cpu_baseline": None}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS))
+    ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS) + sorted(STACKS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference arm's sample")
     ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
@@ -169,6 +363,13 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.workload in STACKS:
+        if args.impl == "reference":
+            if rank == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the oracle on single-layer workloads only"}), flush=True)
+            return
+        run_stack(args, rank, local_rank, world)
+        return
     shape, dtype = I.CONFIGS[args.workload]
 
     if args.impl == "reference":
