@@ -84,6 +84,7 @@ struct SsdArgs {
     float *ssq;
     const float *dA;             // [2][B][H][2][Lp]: Lambda, Lambda' (log2 units)
     const float *ssm_in; float *ssm_out;
+    const __nv_bfloat16 *conv_in;  // [B][k-1][conv_ch] pre-conv rows before the first token (left-to-right layer), or NULL
     ScanDir dir[2];
 };
 
@@ -121,11 +122,13 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
         const uint32_t *col = reinterpret_cast<const uint32_t *>(zx + a.d_inner + cc);      // 4-byte aligned: all widths are even
         const int64_t ld32 = a.d_in_proj / 2;
         const int first = rev ? r0 + rg * 32 + 31 : r0 + rg * 32, step = rev ? -1 : 1;        // first-in-time row of the block
+        const uint32_t *cin = (!rev && a.conv_in) ? reinterpret_cast<const uint32_t *>(a.conv_in + (int64_t)b * (k - 1) * a.conv_ch + cc) : nullptr;
         uint32_t raw[35];
 #pragma unroll
         for (int i = 0; i < 35; ++i) {
             const int t = first + (i - 3) * step;
             raw[i] = (t >= 0 && t < L) ? __ldg(col + (int64_t)t * ld32) : 0u;
+            if (cin && t < 0 && k - 1 + t >= 0) raw[i] = __ldg(cin + (int64_t)(k - 1 + t) * (a.conv_ch / 2));    // carried rows
         }
         __nv_bfloat16 *dst = (cp < 64 ? Bp + 2 * cp : Cp + 2 * (cp - 64)) + seq * L * N;
 #pragma unroll
@@ -402,6 +405,10 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 for (int m = 1; m <= 3; ++m) {
                     const int r = first - m * step + toff;
                     hr[m - 1] = *reinterpret_cast<const uint2 *>(xt + r * 128 + ((colx ^ (r & 7)) << 4) + sub);
+                    if (c == 0 && rb == 0 && !rev && a.conv_in)      // rows before the sequence: the carried conv state (zeros beyond it)
+                        hr[m - 1] = a.k - 1 - m >= 0
+                            ? __ldg(reinterpret_cast<const uint2 *>(a.conv_in + ((int64_t)b * (a.k - 1) + (a.k - 1 - m)) * a.conv_ch + h * P + cg * 4))
+                            : make_uint2(0u, 0u);
                 }
                 h1[0] = bf2_to_f2(hr[0].x); h1[1] = bf2_to_f2(hr[0].y);
                 h2[0] = bf2_to_f2(hr[1].x); h2[1] = bf2_to_f2(hr[1].y);
@@ -674,8 +681,6 @@ Scratch scratch_layout(const ScanArgs &a) {
 bool scan_ssd_supports(const ScanArgs &a) {
     if (a.dtype != DM_BF16 || a.N != N || a.P != P || a.k < 2 || a.k > 4) return false;
     if (a.d_in_proj % 8 || a.d_inner % 8) return false;                  // 16-byte rows for TMA and vector access
-    if (a.conv_in) return false;                                         // carried conv rows take the sequential kernel
-    if (a.L < 64) return false;                                          // short blocks: the sequential kernel is the better fit
     if (a.H > 65535 || a.B > 65535) return false;
     return encode_fn() != nullptr;
 }
@@ -695,7 +700,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     k.B = a.B; k.L = a.L; k.H = a.H; k.d_inner = a.d_inner; k.d_in_proj = a.d_in_proj; k.conv_ch = a.conv_ch; k.k = a.k;
     k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp;
     k.zx = static_cast<const __nv_bfloat16 *>(a.zx); k.ssq = a.ssq; k.dA = dA;
-    k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out;
+    k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out; k.conv_in = static_cast<const __nv_bfloat16 *>(a.conv_in);
     k.dir[0] = a.dir[0]; k.dir[1] = a.dir[1];
     const int ndir = a.dir_mask == DM_DIR_BOTH ? 2 : 1, dir0 = a.dir_mask == DM_DIR_REV ? 1 : 0;
 
