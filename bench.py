@@ -28,9 +28,18 @@ from paper_2511_15927_b200 import inputs as I  # noqa: E402
 METRIC = "denoised tokens/s per bidirectional Mamba layer"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused scan kernel, from the ncu captures
-# summarised under profiles/ (None = not captured for that workload).
-NCU_SCAN_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (taken on
+# cfg3_8k = 8192 tokens; traffic of both kernels grows in proportion to the token count, so other single-layer bf16
+# workloads of the same widths scale it by their tokens; None = no capture applies).
+NCU_TRAFFIC_PER_TOKEN = {"scan": (286.4832e6 + 110.2285e6) / 8192,      # ssd_scan_kernel, profiles/ssd_scan_cfg3_8k.txt
+                         "in_proj": (73.3286e6 + 104.1836e6) / 8192}    # gemm_tc_kernel<256>, one direction, profiles/gemm_tc_cfg3_8k.txt
+NCU_WIDTHS = (2048, 128, 64)                                             # d_model, d_state, heads the captures were taken at
+
+
+def ncu_traffic(kind, shape, dtype, tokens):
+    if dtype != I.BF16 or (shape.d_model, shape.d_state, shape.n_heads) != NCU_WIDTHS or kind not in NCU_TRAFFIC_PER_TOKEN:
+        return None
+    return NCU_TRAFFIC_PER_TOKEN[kind] * tokens
 
 
 def load_peaks():
@@ -483,12 +492,13 @@ def main():
     dominant = max(("in_proj", inp_ms), ("scan", scan_ms), ("out_proj", outp_ms), key=lambda kv: kv[1])[0]
     if dominant == "scan" or dtype != I.BF16:
         roofline = {"kernel": "fused conv+scan+gate", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": scan_gbs / peaks["hbm_gbs"], "traffic": NCU_SCAN_TRAFFIC_BYTES.get(args.workload),
+                    "frac": scan_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic("scan", shape, dtype, T),
                     "peak_source": peaks["source"] + " (sustained copy)"}
     else:
         tf = in_tf if dominant == "in_proj" else out_tf
-        roofline = {"kernel": dominant + " GEMM", "bound": "tensor", "achieved": tf, "peak": tensor_peak, "unit": "TFLOP/s",
-                    "frac": tf / tensor_peak, "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)"}
+        roofline = {"kernel": dominant + " GEMM (one launch per direction)", "bound": "tensor", "achieved": tf, "peak": tensor_peak,
+                    "unit": "TFLOP/s", "frac": tf / tensor_peak, "traffic": ncu_traffic(dominant, shape, dtype, T),
+                    "peak_source": peaks["source"] + " (sustained bf16)"}
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
