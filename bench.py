@@ -199,14 +199,11 @@ def run_stack(args, rank, local_rank, world):
     arg-max).  cfg4_decode: the step covers the 32-token active block of every sequence, starting from the carried
     state of a committed 2048-token prefix; the same stack's full re-encode of prefix + block is timed beside it."""
     import torch
-    import torch.distributed as dist
     from paper_2511_15927_b200 import build
     if rank == 0 or world == 1:
         build.build()
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-        dist.barrier()
+    from paper_2511_15927_b200 import dist_util as D
+    D.init("nccl", local_rank)
     from paper_2511_15927_b200 import binding as dm
     torch.cuda.set_device(local_rank)
     from paper_2511_15927_b200 import torch_io as G
@@ -257,23 +254,16 @@ def run_stack(args, rank, local_rank, world):
         for i in range(args.warmup):
             fn(i)
         dm.dm_check(stream)
-        if world > 1:
-            dist.barrier()
+        D.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for i in range(n):
             fn(i)
         e1.record()
-        if world > 1:
-            dist.barrier()
+        D.barrier()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return D.max_over_ranks(e0.elapsed_time(e1), "cuda")
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     dm.dm_profile_enable(True)
@@ -315,8 +305,7 @@ def run_stack(args, rank, local_rank, world):
         sec = time.perf_counter() - t0
         e2e = {"value": world * T * layers * args.steps / sec, "unit": UNIT, "h2d_bytes_per_step": T * 4, "d2h_bytes_per_step": T * 4}
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        D.shutdown()
         return
     peaks = load_peaks()
     n_calls = max(stage_n[dm.DM_STAGE_SCAN], 1)       # mixer calls profiled (warm-up included)
@@ -350,8 +339,7 @@ def run_stack(args, rank, local_rank, world):
                            **extra),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels, "cpu_baseline": None}
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    D.shutdown()
 
 
 def main():
@@ -386,14 +374,11 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
     from paper_2511_15927_b200 import build
     if rank == 0 or world == 1:
         build.build()
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-        dist.barrier()
+    from paper_2511_15927_b200 import dist_util as D
+    D.init("nccl", local_rank)
     from paper_2511_15927_b200 import binding as dm
     torch.cuda.set_device(local_rank)
     from paper_2511_15927_b200 import torch_io as G
@@ -417,8 +402,7 @@ def main():
         dm.dm_bimamba_forward(cfg, cw, xs[i % n_rot].data_ptr(), y.data_ptr(), ws.data_ptr(), nb, stream)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        D.barrier()
         torch.cuda.synchronize()
 
     for i in range(args.warmup):
@@ -441,12 +425,9 @@ def main():
     dm.dm_profile_enable(False)
     clocks = sampler.stop() if sampler else None
     dm.dm_check(stream)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = D.max_over_ranks(ms_total, "cuda")
     ms_step = ms_total / args.steps
-    value = world * T * args.steps / (ms_total * 1e-3)
+    value = D.whole_job_value(T, args.steps, ms_total)
 
     # ---- end to end through the host entry point: pinned host x in, y out, copies inside the timed region
     e2e = None
@@ -461,16 +442,12 @@ def main():
             dm.dm_bimamba_forward_host(cfg, cw, xh.data_ptr(), yh.data_ptr(), ws.data_ptr(), nb + 2 * act_bytes, stream)
         torch.cuda.synchronize()
         sec = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([sec], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            sec = float(t.item())
-        e2e = {"value": world * T * args.steps / sec, "unit": UNIT, "h2d_bytes_per_step": T * shape.d_model * es,
+        sec = D.max_over_ranks(sec, "cuda")
+        e2e = {"value": D.whole_job_value(T, args.steps, sec * 1e3), "unit": UNIT, "h2d_bytes_per_step": T * shape.d_model * es,
                "d2h_bytes_per_step": T * shape.d_model * es}
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        D.shutdown()
         return
 
     peaks = load_peaks()
@@ -518,8 +495,7 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
             "cpu_baseline": cpu_baseline}
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    D.shutdown()
 
 
 if __name__ == "__main__":
