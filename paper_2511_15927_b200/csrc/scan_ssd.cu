@@ -479,9 +479,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int c = 0; c < nch; ++c) {
             const int sd = c % NDL;
             const uint32_t par = c & 1;
-            if (ok) ok = WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->s_full, par) && WAIT(&misc->w_empty, par ^ 1);
+            // the decay factors depend on Lambda only: they are prepared while S of this chunk is still being computed
+            if (ok) ok = WAIT(&misc->full_dl[sd], (c / NDL) & 1);
             if (!named_all(3 + mg, WG, ok)) { ok = false; break; }
-            fence_after();
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
             const float li = lam[row];
             const float dec = ex2f(lam[rev ? 0 : Q - 1]);
@@ -501,6 +501,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 __syncwarp();
             }
             const f32x2 ri2 = pk2(ri, ri);
+            // validity of the diagonal block's entries as integers: entry jj (0..31) of the block counts iff key(jj) >= 0,
+            // and carries the D skip iff key(jj) == 0
+            const int ksign = rev ? 1 : -1, kbase = rev ? -(row & 31) : (row & 31);
+            if (!(WAIT(&misc->s_full, par) && WAIT(&misc->w_empty, par ^ 1))) { ok = false; continue; }
+            fence_after();
 #pragma unroll 1
             for (int gi = mg; gi < 8; gi += NWG) {        // this group's share of the 8 groups of 16 columns
                 const int jb = gi >> 1, j0 = gi * 16;
@@ -528,10 +533,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         float v[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const int j = j0 + 4 * v4 + e;
-                            float m = ex2f(li - lpv[e]);
-                            if (rev ? j < row : j > row) m = 0.f;
-                            v[e] = fmaf(__uint_as_float(r[4 * v4 + e]), m, j == row ? Dh : 0.f);
+                            const int key = ksign * ((j0 & 31) + 4 * v4 + e) + kbase;
+                            const float m = key >= 0 ? ex2f(li - lpv[e]) : 0.f;
+                            v[e] = fmaf(__uint_as_float(r[4 * v4 + e]), m, key == 0 ? Dh : 0.f);
                         }
                         out[2 * v4] = pack_bf16(v[0], v[1]);
                         out[2 * v4 + 1] = pack_bf16(v[2], v[3]);
