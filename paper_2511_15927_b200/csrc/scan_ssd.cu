@@ -197,7 +197,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_c,
                 const __grid_constant__ CUtensorMap map_g, const SsdArgs a, int dir0, int *status) {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     Misc *misc = reinterpret_cast<Misc *>(smem + OFF_MISC);
     volatile int *abort_flag = &misc->abort;
 
@@ -534,7 +535,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int key = ksign * ((j0 & 31) + 4 * v4 + e) + kbase;
-                            const float m = key >= 0 ? ex2f(li - lpv[e]) : 0.f;
+                            const float m = ex2f(key >= 0 ? li - lpv[e] : -INFINITY);      // 2^-inf = 0: no branch around the exponential
                             v[e] = fmaf(__uint_as_float(r[4 * v4 + e]), m, key == 0 ? Dh : 0.f);
                         }
                         out[2 * v4] = pack_bf16(v[0], v[1]);
