@@ -16,7 +16,7 @@
 // the chunks in descending order and uses the transposed causal mask, so nothing is ever flipped in memory.
 // The CTA is a pipeline of specialised warps that work on different chunks at the same time:
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
-//     warp 1      copies C' into TMEM (tcgen05.cp; it is the A operand of S and Yb) and issues the four tcgen05 products of a chunk:  S = C B^T,  St = B^T (w o x'),  Yb = C h_in,  Ya = W x'
+//     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  Ya = W x',  St = B^T (w o x')
 //     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
 //     warps 4-7   depthwise conv + SiLU of the x tile in place, and the decay-weighted copy w o x'
 //     warps 8-11  mask: S (TMEM, fp32) -> W (TMEM, bf16);  state: h <- exp(Lambda_last) h + St (fp32, kept in TMEM),
@@ -63,11 +63,11 @@ static_assert(OFF_Z % 1024 == 0 && OFF_B % 1024 == 0 && OFF_C % 1024 == 0 && OFF
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 // TMEM columns (all 512 are allocated)
-constexpr uint32_t TM_S = 0, TM_W = 128, TM_CT = 192, TM_YA = 256, TM_YB = 320, TM_ST = 384, TM_HS = 448, TM_COLS = 512;
+constexpr uint32_t TM_S = 0, TM_W = 128, TM_YB1 = 192, TM_YA = 256, TM_YB0 = 320, TM_ST = 384, TM_HS = 448, TM_COLS = 512;    // Yb is double-buffered
 
 struct Misc {
     uint64_t full_x[NX], empty_x[NX], full_z[NZ], empty_z[NZ], full_b[NB], empty_b[NB], full_c, empty_c, full_dl[NDL], empty_dl[NDL];
-    uint64_t xs_full, xs_empty, ct_full, ct_empty, s_full, s_empty, w_full, w_empty, st_full, st_empty, h_full, h_empty, y_full, y_empty;
+    uint64_t xs_full, xs_empty, s_full, s_empty, w_full, w_empty, st_full, st_empty, h_full, h_empty, y_full, ya_empty, yb_empty[2];
     uint32_t tmem_base;
     int abort;
     alignas(16) float norm_w[P];  // the three arrays below are read as float4
@@ -217,12 +217,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int i = 0; i < NDL; ++i) { mbar_init(&misc->full_dl[i], 1); mbar_init(&misc->empty_dl[i], 3 * ROLE); }
         mbar_init(&misc->full_c, 1);   mbar_init(&misc->empty_c, 1);
         mbar_init(&misc->xs_full, ROLE); mbar_init(&misc->xs_empty, 1);
-        mbar_init(&misc->ct_full, WG); mbar_init(&misc->ct_empty, 1);
         mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, ROLE);
         mbar_init(&misc->w_full, ROLE);  mbar_init(&misc->w_empty, 1);
         mbar_init(&misc->st_full, 1);  mbar_init(&misc->st_empty, ROLE);
         mbar_init(&misc->h_full, ROLE);  mbar_init(&misc->h_empty, 1);
-        mbar_init(&misc->y_full, 1);   mbar_init(&misc->y_empty, ROLE);
+        mbar_init(&misc->y_full, 1);   mbar_init(&misc->ya_empty, ROLE);
+        mbar_init(&misc->yb_empty[0], ROLE); mbar_init(&misc->yb_empty[1], ROLE);
         misc->abort = 0;
         mbar_fence_init();
     }
@@ -294,8 +294,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     } else if (warp == 1) {
         // ============================================================ MMA issuer
-        // Order per iteration: S(c), Ya(c-1), St(c), Yb(c): S(c) goes out as soon as the mask of chunk c-1 has
-        // read S(c-1), so the mask group is never waiting for more than one product.
+        // Order per iteration: S(c), Yb(c), Ya(c-1), St(c).  S(c) goes out as soon as the mask of chunk c-1 has read
+        // S(c-1); Yb(c) follows at once (its accumulator is double-buffered, so it does not wait for the epilogue of
+        // chunk c-1), which frees the single C' buffer early enough for the next chunk's load.
         if (lane == 0) {
             // low halves of the operand descriptors; a K step of 16 advances a K-major operand by 32 bytes inside its
             // 64-wide tile (+2) or to the next tile (+T16/16), an MN-major operand by 16 rows (+2048/16)
@@ -306,39 +307,42 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             constexpr uint32_t I128 = idesc_bf16(128, 128, 0, 0), I64 = idesc_bf16(128, 64, 0, 1), I64T = idesc_bf16(128, 64, 1, 1);
             auto issue_ya = [&](int c) -> bool {       // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
                 const int sx = c % NX;
-                if (!WAIT(&misc->w_full, c & 1)) return false;
+                if (!WAIT(&misc->w_full, c & 1) || !WAIT(&misc->ya_empty, (c & 1) ^ 1)) return false;
                 fence_after();
                 const uint32_t dX = dX0 + (uint32_t)sx * (XTILE >> 4);
                 umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
 #pragma unroll
                 for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
-                umma_commit(&misc->y_full);
+                umma_commit(&misc->y_full);              // Yb of the same chunk was issued earlier: it has completed as well
                 umma_commit(&misc->w_empty);
                 umma_commit(&misc->empty_x[sx]);
                 return true;
             };
-            // C' of chunk c: shared memory -> TMEM (A operand of S and Yb), by tcgen05.cp from this thread, so that it is
-            // ordered before the products that follow; the transit buffer is released when the copies have completed
-            auto copy_c = [&](int c) -> bool {
-                if (!WAIT(&misc->full_c, c & 1) || !WAIT(&misc->ct_empty, (c & 1) ^ 1)) return false;
-                fence_after();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) tmem_cp_128x256b_lo(tmem + TM_CT + 8 * kk, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3));
-                umma_commit(&misc->empty_c);
-                return true;
-            };
-            bool ok = copy_c(0);
+            bool ok = true;
             for (int c = 0; c < nch && ok; ++c) {
                 const int sb = c % NB;
                 const uint32_t par = c & 1;
                 const uint32_t dBk = dBk0 + (uint32_t)sb * (2 * T16 >> 4), dBm = dBm0 + (uint32_t)sb * (2 * T16 >> 4);
-                // S = C' B'^T  (A = C' from TMEM, B = B' K-major)
-                if (!WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
+                // S = C' B'^T  (both K-major in shared memory)
+                if (!WAIT(&misc->full_c, par) || !WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
                 fence_after();
-                umma_ts<0>(tmem + TM_S, tmem + TM_CT, dBk, I128);
+                umma_ss<0>(tmem + TM_S, dC, dBk, I128);
 #pragma unroll
-                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_S, tmem + TM_CT + 8 * kk, dBk + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), I128);
+                for (int kk = 1; kk < 8; ++kk) {
+                    const uint32_t o = (kk >> 2) * (T16 >> 4) + 2 * (kk & 3);
+                    umma_ss<1>(tmem + TM_S, dC + o, dBk + o, I128);
+                }
                 umma_commit(&misc->s_full);
+                // Yb = C' h_in  (A = C' K-major, B = bf16 state [n][p] MN-major) into the buffer the epilogue of chunk c-2 has drained;
+                // its completion releases C' (S was issued before it) and the state copy
+                const uint32_t tyb = tmem + (par ? TM_YB1 : TM_YB0);
+                if (!WAIT(&misc->h_full, par) || !WAIT(&misc->yb_empty[par], ((c >> 1) & 1) ^ 1)) break;
+                fence_after();
+                umma_ss<0>(tyb, dC, dH, I64);
+#pragma unroll
+                for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tyb, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), dH + kk * 128, I64);
+                umma_commit(&misc->empty_c);
+                umma_commit(&misc->h_empty);
                 if (c > 0 && !issue_ya(c - 1)) break;
                 // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
                 if (!WAIT(&misc->xs_full, par) || !WAIT(&misc->st_empty, par ^ 1)) break;
@@ -349,16 +353,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&misc->st_full);
                 umma_commit(&misc->xs_empty);
                 umma_commit(&misc->empty_b[sb]);
-                // Yb = C' h_in  (B = bf16 state [n][p], MN-major)
-                if (!WAIT(&misc->h_full, par) || !WAIT(&misc->y_empty, par ^ 1)) break;
-                fence_after();
-                umma_ts<0>(tmem + TM_YB, tmem + TM_CT, dH, I64);
-#pragma unroll
-                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_YB, tmem + TM_CT + 8 * kk, dH + kk * 128, I64);
-                umma_commit(&misc->ct_empty);
-                umma_commit(&misc->h_empty);
                 if (c == nch - 1) ok = issue_ya(c);
-                else ok = copy_c(c + 1);
             }
         }
     } else if (warp < 4 + 4 * NWG) {
@@ -617,9 +612,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int c8 = eg * 4; c8 < eg * 4 + 4; ++c8) {   // 8 channels (one 16-byte chunk of z) at a time
                 uint32_t ya[8], yb[8];
                 tmem_ld_x8(tlane + TM_YA + c8 * 8, ya);
-                tmem_ld_x8(tlane + TM_YB + c8 * 8, yb);
+                tmem_ld_x8(tlane + (par ? TM_YB1 : TM_YB0) + c8 * 8, yb);
                 tmem_wait_ld();
-                if (c8 == eg * 4 + 3) { fence_before(); mbar_arrive(&misc->y_empty); }
+                if (c8 == eg * 4 + 3) { fence_before(); mbar_arrive(&misc->ya_empty); mbar_arrive(&misc->yb_empty[par]); }
                 uint4 *zp = reinterpret_cast<uint4 *>(zt + row * 128 + ((c8 ^ (row & 7)) << 4));
                 const uint4 zv = *zp;
                 const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
