@@ -18,11 +18,11 @@
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
 //     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  Ya = W x',  St = B^T (w o x')
 //     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
-//     warps 4-7   depthwise conv + SiLU of the x tile in place, and the decay-weighted copy w o x'
-//     warps 8-11  mask: S (TMEM, fp32) -> W (TMEM, bf16);  state: h <- exp(Lambda_last) h + St (fp32, kept in TMEM),
-//                 bf16 copy of h for the next chunk's Yb
-//     warps 12-15 epilogue: y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w], per-head sum of squares,
-//                 written over the z tile and stored with TMA
+//     warps 4-11   conv groups: depthwise conv + SiLU of the x tile in place (8-row blocks), and the decay-weighted copy w o x'
+//     warps 12-19  mask groups: S (TMEM, fp32) -> W (TMEM, bf16), the 16-column groups split between the two groups;
+//                  state: h <- exp(Lambda_last) h + St (fp32, kept in TMEM), bf16 copy of h for the next chunk's Yb
+//     warps 20-27  epilogue groups (half of the channels each): y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w],
+//                  per-head sum of squares, written over the z tile and stored with TMA
 // Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
 // device status word, all roles leave their loops, outstanding TMA traffic is waited for (bounded), TMEM is
 // freed and the CTA returns.
