@@ -235,6 +235,10 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's TMEM lane quarter
     const float *dA_head = a.dA + (((int64_t)seq * a.H + h) * 2) * a.Lp;
     auto WAIT = [&](uint64_t *bar, uint32_t parity) { return mbar_wait(bar, parity, abort_flag, status); };
+    auto WAIT2 = [&](uint64_t *b1, uint32_t p1, uint64_t *b2, uint32_t p2) { return mbar_wait2(b1, p1, b2, p2, abort_flag, status); };
+    auto WAIT3 = [&](uint64_t *b1, uint32_t p1, uint64_t *b2, uint32_t p2, uint64_t *b3, uint32_t p3) {
+        return mbar_wait3(b1, p1, b2, p2, b3, p3, abort_flag, status);
+    };
 
     if (warp == 0) {
         // ============================================================ TMA: x tile (+halo) and Lambda, Lambda'
@@ -242,7 +246,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             int issued = 0;
             for (int c = 0; c < nch; ++c) {
                 const int sx = c % NX, sd = c % NDL, pc = rev ? nch - 1 - c : c;
-                if (!WAIT(&misc->empty_x[sx], ((c / NX) & 1) ^ 1) || !WAIT(&misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
+                if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
                 tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * P, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
                 mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
@@ -307,7 +311,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             constexpr uint32_t I128 = idesc_bf16(128, 128, 0, 0), I64 = idesc_bf16(128, 64, 0, 1), I64T = idesc_bf16(128, 64, 1, 1);
             auto issue_ya = [&](int c) -> bool {       // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
                 const int sx = c % NX;
-                if (!WAIT(&misc->w_full, c & 1) || !WAIT(&misc->ya_empty, (c & 1) ^ 1)) return false;
+                if (!WAIT2(&misc->w_full, c & 1, &misc->ya_empty, (c & 1) ^ 1)) return false;
                 fence_after();
                 const uint32_t dX = dX0 + (uint32_t)sx * (XTILE >> 4);
                 umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
@@ -324,7 +328,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const uint32_t par = c & 1;
                 const uint32_t dBk = dBk0 + (uint32_t)sb * (2 * T16 >> 4), dBm = dBm0 + (uint32_t)sb * (2 * T16 >> 4);
                 // S = C' B'^T  (both K-major in shared memory)
-                if (!WAIT(&misc->full_c, par) || !WAIT(&misc->full_b[sb], (c / NB) & 1) || !WAIT(&misc->s_empty, par ^ 1)) break;
+                if (!WAIT3(&misc->full_c, par, &misc->full_b[sb], (c / NB) & 1, &misc->s_empty, par ^ 1)) break;
                 fence_after();
                 umma_ss<0>(tmem + TM_S, dC, dBk, I128);
 #pragma unroll
@@ -336,7 +340,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 // Yb = C' h_in  (A = C' K-major, B = bf16 state [n][p] MN-major) into the buffer the epilogue of chunk c-2 has drained;
                 // its completion releases C' (S was issued before it) and the state copy
                 const uint32_t tyb = tmem + (par ? TM_YB1 : TM_YB0);
-                if (!WAIT(&misc->h_full, par) || !WAIT(&misc->yb_empty[par], ((c >> 1) & 1) ^ 1)) break;
+                if (!WAIT2(&misc->h_full, par, &misc->yb_empty[par], ((c >> 1) & 1) ^ 1)) break;
                 fence_after();
                 umma_ss<0>(tyb, dC, dH, I64);
 #pragma unroll
@@ -345,7 +349,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(&misc->h_empty);
                 if (c > 0 && !issue_ya(c - 1)) break;
                 // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
-                if (!WAIT(&misc->xs_full, par) || !WAIT(&misc->st_empty, par ^ 1)) break;
+                if (!WAIT2(&misc->xs_full, par, &misc->st_empty, par ^ 1)) break;
                 fence_after();
                 umma_ss<0>(tmem + TM_ST, dBm, dXs, I64T);
 #pragma unroll
@@ -388,7 +392,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
             const uint32_t par = c & 1;
-            if (ok) ok = WAIT(&misc->full_x[sx], (c / NX) & 1) && WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->xs_empty, par ^ 1);
+            if (ok) ok = WAIT3(&misc->full_x[sx], (c / NX) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->xs_empty, par ^ 1);
             if (!named_all(1, ROLE, ok)) { ok = false; break; }
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
             // place: they are read before the group barrier; the block's own rows are read just before being replaced.
@@ -500,7 +504,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // validity of the diagonal block's entries as integers: entry jj (0..31) of the block counts iff key(jj) >= 0,
             // and carries the D skip iff key(jj) == 0
             const int ksign = rev ? 1 : -1, kbase = rev ? -(row & 31) : (row & 31);
-            if (!(WAIT(&misc->s_full, par) && WAIT(&misc->w_empty, par ^ 1))) { ok = false; continue; }
+            if (!WAIT2(&misc->s_full, par, &misc->w_empty, par ^ 1)) { ok = false; continue; }
             fence_after();
 #pragma unroll 1
             for (int gi = mg; gi < 8; gi += NWG) {        // this group's share of the 8 groups of 16 columns
@@ -548,7 +552,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_before();
             mbar_arrive(&misc->w_full);
             // ---- state: h <- 2^(Lambda_last) h + St; bf16 copy for the next chunk's Yb
-            if (!(WAIT(&misc->st_full, par) && WAIT(&misc->h_empty, par))) { ok = false; continue; }
+            if (!WAIT2(&misc->st_full, par, &misc->h_empty, par)) { ok = false; continue; }
             fence_after();
             const bool more = c + 1 < nch;
             const f32x2 dec2 = pk2(dec, dec);
@@ -598,7 +602,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int c = 0; c < nch; ++c) {
             const int sz = c % NZ, sd = c % NDL, pc = rev ? nch - 1 - c : c;
             const uint32_t par = c & 1;
-            if (ok) ok = WAIT(&misc->full_z[sz], (c / NZ) & 1) && WAIT(&misc->full_dl[sd], (c / NDL) & 1) && WAIT(&misc->y_full, par);
+            if (ok) ok = WAIT3(&misc->full_z[sz], (c / NZ) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->y_full, par);
             if (!named_all(2, ROLE, ok)) { ok = false; break; }
             fence_after();
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4);

@@ -55,6 +55,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         }
     }
 }
+// Waits on two or three barriers at once: the first probes are issued back to back so that their latencies overlap
+// (a probe of a completed phase costs about a hundred clocks); whatever is not complete yet is then waited for in turn.
+__device__ __forceinline__ bool mbar_wait2(uint64_t *b1, uint32_t p1, uint64_t *b2, uint32_t p2, volatile int *abort_flag, int *status) {
+    const bool r1 = mbar_try_wait(b1, p1), r2 = mbar_try_wait(b2, p2);
+    return (r1 || mbar_wait(b1, p1, abort_flag, status)) && (r2 || mbar_wait(b2, p2, abort_flag, status));
+}
+__device__ __forceinline__ bool mbar_wait3(uint64_t *b1, uint32_t p1, uint64_t *b2, uint32_t p2, uint64_t *b3, uint32_t p3,
+                                           volatile int *abort_flag, int *status) {
+    const bool r1 = mbar_try_wait(b1, p1), r2 = mbar_try_wait(b2, p2), r3 = mbar_try_wait(b3, p3);
+    return (r1 || mbar_wait(b1, p1, abort_flag, status)) && (r2 || mbar_wait(b2, p2, abort_flag, status)) &&
+           (r3 || mbar_wait(b3, p3, abort_flag, status));
+}
 // Wait with its own short limit and no side effect (used while tearing down after an abort).
 __device__ __forceinline__ void mbar_wait_quiet(uint64_t *bar, uint32_t parity, uint64_t limit_ns) {
     const uint64_t t0 = globaltimer_ns();
