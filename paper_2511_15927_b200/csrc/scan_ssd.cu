@@ -67,7 +67,7 @@ constexpr uint32_t TM_S = 0, TM_W = 128, TM_YB1 = 192, TM_YA = 256, TM_YB0 = 320
 
 struct Misc {
     uint64_t full_x[NX], empty_x[NX], full_z[NZ], empty_z[NZ], full_b[NB], empty_b[NB], full_c, empty_c, full_dl[NDL], empty_dl[NDL];
-    uint64_t xs_full, xs_empty, s_full, s_empty, w_full, w_empty, st_full, st_empty, h_full, h_empty, y_full, ya_empty, yb_empty[2];
+    uint64_t xs_full, s_full, s_empty, w_full, st_full, st_empty, h_full, y_full, ya_empty, yb_empty[2];
     uint32_t tmem_base;
     int abort;
     alignas(16) float norm_w[P];  // the three arrays below are read as float4
@@ -216,11 +216,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int i = 0; i < NB; ++i) { mbar_init(&misc->full_b[i], 1); mbar_init(&misc->empty_b[i], 1); }
         for (int i = 0; i < NDL; ++i) { mbar_init(&misc->full_dl[i], 1); mbar_init(&misc->empty_dl[i], 3 * ROLE); }
         mbar_init(&misc->full_c, 1);   mbar_init(&misc->empty_c, 1);
-        mbar_init(&misc->xs_full, ROLE); mbar_init(&misc->xs_empty, 1);
+        mbar_init(&misc->xs_full, ROLE);
         mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, ROLE);
-        mbar_init(&misc->w_full, ROLE);  mbar_init(&misc->w_empty, 1);
+        mbar_init(&misc->w_full, ROLE);
         mbar_init(&misc->st_full, 1);  mbar_init(&misc->st_empty, ROLE);
-        mbar_init(&misc->h_full, ROLE);  mbar_init(&misc->h_empty, 1);
+        mbar_init(&misc->h_full, ROLE);
         mbar_init(&misc->y_full, 1);   mbar_init(&misc->ya_empty, ROLE);
         mbar_init(&misc->yb_empty[0], ROLE); mbar_init(&misc->yb_empty[1], ROLE);
         misc->abort = 0;
@@ -317,8 +317,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
 #pragma unroll
                 for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
-                umma_commit(&misc->y_full);              // Yb of the same chunk was issued earlier: it has completed as well
-                umma_commit(&misc->w_empty);
+                umma_commit(&misc->y_full);              // Yb of the same chunk was issued earlier: it has completed as well; also frees W
                 umma_commit(&misc->empty_x[sx]);
                 return true;
             };
@@ -345,8 +344,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_ss<0>(tyb, dC, dH, I64);
 #pragma unroll
                 for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tyb, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), dH + kk * 128, I64);
-                umma_commit(&misc->empty_c);
-                umma_commit(&misc->h_empty);
+                umma_commit(&misc->empty_c);             // also releases the bf16 state copy
                 if (c > 0 && !issue_ya(c - 1)) break;
                 // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
                 if (!WAIT2(&misc->xs_full, par, &misc->st_empty, par ^ 1)) break;
@@ -354,8 +352,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_ss<0>(tmem + TM_ST, dBm, dXs, I64T);
 #pragma unroll
                 for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tmem + TM_ST, dBm + kk * 128, dXs + kk * 128, I64T);
-                umma_commit(&misc->st_full);
-                umma_commit(&misc->xs_empty);
+                umma_commit(&misc->st_full);             // also frees the w o x' buffer
                 umma_commit(&misc->empty_b[sb]);
                 if (c == nch - 1) ok = issue_ya(c);
             }
@@ -392,7 +389,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
             const uint32_t par = c & 1;
-            if (ok) ok = WAIT3(&misc->full_x[sx], (c / NX) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->xs_empty, par ^ 1);
+            if (ok) ok = WAIT3(&misc->full_x[sx], (c / NX) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->st_full, par ^ 1);
             if (!named_all(1, ROLE, ok)) { ok = false; break; }
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
             // place: they are read before the group barrier; the block's own rows are read just before being replaced.
@@ -504,7 +501,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // validity of the diagonal block's entries as integers: entry jj (0..31) of the block counts iff key(jj) >= 0,
             // and carries the D skip iff key(jj) == 0
             const int ksign = rev ? 1 : -1, kbase = rev ? -(row & 31) : (row & 31);
-            if (!WAIT2(&misc->s_full, par, &misc->w_empty, par ^ 1)) { ok = false; continue; }
+            if (!WAIT2(&misc->s_full, par, &misc->y_full, par ^ 1)) { ok = false; continue; }
             fence_after();
 #pragma unroll 1
             for (int gi = mg; gi < 8; gi += NWG) {        // this group's share of the 8 groups of 16 columns
@@ -552,7 +549,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_before();
             mbar_arrive(&misc->w_full);
             // ---- state: h <- 2^(Lambda_last) h + St; bf16 copy for the next chunk's Yb
-            if (!WAIT2(&misc->st_full, par, &misc->h_empty, par)) { ok = false; continue; }
+            if (!WAIT2(&misc->st_full, par, &misc->empty_c, par)) { ok = false; continue; }
             fence_after();
             const bool more = c + 1 < nch;
             const f32x2 dec2 = pk2(dec, dec);
