@@ -18,9 +18,9 @@
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
 //     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  Ya = W x',  St = B^T (w o x')
 //     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
-//     warps 4-11   conv groups: depthwise conv + SiLU of the x tile in place (8-row blocks), and the decay-weighted copy w o x'
-//     warps 12-19  mask groups: S (TMEM, fp32) -> W (TMEM, bf16), the 16-column groups split between the two groups;
-//                  state: h <- exp(Lambda_last) h + St (fp32, kept in TMEM), bf16 copy of h for the next chunk's Yb
+//     warps 4-11   conv groups: state update of the previous chunk, h <- exp(Lambda_last) h + St (fp32, kept in TMEM) with its
+//                  bf16 copy for the next Yb; depthwise conv + SiLU of the x tile in place (8-row blocks); the decay-weighted copy w o x'
+//     warps 12-19  mask groups: S (TMEM, fp32) -> W (TMEM, bf16), the 16-column groups split between the two groups
 //     warps 20-27  epilogue groups (half of the channels each): y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w],
 //                  per-head sum of squares, written over the z tile and stored with TMA
 // Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
@@ -358,7 +358,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
         }
     } else if (warp < 4 + 4 * NWG) {
-        // ============================================================ conv + SiLU of the x tile; w o x'
+        // ============================================================ state update; conv + SiLU of the x tile; w o x'
         constexpr int RB = Q * 16 / ROLE;               // rows per thread
         const int t = tid - 4 * 32;                     // 0..ROLE-1
         const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of RB rows
@@ -385,12 +385,68 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const f32x2 half2 = pk2(0.5f, 0.5f);
         const int first = rev ? rb * RB + RB - 1 : rb * RB, step = rev ? -1 : 1;   // first-in-time chunk row of the block
         const int toff = rev ? 0 : HALO;                                          // tile row = chunk row + toff
+        const int srow = t & (WG - 1), sh = t >> 7;      // state row and column half of this thread
+        // incoming state -> TMEM (fp32) and shared memory (bf16)
+        {
+            const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * N + srow : nullptr;
+            {
+                const int half = sh;                     // this group's half of the state columns
+                uint32_t hs[32];
+#pragma unroll
+                for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * N]) : 0u;
+                tmem_st_x32(tlane + TM_HS + half * 32, hs);
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4)
+                    *reinterpret_cast<uint4 *>(smem + OFF_H + srow * 128 + (((half * 4 + c4) ^ (srow & 7)) << 4)) =
+                        make_uint4(pack_bf16(__uint_as_float(hs[c4 * 8]), __uint_as_float(hs[c4 * 8 + 1])),
+                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 2]), __uint_as_float(hs[c4 * 8 + 3])),
+                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 4]), __uint_as_float(hs[c4 * 8 + 5])),
+                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 6]), __uint_as_float(hs[c4 * 8 + 7])));
+            }
+            fence_proxy_async();
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(&misc->h_full);
+        }
+        // state: h <- 2^(Lambda_last) h + St (fp32, kept in TMEM); bf16 copy for the next chunk's Yb.  Thread = state row, half of the columns.
+        auto state_update = [&](float dec, bool more) {
+            fence_after();
+            const f32x2 dec2 = pk2(dec, dec);
+#pragma unroll 1
+            for (int c8 = sh * 4; c8 < sh * 4 + 4; ++c8) {   // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
+                uint32_t st[8], hs[8];
+                tmem_ld_x8(tlane + TM_ST + c8 * 8, st);
+                tmem_ld_x8(tlane + TM_HS + c8 * 8, hs);
+                tmem_wait_ld();
+                uint32_t hb[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    const f32x2 hn = fma2(dec2, pk2(__uint_as_float(hs[2 * e2]), __uint_as_float(hs[2 * e2 + 1])),
+                                          pk2(__uint_as_float(st[2 * e2]), __uint_as_float(st[2 * e2 + 1])));
+                    float lo, hi;
+                    upk2(hn, lo, hi);
+                    hs[2 * e2] = __float_as_uint(lo); hs[2 * e2 + 1] = __float_as_uint(hi);
+                    hb[e2] = pack_bf16(lo, hi);
+                }
+                tmem_st_x8(tlane + TM_HS + c8 * 8, hs);
+                if (more) *reinterpret_cast<uint4 *>(smem + OFF_H + srow * 128 + ((c8 ^ (srow & 7)) << 4)) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
+            }
+            fence_before();
+            mbar_arrive(&misc->st_empty);
+            fence_proxy_async();
+            tmem_wait_st();
+            fence_before();
+            if (more) mbar_arrive(&misc->h_full);
+        };
+        float dec_prev = 0.f;
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
             const uint32_t par = c & 1;
             if (ok) ok = WAIT3(&misc->full_x[sx], (c / NX) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->st_full, par ^ 1);
             if (!named_all(1, ROLE, ok)) { ok = false; break; }
+            // St of the previous chunk has completed (so has its Yb, issued before it): update the state first, the next Yb waits for it
+            if (c > 0) state_update(dec_prev, true);
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
             // place: they are read before the group barrier; the block's own rows are read just before being replaced.
             uint8_t *xt = smem + OFF_X + sx * XTILE;
@@ -411,6 +467,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 h2[0] = bf2_to_f2(hr[1].x); h2[1] = bf2_to_f2(hr[1].y);
                 h3[0] = bf2_to_f2(hr[2].x); h3[1] = bf2_to_f2(hr[2].y);
             }
+            const float dec_cur = ex2f(lam[rev ? 0 : Q - 1]);   // this chunk's total decay, for the state update at the next iteration
             if (t < Q) misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
             mbar_arrive(&misc->empty_dl[sd]);
             named_sync(1, ROLE);                           // halo rows are in registers; wbuf is visible
@@ -440,9 +497,22 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
             fence_proxy_async();
             mbar_arrive(&misc->xs_full);
+            dec_prev = dec_cur;
+        }
+        if (ok && WAIT(&misc->st_full, (nch - 1) & 1)) state_update(dec_prev, false); else ok = false;
+        if (ok && !rev && a.ssm_out) {
+            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * N + srow;
+            {
+                const int half = sh;
+                uint32_t hs[32];
+                tmem_ld_x32(tlane + TM_HS + half * 32, hs);
+                tmem_wait_ld();
+#pragma unroll
+                for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * N] = __uint_as_float(hs[p]);
+            }
         }
     } else if (warp < 4 + 8 * NWG) {
-        // ============================================================ mask S -> W; state update
+        // ============================================================ mask S -> W
         // The NWG groups share every row: group g takes the 16-column groups gi = g, g + NWG, ... of the mask and the
         // state columns [g, g+1) * P / NWG, so the triangular mask is split evenly between them.
         const int mg = (warp - 4 - 4 * NWG) >> 2;       // group index
@@ -450,28 +520,6 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int q = warp & 3;
         const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
         float *cbuf = misc->cbuf[mg][q];
-        // incoming state -> TMEM (fp32) and shared memory (bf16)
-        {
-            const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * N + row : nullptr;
-            {
-                const int half = mg;                     // this group's half of the state columns
-                uint32_t hs[32];
-#pragma unroll
-                for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * N]) : 0u;
-                tmem_st_x32(tlane + TM_HS + half * 32, hs);
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4)
-                    *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + (((half * 4 + c4) ^ (row & 7)) << 4)) =
-                        make_uint4(pack_bf16(__uint_as_float(hs[c4 * 8]), __uint_as_float(hs[c4 * 8 + 1])),
-                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 2]), __uint_as_float(hs[c4 * 8 + 3])),
-                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 4]), __uint_as_float(hs[c4 * 8 + 5])),
-                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 6]), __uint_as_float(hs[c4 * 8 + 7])));
-            }
-            fence_proxy_async();
-            tmem_wait_st();
-            fence_before();
-            mbar_arrive(&misc->h_full);
-        }
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sd = c % NDL;
@@ -481,7 +529,6 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (!named_all(3 + mg, WG, ok)) { ok = false; break; }
             const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
             const float li = lam[row];
-            const float dec = ex2f(lam[rev ? 0 : Q - 1]);
             // ---- W_ij = S_ij 2^(Lambda_i - Lambda'_j) for j not after i in time, + D on the diagonal; 0 elsewhere.
             // Blocks of 32 x 32: the block on the diagonal takes one exponential per entry; a block before it (in
             // time) uses 2^(Lambda_i - Lambda_ref) * 2^(Lambda_ref - Lambda'_j) with Lambda_ref the last row before this
@@ -548,48 +595,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             tmem_wait_st();
             fence_before();
             mbar_arrive(&misc->w_full);
-            // ---- state: h <- 2^(Lambda_last) h + St; bf16 copy for the next chunk's Yb
-            if (!WAIT2(&misc->st_full, par, &misc->empty_c, par)) { ok = false; continue; }
-            fence_after();
-            const bool more = c + 1 < nch;
-            const f32x2 dec2 = pk2(dec, dec);
-#pragma unroll 1
-            for (int c8 = mg * 4; c8 < mg * 4 + 4; ++c8) {   // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
-                uint32_t st[8], hs[8];
-                tmem_ld_x8(tlane + TM_ST + c8 * 8, st);
-                tmem_ld_x8(tlane + TM_HS + c8 * 8, hs);
-                tmem_wait_ld();
-                uint32_t hb[4];
-#pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) {
-                    const f32x2 hn = fma2(dec2, pk2(__uint_as_float(hs[2 * e2]), __uint_as_float(hs[2 * e2 + 1])),
-                                          pk2(__uint_as_float(st[2 * e2]), __uint_as_float(st[2 * e2 + 1])));
-                    float lo, hi;
-                    upk2(hn, lo, hi);
-                    hs[2 * e2] = __float_as_uint(lo); hs[2 * e2 + 1] = __float_as_uint(hi);
-                    hb[e2] = pack_bf16(lo, hi);
-                }
-                tmem_st_x8(tlane + TM_HS + c8 * 8, hs);
-                if (more) *reinterpret_cast<uint4 *>(smem + OFF_H + row * 128 + ((c8 ^ (row & 7)) << 4)) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
-            }
             mbar_arrive(&misc->empty_dl[sd]);
-            fence_before();
-            mbar_arrive(&misc->st_empty);
-            fence_proxy_async();
-            tmem_wait_st();
-            fence_before();
-            if (more) mbar_arrive(&misc->h_full);
-        }
-        if (ok && !rev && a.ssm_out) {
-            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * N + row;
-            {
-                const int half = mg;
-                uint32_t hs[32];
-                tmem_ld_x32(tlane + TM_HS + half * 32, hs);
-                tmem_wait_ld();
-#pragma unroll
-                for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * N] = __uint_as_float(hs[p]);
-            }
         }
     } else {
         // ============================================================ epilogue
