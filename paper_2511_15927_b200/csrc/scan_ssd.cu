@@ -90,12 +90,15 @@ struct SsdArgs {
 
 __device__ __forceinline__ float silu_fast(float v) { return v / (1.f + __expf(-v)); }
 // --------------------------------------------------------------------------------------------------
-// Launch 1: B', C' (bf16) and Lambda, Lambda' (fp32, log2 units) for one physical chunk of one (direction, batch row).
+// Launch 1: B', C' (bf16) and Lambda, Lambda' (fp32, log2 units).  A CTA takes one quarter of one physical chunk of one
+// (direction, batch row): 32 of its rows for B' and C', 16 of every 64 heads for the decays.  The work per CTA is a
+// chain of dependent memory round trips, so many small CTAs per SM hide it better than few large ones.
 // --------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(512)
+constexpr int PREP_PARTS = 4, PREP_THREADS = 128, PREP_HEADS = 64 / PREP_PARTS;
+__global__ void __launch_bounds__(PREP_THREADS)
 ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, int dir0) {
-    __shared__ float dsm[Q][65];
-    const int pc = blockIdx.x, b = blockIdx.y, dir = dir0 + blockIdx.z;
+    __shared__ float dsm[Q][PREP_HEADS + 1];
+    const int pc = blockIdx.x / PREP_PARTS, part = blockIdx.x % PREP_PARTS, b = blockIdx.y, dir = dir0 + blockIdx.z;
     const bool rev = dir == 1;
     const int L = a.L, k = a.k, tid = threadIdx.x;
     const ScanDir &w = a.dir[dir];
@@ -104,9 +107,9 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
     const int r0 = pc * Q;
     const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
 
-    // ---- B and C channels: thread = (channel pair, block of 32 rows); the 35-row window is loaded up front
+    // ---- B and C channels: thread = channel pair, over this CTA's block of 32 rows; the 35-row window is loaded up front
     {
-        const int cp = tid & 127, rg = tid >> 7;
+        const int cp = tid, rg = part;
         const int cc = a.d_inner + 2 * cp;                               // conv channel of the pair's first member
         const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)cc * k;
         float wl[2][4];                                                  // wl[e][m]: weight of the row m steps back in time
@@ -148,8 +151,8 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
     for (int h0 = 0; h0 < a.H; h0 += 64) {
         __syncthreads();
 #pragma unroll 4
-        for (int i = 0; i < 16; ++i) {
-            const int idx = tid + 512 * i, hh = idx & 63, r = idx >> 6, t = r0 + r, h = h0 + hh;
+        for (int i = 0; i < Q * PREP_HEADS / PREP_THREADS; ++i) {
+            const int idx = tid + PREP_THREADS * i, hh = idx % PREP_HEADS, r = idx / PREP_HEADS, t = r0 + r, h = h0 + part * PREP_HEADS + hh;
             float d = 0.f;
             if (t < L && h < a.H) {
                 const float v = __bfloat162float(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h]) + w.dt_bias[h];
@@ -159,8 +162,8 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
         }
         __syncthreads();
         const int warp = tid >> 5, lane = tid & 31;
-        for (int hh = warp; hh < 64 && h0 + hh < a.H; hh += 16) {
-            const int h = h0 + hh;
+        for (int hh = warp; hh < PREP_HEADS && h0 + part * PREP_HEADS + hh < a.H; hh += PREP_THREADS / 32) {
+            const int h = h0 + part * PREP_HEADS + hh;
             const float Ah = -expf(w.A_log[h]) * LOG2E;
             float d[4], cum[4];
 #pragma unroll
@@ -471,13 +474,18 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (t < Q) misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
             mbar_arrive(&misc->empty_dl[sd]);
             named_sync(1, ROLE);                           // halo rows are in registers; wbuf is visible
+            // Row j of the block sits at j * 128 + ((colx ^ (j & 7)) << 4) in both tiles; with j & 7 = jx this is
+            // ((9 jx) ^ colx) << 4, so one running counter k = 144 jx and one exclusive-or give the offset of every row.
+            uint8_t *bx = xt + (toff + rb * RB) * 128 + sub, *bs = smem + OFF_XS + rb * RB * 128 + sub;
+            const uint8_t *wp = reinterpret_cast<const uint8_t *>(misc->wbuf + rb * RB + (rev ? RB - 1 : 0));
+            uint32_t k = rev ? (RB - 1) * 144u : 0u;
 #pragma unroll 2
             for (int tau = 0; tau < RB; ++tau) {
-                const int j = first + tau * step, xr = j + toff;
-                uint2 *xp = reinterpret_cast<uint2 *>(xt + xr * 128 + ((colx ^ (xr & 7)) << 4) + sub);
+                const uint32_t off = k ^ (colx << 4);
+                uint2 *xp = reinterpret_cast<uint2 *>(bx + off);
                 const uint2 rw = *xp;
                 const f32x2 cur[2] = {bf2_to_f2(rw.x), bf2_to_f2(rw.y)};
-                const float wj = misc->wbuf[j];
+                const float wj = *reinterpret_cast<const float *>(wp);
                 const f32x2 w2 = pk2(wj, wj);
                 uint32_t ox[2], os[2];
 #pragma unroll
@@ -493,7 +501,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     h3[e2] = h2[e2]; h2[e2] = h1[e2]; h1[e2] = cur[e2];
                 }
                 *xp = make_uint2(ox[0], ox[1]);
-                *reinterpret_cast<uint2 *>(smem + OFF_XS + j * 128 + ((colx ^ (j & 7)) << 4) + sub) = make_uint2(os[0], os[1]);
+                *reinterpret_cast<uint2 *>(bs + off) = make_uint2(os[0], os[1]);
+                k += rev ? -144u : 144u;
+                wp += rev ? -4 : 4;
             }
             fence_proxy_async();
             mbar_arrive(&misc->xs_full);
@@ -733,7 +743,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
 
-    ssd_prep_kernel<<<dim3(l.nch, a.B, ndir), 512, 0, s>>>(k, Bp, Cp, dA, dir0);
+    ssd_prep_kernel<<<dim3(l.nch * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, dir0);
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
