@@ -80,6 +80,7 @@ static_assert(offsetof(Misc, norm_w) % 16 == 0 && offsetof(Misc, wbuf) % 16 == 0
 
 struct SsdArgs {
     int B, L, H, d_inner, d_in_proj, conv_ch, k, flags, nch, Lp;
+    int Nr;                      // d_state of the model (<= N); B', C' and the state are zero-padded to N
     const __nv_bfloat16 *zx;
     float *ssq;
     const float *dA;             // [2][B][H][2][Lp]: Lambda, Lambda' (log2 units)
@@ -110,15 +111,18 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
     // ---- B and C channels: thread = channel pair, over this CTA's block of 32 rows; the 35-row window is loaded up front
     {
         const int cp = tid, rg = part;
-        const int cc = a.d_inner + 2 * cp;                               // conv channel of the pair's first member
+        const bool isC = cp >= N / 2;
+        const int pi = cp & (N / 2 - 1);                                 // pair index inside B or C
+        const bool valid = 2 * pi < a.Nr;                                // beyond the model's d_state: zero padding
+        const int cc = a.d_inner + (isC ? a.Nr : 0) + (valid ? 2 * pi : 0);   // conv channel of the pair's first member
         const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)cc * k;
         float wl[2][4];                                                  // wl[e][m]: weight of the row m steps back in time
 #pragma unroll
         for (int e = 0; e < 2; ++e)
 #pragma unroll
-            for (int m = 0; m < 4; ++m) wl[e][m] = m < k ? __bfloat162float(cw[e * k + k - 1 - m]) : 0.f;
+            for (int m = 0; m < 4; ++m) wl[e][m] = (m < k && valid) ? __bfloat162float(cw[e * k + k - 1 - m]) : 0.f;
         float bias[2] = {0.f, 0.f};
-        if (has_bias) {
+        if (has_bias && valid) {
             bias[0] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc]);
             bias[1] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc + 1]);
         }
@@ -130,10 +134,10 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
 #pragma unroll
         for (int i = 0; i < 35; ++i) {
             const int t = first + (i - 3) * step;
-            raw[i] = (t >= 0 && t < L) ? __ldg(col + (int64_t)t * ld32) : 0u;
-            if (cin && t < 0 && k - 1 + t >= 0) raw[i] = __ldg(cin + (int64_t)(k - 1 + t) * (a.conv_ch / 2));    // carried rows
+            raw[i] = (valid && t >= 0 && t < L) ? __ldg(col + (int64_t)t * ld32) : 0u;
+            if (valid && cin && t < 0 && k - 1 + t >= 0) raw[i] = __ldg(cin + (int64_t)(k - 1 + t) * (a.conv_ch / 2));    // carried rows
         }
-        __nv_bfloat16 *dst = (cp < 64 ? Bp + 2 * cp : Cp + 2 * (cp - 64)) + seq * L * N;
+        __nv_bfloat16 *dst = (isC ? Cp : Bp) + 2 * pi + seq * L * N;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             const int t = first + i * step;
@@ -391,12 +395,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int srow = t & (WG - 1), sh = t >> 7;      // state row and column half of this thread
         // incoming state -> TMEM (fp32) and shared memory (bf16)
         {
-            const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * N + srow : nullptr;
+            const float *h0 = (!rev && a.ssm_in && srow < a.Nr) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * a.Nr + srow : nullptr;
             {
                 const int half = sh;                     // this group's half of the state columns
                 uint32_t hs[32];
 #pragma unroll
-                for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * N]) : 0u;
+                for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * a.Nr]) : 0u;
                 tmem_st_x32(tlane + TM_HS + half * 32, hs);
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4)
@@ -511,14 +515,14 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
         if (ok && WAIT(&misc->st_full, (nch - 1) & 1)) state_update(dec_prev, false); else ok = false;
         if (ok && !rev && a.ssm_out) {
-            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * N + srow;
-            {
-                const int half = sh;
-                uint32_t hs[32];
-                tmem_ld_x32(tlane + TM_HS + half * 32, hs);
-                tmem_wait_ld();
+            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * a.Nr + srow;
+            const int half = sh;
+            uint32_t hs[32];
+            tmem_ld_x32(tlane + TM_HS + half * 32, hs);          // warp-wide: every lane takes part
+            tmem_wait_ld();
+            if (srow < a.Nr) {                                   // rows beyond the model's d_state are padding (exact zeros)
 #pragma unroll
-                for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * N] = __uint_as_float(hs[p]);
+                for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * a.Nr] = __uint_as_float(hs[p]);
             }
         }
     } else if (warp < 4 + 8 * NWG) {
@@ -696,14 +700,14 @@ Scratch scratch_layout(const ScanArgs &a) {
 }  // namespace
 
 bool scan_ssd_supports(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N != N || a.P != P || a.k < 2 || a.k > 4) return false;
+    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || a.P != P || a.k < 2 || a.k > 4) return false;   // smaller d_state: zero-padded to N
     if (a.d_in_proj % 8 || a.d_inner % 8) return false;                  // 16-byte rows for TMA and vector access
     if (a.H > 65535 || a.B > 65535) return false;
     return encode_fn() != nullptr;
 }
 
 size_t scan_ssd_workspace_bytes(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N != N || a.P != P) return 0;
+    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || a.P != P) return 0;
     return scratch_layout(a).total;
 }
 
@@ -715,7 +719,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     float *dA = reinterpret_cast<float *>(base + l.da);
     SsdArgs k{};
     k.B = a.B; k.L = a.L; k.H = a.H; k.d_inner = a.d_inner; k.d_in_proj = a.d_in_proj; k.conv_ch = a.conv_ch; k.k = a.k;
-    k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp;
+    k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp; k.Nr = a.N;
     k.zx = static_cast<const __nv_bfloat16 *>(a.zx); k.ssq = a.ssq; k.dA = dA;
     k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out; k.conv_in = static_cast<const __nv_bfloat16 *>(a.conv_in);
     k.dir[0] = a.dir[0]; k.dir[1] = a.dir[1];

@@ -89,3 +89,22 @@ def test_state_in_and_out(G):
     y2, s2_, _ = G.run_block_step(half, I.BF16, wf, wr, np.ascontiguousarray(x2[:, 128:]), s1.astype(np.float32), c1.astype(np.float32), dir_mask=1)
     assert G.rel_l2(np.concatenate([y1, y2], axis=1), whole) <= 5e-3
     assert G.rel_l2(s2_, s_whole) <= 5e-3
+
+
+@pytest.mark.parametrize("N,H", [(16, 8), (32, 8), (64, 8)])
+def test_smaller_d_state_runs_zero_padded(G, N, H):
+    """d_state below 128 takes the same kernel with B', C' and the state zero-padded: parity of the output, and the
+    carried state in the model's own [B, H, P, d_state] layout, in and out."""
+    shape = I.MixerShape(2, 300, 32 * H, 2, N, 4, H)
+    assert shape.d_in_proj % 8 == 0                         # 16-byte rows: the tensor-core path takes the shape
+    wf, wr = I.make_mixer_weights(shape, 20 + N, I.BF16, perturb=True)
+    x = I.make_activations(shape, 20 + N, I.BF16)
+    kw = G.oracle_kwargs(shape)
+    _check(G, G.run_forward(shape, I.BF16, wf, wr, x), O.bimamba_forward(x, wf, wr, **kw))
+    ssm_in, conv_in = I.make_states(shape, 20 + N, I.BF16)
+    y_o, s_o, c_o = O.bimamba_block_step(x, wf, wr, ssm_state_in=ssm_in, conv_state_in=conv_in, **kw)
+    y_g, s_g, c_g = G.run_block_step(shape, I.BF16, wf, wr, x, ssm_in, conv_in)
+    assert s_g.shape == s_o.shape == (2, H, 64, N)
+    _check(G, y_g, y_o)
+    _check(G, s_g, s_o)
+    _check(G, c_g, c_o)
