@@ -30,6 +30,7 @@ struct EpiArgs {
     void *C; int64_t ldc; int c_is_f32;
     const float *row_scale; const float *addend; int64_t ld_add;
     int M, N, K;
+    int n_fast;      // tile order: consecutive tiles step along N (the A rows are streamed once, B stays in L2) or along M
 };
 
 template <int BN>
@@ -68,7 +69,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+                const int m0 = (ep.n_fast ? tile / tiles_n : tile % tiles_m) * BM, n0 = (ep.n_fast ? tile % tiles_n : tile / tiles_m) * BN;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!(ok = mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, status))) break;
@@ -118,7 +119,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
             const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
-            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+            const int m0 = (ep.n_fast ? tile / tiles_n : tile % tiles_m) * BM, n0 = (ep.n_fast ? tile % tiles_n : tile / tiles_m) * BN;
             ok = mbar_wait(&bars->tmem_full[buf], bph, abort_flag, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -202,7 +203,8 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     if (!status) return cudaErrorUnknown;
     const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K};
+    // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
+    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.M > a.N ? 1 : 0};
     gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma, mb, ep, status);
     count_launch();
     return cudaGetLastError();
