@@ -115,6 +115,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // ------------------------------------------------------------ epilogue: 4 warps, one TMEM lane quarter each
         const int q = warp & 3;                            // warps 2,3,4,5 -> quarters 2,3,0,1
+        // 32-byte stores and loads (one full sector per thread) when every row of C / of the addend starts on a 32-byte boundary
+        const int c_es = ep.c_is_f32 ? 4 : 2;
+        const bool wide_c = (reinterpret_cast<uintptr_t>(ep.C) & 31u) == 0 && ((ep.ldc * c_es) & 31) == 0;
+        const bool wide_add = ep.addend && (reinterpret_cast<uintptr_t>(ep.addend) & 31u) == 0 && ((ep.ld_add * 4) & 31) == 0;
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
@@ -140,7 +144,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * sc;
                 const bool full = col + 32 <= ep.N;
                 if (add_row) {
-                    if (full && (ep.ld_add & 3) == 0) {
+                    if (full && wide_add) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint32_t a8[8];
+                            ld_global_256(add_row + col + j, a8);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) v[j + e] += __uint_as_float(a8[e]);
+                        }
+                    } else if (full && (ep.ld_add & 3) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             const float4 a4 = *reinterpret_cast<const float4 *>(add_row + col + j);
@@ -152,7 +164,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 if (ep.c_is_f32) {
                     float *crow = static_cast<float *>(ep.C) + (int64_t)row * ep.ldc + col;
-                    if (full && (ep.ldc & 3) == 0) {
+                    if (full && wide_c) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint32_t o[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(v[j + e]);
+                            st_global_256(crow + j, o);
+                        }
+                    } else if (full && (ep.ldc & 3) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4 *>(crow + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                     } else {
@@ -160,7 +180,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 } else {
                     __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(ep.C) + (int64_t)row * ep.ldc + col;
-                    if (full && (ep.ldc & 7) == 0) {
+                    if (full && wide_c) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 16) {
+                            uint32_t o[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] = pack_bf16(v[j + 2 * e], v[j + 2 * e + 1]);
+                            st_global_256(crow + j, o);
+                        }
+                    } else if (full && (ep.ldc & 7) == 0) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 8)
                             *reinterpret_cast<uint4 *>(crow + j) = make_uint4(pack_bf16(v[j], v[j + 1]), pack_bf16(v[j + 2], v[j + 3]),
