@@ -158,16 +158,6 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
     const bool norm_on = (c->flags & DM_FLAG_GATED_RMSNORM) != 0;
     cudaError_t e;
 
-    for (int dir = 0; dir < 2; ++dir) {
-        if (!(c->dir_mask & (1 << dir))) continue;
-        StageTimer tm(DM_STAGE_IN_PROJ, s);
-        GemmArgs a{};
-        a.A = x; a.lda = m.d; a.B = w[dir].w_in; a.ldb = m.d;
-        a.C = zx + (size_t)dir * m.T * m.d_in_proj * m.es; a.ldc = m.d_in_proj;
-        a.in_dtype = c->dtype; a.c_dtype = c->dtype; a.M = (int)m.T; a.N = m.d_in_proj; a.K = m.d;
-        if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "in_proj");
-    }
-
     ScanArgs sa{};
     sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
     sa.d_in_proj = m.d_in_proj; sa.conv_ch = m.conv_ch;
@@ -178,9 +168,25 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         sa.dir[dir].dt_bias = w[dir].dt_bias; sa.dir[dir].A_log = w[dir].A_log; sa.dir[dir].D = w[dir].D;
     }
     sa.ssm_in = ssm_in; sa.conv_in = conv_in; sa.ssm_out = ssm_out;
+    // The tensor-core scan is bound by instruction issue while the GEMM's epilogue warps mostly wait: on that path the
+    // gate's SiLU(z) (Sec. 3.2) is applied to the z columns by the in_proj epilogue.
+    sa.z_gated = 1;
+    const bool ssd = scan_ssd_supports(sa);
+    sa.z_gated = ssd ? 1 : 0;
+
+    for (int dir = 0; dir < 2; ++dir) {
+        if (!(c->dir_mask & (1 << dir))) continue;
+        StageTimer tm(DM_STAGE_IN_PROJ, s);
+        GemmArgs a{};
+        a.A = x; a.lda = m.d; a.B = w[dir].w_in; a.ldb = m.d;
+        a.C = zx + (size_t)dir * m.T * m.d_in_proj * m.es; a.ldc = m.d_in_proj;
+        a.in_dtype = c->dtype; a.c_dtype = c->dtype; a.M = (int)m.T; a.N = m.d_in_proj; a.K = m.d;
+        a.silu_cols = ssd ? m.d_inner : 0;
+        if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "in_proj");
+    }
     {
         StageTimer tm(DM_STAGE_SCAN, s);
-        if (scan_ssd_supports(sa)) e = scan_ssd(sa, ws + l.scan, s);
+        if (ssd) e = scan_ssd(sa, ws + l.scan, s);
         else e = scan_sequential(sa, ws + l.scan, s);
     }
     if (e != cudaSuccess) return cuda_fail(e, "scan");

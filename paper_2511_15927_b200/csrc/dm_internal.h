@@ -32,6 +32,7 @@ struct GemmArgs {
     int M, N, K;
     const float *row_scale;
     const float *addend; int64_t ld_add;
+    int silu_cols;           // output columns [0, silu_cols) get SiLU applied after scale and addend (0 = none)
 };
 cudaError_t gemm_simple(const GemmArgs &a, cudaStream_t s);
 // Tensor-core path (tcgen05 + TMEM + TMA).  Returns cudaErrorNotSupported for shapes it does not take.
@@ -49,6 +50,7 @@ struct ScanArgs {
     int B, L, d_inner, H, P, N, k, d_in_proj, conv_ch;
     int dtype, flags, dir_mask, chunk;
     const void *zx;          // [2][B*L][d_in_proj] dtype: in_proj output of each direction
+    int z_gated;             // the z columns of zx already hold SiLU(z) (applied by the in_proj epilogue); the tensor-core scan requires it
     void *g;                 // [2][B*L][d_inner]   dtype: gated output (times norm_w when the norm is on)
     float *ssq;              // [2][B*L][H] per-head sum of squares of the gated output (norm on), or NULL
     ScanDir dir[2];

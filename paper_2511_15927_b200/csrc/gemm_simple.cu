@@ -15,7 +15,7 @@ template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(256)
 gemm_simple_kernel(const TIn *__restrict__ A, int64_t lda, const TIn *__restrict__ B, int64_t ldb,
                    TOut *C, int64_t ldc, int M, int N, int K,
-                   const float *__restrict__ row_scale, const float *addend, int64_t ld_add) {
+                   const float *__restrict__ row_scale, const float *addend, int64_t ld_add, int silu_cols) {
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -57,6 +57,7 @@ gemm_simple_kernel(const TIn *__restrict__ A, int64_t lda, const TIn *__restrict
             if (gn >= N) continue;
             float v = acc[i][j] * sc;
             if (addend) v += addend[(int64_t)gm * ld_add + gn];
+            if (gn < silu_cols) v = v / (1.f + __expf(-v));
             if constexpr (sizeof(TOut) == 4) C[(int64_t)gm * ldc + gn] = v;
             else C[(int64_t)gm * ldc + gn] = __float2bfloat16_rn(v);
         }
@@ -68,7 +69,7 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM);
     gemm_simple_kernel<TIn, TOut><<<grid, 256, 0, s>>>(
         static_cast<const TIn *>(a.A), a.lda, static_cast<const TIn *>(a.B), a.ldb,
-        static_cast<TOut *>(a.C), a.ldc, a.M, a.N, a.K, a.row_scale, a.addend, a.ld_add);
+        static_cast<TOut *>(a.C), a.ldc, a.M, a.N, a.K, a.row_scale, a.addend, a.ld_add, a.silu_cols);
     count_launch();
     return cudaGetLastError();
 }

@@ -30,6 +30,7 @@ struct EpiArgs {
     void *C; int64_t ldc; int c_is_f32;
     const float *row_scale; const float *addend; int64_t ld_add;
     int M, N, K;
+    int silu_cols;   // SiLU on output columns below this one
     int n_fast;      // tile order: consecutive tiles step along N (the A rows are streamed once, B stays in L2) or along M
 };
 
@@ -162,6 +163,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int j = 0; j < 32; ++j) if (col + j < ep.N) v[j] += add_row[col + j];
                     }
                 }
+                if (col < ep.silu_cols) {                  // gate columns: SiLU here, where the ALUs idle, not in the scan
+                    if (col + 32 <= ep.silu_cols) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) { const float hv = 0.5f * v[j]; v[j] = fmaf(hv, tanh_fast(hv), hv); }   // SiLU(v) = v/2 + v/2 tanh(v/2)
+                    } else {
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < ep.silu_cols) { const float hv = 0.5f * v[j]; v[j] = fmaf(hv, tanh_fast(hv), hv); }
+                    }
+                }
                 if (ep.c_is_f32) {
                     float *crow = static_cast<float *>(ep.C) + (int64_t)row * ep.ldc + col;
                     if (full && wide_c) {
@@ -232,7 +242,7 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
     const int grid = tiles < sm_count() ? tiles : sm_count();
     // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
-    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.M > a.N ? 1 : 0};
+    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols, a.M > a.N ? 1 : 0};
     gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma, mb, ep, status);
     count_launch();
     return cudaGetLastError();

@@ -21,8 +21,8 @@
 //     warps 4-11   conv groups: state update of the previous chunk, h <- exp(Lambda_last) h + St (fp32, kept in TMEM) with its
 //                  bf16 copy for the next Yb; depthwise conv + SiLU of the x tile in place (8-row blocks); the decay-weighted copy w o x'
 //     warps 12-19  mask groups: S (TMEM, fp32) -> W (TMEM, bf16), the 16-column groups split between the two groups
-//     warps 20-27  epilogue groups (half of the channels each): y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w],
-//                  per-head sum of squares, written over the z tile and stored with TMA
+//     warps 20-27  epilogue groups (half of the channels each): y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w] (the z
+//                  tile arrives as SiLU(z): the in_proj epilogue applies it), per-head sum of squares, written over the z tile and stored with TMA
 // Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
 // device status word, all roles leave their loops, outstanding TMA traffic is waited for (bounded), TMEM is
 // freed and the CTA returns.
@@ -627,7 +627,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             mbar_arrive(&misc->empty_dl[sd]);
             const int t = pc * Q + row;
             uint8_t *zt = smem + OFF_Z + sz * T16;
-            const f32x2 ei2 = pk2(ei, ei), half2 = pk2(0.5f, 0.5f);
+            const f32x2 ei2 = pk2(ei, ei);
             f32x2 ss2 = pk2(0.f, 0.f);
 #pragma unroll 1
             for (int c8 = eg * 4; c8 < eg * 4 + 4; ++c8) {   // 8 channels (one 16-byte chunk of z) at a time
@@ -646,10 +646,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 for (int e2 = 0; e2 < 4; ++e2) {
                     const f32x2 y = fma2(ei2, pk2(__uint_as_float(yb[2 * e2]), __uint_as_float(yb[2 * e2 + 1])),
                                          pk2(__uint_as_float(ya[2 * e2]), __uint_as_float(ya[2 * e2 + 1])));
-                    const f32x2 hh = mul2(bf2_to_f2(zw[e2]), half2);     // SiLU(z) = z/2 + z/2 tanh(z/2)
-                    float ha, hb;
-                    upk2(hh, ha, hb);
-                    const f32x2 g = mul2(y, fma2(hh, pk2(tanh_fast(ha), tanh_fast(hb)), hh));
+                    const f32x2 g = mul2(y, bf2_to_f2(zw[e2]));          // the z tile holds SiLU(z): the in_proj epilogue applied it
                     ss2 = fma2(g, g, ss2);
                     ow[e2] = f2_to_bf2(mul2(g, nw[e2]));
                 }
@@ -700,7 +697,8 @@ Scratch scratch_layout(const ScanArgs &a) {
 }  // namespace
 
 bool scan_ssd_supports(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || a.P != P || a.k < 2 || a.k > 4) return false;   // smaller d_state: zero-padded to N
+    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || a.P != P || a.k < 2 || a.k > 4) return false;
+    if (!a.z_gated) return false;                                         // the gate's SiLU is the in_proj epilogue's job on this path   // smaller d_state: zero-padded to N
     if (a.d_in_proj % 8 || a.d_inner % 8) return false;                  // 16-byte rows for TMA and vector access
     if (a.H > 65535 || a.B > 65535) return false;
     return encode_fn() != nullptr;
