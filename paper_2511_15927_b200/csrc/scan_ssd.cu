@@ -18,8 +18,9 @@
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
 //     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  Ya = W x',  St = B^T (w o x')
 //     warp 2      TMA loads of the z tile        warp 3   TMA loads of the B' and C' tiles
-//     warps 4-11   conv groups: state update of the previous chunk, h <- exp(Lambda_last) h + St (fp32, kept in TMEM) with its
-//                  bf16 copy for the next Yb; depthwise conv + SiLU of the x tile in place (8-row blocks); the decay-weighted copy w o x'
+//     warps 4-11   conv groups: state hand-over (the fp32 state stays in TMEM and St accumulates onto it: its bf16 copy for Yb is
+//                  taken and it is scaled by exp(Lambda_last) before St is issued); depthwise conv + SiLU of the x tile in place
+//                  (8-row blocks); the decay-weighted copy w o x'
 //     warps 12-19  mask groups: S (TMEM, fp32) -> W (TMEM, bf16), the 16-column groups split between the two groups
 //     warps 20-27  epilogue groups (half of the channels each): y = Ya + exp(Lambda_i) Yb,  g = y SiLU(z) [* norm_w] (the z
 //                  tile arrives as SiLU(z): the in_proj epilogue applies it), per-head sum of squares, written over the z tile and stored with TMA
@@ -63,11 +64,11 @@ static_assert(OFF_Z % 1024 == 0 && OFF_B % 1024 == 0 && OFF_C % 1024 == 0 && OFF
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 // TMEM columns (all 512 are allocated)
-constexpr uint32_t TM_S = 0, TM_W = 128, TM_YB1 = 192, TM_YA = 256, TM_YB0 = 320, TM_ST = 384, TM_HS = 448, TM_COLS = 512;    // Yb is double-buffered
+constexpr uint32_t TM_S = 0, TM_W = 128, TM_YB1 = 192, TM_YA = 256, TM_YB0 = 320, TM_HS = 448, TM_COLS = 512;    // Yb is double-buffered; columns 384..447 are unused
 
 struct Misc {
     uint64_t full_x[NX], empty_x[NX], full_z[NZ], empty_z[NZ], full_b[NB], empty_b[NB], full_c, empty_c, full_dl[NDL], empty_dl[NDL];
-    uint64_t xs_full, s_full, s_empty, w_full, st_full, st_empty, h_full, y_full, ya_empty, yb_empty[2];
+    uint64_t xs_full, s_full, s_empty, w_full, st_full, hs_ready, h_full, y_full, ya_empty, yb_empty[2];
     uint32_t tmem_base;
     int abort;
     alignas(16) float norm_w[P];  // the three arrays below are read as float4
@@ -226,7 +227,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         mbar_init(&misc->xs_full, ROLE);
         mbar_init(&misc->s_full, 1);   mbar_init(&misc->s_empty, ROLE);
         mbar_init(&misc->w_full, ROLE);
-        mbar_init(&misc->st_full, 1);  mbar_init(&misc->st_empty, ROLE);
+        mbar_init(&misc->st_full, 1);  mbar_init(&misc->hs_ready, ROLE);
         mbar_init(&misc->h_full, ROLE);
         mbar_init(&misc->y_full, 1);   mbar_init(&misc->ya_empty, ROLE);
         mbar_init(&misc->yb_empty[0], ROLE); mbar_init(&misc->yb_empty[1], ROLE);
@@ -353,12 +354,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tyb, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), dH + kk * 128, I64);
                 umma_commit(&misc->empty_c);             // also releases the bf16 state copy
                 if (c > 0 && !issue_ya(c - 1)) break;
-                // St = B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major)
-                if (!WAIT2(&misc->xs_full, par, &misc->st_empty, par ^ 1)) break;
+                // h += B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major), onto the state the conv groups have scaled
+                if (!WAIT2(&misc->xs_full, par, &misc->hs_ready, par)) break;
                 fence_after();
-                umma_ss<0>(tmem + TM_ST, dBm, dXs, I64T);
+                umma_ss<1>(tmem + TM_HS, dBm, dXs, I64T);
 #pragma unroll
-                for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tmem + TM_ST, dBm + kk * 128, dXs + kk * 128, I64T);
+                for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tmem + TM_HS, dBm + kk * 128, dXs + kk * 128, I64T);
                 umma_commit(&misc->st_full);             // also frees the w o x' buffer
                 umma_commit(&misc->empty_b[sb]);
                 if (c == nch - 1) ok = issue_ya(c);
@@ -393,71 +394,56 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int first = rev ? rb * RB + RB - 1 : rb * RB, step = rev ? -1 : 1;   // first-in-time chunk row of the block
         const int toff = rev ? 0 : HALO;                                          // tile row = chunk row + toff
         const int srow = t & (WG - 1), sh = t >> 7;      // state row and column half of this thread
-        // incoming state -> TMEM (fp32) and shared memory (bf16)
+        // incoming state -> TMEM (fp32)
         {
             const float *h0 = (!rev && a.ssm_in && srow < a.Nr) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * a.Nr + srow : nullptr;
-            {
-                const int half = sh;                     // this group's half of the state columns
-                uint32_t hs[32];
+            uint32_t hs[32];
 #pragma unroll
-                for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(half * 32 + p) * a.Nr]) : 0u;
-                tmem_st_x32(tlane + TM_HS + half * 32, hs);
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4)
-                    *reinterpret_cast<uint4 *>(smem + OFF_H + srow * 128 + (((half * 4 + c4) ^ (srow & 7)) << 4)) =
-                        make_uint4(pack_bf16(__uint_as_float(hs[c4 * 8]), __uint_as_float(hs[c4 * 8 + 1])),
-                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 2]), __uint_as_float(hs[c4 * 8 + 3])),
-                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 4]), __uint_as_float(hs[c4 * 8 + 5])),
-                                   pack_bf16(__uint_as_float(hs[c4 * 8 + 6]), __uint_as_float(hs[c4 * 8 + 7])));
-            }
-            fence_proxy_async();
+            for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(sh * 32 + p) * a.Nr]) : 0u;
+            tmem_st_x32(tlane + TM_HS + sh * 32, hs);
             tmem_wait_st();
-            fence_before();
-            mbar_arrive(&misc->h_full);
         }
-        // state: h <- 2^(Lambda_last) h + St (fp32, kept in TMEM); bf16 copy for the next chunk's Yb.  Thread = state row, half of the columns.
-        auto state_update = [&](float dec, bool more) {
+        // The fp32 state lives in TMEM and St accumulates onto it: before chunk c's St is issued, the state entering the
+        // chunk is copied to shared memory as bf16 (B operand of Yb) and scaled in place by the chunk's total decay, so
+        // that after St it reads h <- 2^(Lambda_last) h + B'^T (w o x').  Thread = state row, half of the columns.
+        auto state_prepare = [&](float dec) {
             fence_after();
             const f32x2 dec2 = pk2(dec, dec);
 #pragma unroll 1
             for (int c8 = sh * 4; c8 < sh * 4 + 4; ++c8) {   // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
-                uint32_t st[8], hs[8];
-                tmem_ld_x8(tlane + TM_ST + c8 * 8, st);
+                uint32_t hs[8];
                 tmem_ld_x8(tlane + TM_HS + c8 * 8, hs);
                 tmem_wait_ld();
                 uint32_t hb[4];
 #pragma unroll
                 for (int e2 = 0; e2 < 4; ++e2) {
-                    const f32x2 hn = fma2(dec2, pk2(__uint_as_float(hs[2 * e2]), __uint_as_float(hs[2 * e2 + 1])),
-                                          pk2(__uint_as_float(st[2 * e2]), __uint_as_float(st[2 * e2 + 1])));
+                    const f32x2 hv = pk2(__uint_as_float(hs[2 * e2]), __uint_as_float(hs[2 * e2 + 1]));
+                    hb[e2] = f2_to_bf2(hv);
                     float lo, hi;
-                    upk2(hn, lo, hi);
+                    upk2(mul2(dec2, hv), lo, hi);
                     hs[2 * e2] = __float_as_uint(lo); hs[2 * e2 + 1] = __float_as_uint(hi);
-                    hb[e2] = pack_bf16(lo, hi);
                 }
                 tmem_st_x8(tlane + TM_HS + c8 * 8, hs);
-                if (more) *reinterpret_cast<uint4 *>(smem + OFF_H + srow * 128 + ((c8 ^ (srow & 7)) << 4)) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
+                *reinterpret_cast<uint4 *>(smem + OFF_H + srow * 128 + ((c8 ^ (srow & 7)) << 4)) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
             }
-            fence_before();
-            mbar_arrive(&misc->st_empty);
             fence_proxy_async();
             tmem_wait_st();
             fence_before();
-            if (more) mbar_arrive(&misc->h_full);
+            mbar_arrive(&misc->hs_ready);
+            mbar_arrive(&misc->h_full);
         };
-        float dec_prev = 0.f;
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sx = c % NX, sd = c % NDL;
             const uint32_t par = c & 1;
             if (ok) ok = WAIT3(&misc->full_x[sx], (c / NX) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->st_full, par ^ 1);
             if (!named_all(1, ROLE, ok)) { ok = false; break; }
-            // St of the previous chunk has completed (so has its Yb, issued before it): update the state first, the next Yb waits for it
-            if (c > 0) state_update(dec_prev, true);
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
+            // St of the previous chunk has completed (so has its Yb, issued before it): hand the state over first, Yb and St wait for it
+            state_prepare(ex2f(lam[rev ? 0 : Q - 1]));
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
             // place: they are read before the group barrier; the block's own rows are read just before being replaced.
             uint8_t *xt = smem + OFF_X + sx * XTILE;
-            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
             f32x2 h1[2], h2[2], h3[2];
             {
                 uint2 hr[3];
@@ -474,7 +460,6 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 h2[0] = bf2_to_f2(hr[1].x); h2[1] = bf2_to_f2(hr[1].y);
                 h3[0] = bf2_to_f2(hr[2].x); h3[1] = bf2_to_f2(hr[2].y);
             }
-            const float dec_cur = ex2f(lam[rev ? 0 : Q - 1]);   // this chunk's total decay, for the state update at the next iteration
             if (t < Q) misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
             mbar_arrive(&misc->empty_dl[sd]);
             named_sync(1, ROLE);                           // halo rows are in registers; wbuf is visible
@@ -511,9 +496,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             }
             fence_proxy_async();
             mbar_arrive(&misc->xs_full);
-            dec_prev = dec_cur;
         }
-        if (ok && WAIT(&misc->st_full, (nch - 1) & 1)) state_update(dec_prev, false); else ok = false;
+        if (!(ok && WAIT(&misc->st_full, (nch - 1) & 1))) ok = false;     // the last St has landed: TMEM holds the outgoing state
+        fence_after();
         if (ok && !rev && a.ssm_out) {
             float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * a.Nr + srow;
             const int half = sh;
