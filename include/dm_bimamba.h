@@ -165,8 +165,12 @@ int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype,
               int64_t rows, int32_t in_features, int32_t out_features,
               const float *row_scale, const float *addend, void *cuda_stream);
 
-/* Same as dm_bimamba_forward, but x and y are HOST buffers (pageable or pinned): the call copies x to
- * the device, runs the mixer and copies y back, all on `cuda_stream`, then synchronises it.
+/* Same as dm_bimamba_forward, but x and y are HOST buffers (pageable or pinned; pinned lets the copies
+ * overlap): the call copies x to the device, runs the mixer and copies y back, then synchronises
+ * `cuda_stream`.  Batch rows are independent, so the batch is cut into up to 8 pieces of whole rows (about 4096 tokens or more each) and the
+ * copy-in of the next piece and the copy-out of the previous one run on two internal streams (created on
+ * the first call on a device) while the current piece is computed on `cuda_stream`; the work is ordered
+ * after whatever was enqueued on `cuda_stream` before.  Calls on the same device must not overlap.
  * `workspace` must hold dm_bimamba_workspace_bytes + 2*B*L*d_model*sizeof(dtype) bytes. */
 int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
                             const void *x_host, void *y_host,

@@ -485,6 +485,35 @@ int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype, int
     return DM_OK;
 }
 
+// Copy streams and events of the host-buffer entry point, one set per device, created on first use.
+namespace {
+constexpr int HOST_PIECES = 8, MAX_DEVICES = 64;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, copied[HOST_PIECES] = {}, computed[HOST_PIECES] = {};
+};
+HostPipe *host_pipe() {
+    static HostPipe pipes[MAX_DEVICES];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    HostPipe &p = pipes[dev];
+    if (p.ready) return &p;
+    bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < HOST_PIECES && ok; ++i)
+        ok = cudaEventCreateWithFlags(&p.copied[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&p.computed[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    p.ready = true;
+    return &p;
+}
+}  // namespace
+
 int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], const void *x_host, void *y_host,
                             void *workspace, size_t workspace_bytes, void *cuda_stream) {
     Dims m;
@@ -496,12 +525,40 @@ int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], 
     if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;
     char *ws = static_cast<char *>(workspace);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    void *xd = ws, *yd = ws + act;
-    cudaError_t e = cudaMemcpyAsync(xd, x_host, (size_t)m.T * m.d * m.es, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(e, "copy x to the device");
-    st = dm_bimamba_forward(cfg, w, xd, yd, ws + 2 * act, workspace_bytes - 2 * act, cuda_stream);
-    if (st != DM_OK) return st;
-    if ((e = cudaMemcpyAsync(y_host, yd, (size_t)m.T * m.d * m.es, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e, "copy y to the host");
+    char *xd = ws, *yd = ws + act;
+    HostPipe *hp = host_pipe();
+    if (!hp) return fail(DM_ERR_CUDA, "could not create the copy streams");
+    // Batch rows are independent (Sec. 3.2: the mixer acts on each sequence separately), so the batch is cut into
+    // pieces of whole rows: while piece i is computed on the caller's stream, piece i+1 is on its way in and piece
+    // i-1 on its way out.  The pieces share the mixer workspace (they run one after the other on `cuda_stream`).
+    // at least ~4096 tokens per piece (smaller pieces run the kernels below their full-size efficiency), at most HOST_PIECES pieces
+    int rows = (int)((4096 + m.L - 1) / m.L);
+    if (rows < (m.B + HOST_PIECES - 1) / HOST_PIECES) rows = (m.B + HOST_PIECES - 1) / HOST_PIECES;
+    if (rows > m.B) rows = m.B;
+    const int pieces = (m.B + rows - 1) / rows;
+    const size_t row_bytes = (size_t)m.L * m.d * m.es;
+    cudaError_t e;
+    if ((e = cudaEventRecord(hp->start, s)) != cudaSuccess) return cuda_fail(e, "record");
+    if ((e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess) return cuda_fail(e, "wait");      // after the caller's earlier work
+    if ((e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess) return cuda_fail(e, "wait");
+    dm_mixer_cfg piece_cfg = *cfg;
+    for (int i = 0; i < pieces; ++i) {
+        const int r0 = i * rows, nr = (r0 + rows <= m.B) ? rows : m.B - r0;
+        const size_t off = (size_t)r0 * row_bytes, bytes = (size_t)nr * row_bytes;
+        if ((e = cudaMemcpyAsync(xd + off, static_cast<const char *>(x_host) + off, bytes, cudaMemcpyHostToDevice, hp->in)) != cudaSuccess)
+            return cuda_fail(e, "copy x to the device");
+        if ((e = cudaEventRecord(hp->copied[i], hp->in)) != cudaSuccess) return cuda_fail(e, "record");
+        if ((e = cudaStreamWaitEvent(s, hp->copied[i], 0)) != cudaSuccess) return cuda_fail(e, "wait");
+        piece_cfg.batch = nr;
+        st = dm_bimamba_forward(&piece_cfg, w, xd + off, yd + off, ws + 2 * act, workspace_bytes - 2 * act, cuda_stream);
+        if (st != DM_OK) return st;
+        if ((e = cudaEventRecord(hp->computed[i], s)) != cudaSuccess) return cuda_fail(e, "record");
+        if ((e = cudaStreamWaitEvent(hp->out, hp->computed[i], 0)) != cudaSuccess) return cuda_fail(e, "wait");
+        if ((e = cudaMemcpyAsync(static_cast<char *>(y_host) + off, yd + off, bytes, cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
+            return cuda_fail(e, "copy y to the host");
+    }
+    if ((e = cudaEventRecord(hp->done, hp->out)) != cudaSuccess) return cuda_fail(e, "record");
+    if ((e = cudaStreamWaitEvent(s, hp->done, 0)) != cudaSuccess) return cuda_fail(e, "wait");
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e, "synchronize");
     return DM_OK;
 }

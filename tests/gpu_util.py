@@ -25,6 +25,24 @@ def run_forward(shape, dtype, wf, wr, x, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.
     return yd.float().cpu().numpy().astype(np.float64)
 
 
+def run_forward_host(shape, dtype, wf, wr, x, pinned=True):
+    """dm_bimamba_forward_host: x and y live in host memory, the library stages them through its workspace."""
+    cfg = cfg_of(shape, dtype)
+    dwf, dwr = dev_dir_weights(wf, dtype), dev_dir_weights(wr, dtype)
+    xh = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(tdtype(dtype))
+    yh = torch.empty_like(xh)
+    if pinned:
+        xh, yh = xh.pin_memory(), yh.pin_memory()
+    act = (xh.numel() * xh.element_size() + 255) // 256 * 256
+    nb = dm.dm_bimamba_workspace_bytes(cfg) + 2 * act
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_bimamba_forward_host(cfg, (dm.make_dir_weights(dwf), dm.make_dir_weights(dwr)), xh.data_ptr(), yh.data_ptr(),
+                               ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    return yh.float().numpy().astype(np.float64)
+
+
 def run_block_step(shape, dtype, wf, wr, x_blk, ssm_in=None, conv_in=None, want_state=True, flags=dm.DM_FLAGS_DEFAULT,
                    dir_mask=dm.DM_DIR_BOTH, chunk=0):
     cfg = cfg_of(shape, dtype, flags, dir_mask, chunk)

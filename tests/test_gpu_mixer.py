@@ -178,3 +178,14 @@ def test_unsupported_and_error_paths_do_not_launch(G):
         dm.dm_bimamba_forward(cfg, (dm.dm_dir_weights(), dm.dm_dir_weights()), 0, 0, 0, 0)
     assert dm.dm_kernel_launch_count() == before
     dm.dm_check(0)
+
+
+@pytest.mark.parametrize("B,pinned", [(1, True), (5, True), (20, True), (3, False)])
+def test_host_buffer_entry_equals_device_entry(G, B, pinned):
+    """The host-buffer call cuts the batch into pieces of whole rows and overlaps their copies with the compute;
+    rows are independent, so its result is the device call's, bit for bit (uneven last piece included)."""
+    shape = I.MixerShape(B, 2100, 128, 2, 128, 4, 4)          # pieces of 2 rows (3 rows at B = 20), the last one shorter
+    wf, wr, x = _case(shape, I.BF16, seed=30 + B)
+    want = G.run_forward(shape, I.BF16, wf, wr, x)
+    for _ in range(2):                                        # second call reuses the library's copy streams
+        np.testing.assert_array_equal(G.run_forward_host(shape, I.BF16, wf, wr, x, pinned), want)
