@@ -27,6 +27,13 @@ nothing printed can confirm -- the gated RMS norm inside each direction (both se
 implemented and tested), when the carried state is committed, and the stack's plain RMSNorm
 pre-norm without the MLP sublayer.  For those three: parity unpinned (by the paper); they follow
 the stated readings.
+
+The timestep-conditioned block of App. A.1 (AdaLN before the mixer and before the MLP, Eq. "AdaLN" and
+the two equations after it) is `diffusion_block` / `denoise_step_cond`.  Its arithmetic is pinned
+(standardisation, identities, brute force, the FLOP rows "MLP" and "AdaLN" of App. C); what the paper
+leaves open there -- the third modulation vector per sublayer that App. C's 6*d count implies and the
+equation does not show (read as a gate on the sublayer's output), the MLP's activation (GELU, tanh
+form) and the epsilon of the normalisation -- is parity unpinned (by the paper) as well.
 """
 from __future__ import annotations
 
@@ -297,3 +304,84 @@ def denoise_step(tokens, sw: dict, *, rms_eps: float = 1e-5, states_in=None, ret
     if return_hidden:
         res += (hidden,)
     return res[0] if len(res) == 1 else res
+
+
+# --------------------------------------------------------------------------------------------
+# Timestep-conditioned block (App. A.1): AdaLN -> mixer -> residual, AdaLN -> MLP -> residual
+# --------------------------------------------------------------------------------------------
+def layernorm_plain(x, eps: float = 1e-5):
+    """(x - mu(x)) / sigma(x) over the channel axis (App. A.1, Eq. "AdaLN"): population variance,
+    epsilon under the root, no learned affine."""
+    x = np.asarray(x, F64)
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps)
+
+
+def adaln(x, gamma, beta, eps: float = 1e-5):
+    """AdaLN(x; tau) = gamma_t * (x - mu) / sigma + beta_t (App. A.1); gamma, beta: [B, d], one pair per
+    sequence (the timestep is per sequence), x: [B, L, d]."""
+    return np.asarray(gamma, F64)[:, None, :] * layernorm_plain(x, eps) + np.asarray(beta, F64)[:, None, :]
+
+
+def gelu_tanh(v):
+    v = np.asarray(v, F64)
+    return 0.5 * v * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (v + 0.044715 * v ** 3)))
+
+
+def modulation(tau, w_cond, b_cond=None):
+    """W_cond tau_t (+ bias): [B, d_c] -> six vectors of d channels per sequence (App. C counts
+    2 * 6d * d_c FLOPs per layer).  Order: (beta, gamma, gate) of the mixer sublayer, then of the MLP
+    sublayer."""
+    tau = np.asarray(tau, F64)
+    m = tau @ np.asarray(w_cond, F64).T
+    if b_cond is not None:
+        m = m + np.asarray(b_cond, F64)
+    d = m.shape[1] // 6
+    return tuple(m[:, i * d:(i + 1) * d] for i in range(6))
+
+
+def mlp(u, w_up, w_down, b_up=None, b_down=None):
+    """Two linear layers, d -> d_ff -> d (App. C: 4 * d * d_ff FLOPs), GELU between them."""
+    hmid = np.asarray(u, F64) @ np.asarray(w_up, F64).T
+    if b_up is not None:
+        hmid = hmid + np.asarray(b_up, F64)
+    out = gelu_tanh(hmid) @ np.asarray(w_down, F64).T
+    if b_down is not None:
+        out = out + np.asarray(b_down, F64)
+    return out
+
+
+def diffusion_block(x, tau, layer: dict, *, ln_eps: float = 1e-5, ssm_state_in=None, conv_state_in=None,
+                    return_state: bool = False, **kw):
+    """y_mixer = x + g1 * Mamba(AdaLN(x; tau)),  y_mlp = y_mixer + g2 * MLP(AdaLN(y_mixer; tau))  (App. A.1;
+    g1 = g2 = 1 gives the equations exactly as printed)."""
+    x = np.asarray(x, F64)
+    b1, s1, g1, b2, s2, g2 = modulation(tau, layer["w_cond"], layer.get("b_cond"))
+    u = adaln(x, s1, b1, ln_eps)
+    if return_state or ssm_state_in is not None or conv_state_in is not None:
+        m, s_out, c_out = bimamba_block_step(u, layer["fwd"], layer["rev"], ssm_state_in=ssm_state_in,
+                                             conv_state_in=conv_state_in, **kw)
+    else:
+        m, s_out, c_out = bimamba_forward(u, layer["fwd"], layer["rev"], **kw), None, None
+    y = x + g1[:, None, :] * m
+    y = y + g2[:, None, :] * mlp(adaln(y, s2, b2, ln_eps), layer["w_up"], layer["w_down"], layer.get("b_up"), layer.get("b_down"))
+    return (y, s_out, c_out) if return_state else y
+
+
+def denoise_step_cond(tokens, tau, sw: dict, *, rms_eps: float = 1e-5, ln_eps: float = 1e-5, states_in=None,
+                      return_states: bool = False, **kw):
+    """z = OutputProj(B_N(... B_1(E(x_t), tau_t) ...))  (App. A.1), OutputProj = final RMSNorm + unembedding
+    (App. C).  tau: [B, d_c], the timestep embedding of each sequence."""
+    r = np.asarray(sw["embed"], F64)[np.asarray(tokens)]
+    states_out = []
+    for i, layer in enumerate(sw["layers"]):
+        if states_in is None and not return_states:
+            r = diffusion_block(r, tau, layer, ln_eps=ln_eps, **kw)
+        else:
+            s_in, c_in = (None, None) if states_in is None or states_in[i] is None else states_in[i]
+            r, s_out, c_out = diffusion_block(r, tau, layer, ln_eps=ln_eps, ssm_state_in=s_in, conv_state_in=c_in,
+                                              return_state=True, **kw)
+            states_out.append((s_out, c_out))
+    logits = rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T
+    return (logits, states_out) if return_states else logits

@@ -159,6 +159,28 @@ def make_stack_weights(shape: MixerShape, n_layers: int, vocab: int, seed: int =
     return sw
 
 
+def add_block_weights(sw: dict, shape: MixerShape, d_ff: int, d_cond: int, seed: int = 0, dtype: str = F32) -> dict:
+    """Adds the timestep-conditioned block's parameters to every layer of `sw` (App. A.1): the modulation
+    map W_cond [6 d, d_c] with its bias (shift rows start at 0, scale and gate rows at 1, so that the block
+    is not degenerate at tau = 0) and the MLP d -> d_ff -> d with biases."""
+    d = shape.d_model
+    for i, layer in enumerate(sw["layers"]):
+        g = lambda name: _rng(seed, f"L{i}.{name}")
+        layer["w_cond"] = _typed(0.02 * g("w_cond").standard_normal((6 * d, d_cond), dtype=np.float32), dtype)
+        base = np.tile(np.repeat(np.array([0.0, 1.0, 1.0], np.float32), d), 2)
+        layer["b_cond"] = (base + 0.1 * g("b_cond").standard_normal((6 * d,), dtype=np.float32)).astype(np.float32)
+        layer["w_up"] = _typed(0.02 * g("w_up").standard_normal((d_ff, d), dtype=np.float32), dtype)
+        layer["b_up"] = (0.02 * g("b_up").standard_normal((d_ff,), dtype=np.float32)).astype(np.float32)
+        layer["w_down"] = _typed(0.02 * g("w_down").standard_normal((d, d_ff), dtype=np.float32), dtype)
+        layer["b_down"] = (0.02 * g("b_down").standard_normal((d,), dtype=np.float32)).astype(np.float32)
+    return sw
+
+
+def make_timestep_embedding(batch: int, d_cond: int, seed: int = 0) -> np.ndarray:
+    """tau_t of each sequence, [B, d_c] fp32 (stands in for the output of the paper's timestep MLP)."""
+    return _rng(seed, "tau").standard_normal((batch, d_cond), dtype=np.float32)
+
+
 # The benchmark configurations (batch, L, d_model, heads, d_state) with their I/O dtype.
 CONFIGS = {
     "cfg0": (MixerShape(1, 256, 128, 2, 16, 4, 8), F32),

@@ -421,3 +421,118 @@ def test_stack_block_mode_matches_prefix_pass_for_forward_direction():
     tail, st2 = O.denoise_step(tok[:, 5:], sw, states_in=st, return_states=True, **kw)
     np.testing.assert_allclose(tail, whole[:, 5:], rtol=1e-10, atol=1e-12)
     assert len(st2) == 2 and st2[0][0].shape == (1, 4, 3, 3)
+
+
+# ------------------------------------------------------------------ timestep-conditioned block (App. A.1)
+
+def _tiny_cond_stack(n_layers=2, d=6, d_ff=12, d_c=5, seed=40):
+    sw = _tiny_stack(n_layers, d=d, seed=seed)
+    r = np.random.default_rng(seed + 100)
+    for layer in sw["layers"]:
+        layer.update(w_cond=r.standard_normal((6 * d, d_c)), b_cond=r.standard_normal(6 * d),
+                     w_up=r.standard_normal((d_ff, d)), b_up=r.standard_normal(d_ff),
+                     w_down=r.standard_normal((d, d_ff)), b_down=r.standard_normal(d))
+    return sw, r.standard_normal((2, d_c))
+
+
+def test_layernorm_standardises_and_adaln_is_affine_in_its_modulation():
+    x = rng.standard_normal((2, 5, 9)) * 3 + 7
+    n = O.layernorm_plain(x, eps=0.0)
+    np.testing.assert_allclose(n.mean(-1), 0, atol=1e-13)
+    np.testing.assert_allclose((n ** 2).mean(-1), 1, rtol=1e-12)
+    np.testing.assert_allclose(O.layernorm_plain(4.0 * x - 11.0, eps=0.0), n, rtol=1e-10, atol=1e-12)   # shift and scale invariant
+    for bb in range(2):                                           # the textbook z-score, element by element
+        for t in range(5):
+            row = x[bb, t]
+            mu = sum(row) / 9
+            sd = (sum((v - mu) ** 2 for v in row) / 9 + 1e-5) ** 0.5
+            np.testing.assert_allclose(O.layernorm_plain(x)[bb, t], [(v - mu) / sd for v in row], rtol=1e-12)
+    g, b = rng.standard_normal((2, 9)), rng.standard_normal((2, 9))
+    np.testing.assert_allclose(O.adaln(x, np.ones((2, 9)), np.zeros((2, 9)), 0.0), n, rtol=1e-13)
+    np.testing.assert_allclose(O.adaln(x, g, b, 0.0), g[:, None] * n + b[:, None], rtol=1e-13)
+    assert np.all(O.adaln(x, g, b)[0, :, 0] != O.adaln(x, g, b)[1, :, 0])      # one modulation per sequence
+
+
+def test_gelu_against_the_exact_form_and_its_symmetry():
+    v = np.linspace(-8, 8, 1601)
+    exact = 0.5 * v * (1 + special.erf(v / np.sqrt(2)))
+    assert np.max(np.abs(O.gelu_tanh(v) - exact)) < 5e-4          # the tanh form's known distance from the erf form
+    np.testing.assert_allclose(O.gelu_tanh(v) - O.gelu_tanh(-v), v, atol=1e-14)   # gelu(x) - gelu(-x) = x
+    assert O.gelu_tanh(0.0) == 0.0 and abs(O.gelu_tanh(30.0) - 30.0) < 1e-12 and abs(O.gelu_tanh(-30.0)) < 1e-12
+
+
+def test_modulation_and_mlp_by_loops():
+    sw, tau = _tiny_cond_stack()
+    L0 = sw["layers"][0]
+    parts = O.modulation(tau, L0["w_cond"], L0["b_cond"])
+    assert len(parts) == 6 and all(p.shape == (2, 6) for p in parts)
+    for k in range(6):
+        for bb in range(2):
+            for j in range(6):
+                want = L0["b_cond"][k * 6 + j] + sum(L0["w_cond"][k * 6 + j, c] * tau[bb, c] for c in range(5))
+                assert parts[k][bb, j] == pytest.approx(want, rel=1e-12, abs=1e-13)
+    np.testing.assert_allclose(np.concatenate(O.modulation(0 * tau, L0["w_cond"], L0["b_cond"]), 1), np.tile(L0["b_cond"], (2, 1)))
+    u = rng.standard_normal((2, 3, 6))
+    got = O.mlp(u, L0["w_up"], L0["w_down"], L0["b_up"], L0["b_down"])
+    for bb in range(2):
+        for t in range(3):
+            hid = [O.gelu_tanh(L0["b_up"][f] + sum(L0["w_up"][f, c] * u[bb, t, c] for c in range(6))) for f in range(12)]
+            for j in range(6):
+                assert got[bb, t, j] == pytest.approx(L0["b_down"][j] + sum(L0["w_down"][j, f] * hid[f] for f in range(12)), rel=1e-11)
+    # FLOP rows "MLP" and "AdaLN" of App. C from the weight shapes a 1.3B layer would have (2mn per linear layer)
+    g = _golden("appC_mamba_layer_flops.txt")
+    d, d_ff, d_c = 1920, 3840, 128
+    assert round((2 * d_ff * d + 2 * d * d_ff) / 1e6, 2) == g["mlp_M"] and round(2 * (6 * d) * d_c / 1e6, 2) == g["adaln_M"]
+
+
+def test_diffusion_block_structure():
+    sw, tau = _tiny_cond_stack()
+    L0 = sw["layers"][0]
+    x = rng.standard_normal((2, 7, 6))
+    d = 6
+    def with_bias(vec):                                           # modulation independent of tau: W_cond = 0, bias = vec
+        return {**L0, "w_cond": 0 * L0["w_cond"], "b_cond": np.asarray(vec, float)}
+    one, zero = np.ones(d), np.zeros(d)
+    # both gates shut: the block is the identity
+    np.testing.assert_array_equal(O.diffusion_block(x, tau, with_bias(np.r_[zero, one, zero, zero, one, zero]), **KW), x)
+    # gamma = 1, beta = 0, gates = 1: the two equations as printed
+    y = O.diffusion_block(x, tau, with_bias(np.r_[zero, one, one, zero, one, one]), **KW)
+    ym = x + O.bimamba_forward(O.layernorm_plain(x), L0["fwd"], L0["rev"], **KW)
+    want = ym + O.mlp(O.layernorm_plain(ym), L0["w_up"], L0["w_down"], L0["b_up"], L0["b_down"])
+    np.testing.assert_allclose(y, want, rtol=1e-11, atol=1e-12)
+    # MLP gate shut: what remains is linear in the mixer gate
+    y1 = O.diffusion_block(x, tau, with_bias(np.r_[zero, one, one, zero, one, zero]), **KW)
+    y3 = O.diffusion_block(x, tau, with_bias(np.r_[zero, one, 3 * one, zero, one, zero]), **KW)
+    np.testing.assert_allclose(y3 - x, 3 * (y1 - x), rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(y1, ym, rtol=1e-11, atol=1e-12)
+    # the general case, assembled from the pinned parts
+    b1, s1, g1, b2, s2, g2 = O.modulation(tau, L0["w_cond"], L0["b_cond"])
+    ym = x + g1[:, None] * O.bimamba_forward(O.adaln(x, s1, b1), L0["fwd"], L0["rev"], **KW)
+    want = ym + g2[:, None] * O.mlp(O.adaln(ym, s2, b2), L0["w_up"], L0["w_down"], L0["b_up"], L0["b_down"])
+    np.testing.assert_allclose(O.diffusion_block(x, tau, L0, **KW), want, rtol=1e-11, atol=1e-12)
+    # sequences do not interact and each sees its own timestep
+    tau2 = tau.copy(); tau2[1] += 1.0
+    ya, yb = O.diffusion_block(x, tau, L0, **KW), O.diffusion_block(x, tau2, L0, **KW)
+    np.testing.assert_array_equal(ya[0], yb[0]); assert np.any(ya[1] != yb[1])
+
+
+def test_conditioned_stack_and_its_block_mode():
+    sw, tau = _tiny_cond_stack()
+    tok = rng.integers(0, 11, (2, 8))
+    logits = O.denoise_step_cond(tok, tau, sw, **KW)
+    r = sw["embed"][tok]
+    for layer in sw["layers"]:
+        r = O.diffusion_block(r, tau, layer, **KW)
+    np.testing.assert_allclose(logits, O.rmsnorm(r, sw["final_norm_w"]) @ sw["w_vocab"].T, rtol=1e-12)
+    # all gates shut: a table lookup followed by the head
+    shut = {**sw, "layers": [{**l, "w_cond": 0 * l["w_cond"], "b_cond": 0 * l["b_cond"]} for l in sw["layers"]]}
+    e = sw["embed"][tok]
+    head = e / np.sqrt(np.mean(e ** 2, -1, keepdims=True) + 1e-5) * sw["final_norm_w"] @ sw["w_vocab"].T
+    np.testing.assert_allclose(O.denoise_step_cond(tok, tau, shut, **KW), head, rtol=1e-12)
+    # block mode, left-to-right direction only: two blocks through the carried state == one pass (Sec. 4.3);
+    # the AdaLN statistics are per token, so they do not couple the blocks
+    kw = dict(KW, dir_mask=O.DIR_FWD)
+    whole = O.denoise_step_cond(tok, tau, sw, **kw)
+    l1, st = O.denoise_step_cond(tok[:, :5], tau, sw, return_states=True, **kw)
+    l2, _ = O.denoise_step_cond(tok[:, 5:], tau, sw, states_in=st, return_states=True, **kw)
+    np.testing.assert_allclose(np.concatenate([l1, l2], 1), whole, rtol=1e-9, atol=1e-11)
