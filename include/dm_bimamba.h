@@ -96,6 +96,29 @@ typedef struct {
     const void             *w_vocab;       /* [vocab, d_model] dtype */
 } dm_stack_weights;
 
+/* The timestep-conditioned block of App. A.1 around the mixer (used by dm_denoise_step_cond):
+ *     y_mixer = x + g1 * Mamba(AdaLN1(x; tau)),     y_mlp = y_mixer + g2 * MLP(AdaLN2(y_mixer; tau)),
+ *     AdaLN(x; tau) = gamma * (x - mean(x)) / sqrt(var(x) + ln_eps) + beta   over the channels of each token,
+ *     [beta1 | gamma1 | g1 | beta2 | gamma2 | g2] = W_cond tau + b_cond      (6 * d_model values per sequence),
+ *     MLP(u) = W_down GELU(W_up u + b_up) + b_down   (GELU in its tanh form).
+ * The paper's equations show gamma and beta only; its FLOP table counts 6 * d_model modulation outputs
+ * per layer, read here as a third vector per sublayer that gates the sublayer's output (g = 1 gives the
+ * equations as printed). */
+typedef struct {
+    int32_t d_ff;      /* hidden width of the MLP (the paper: 2 * d_model) */
+    int32_t d_cond;    /* width of the timestep embedding tau (the paper: 128) */
+    float   ln_eps;
+} dm_block_cfg;
+
+typedef struct {
+    const void  *w_cond;   /* [6 * d_model, d_cond] dtype */
+    const float *b_cond;   /* [6 * d_model] fp32 or NULL */
+    const void  *w_up;     /* [d_ff, d_model] dtype */
+    const float *b_up;     /* [d_ff] fp32 or NULL */
+    const void  *w_down;   /* [d_model, d_ff] dtype */
+    const float *b_down;   /* [d_model] fp32 or NULL */
+} dm_block_weights;
+
 /* Carried state of one layer in block mode (Sec. 4.3): only the left-to-right direction has one.
  * *_in == NULL means zeros (no prefix yet); *_out == NULL means "do not commit".  in and out must not
  * be the same buffer. */
@@ -154,6 +177,18 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights,
                     const int32_t *tokens, void *logits, int32_t *argmax_out,
                     const dm_layer_state *states,
                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* dm_denoise_step with the timestep-conditioned block of App. A.1 in every layer (see dm_block_cfg):
+ *     r_0 = E[tokens];  r_{l+1} = Block_l(r_l, tau);  logits = W_vocab RMSNorm(r_N) * final_norm_w.
+ * block_weights: HOST array of cfg->n_layers entries (device pointers inside); weights->layers[l].norm_w
+ * is not used.  tau: [B, d_cond] fp32 on the device, the timestep embedding of each sequence (the output
+ * of the paper's timestep MLP, computed by the caller).  Everything else as in dm_denoise_step, block
+ * mode included; the workspace size comes from dm_denoise_cond_workspace_bytes. */
+int dm_denoise_cond_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes);
+int dm_denoise_step_cond(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights,
+                         const dm_block_weights *block_weights, const int32_t *tokens, const float *tau,
+                         void *logits, int32_t *argmax_out, const dm_layer_state *states,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* One dense projection as the mixer uses it (App. C counts 2mn FLOPs per token for a weight W in R^{m x n}):
  *     y[r, :] = row_scale[r] * (W x[r, :]) + addend[r, :]

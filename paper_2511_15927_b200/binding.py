@@ -47,6 +47,14 @@ class dm_layer_state(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("ssm_in", "conv_in", "ssm_out", "conv_out")]
 
 
+class dm_block_cfg(C.Structure):
+    _fields_ = [("d_ff", C.c_int32), ("d_cond", C.c_int32), ("ln_eps", C.c_float)]
+
+
+class dm_block_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_cond", "b_cond", "w_up", "b_up", "w_down", "b_down")]
+
+
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2511_15927_b200.build` "
                       "(or __graft_entry__.build()); there is no fallback path")
@@ -70,6 +78,11 @@ _lib.dm_bimamba_block_step.argtypes = [C.POINTER(dm_mixer_cfg), C.POINTER(dm_dir
                                        _vp, _sz, _vp]
 _lib.dm_denoise_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_stack_weights), _vp, _vp, _vp,
                                  C.POINTER(dm_layer_state), _vp, _sz, _vp]
+_lib.dm_denoise_cond_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(_sz)]
+_lib.dm_denoise_cond_workspace_bytes.restype = C.c_int
+_lib.dm_denoise_step_cond.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_stack_weights),
+                                      C.POINTER(dm_block_weights), _vp, _vp, _vp, _vp, C.POINTER(dm_layer_state), _vp, _sz, _vp]
+_lib.dm_denoise_step_cond.restype = C.c_int
 _lib.dm_linear.argtypes = [C.c_int, _vp, _vp, _vp, C.c_int, C.c_int64, C.c_int32, C.c_int32, _vp, _vp, _vp]
 _lib.dm_linear.restype = C.c_int
 _lib.dm_profile_enable.argtypes = [C.c_int]
@@ -80,7 +93,8 @@ for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes",
 
 EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
-           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static")
+           "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
+           "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -177,6 +191,20 @@ def dm_denoise_step(cfg, weights, tokens: int, logits: int, argmax_out: int, sta
                              states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
 
 
+def dm_denoise_cond_workspace_bytes(cfg: dm_stack_cfg, blk: dm_block_cfg) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_denoise_cond_workspace_bytes(C.byref(cfg), C.byref(blk), C.byref(n)))
+    return n.value
+
+
+def dm_denoise_step_cond(cfg, blk, weights, block_weights, tokens: int, tau: int, logits: int, argmax_out: int, states,
+                         workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    """`block_weights`: ctypes array (dm_block_weights * n_layers); `states`: None or (dm_layer_state * n_layers)."""
+    _ok(_lib.dm_denoise_step_cond(C.byref(cfg), C.byref(blk), C.byref(weights), block_weights, _vp(tokens), _vp(tau),
+                                  _vp(logits or None), _vp(argmax_out or None), states, _vp(workspace), _sz(workspace_bytes),
+                                  _vp(cuda_stream)))
+
+
 # ------------------------------------------------------------------------------------------------
 # Marshalling helpers (no arithmetic): build the C structs from shapes and from dicts of tensors.
 # ------------------------------------------------------------------------------------------------
@@ -205,3 +233,13 @@ def make_stack_weights(t: dict):
     sw = dm_stack_weights(t["embed"].data_ptr(), C.cast(arr, C.POINTER(dm_layer_weights)), t["final_norm_w"].data_ptr(),
                           t["w_vocab"].data_ptr())
     return sw, arr
+
+
+def make_block_weights(layers):
+    """layers: list of {"w_cond", "b_cond", "w_up", "b_up", "w_down", "b_down"} of device tensors (biases may be None).
+    Returns the ctypes array (dm_block_weights * n_layers)."""
+    arr = (dm_block_weights * len(layers))()
+    for i, l in enumerate(layers):
+        arr[i] = dm_block_weights(*[(l[n].data_ptr() if l.get(n) is not None else None)
+                                    for n in ("w_cond", "b_cond", "w_up", "b_up", "w_down", "b_down")])
+    return arr

@@ -145,6 +145,7 @@ static cudaError_t gemm(const GemmArgs &a, cudaStream_t s) {
 
 struct MixerOut {
     void *y; int y_dtype; const float *addend; int64_t ld_add;
+    const float *col_scale = nullptr; int cs_rows = 0; int64_t ld_cs = 0;   // per-sequence gate on the mixer's output (App. A.1), or NULL
 };
 
 // in_proj -> fused conv/scan/gate -> out_proj of both directions, summed (Sec. 3.2).
@@ -213,6 +214,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         a.in_dtype = c->dtype; a.M = (int)m.T; a.N = m.d; a.K = m.d_inner;
         a.row_scale = norm_on ? rstd + (size_t)dir * m.T : nullptr;
         a.addend = carry; a.ld_add = ld_carry;
+        a.col_scale = out.col_scale; a.cs_rows = out.cs_rows; a.ld_cs = out.ld_cs;   // the gate distributes over the sum of the directions
         if (last) { a.C = out.y; a.ldc = m.d; a.c_dtype = out.y_dtype; }
         else { a.C = ytmp; a.ldc = m.d; a.c_dtype = DM_F32; carry = ytmp; ld_carry = m.d; }
         if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "out_proj");
@@ -228,11 +230,11 @@ static int check_ws(const void *ws, size_t have, size_t need) {
 }
 
 struct StackWs {
-    size_t r, u, logits, mixer, total;
+    size_t r, u, logits, mixer, mod, hmid, total;
     int logits_rows;
 };
 
-static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m) {
+static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg *blk = nullptr) {
     StackWs w;
     size_t off = 0;
     w.r = off; off += align_up((size_t)m.T * m.d * sizeof(float));
@@ -240,6 +242,11 @@ static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m) {
     w.logits_rows = (int)(m.T < 2048 ? m.T : 2048);
     w.logits = off; off += align_up((size_t)w.logits_rows * c->vocab * m.es);
     w.mixer = off; off += mixer_ws(&c->mixer, m).total;
+    w.mod = w.hmid = off;
+    if (blk) {
+        w.mod = off; off += align_up((size_t)m.B * 6 * m.d * sizeof(float));
+        w.hmid = off; off += align_up((size_t)m.T * blk->d_ff * m.es);
+    }
     w.total = off;
     return w;
 }
@@ -406,9 +413,14 @@ int dm_bimamba_block_step(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], co
                      static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
 }
 
-int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, const int32_t *tokens, void *logits,
-                    int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
-                    void *cuda_stream) {
+}  // extern "C"
+
+// One denoiser evaluation.  blk == NULL: RMSNorm pre-norm + mixer per layer; otherwise the timestep-conditioned block of
+// App. A.1 (AdaLN -> mixer -> gated residual, AdaLN -> MLP -> gated residual) with the modulation of each layer from tau.
+static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights, const dm_block_weights *bw,
+                        const int32_t *tokens, const float *tau, void *logits,
+                        int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream) {
     Dims m;
     if (!cfg || !weights) return fail(DM_ERR_INVALID_ARG, "cfg or weights is NULL");
     int st = check_cfg(&cfg->mixer, &m);
@@ -422,8 +434,20 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, co
     if (!aligned16(weights->embed) || !aligned16(weights->w_vocab) || !aligned16(logits))
         return fail(DM_ERR_INVALID_ARG, "embed, w_vocab and logits must be 16-byte aligned");
     if (logits && (((size_t)cfg->vocab * m.es) % 16)) return fail(DM_ERR_UNSUPPORTED, "vocab*sizeof(dtype) must be a multiple of 16");
+    if (blk) {
+        if (!bw || !tau) return fail(DM_ERR_INVALID_ARG, "block weights or tau is NULL");
+        if (blk->d_ff <= 0 || blk->d_cond <= 0 || !(blk->ln_eps >= 0.f)) return fail(DM_ERR_INVALID_ARG, "d_ff and d_cond must be positive, ln_eps >= 0");
+        if (m.d % 4) return fail(DM_ERR_UNSUPPORTED, "the conditioned block needs d_model to be a multiple of 4");
+        if (!aligned16(tau)) return fail(DM_ERR_INVALID_ARG, "tau must be 16-byte aligned");
+        for (int i = 0; i < cfg->n_layers; ++i) {
+            const dm_block_weights &q = bw[i];
+            if (!q.w_cond || !q.w_up || !q.w_down) return fail(DM_ERR_INVALID_ARG, "layer %d: NULL pointer in block weights", i);
+            if (!aligned16(q.w_cond) || !aligned16(q.w_up) || !aligned16(q.w_down) || !aligned16(q.b_cond) || !aligned16(q.b_up) || !aligned16(q.b_down))
+                return fail(DM_ERR_INVALID_ARG, "layer %d: block weights must be 16-byte aligned", i);
+        }
+    }
     for (int i = 0; i < cfg->n_layers; ++i) {
-        if (!weights->layers[i].norm_w) return fail(DM_ERR_INVALID_ARG, "layer %d: norm_w is NULL", i);
+        if (!blk && !weights->layers[i].norm_w) return fail(DM_ERR_INVALID_ARG, "layer %d: norm_w is NULL", i);
         if ((st = check_weights(&cfg->mixer, weights->layers[i].dir)) != DM_OK) return st;
         if (states) {
             const dm_layer_state &q = states[i];
@@ -435,10 +459,11 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, co
                 return fail(DM_ERR_INVALID_ARG, "state_out needs the left-to-right direction");
         }
     }
-    const StackWs l = stack_ws(cfg, m);
+    const StackWs l = stack_ws(cfg, m, blk);
     if ((st = check_ws(workspace, workspace_bytes, l.total)) != DM_OK) return st;
     char *ws = static_cast<char *>(workspace);
     float *r = reinterpret_cast<float *>(ws + l.r);
+    float *mod = reinterpret_cast<float *>(ws + l.mod);
     void *u = ws + l.u;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const int dtype = cfg->mixer.dtype;
@@ -447,12 +472,35 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, co
     if ((e = embed_gather(weights->embed, dtype, tokens, r, (int)m.T, m.d, cfg->vocab, s)) != cudaSuccess) return cuda_fail(e, "embed");
     for (int i = 0; i < cfg->n_layers; ++i) {
         const dm_layer_weights &lw = weights->layers[i];
-        if ((e = rmsnorm_rows(r, lw.norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "rmsnorm");
         MixerOut out{r, DM_F32, r, m.d};          // r <- r + Mamba(u): the residual add rides in the out_proj epilogue
+        const int64_t ldm = 6 * (int64_t)m.d;     // modulation row: [beta1 | gamma1 | gate1 | beta2 | gamma2 | gate2]
+        if (blk) {
+            if ((e = modulation_rows(tau, bw[i].w_cond, bw[i].b_cond, mod, dtype, m.B, 6 * m.d, blk->d_cond, s)) != cudaSuccess) return cuda_fail(e, "modulation");
+            if ((e = adaln_rows(r, mod + m.d, mod, ldm, u, dtype, (int)m.T, m.L, m.d, blk->ln_eps, s)) != cudaSuccess) return cuda_fail(e, "adaln");
+            out.col_scale = mod + 2 * m.d; out.cs_rows = m.L; out.ld_cs = ldm;
+        } else {
+            if ((e = rmsnorm_rows(r, lw.norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "rmsnorm");
+        }
         const dm_layer_state *q = states ? &states[i] : nullptr;
         st = run_mixer(&cfg->mixer, m, lw.dir, u, out, q ? q->ssm_in : nullptr, q ? q->conv_in : nullptr,
                        q ? q->ssm_out : nullptr, q ? q->conv_out : nullptr, ws + l.mixer, s);
         if (st != DM_OK) return st;
+        if (blk) {
+            // r <- r + gate2 * (W_down GELU(W_up AdaLN(r) + b_up) + b_down): activation, bias, gate and residual ride in the epilogues
+            if ((e = adaln_rows(r, mod + 4 * m.d, mod + 3 * m.d, ldm, u, dtype, (int)m.T, m.L, m.d, blk->ln_eps, s)) != cudaSuccess) return cuda_fail(e, "adaln");
+            void *hmid = ws + l.hmid;
+            GemmArgs up{};
+            up.A = u; up.lda = m.d; up.B = bw[i].w_up; up.ldb = m.d; up.C = hmid; up.ldc = blk->d_ff;
+            up.in_dtype = dtype; up.c_dtype = dtype; up.M = (int)m.T; up.N = blk->d_ff; up.K = m.d;
+            up.col_bias = bw[i].b_up; up.gelu = 1;
+            if ((e = gemm(up, s)) != cudaSuccess) return cuda_fail(e, "mlp up");
+            GemmArgs dn{};
+            dn.A = hmid; dn.lda = blk->d_ff; dn.B = bw[i].w_down; dn.ldb = blk->d_ff; dn.C = r; dn.ldc = m.d;
+            dn.in_dtype = dtype; dn.c_dtype = DM_F32; dn.M = (int)m.T; dn.N = m.d; dn.K = blk->d_ff;
+            dn.col_bias = bw[i].b_down; dn.col_scale = mod + 5 * m.d; dn.cs_rows = m.L; dn.ld_cs = ldm;
+            dn.addend = r; dn.ld_add = m.d;
+            if ((e = gemm(dn, s)) != cudaSuccess) return cuda_fail(e, "mlp down");
+        }
     }
     if ((e = rmsnorm_rows(r, weights->final_norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "final norm");
     const int64_t rows_per = logits ? m.T : l.logits_rows;
@@ -467,6 +515,32 @@ int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, co
         if (argmax_out && (e = argmax_rows(a.C, dtype, argmax_out + t0, rows, cfg->vocab, s)) != cudaSuccess) return cuda_fail(e, "argmax");
     }
     return DM_OK;
+}
+
+extern "C" {
+
+int dm_denoise_step(const dm_stack_cfg *cfg, const dm_stack_weights *weights, const int32_t *tokens, void *logits,
+                    int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
+                    void *cuda_stream) {
+    return denoise_impl(cfg, nullptr, weights, nullptr, tokens, nullptr, logits, argmax_out, states, workspace, workspace_bytes, cuda_stream);
+}
+
+int dm_denoise_cond_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes) {
+    Dims m;
+    if (!cfg || !blk || !bytes) return fail(DM_ERR_INVALID_ARG, "NULL argument");
+    int st = check_cfg(&cfg->mixer, &m);
+    if (st != DM_OK) return st;
+    if (cfg->vocab <= 0 || blk->d_ff <= 0) return fail(DM_ERR_INVALID_ARG, "vocab and d_ff must be positive");
+    *bytes = stack_ws(cfg, m, blk).total;
+    return DM_OK;
+}
+
+int dm_denoise_step_cond(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights,
+                         const dm_block_weights *block_weights, const int32_t *tokens, const float *tau, void *logits,
+                         int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream) {
+    if (!blk) return fail(DM_ERR_INVALID_ARG, "block configuration is NULL");
+    return denoise_impl(cfg, blk, weights, block_weights, tokens, tau, logits, argmax_out, states, workspace, workspace_bytes, cuda_stream);
 }
 
 int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype, int64_t rows, int32_t in_features,

@@ -32,7 +32,13 @@ struct GemmArgs {
     int M, N, K;
     const float *row_scale;
     const float *addend; int64_t ld_add;
-    int silu_cols;           // output columns [0, silu_cols) get SiLU applied after scale and addend (0 = none)
+    int silu_cols;           // output columns [0, silu_cols) get SiLU applied (0 = none)
+    // Epilogue order: v = acc * row_scale[r] + col_bias[c];  v = act(v);  v *= col_scale[(r / cs_rows) * ld_cs + c];  v += addend[r, c]
+    const float *col_bias;   // [N] or NULL
+    int gelu;                // GELU (tanh form) on every output column
+    const float *col_scale;  // [ceil(M / cs_rows), ld_cs] or NULL: one scale vector per group of cs_rows consecutive rows
+    int cs_rows;
+    int64_t ld_cs;           // row pitch of col_scale (0 = N)
 };
 cudaError_t gemm_simple(const GemmArgs &a, cudaStream_t s);
 // Tensor-core path (tcgen05 + TMEM + TMA).  Returns cudaErrorNotSupported for shapes it does not take.
@@ -73,6 +79,12 @@ cudaError_t rstd_from_ssq(const float *ssq, float *rstd, int rows, int H, int d_
 cudaError_t embed_gather(const void *embed, int dtype, const int32_t *tokens, float *r, int T, int d, int vocab, cudaStream_t s);
 // u[t, :] = r[t, :] * rsqrt(mean(r[t]^2) + eps) * w
 cudaError_t rmsnorm_rows(const float *r, const void *w, void *u, int dtype, int T, int d, float eps, cudaStream_t s);
+// u[t, :] = gamma[t / L, :] * (r[t, :] - mean) / sqrt(var + eps) + beta[t / L, :]   (gamma, beta: rows of pitch ld_mod)
+cudaError_t adaln_rows(const float *r, const float *gamma, const float *beta, int64_t ld_mod, void *u, int dtype, int T, int L, int d,
+                       float eps, cudaStream_t s);
+// mod[b, :] = b_cond + W_cond tau[b, :]   (W_cond [n_out, d_c] dtype, b_cond [n_out] fp32 or NULL, tau [B, d_c] fp32)
+cudaError_t modulation_rows(const float *tau, const void *w_cond, const float *b_cond, float *mod, int dtype, int B, int n_out, int d_c,
+                            cudaStream_t s);
 // out[t] = argmax_v logits[t, v], lowest index on ties
 cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s);
 // conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])

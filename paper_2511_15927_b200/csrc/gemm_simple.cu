@@ -15,7 +15,8 @@ template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(256)
 gemm_simple_kernel(const TIn *__restrict__ A, int64_t lda, const TIn *__restrict__ B, int64_t ldb,
                    TOut *C, int64_t ldc, int M, int N, int K,
-                   const float *__restrict__ row_scale, const float *addend, int64_t ld_add, int silu_cols) {
+                   const float *__restrict__ row_scale, const float *addend, int64_t ld_add, int silu_cols,
+                   const float *__restrict__ col_bias, int gelu, const float *__restrict__ col_scale, int cs_rows, int64_t ld_cs) {
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -56,8 +57,11 @@ gemm_simple_kernel(const TIn *__restrict__ A, int64_t lda, const TIn *__restrict
             const int gn = n0 + tx * TN + j;
             if (gn >= N) continue;
             float v = acc[i][j] * sc;
-            if (addend) v += addend[(int64_t)gm * ld_add + gn];
+            if (col_bias) v += col_bias[gn];
             if (gn < silu_cols) v = v / (1.f + __expf(-v));
+            if (gelu) v = 0.5f * v * (1.f + tanhf(0.7978845608028654f * (v + 0.044715f * v * v * v)));
+            if (col_scale) v *= col_scale[(int64_t)(gm / cs_rows) * ld_cs + gn];
+            if (addend) v += addend[(int64_t)gm * ld_add + gn];
             if constexpr (sizeof(TOut) == 4) C[(int64_t)gm * ldc + gn] = v;
             else C[(int64_t)gm * ldc + gn] = __float2bfloat16_rn(v);
         }
@@ -69,7 +73,8 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM);
     gemm_simple_kernel<TIn, TOut><<<grid, 256, 0, s>>>(
         static_cast<const TIn *>(a.A), a.lda, static_cast<const TIn *>(a.B), a.ldb,
-        static_cast<TOut *>(a.C), a.ldc, a.M, a.N, a.K, a.row_scale, a.addend, a.ld_add, a.silu_cols);
+        static_cast<TOut *>(a.C), a.ldc, a.M, a.N, a.K, a.row_scale, a.addend, a.ld_add, a.silu_cols,
+        a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : a.N);
     count_launch();
     return cudaGetLastError();
 }

@@ -31,6 +31,7 @@ struct EpiArgs {
     const float *row_scale; const float *addend; int64_t ld_add;
     int M, N, K;
     int silu_cols;   // SiLU on output columns below this one
+    const float *col_bias; int gelu; const float *col_scale; int cs_rows; int64_t ld_cs;   // see GemmArgs
     int n_fast;      // tile order: consecutive tiles step along N (the A rows are streamed once, B stays in L2) or along M
 };
 
@@ -144,6 +145,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * sc;
                 const bool full = col + 32 <= ep.N;
+                if (ep.col_bias) {
+                    if (full) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 b4 = *reinterpret_cast<const float4 *>(ep.col_bias + col + j);
+                            v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+                        }
+                    } else {
+                        for (int j = 0; j < 32; ++j) if (col + j < ep.N) v[j] += ep.col_bias[col + j];
+                    }
+                }
+                if (col < ep.silu_cols) {                  // gate columns: SiLU here, where the ALUs idle, not in the scan
+                    if (col + 32 <= ep.silu_cols) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) { const float hv = 0.5f * v[j]; v[j] = fmaf(hv, tanh_fast(hv), hv); }   // SiLU(v) = v/2 + v/2 tanh(v/2)
+                    } else {
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < ep.silu_cols) { const float hv = 0.5f * v[j]; v[j] = fmaf(hv, tanh_fast(hv), hv); }
+                    }
+                }
+                if (ep.gelu) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {                  // GELU, tanh form
+                        const float x = v[j], hx = 0.5f * x;
+                        v[j] = fmaf(hx, tanh_fast(0.7978845608028654f * fmaf(0.044715f * x, x * x, x)), hx);
+                    }
+                }
+                if (ep.col_scale) {
+                    const float *cs = ep.col_scale + (int64_t)(row / ep.cs_rows) * ep.ld_cs + col;
+                    if (full) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 c4 = *reinterpret_cast<const float4 *>(cs + j);
+                            v[j] *= c4.x; v[j + 1] *= c4.y; v[j + 2] *= c4.z; v[j + 3] *= c4.w;
+                        }
+                    } else {
+                        for (int j = 0; j < 32; ++j) if (col + j < ep.N) v[j] *= cs[j];
+                    }
+                }
                 if (add_row) {
                     if (full && wide_add) {
 #pragma unroll
@@ -161,15 +201,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     } else {
                         for (int j = 0; j < 32; ++j) if (col + j < ep.N) v[j] += add_row[col + j];
-                    }
-                }
-                if (col < ep.silu_cols) {                  // gate columns: SiLU here, where the ALUs idle, not in the scan
-                    if (col + 32 <= ep.silu_cols) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) { const float hv = 0.5f * v[j]; v[j] = fmaf(hv, tanh_fast(hv), hv); }   // SiLU(v) = v/2 + v/2 tanh(v/2)
-                    } else {
-                        for (int j = 0; j < 32; ++j)
-                            if (col + j < ep.silu_cols) { const float hv = 0.5f * v[j]; v[j] = fmaf(hv, tanh_fast(hv), hv); }
                     }
                 }
                 if (ep.c_is_f32) {
@@ -242,7 +273,8 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
     const int grid = tiles < sm_count() ? tiles : sm_count();
     // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
-    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols, a.M > a.N ? 1 : 0};
+    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols,
+               a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.M > a.N ? 1 : 0};
     gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma, mb, ep, status);
     count_launch();
     return cudaGetLastError();
@@ -257,6 +289,8 @@ bool gemm_tcgen05_supports(const GemmArgs &a) {
     if ((reinterpret_cast<uintptr_t>(a.A) & 15u) || (reinterpret_cast<uintptr_t>(a.B) & 15u)) return false;
     if (a.c_dtype == DM_BF16 ? (reinterpret_cast<uintptr_t>(a.C) & 15u) : (reinterpret_cast<uintptr_t>(a.C) & 15u)) return false;
     if (a.addend && (reinterpret_cast<uintptr_t>(a.addend) & 15u)) return false;
+    if (a.col_bias && (reinterpret_cast<uintptr_t>(a.col_bias) & 15u)) return false;
+    if (a.col_scale && ((reinterpret_cast<uintptr_t>(a.col_scale) & 15u) || ((a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N) & 3))) return false;
     return encode_fn() != nullptr;
 }
 

@@ -50,6 +50,37 @@ __global__ void rmsnorm_kernel(const float *__restrict__ r, const T *__restrict_
     for (int c = threadIdx.x; c < d; c += blockDim.x) stf(u + t * d + c, r[t * d + c] * rs * ldf(w + c));
 }
 
+// u[t, :] = gamma[b, :] * (r[t, :] - mean) / sqrt(var + eps) + beta[b, :], b = t / L  (App. A.1, Eq. "AdaLN");
+// gamma and beta are rows of the per-sequence modulation table (row pitch ld_mod).
+template <typename T>
+__global__ void adaln_kernel(const float *__restrict__ r, const float *__restrict__ gamma, const float *__restrict__ beta, int64_t ld_mod,
+                             T *__restrict__ u, int L, int d, float eps) {
+    __shared__ float red[32];
+    const int64_t t = blockIdx.x, b = t / L;
+    float s = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) s += r[t * d + c];
+    const float mu = block_sum(s, red) / (float)d;
+    __syncthreads();
+    float q = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = r[t * d + c] - mu; q = fmaf(v, v, q); }
+    const float rs = rsqrtf(block_sum(q, red) / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x)
+        stf(u + t * d + c, fmaf(gamma[b * ld_mod + c], (r[t * d + c] - mu) * rs, beta[b * ld_mod + c]));
+}
+
+// mod[b, j] = bias[j] + sum_c w[j, c] tau[b, c]: the modulation vectors of one layer (App. A.1: (gamma, beta) = W_cond tau).
+// One warp per output element.
+template <typename T>
+__global__ void modulation_kernel(const float *__restrict__ tau, const T *__restrict__ w, const float *__restrict__ bias,
+                                  float *__restrict__ mod, int n_out, int d_c) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31, b = blockIdx.y;
+    if (warp >= n_out) return;
+    float s = 0.f;
+    for (int c = lane; c < d_c; c += 32) s = fmaf(ldf(w + (int64_t)warp * d_c + c), tau[(int64_t)b * d_c + c], s);
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0) mod[(int64_t)b * n_out + warp] = s + (bias ? bias[warp] : 0.f);
+}
+
 template <typename T>
 __global__ void argmax_kernel(const T *__restrict__ logits, int32_t *__restrict__ out, int V) {
     __shared__ float bv[32];
@@ -114,6 +145,23 @@ cudaError_t embed_gather(const void *embed, int dtype, const int32_t *tokens, fl
 cudaError_t rmsnorm_rows(const float *r, const void *w, void *u, int dtype, int T, int d, float eps, cudaStream_t s) {
     if (dtype == DM_BF16) rmsnorm_kernel<<<T, 256, 0, s>>>(r, static_cast<const __nv_bfloat16 *>(w), static_cast<__nv_bfloat16 *>(u), d, eps);
     else rmsnorm_kernel<<<T, 256, 0, s>>>(r, static_cast<const float *>(w), static_cast<float *>(u), d, eps);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t adaln_rows(const float *r, const float *gamma, const float *beta, int64_t ld_mod, void *u, int dtype, int T, int L, int d,
+                       float eps, cudaStream_t s) {
+    if (dtype == DM_BF16) adaln_kernel<<<T, 256, 0, s>>>(r, gamma, beta, ld_mod, static_cast<__nv_bfloat16 *>(u), L, d, eps);
+    else adaln_kernel<<<T, 256, 0, s>>>(r, gamma, beta, ld_mod, static_cast<float *>(u), L, d, eps);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t modulation_rows(const float *tau, const void *w_cond, const float *b_cond, float *mod, int dtype, int B, int n_out, int d_c,
+                            cudaStream_t s) {
+    dim3 grid((n_out * 32 + 255) / 256, B);
+    if (dtype == DM_BF16) modulation_kernel<<<grid, 256, 0, s>>>(tau, static_cast<const __nv_bfloat16 *>(w_cond), b_cond, mod, n_out, d_c);
+    else modulation_kernel<<<grid, 256, 0, s>>>(tau, static_cast<const float *>(w_cond), b_cond, mod, n_out, d_c);
     count_launch();
     return cudaGetLastError();
 }

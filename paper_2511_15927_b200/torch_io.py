@@ -46,3 +46,11 @@ def dev_stack_weights(sw: dict, dtype) -> dict:
                         "rev": dev_dir_weights(l["rev"], dtype)} for l in sw["layers"]]}
 
 
+def dev_block_weights(sw: dict, dtype) -> list:
+    """The timestep-conditioned block's parameters of every layer: matrices in the I/O dtype, biases in fp32."""
+    f32 = lambda a: None if a is None else dev(np.asarray(a, np.float32))
+    return [{"w_cond": dev(l["w_cond"], dtype), "b_cond": f32(l.get("b_cond")), "w_up": dev(l["w_up"], dtype),
+             "b_up": f32(l.get("b_up")), "w_down": dev(l["w_down"], dtype), "b_down": f32(l.get("b_down"))}
+            for l in sw["layers"]]
+
+

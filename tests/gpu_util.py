@@ -7,8 +7,8 @@ import torch
 
 from paper_2511_15927_b200 import binding as dm
 from paper_2511_15927_b200 import inputs as I
-from paper_2511_15927_b200.torch_io import (cfg_of, dev, dev_dir_weights, dev_stack_weights, dm_dtype, tdtype,  # noqa: F401
-                                            workspace)
+from paper_2511_15927_b200.torch_io import (cfg_of, dev, dev_block_weights, dev_dir_weights, dev_stack_weights, dm_dtype,  # noqa: F401
+                                            tdtype, workspace)
 
 
 def run_forward(shape, dtype, wf, wr, x, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, chunk=0):
@@ -65,7 +65,8 @@ def run_block_step(shape, dtype, wf, wr, x_blk, ssm_in=None, conv_in=None, want_
 
 
 def run_denoise(shape, dtype, sw, tokens, vocab, want_logits=True, want_argmax=True, states_in=None, want_states=False,
-                flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, rms_eps=1e-5):
+                flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, rms_eps=1e-5, tau=None, d_ff=0, ln_eps=1e-5):
+    """tau given: the timestep-conditioned stack (dm_denoise_step_cond), whose block weights are in sw's layers."""
     n_layers = len(sw["layers"])
     scfg = dm.dm_stack_cfg(cfg_of(shape, dtype, flags, dir_mask), n_layers, vocab, rms_eps)
     dsw = dev_stack_weights(sw, dtype)
@@ -87,11 +88,21 @@ def run_denoise(shape, dtype, sw, tokens, vocab, want_logits=True, want_argmax=T
             bufs.append((s_in, c_in, s_out, c_out))
             p = lambda t: t.data_ptr() if t is not None else None
             states[i] = dm.dm_layer_state(p(s_in), p(c_in), p(s_out), p(c_out))
-    nb = dm.dm_denoise_workspace_bytes(scfg)
-    ws = workspace(nb)
     st = torch.cuda.current_stream().cuda_stream
-    dm.dm_denoise_step(scfg, csw, tok.data_ptr(), logits.data_ptr() if want_logits else 0,
-                       amax.data_ptr() if want_argmax else 0, states, ws.data_ptr(), nb, st)
+    if tau is None:
+        nb = dm.dm_denoise_workspace_bytes(scfg)
+        ws = workspace(nb)
+        dm.dm_denoise_step(scfg, csw, tok.data_ptr(), logits.data_ptr() if want_logits else 0,
+                           amax.data_ptr() if want_argmax else 0, states, ws.data_ptr(), nb, st)
+    else:
+        blk = dm.dm_block_cfg(d_ff, tau.shape[1], ln_eps)
+        dbw = dev_block_weights(sw, dtype)
+        cbw = dm.make_block_weights(dbw)
+        taud = dev(np.asarray(tau, np.float32))
+        nb = dm.dm_denoise_cond_workspace_bytes(scfg, blk)
+        ws = workspace(nb)
+        dm.dm_denoise_step_cond(scfg, blk, csw, cbw, tok.data_ptr(), taud.data_ptr(), logits.data_ptr() if want_logits else 0,
+                                amax.data_ptr() if want_argmax else 0, states, ws.data_ptr(), nb, st)
     dm.dm_check(st)
     f = lambda t: None if t is None else t.float().cpu().numpy().astype(np.float64)
     out_states = [(f(b[2]), f(b[3])) for b in bufs] if want_states else None
