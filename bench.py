@@ -165,10 +165,12 @@ STACKS = {
     "cfg2_stack": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304),
     "cfg2_stack_n128": dict(shape=I.MixerShape(4, 4096, 1024, 2, 128, 4, 32), layers=24, vocab=50304),
     "cfg4_decode": dict(shape=I.MixerShape(16, 32, 2048, 2, 128, 4, 64), layers=24, vocab=50304, prefix=2048),
+    # the same stack with the timestep-conditioned block of App. A.1 in every layer (AdaLN, mixer, AdaLN, MLP with d_ff = 2 d)
+    "cfg2_stack_cond": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, cond=dict(d_ff=2048, d_cond=128)),
 }
 
 
-def device_stack_weights(torch, shape, layers, vocab, seed=0):
+def device_stack_weights(torch, shape, layers, vocab, seed=0, cond=None):
     """Random-init bf16 weights of a stack, drawn on the device with the distributions of inputs.py (the host
     generator would take minutes at these sizes).  Returns the dict layout make_stack_weights() of the binding takes."""
     g = torch.Generator(device="cuda").manual_seed(seed)
@@ -188,15 +190,25 @@ def device_stack_weights(torch, shape, layers, vocab, seed=0):
                 "dt_bias": dt + torch.log(-torch.expm1(-dt)), "D": torch.ones(s.n_heads, device="cuda"),
                 "norm_w": torch.ones(s.d_inner, device="cuda", dtype=bf), "w_out": normal(s.d_model, s.d_inner)}
 
-    return {"embed": normal(vocab, s.d_model), "w_vocab": normal(vocab, s.d_model),
-            "final_norm_w": torch.ones(s.d_model, device="cuda", dtype=bf),
-            "layers": [{"norm_w": torch.ones(s.d_model, device="cuda", dtype=bf), "fwd": direction(), "rev": direction()}
-                       for _ in range(layers)]}
+    def block():
+        d, d_ff, d_c = s.d_model, cond["d_ff"], cond["d_cond"]
+        base = torch.tensor([0.0, 1.0, 1.0], device="cuda").repeat_interleave(d).repeat(2)      # shift 0, scale 1, gate 1
+        return {"w_cond": normal(6 * d, d_c), "b_cond": base + 0.1 * torch.randn(6 * d, generator=g, device="cuda"),
+                "w_up": normal(d_ff, d), "b_up": 0.02 * torch.randn(d_ff, generator=g, device="cuda"),
+                "w_down": normal(d, d_ff), "b_down": 0.02 * torch.randn(d, generator=g, device="cuda")}
+
+    out = {"embed": normal(vocab, s.d_model), "w_vocab": normal(vocab, s.d_model),
+           "final_norm_w": torch.ones(s.d_model, device="cuda", dtype=bf),
+           "layers": [{"norm_w": torch.ones(s.d_model, device="cuda", dtype=bf), "fwd": direction(), "rev": direction()}
+                      for _ in range(layers)]}
+    if cond:
+        out["blocks"] = [block() for _ in range(layers)]
+    return out
 
 
 def run_stack(args, rank, local_rank, world):
     """One step = one dm_denoise_step (embedding, 24 x (RMSNorm, mixer, residual), final norm, vocabulary projection,
-    arg-max).  cfg4_decode: the step covers the 32-token active block of every sequence, starting from the carried
+    arg-max); cfg2_stack_cond: one dm_denoise_step_cond (24 x the timestep-conditioned block instead).  cfg4_decode: the step covers the 32-token active block of every sequence, starting from the carried
     state of a committed 2048-token prefix; the same stack's full re-encode of prefix + block is timed beside it."""
     import torch
     from paper_2511_15927_b200 import build
@@ -210,9 +222,23 @@ def run_stack(args, rank, local_rank, world):
     spec = STACKS[args.workload]
     shape, layers, vocab, prefix = spec["shape"], spec["layers"], spec["vocab"], spec.get("prefix")
     B, Lb = shape.batch, shape.seqlen
-    w = device_stack_weights(torch, shape, layers, vocab)
+    cond = spec.get("cond")
+    w = device_stack_weights(torch, shape, layers, vocab, cond=cond)
     csw, keep = dm.make_stack_weights(w)
     stream = torch.cuda.current_stream().cuda_stream
+    if cond:
+        blk = dm.dm_block_cfg(cond["d_ff"], cond["d_cond"], 1e-5)
+        cbw = dm.make_block_weights(w["blocks"])
+        tau = torch.from_numpy(I.make_timestep_embedding(B, cond["d_cond"], seed=0)).cuda()
+
+    def ws_bytes(cfg):
+        return dm.dm_denoise_cond_workspace_bytes(cfg, blk) if cond else dm.dm_denoise_workspace_bytes(cfg)
+
+    def denoise(cfg, tok_ptr, amax_ptr, st):
+        if cond:
+            dm.dm_denoise_step_cond(cfg, blk, csw, cbw, tok_ptr, tau.data_ptr(), 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
+        else:
+            dm.dm_denoise_step(cfg, csw, tok_ptr, 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
 
     def stack_cfg(L):
         sh = I.MixerShape(B, L, shape.d_model, shape.expand, shape.d_state, shape.d_conv, shape.n_heads)
@@ -222,14 +248,14 @@ def run_stack(args, rank, local_rank, world):
         return [torch.from_numpy(I.make_tokens(B, L, 50257, 50257, seed=i)).cuda() for i in range(n)]
 
     scfg = stack_cfg(Lb)
-    nb = dm.dm_denoise_workspace_bytes(scfg)
+    nb = ws_bytes(scfg)
     states = None
     extra = {}
     if prefix:
         # commit the prefix once (block step over the prefix, NULL state in), then time steps over the active block
         pcfg = stack_cfg(prefix)
-        nbp = dm.dm_denoise_workspace_bytes(pcfg)
-        ws = G.workspace(max(nb, nbp, dm.dm_denoise_workspace_bytes(stack_cfg(prefix + Lb))))
+        nbp = ws_bytes(pcfg)
+        ws = G.workspace(max(nb, nbp, ws_bytes(stack_cfg(prefix + Lb))))
         st_bufs = [(torch.empty((B, shape.n_heads, shape.headdim, shape.d_state), device="cuda"),
                     torch.empty((B, shape.d_conv - 1, shape.conv_ch), device="cuda", dtype=torch.bfloat16)) for _ in range(layers)]
         pst = (dm.dm_layer_state * layers)()
@@ -237,7 +263,7 @@ def run_stack(args, rank, local_rank, world):
             pst[i] = dm.dm_layer_state(None, None, sb.data_ptr(), cb.data_ptr())
         ptok = tokens(prefix, 1)[0]
         amax_p = torch.empty((B, prefix), device="cuda", dtype=torch.int32)
-        dm.dm_denoise_step(pcfg, csw, ptok.data_ptr(), 0, amax_p.data_ptr(), pst, ws.data_ptr(), ws.numel(), stream)
+        denoise(pcfg, ptok.data_ptr(), amax_p.data_ptr(), pst)
         dm.dm_check(stream)
         states = (dm.dm_layer_state * layers)()
         for i, (sb, cb) in enumerate(st_bufs):
@@ -248,7 +274,7 @@ def run_stack(args, rank, local_rank, world):
     amax = torch.empty((B, Lb), device="cuda", dtype=torch.int32)
 
     def step(i):
-        dm.dm_denoise_step(scfg, csw, toks[i % 4].data_ptr(), 0, amax.data_ptr(), states, ws.data_ptr(), ws.numel(), stream)
+        denoise(scfg, toks[i % 4].data_ptr(), amax.data_ptr(), states)
 
     def timed(fn, n):
         for i in range(args.warmup):
@@ -282,8 +308,7 @@ def run_stack(args, rank, local_rank, world):
         fcfg = stack_cfg(prefix + Lb)
         ftok = tokens(prefix + Lb, 2)
         famax = torch.empty((B, prefix + Lb), device="cuda", dtype=torch.int32)
-        ms_full = timed(lambda i: dm.dm_denoise_step(fcfg, csw, ftok[i % 2].data_ptr(), 0, famax.data_ptr(), None, ws.data_ptr(),
-                                                      ws.numel(), stream), max(2, args.steps // 4)) / max(2, args.steps // 4)
+        ms_full = timed(lambda i: denoise(fcfg, ftok[i % 2].data_ptr(), famax.data_ptr(), None), max(2, args.steps // 4)) / max(2, args.steps // 4)
         extra = {"prefix": prefix, "full_reencode_ms_per_step": ms_full, "state_carry_speedup": ms_full / ms_step}
     # end to end: token ids from pinned host memory in, arg-max ids back, inside the timed region
     e2e = None
@@ -294,7 +319,7 @@ def run_stack(args, rank, local_rank, world):
 
         def host_step(i):
             td.copy_(th, non_blocking=True)
-            dm.dm_denoise_step(scfg, csw, td.data_ptr(), 0, amax.data_ptr(), states, ws.data_ptr(), ws.numel(), stream)
+            denoise(scfg, td.data_ptr(), amax.data_ptr(), states)
             ah.copy_(amax, non_blocking=True)
             torch.cuda.synchronize()
         for i in range(2):
@@ -333,7 +358,7 @@ def run_stack(args, rank, local_rank, world):
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": dict({"workload": args.workload, "batch": B, "seq_len": Lb, "d_model": shape.d_model, "d_state": shape.d_state,
-                            "heads": shape.n_heads, "layers": layers, "vocab": vocab, "tokens_per_s_whole_stack": world * T / (ms_step * 1e-3),
+                            "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T / (ms_step * 1e-3),
                             "parallelism": "replicas only" if world > 1 else "1 GPU",
                             "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
                            **extra),
