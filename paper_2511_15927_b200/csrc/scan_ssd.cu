@@ -82,6 +82,8 @@ static_assert(offsetof(Misc, norm_w) % 16 == 0 && offsetof(Misc, wbuf) % 16 == 0
 struct SsdArgs {
     int B, L, H, d_inner, d_in_proj, conv_ch, k, flags, nch, Lp;
     int Nr;                      // d_state of the model (<= N); B', C' and the state are zero-padded to N
+    int Pr;                      // headdim of the model: P, or P / 2 (the CTA then carries the next head's channels as unused padding)
+    __nv_bfloat16 *g;            // [2][B*L][d_inner] gated output (written with plain stores when Pr < P, else through map_g)
     const __nv_bfloat16 *zx;
     float *ssq;
     const float *dA;             // [2][B][H][2][Lp]: Lambda, Lambda' (log2 units)
@@ -234,7 +236,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         misc->abort = 0;
         mbar_fence_init();
     }
-    if (tid < P) misc->norm_w[tid] = (norm_on && w.norm_w) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * P + tid]) : 1.f;
+    const int Pr = a.Pr;                 // channels of this head; the tile's remaining P - Pr columns are padding and never leave the CTA
+    if (tid < P) misc->norm_w[tid] = (norm_on && w.norm_w && tid < Pr) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * Pr + tid]) : 1.f;
     if (warp == 1) tmem_alloc(&misc->tmem_base, TM_COLS);
     fence_before();
     __syncthreads();
@@ -256,7 +259,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const int sx = c % NX, sd = c % NDL, pc = rev ? nch - 1 - c : c;
                 if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
-                tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * P, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
+                tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
                 mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
                 bulk_load(smem + OFF_DL + sd * 2 * Q * 4, dA_head + pc * Q, Q * 4, &misc->full_dl[sd]);
                 bulk_load(smem + OFF_DL + sd * 2 * Q * 4 + Q * 4, dA_head + a.Lp + pc * Q, Q * 4, &misc->full_dl[sd]);
@@ -276,7 +279,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const int sz = c % NZ, pc = rev ? nch - 1 - c : c;
                 if (!WAIT(&misc->empty_z[sz], ((c / NZ) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_z[sz], T16);
-                tma_load_3d(smem + OFF_Z + sz * T16, &map_z, h * P, pc * Q, seq, &misc->full_z[sz]);
+                tma_load_3d(smem + OFF_Z + sz * T16, &map_z, h * Pr, pc * Q, seq, &misc->full_z[sz]);
                 issued = c + 1;
             }
             if (*abort_flag)
@@ -377,7 +380,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             float wl[4][4], cbias[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int ch = h * P + cg * 4 + e;
+                const int ch = min(h * Pr + cg * 4 + e, a.conv_ch - 1);      // padding columns read some valid weight: their results are unused
                 const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)ch * a.k;
 #pragma unroll
                 for (int m = 0; m < 4; ++m) wl[e][m] = m < a.k ? __bfloat162float(cw[a.k - 1 - m]) : 0.f;
@@ -396,7 +399,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int srow = t & (WG - 1), sh = t >> 7;      // state row and column half of this thread
         // incoming state -> TMEM (fp32)
         {
-            const float *h0 = (!rev && a.ssm_in && srow < a.Nr) ? a.ssm_in + (((int64_t)b * a.H + h) * P) * a.Nr + srow : nullptr;
+            const float *h0 = (!rev && a.ssm_in && srow < a.Nr && sh * 32 < Pr) ? a.ssm_in + (((int64_t)b * a.H + h) * Pr) * a.Nr + srow : nullptr;
             uint32_t hs[32];
 #pragma unroll
             for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(sh * 32 + p) * a.Nr]) : 0u;
@@ -453,7 +456,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     hr[m - 1] = *reinterpret_cast<const uint2 *>(xt + r * 128 + ((colx ^ (r & 7)) << 4) + sub);
                     if (c == 0 && rb == 0 && !rev && a.conv_in)      // rows before the sequence: the carried conv state (zeros beyond it)
                         hr[m - 1] = a.k - 1 - m >= 0
-                            ? __ldg(reinterpret_cast<const uint2 *>(a.conv_in + ((int64_t)b * (a.k - 1) + (a.k - 1 - m)) * a.conv_ch + h * P + cg * 4))
+                            ? __ldg(reinterpret_cast<const uint2 *>(a.conv_in + ((int64_t)b * (a.k - 1) + (a.k - 1 - m)) * a.conv_ch + h * Pr + cg * 4))
                             : make_uint2(0u, 0u);
                 }
                 h1[0] = bf2_to_f2(hr[0].x); h1[1] = bf2_to_f2(hr[0].y);
@@ -500,12 +503,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         if (!(ok && WAIT(&misc->st_full, (nch - 1) & 1))) ok = false;     // the last St has landed: TMEM holds the outgoing state
         fence_after();
         if (ok && !rev && a.ssm_out) {
-            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * P) * a.Nr + srow;
+            float *ho = a.ssm_out + (((int64_t)b * a.H + h) * Pr) * a.Nr + srow;
             const int half = sh;
             uint32_t hs[32];
             tmem_ld_x32(tlane + TM_HS + half * 32, hs);          // warp-wide: every lane takes part
             tmem_wait_ld();
-            if (srow < a.Nr) {                                   // rows beyond the model's d_state are padding (exact zeros)
+            if (srow < a.Nr && half * 32 < Pr) {                 // rows beyond the model's d_state and columns beyond its headdim are padding
 #pragma unroll
                 for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * a.Nr] = __uint_as_float(hs[p]);
             }
@@ -635,7 +638,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     ss2 = fma2(g, g, ss2);
                     ow[e2] = f2_to_bf2(mul2(g, nw[e2]));
                 }
-                *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                if (Pr == P) *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                else if (eg == 0 && t < L)      // half-width head: its 32 channels go out with plain stores, 64 bytes per token
+                    *reinterpret_cast<uint4 *>(a.g + ((int64_t)seq * L + t) * a.d_inner + h * Pr + c8 * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
             }
             float ss, ss_hi;
             upk2(ss2, ss, ss_hi);
@@ -643,11 +648,13 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (eg == 1) misc->ssq_part[row] = ss;
             fence_proxy_async();
             named_sync(2, ROLE);
-            if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + misc->ssq_part[row];
+            if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + (Pr == P ? misc->ssq_part[row] : 0.f);
             if (eg == 0 && row == 0) {
-                tma_store_3d(&map_g, zt, h * P, pc * Q, seq);    // rows past the end of the sequence are clipped
-                bulk_commit();
-                bulk_wait_read0();
+                if (Pr == P) {
+                    tma_store_3d(&map_g, zt, h * P, pc * Q, seq);    // rows past the end of the sequence are clipped
+                    bulk_commit();
+                    bulk_wait_read0();
+                }
                 mbar_arrive(&misc->empty_z[sz]);
             }
         }
@@ -682,7 +689,8 @@ Scratch scratch_layout(const ScanArgs &a) {
 }  // namespace
 
 bool scan_ssd_supports(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || a.P != P || a.k < 2 || a.k > 4) return false;
+    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || (a.P != P && a.P != P / 2) || a.k < 2 || a.k > 4) return false;
+    if (a.P != P && 2 * a.N < P / 2) return false;                        // a half-width head's tile reaches P/2 columns past the last head: they must exist in the row
     if (!a.z_gated) return false;                                         // the gate's SiLU is the in_proj epilogue's job on this path   // smaller d_state: zero-padded to N
     if (a.d_in_proj % 8 || a.d_inner % 8) return false;                  // 16-byte rows for TMA and vector access
     if (a.H > 65535 || a.B > 65535) return false;
@@ -690,7 +698,7 @@ bool scan_ssd_supports(const ScanArgs &a) {
 }
 
 size_t scan_ssd_workspace_bytes(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || a.P != P) return 0;
+    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || (a.P != P && a.P != P / 2)) return 0;
     return scratch_layout(a).total;
 }
 
@@ -702,7 +710,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     float *dA = reinterpret_cast<float *>(base + l.da);
     SsdArgs k{};
     k.B = a.B; k.L = a.L; k.H = a.H; k.d_inner = a.d_inner; k.d_in_proj = a.d_in_proj; k.conv_ch = a.conv_ch; k.k = a.k;
-    k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp; k.Nr = a.N;
+    k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp; k.Nr = a.N; k.Pr = a.P; k.g = static_cast<__nv_bfloat16 *>(a.g);
     k.zx = static_cast<const __nv_bfloat16 *>(a.zx); k.ssq = a.ssq; k.dA = dA;
     k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out; k.conv_in = static_cast<const __nv_bfloat16 *>(a.conv_in);
     k.dir[0] = a.dir[0]; k.dir[1] = a.dir[1];

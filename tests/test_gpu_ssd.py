@@ -108,3 +108,25 @@ def test_smaller_d_state_runs_zero_padded(G, N, H):
     _check(G, y_g, y_o)
     _check(G, s_g, s_o)
     _check(G, c_g, c_o)
+
+
+@pytest.mark.parametrize("N", [128, 16])
+def test_half_width_heads_run_with_padded_channels(G, N):
+    """headdim 32 (the paper's 1.3B shape: 120 heads of 32, App. A.1) takes the same kernel: a CTA loads 64 channels, of
+    which the second half (the next head's) is padding that never leaves it.  Parity of the output, the last head
+    included, and of the carried state in the model's [B, H, 32, d_state] layout."""
+    H = 8
+    shape = I.MixerShape(2, 300, 128, 2, N, 4, H)           # d_inner 256 = 8 heads of 32
+    assert shape.headdim == 32 and shape.d_in_proj % 8 == 0
+    wf, wr = I.make_mixer_weights(shape, 40 + N, I.BF16, perturb=True)
+    x = I.make_activations(shape, 40 + N, I.BF16)
+    kw = G.oracle_kwargs(shape)
+    for flags in (7, 6):                                    # with and without the gated norm (its sum of squares covers 32 channels)
+        _check(G, G.run_forward(shape, I.BF16, wf, wr, x, flags=flags), O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape, flags)))
+    ssm_in, conv_in = I.make_states(shape, 40 + N, I.BF16)
+    y_o, s_o, c_o = O.bimamba_block_step(x, wf, wr, ssm_state_in=ssm_in, conv_state_in=conv_in, **kw)
+    y_g, s_g, c_g = G.run_block_step(shape, I.BF16, wf, wr, x, ssm_in, conv_in)
+    assert s_g.shape == s_o.shape == (2, H, 32, N)
+    _check(G, y_g, y_o)
+    _check(G, s_g, s_o)
+    _check(G, c_g, c_o)
