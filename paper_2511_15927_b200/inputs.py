@@ -192,4 +192,5 @@ CONFIGS = {
     "cfg3_64k": (MixerShape(1, 65536, 2048, 2, 128, 4, 64), BF16),      # the longest context of the paper's throughput sweep (Sec. 4.3)
     "cfg4_block": (MixerShape(16, 32, 2048, 2, 128, 4, 64), BF16),
     "paper_1p3b": (MixerShape(1, 1024, 1920, 2, 128, 4, 120), BF16),
+    "paper_1p3b_8k": (MixerShape(1, 8192, 1920, 2, 128, 4, 120), BF16),
 }
