@@ -385,3 +385,61 @@ def denoise_step_cond(tokens, tau, sw: dict, *, rms_eps: float = 1e-5, ln_eps: f
             states_out.append((s_out, c_out))
     logits = rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T
     return (logits, states_out) if return_states else logits
+
+
+# --------------------------------------------------------------------------------------------
+# Reverse step of the masked diffusion (Sec. 2, Eq. 3): from noise level t to s < t
+# --------------------------------------------------------------------------------------------
+def reverse_step_probabilities(logits_row, is_masked: bool, token: int, keep_prob: float, mask_id: int):
+    """q_{s|t}(. | x_t) of one position as a vector over the vocabulary (Eq. 3), keep_prob = s / t:
+    an unmasked token stays with probability 1; a masked one stays masked with probability s/t and
+    otherwise becomes token v with probability (1 - s/t) * q_{0|t}(v), where q_{0|t} is the softmax of
+    the logits with the mask token excluded (the substitution parameterisation of App. A.1: the
+    model never predicts [MASK])."""
+    z = np.asarray(logits_row, F64)
+    q = np.zeros_like(z)
+    if not is_masked:
+        q[token] = 1.0
+        return q
+    zz = z.copy()
+    zz[mask_id] = -np.inf
+    p = np.exp(zz - zz[np.isfinite(zz)].max())
+    p /= p.sum()
+    q = (1.0 - keep_prob) * p
+    q[mask_id] = keep_prob
+    return q
+
+
+def reverse_step(tokens, logits, u_keep, u_cat, keep_prob: float, mask_id: int):
+    """One draw from Eq. 3 for every position, driven by two uniforms per position (inputs, so that the
+    draw is a function): a masked position stays masked iff u_keep < s/t; otherwise its token is the
+    inverse-CDF sample of q_{0|t} at u_cat: the first v (mask excluded) whose cumulative probability
+    reaches u_cat.  tokens [B, L] int, logits [B, L, V], u_* [B, L] in [0, 1)."""
+    tokens = np.asarray(tokens)
+    out = tokens.copy()
+    B, L = tokens.shape
+    for b in range(B):
+        for t in range(L):
+            if tokens[b, t] != mask_id:
+                continue                                   # case 1: carried over
+            if np.float32(u_keep[b, t]) < np.float32(keep_prob):
+                continue                                   # case 2: stays masked
+            z = np.asarray(logits[b, t], F64).copy()
+            z[mask_id] = -np.inf
+            p = np.exp(z - z[np.isfinite(z)].max())
+            cdf = np.cumsum(p)
+            target = np.float64(u_cat[b, t]) * cdf[-1]
+            v = int(np.searchsorted(cdf, target, side="right"))     # first v with cdf[v] > target
+            v = min(v, len(cdf) - 1)
+            while p[v] == 0.0:                             # u_cat == 0 with zero-probability leading entries
+                v += 1
+            out[b, t] = v
+    return out
+
+
+def noise_schedule(K: int, eps: float = 1e-3):
+    """Noise levels of a K-step generation, t_0 = 1 > ... > t_K = eps (App. A.1: sampling eps 1e-3), uniformly
+    spaced; step k goes from t_k to s = t_{k+1} and keeps a masked token masked with probability s / t_k
+    (the last step, to eps, still leaves s / t of the masked tokens to a final clean-up pass with keep 0)."""
+    t = 1.0 - (1.0 - eps) * np.arange(K + 1) / K
+    return t

@@ -536,3 +536,47 @@ def test_conditioned_stack_and_its_block_mode():
     l1, st = O.denoise_step_cond(tok[:, :5], tau, sw, return_states=True, **kw)
     l2, _ = O.denoise_step_cond(tok[:, 5:], tau, sw, states_in=st, return_states=True, **kw)
     np.testing.assert_allclose(np.concatenate([l1, l2], 1), whole, rtol=1e-9, atol=1e-11)
+
+
+# ------------------------------------------------------------------ reverse step (Sec. 2, Eq. 3)
+
+def test_reverse_step_cases_and_probabilities():
+    V, mask = 7, 6
+    z = rng.standard_normal(V) * 2
+    # the three cases of Eq. 3 as a probability vector
+    q = O.reverse_step_probabilities(z, False, 3, 0.4, mask)
+    assert q[3] == 1.0 and q.sum() == 1.0
+    q = O.reverse_step_probabilities(z, True, mask, 0.4, mask)
+    soft = np.exp(z[:mask]) / np.exp(z[:mask]).sum()                      # softmax over the real tokens only
+    np.testing.assert_allclose(q[:mask], 0.6 * soft, rtol=1e-12)
+    assert q[mask] == pytest.approx(0.4) and q.sum() == pytest.approx(1.0)
+    # the draw realises those probabilities: sweep both uniforms over a fine grid (a deterministic integral)
+    n = 400
+    uk, uc = np.meshgrid((np.arange(n) + 0.5) / n, (np.arange(n) + 0.5) / n, indexing="ij")
+    tok = np.full((1, n * n), mask)
+    logits = np.broadcast_to(z, (1, n * n, V))
+    out = O.reverse_step(tok, logits, uk.reshape(1, -1), uc.reshape(1, -1), 0.4, mask)
+    freq = np.bincount(out.ravel(), minlength=V) / (n * n)
+    np.testing.assert_allclose(freq, q, atol=2.0 / n)
+    # unmasked tokens are carried over whatever the uniforms say; the mask token is never drawn
+    tok2 = np.array([[0, mask, 5, mask]])
+    lg = rng.standard_normal((1, 4, V))
+    o2 = O.reverse_step(tok2, lg, np.array([[0.0, 0.9, 0.0, 0.1]]), np.array([[0.5, 0.5, 0.5, 0.5]]), 0.4, mask)
+    assert o2[0, 0] == 0 and o2[0, 2] == 5 and o2[0, 3] == mask and o2[0, 1] != mask
+    # extremes of the inverse CDF: u -> 0 picks the first token with probability, u -> 1 the last one
+    lg3 = np.zeros((1, 2, V)); lg3[0, :, 0] = -np.inf
+    o3 = O.reverse_step(np.full((1, 2), mask), lg3, np.ones((1, 2)) * 0.99, np.array([[0.0, 1.0 - 1e-12]]), 0.4, mask)
+    assert o3[0, 0] == 1 and o3[0, 1] == mask - 1
+    # keep_prob 0 unmasks everything, keep_prob 1 nothing
+    full = O.reverse_step(np.full((1, 50), mask), rng.standard_normal((1, 50, V)), rng.random((1, 50)), rng.random((1, 50)), 0.0, mask)
+    assert np.all(full != mask)
+    none = O.reverse_step(np.full((1, 50), mask), rng.standard_normal((1, 50, V)), rng.random((1, 50)), rng.random((1, 50)), 1.0, mask)
+    assert np.all(none == mask)
+
+
+def test_noise_schedule_endpoints_and_expected_unmasking():
+    t = O.noise_schedule(8)
+    assert t[0] == 1.0 and t[-1] == pytest.approx(1e-3) and np.all(np.diff(t) < 0)
+    np.testing.assert_allclose(np.diff(t), np.diff(t)[0])                  # uniform spacing: K = L / p steps of equal size (Sec. 4.3)
+    # the chance that a token is still masked after k steps telescopes to t_k (Eq. 1's marginal: masked w.p. t)
+    np.testing.assert_allclose(np.cumprod(t[1:] / t[:-1]), t[1:], rtol=1e-12)
