@@ -190,6 +190,29 @@ int dm_denoise_step_cond(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const
                          void *logits, int32_t *argmax_out, const dm_layer_state *states,
                          void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* One reverse step of the masked diffusion, Sec. 2 Eq. 3, from noise level t to s < t: the denoiser runs on
+ * tokens_in (as dm_denoise_step when blk == NULL, else as dm_denoise_step_cond), then every position
+ *   - that is not mask_id keeps its token;
+ *   - that is masked stays masked when u_keep[pos] < keep_prob (= s / t);
+ *   - otherwise receives the inverse-CDF draw at u_cat[pos] from softmax(logits[pos, 0..vocab_real)) with mask_id
+ *     excluded (the model never predicts the mask token): the first v whose cumulative probability exceeds
+ *     u_cat[pos].  Both uniforms are in [0, 1) and come from the caller, so the step is a function of its inputs.
+ * Only the drawn positions go through the vocabulary projection (their number is never brought to the host), and
+ * the logits are not stored.  tokens_in, tokens_out [B, L] int32 (different buffers); u_keep, u_cat [B, L] fp32;
+ * all on the device.  The probabilities are accumulated in fp32 in vocabulary order; a draw whose u_cat falls
+ * within rounding distance of a boundary of the cumulative distribution may land on either neighbour. */
+typedef struct {
+    int32_t mask_id;      /* id of [MASK], < vocab */
+    int32_t vocab_real;   /* ids [0, vocab_real) can be drawn; rows of w_vocab beyond are padding */
+    float   keep_prob;    /* s / t of this step, in [0, 1] */
+} dm_sample_cfg;
+int dm_denoise_sample_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes);
+int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights,
+                           const dm_block_weights *block_weights, const int32_t *tokens_in, const float *tau,
+                           const dm_sample_cfg *sample, const float *u_keep, const float *u_cat,
+                           int32_t *tokens_out, const dm_layer_state *states,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* One dense projection as the mixer uses it (App. C counts 2mn FLOPs per token for a weight W in R^{m x n}):
  *     y[r, :] = row_scale[r] * (W x[r, :]) + addend[r, :]
  * x [rows, in_features] dtype; w [out_features, in_features] dtype; y [rows, out_features] of y_dtype

@@ -51,6 +51,10 @@ class dm_block_cfg(C.Structure):
     _fields_ = [("d_ff", C.c_int32), ("d_cond", C.c_int32), ("ln_eps", C.c_float)]
 
 
+class dm_sample_cfg(C.Structure):
+    _fields_ = [("mask_id", C.c_int32), ("vocab_real", C.c_int32), ("keep_prob", C.c_float)]
+
+
 class dm_block_weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_cond", "b_cond", "w_up", "b_up", "w_down", "b_down")]
 
@@ -83,6 +87,12 @@ _lib.dm_denoise_cond_workspace_bytes.restype = C.c_int
 _lib.dm_denoise_step_cond.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_stack_weights),
                                       C.POINTER(dm_block_weights), _vp, _vp, _vp, _vp, C.POINTER(dm_layer_state), _vp, _sz, _vp]
 _lib.dm_denoise_step_cond.restype = C.c_int
+_lib.dm_denoise_sample_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(_sz)]
+_lib.dm_denoise_sample_workspace_bytes.restype = C.c_int
+_lib.dm_denoise_sample_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_stack_weights),
+                                        C.POINTER(dm_block_weights), _vp, _vp, C.POINTER(dm_sample_cfg), _vp, _vp, _vp,
+                                        C.POINTER(dm_layer_state), _vp, _sz, _vp]
+_lib.dm_denoise_sample_step.restype = C.c_int
 _lib.dm_linear.argtypes = [C.c_int, _vp, _vp, _vp, C.c_int, C.c_int64, C.c_int32, C.c_int32, _vp, _vp, _vp]
 _lib.dm_linear.restype = C.c_int
 _lib.dm_profile_enable.argtypes = [C.c_int]
@@ -94,7 +104,7 @@ for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes",
 EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
            "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
-           "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond")
+           "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -203,6 +213,20 @@ def dm_denoise_step_cond(cfg, blk, weights, block_weights, tokens: int, tau: int
     _ok(_lib.dm_denoise_step_cond(C.byref(cfg), C.byref(blk), C.byref(weights), block_weights, _vp(tokens), _vp(tau),
                                   _vp(logits or None), _vp(argmax_out or None), states, _vp(workspace), _sz(workspace_bytes),
                                   _vp(cuda_stream)))
+
+
+def dm_denoise_sample_workspace_bytes(cfg: dm_stack_cfg, blk=None) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_denoise_sample_workspace_bytes(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(n)))
+    return n.value
+
+
+def dm_denoise_sample_step(cfg, blk, weights, block_weights, tokens_in: int, tau: int, sample: dm_sample_cfg, u_keep: int,
+                           u_cat: int, tokens_out: int, states, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    """blk / block_weights / tau: None (or 0) for the plain stack, else as in dm_denoise_step_cond."""
+    _ok(_lib.dm_denoise_sample_step(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(weights), block_weights,
+                                    _vp(tokens_in), _vp(tau or None), C.byref(sample), _vp(u_keep), _vp(u_cat), _vp(tokens_out),
+                                    states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
 
 
 # ------------------------------------------------------------------------------------------------

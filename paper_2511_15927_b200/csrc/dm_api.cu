@@ -230,11 +230,11 @@ static int check_ws(const void *ws, size_t have, size_t need) {
 }
 
 struct StackWs {
-    size_t r, u, logits, mixer, mod, hmid, total;
+    size_t r, u, logits, mixer, mod, hmid, idx, count, ug, total;
     int logits_rows;
 };
 
-static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg *blk = nullptr) {
+static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg *blk = nullptr, bool sampler = false) {
     StackWs w;
     size_t off = 0;
     w.r = off; off += align_up((size_t)m.T * m.d * sizeof(float));
@@ -246,6 +246,12 @@ static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg
     if (blk) {
         w.mod = off; off += align_up((size_t)m.B * 6 * m.d * sizeof(float));
         w.hmid = off; off += align_up((size_t)m.T * blk->d_ff * m.es);
+    }
+    w.idx = w.count = w.ug = off;
+    if (sampler) {
+        w.idx = off; off += align_up((size_t)m.T * sizeof(int32_t));
+        w.count = off; off += align_up(sizeof(int));
+        w.ug = off; off += align_up((size_t)m.T * m.d * m.es);
     }
     w.total = off;
     return w;
@@ -417,10 +423,14 @@ int dm_bimamba_block_step(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], co
 
 // One denoiser evaluation.  blk == NULL: RMSNorm pre-norm + mixer per layer; otherwise the timestep-conditioned block of
 // App. A.1 (AdaLN -> mixer -> gated residual, AdaLN -> MLP -> gated residual) with the modulation of each layer from tau.
+struct SampleArgs {
+    const dm_sample_cfg *cfg; const float *u_keep, *u_cat; int32_t *tokens_out;
+};
+
 static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights, const dm_block_weights *bw,
                         const int32_t *tokens, const float *tau, void *logits,
                         int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
-                        void *cuda_stream) {
+                        void *cuda_stream, const SampleArgs *smp = nullptr) {
     Dims m;
     if (!cfg || !weights) return fail(DM_ERR_INVALID_ARG, "cfg or weights is NULL");
     int st = check_cfg(&cfg->mixer, &m);
@@ -428,7 +438,16 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
     if (cfg->n_layers <= 0 || cfg->vocab <= 0) return fail(DM_ERR_INVALID_ARG, "n_layers and vocab must be positive");
     if (!(cfg->rms_eps >= 0.f)) return fail(DM_ERR_INVALID_ARG, "rms_eps must be >= 0");
     if (!tokens) return fail(DM_ERR_INVALID_ARG, "tokens is NULL");
-    if (!logits && !argmax_out) return fail(DM_ERR_INVALID_ARG, "logits and argmax_out are both NULL");
+    if (!logits && !argmax_out && !smp) return fail(DM_ERR_INVALID_ARG, "logits and argmax_out are both NULL");
+    if (smp) {
+        if (!smp->cfg || !smp->u_keep || !smp->u_cat || !smp->tokens_out) return fail(DM_ERR_INVALID_ARG, "NULL pointer in the sampling arguments");
+        if (smp->tokens_out == tokens) return fail(DM_ERR_INVALID_ARG, "tokens_out must not be tokens_in");
+        const dm_sample_cfg &q = *smp->cfg;
+        if (q.vocab_real <= 0 || q.vocab_real > cfg->vocab || q.mask_id < 0 || q.mask_id >= cfg->vocab)
+            return fail(DM_ERR_INVALID_ARG, "vocab_real must be in (0, vocab], mask_id in [0, vocab)");
+        if (q.vocab_real == 1 && q.mask_id == 0) return fail(DM_ERR_INVALID_ARG, "no token left to draw");
+        if (!(q.keep_prob >= 0.f && q.keep_prob <= 1.f)) return fail(DM_ERR_INVALID_ARG, "keep_prob must be in [0, 1]");
+    }
     if (!weights->embed || !weights->layers || !weights->final_norm_w || !weights->w_vocab)
         return fail(DM_ERR_INVALID_ARG, "NULL pointer in stack weights");
     if (!aligned16(weights->embed) || !aligned16(weights->w_vocab) || !aligned16(logits))
@@ -459,7 +478,7 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
                 return fail(DM_ERR_INVALID_ARG, "state_out needs the left-to-right direction");
         }
     }
-    const StackWs l = stack_ws(cfg, m, blk);
+    const StackWs l = stack_ws(cfg, m, blk, smp != nullptr);
     if ((st = check_ws(workspace, workspace_bytes, l.total)) != DM_OK) return st;
     char *ws = static_cast<char *>(workspace);
     float *r = reinterpret_cast<float *>(ws + l.r);
@@ -503,6 +522,28 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
         }
     }
     if ((e = rmsnorm_rows(r, weights->final_norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "final norm");
+    if (smp) {
+        // Eq. 3: only the positions drawn this step go through the vocabulary projection; how many there are stays on the device
+        int32_t *idx = reinterpret_cast<int32_t *>(ws + l.idx);
+        int *count = reinterpret_cast<int *>(ws + l.count);
+        void *ug = ws + l.ug;
+        const dm_sample_cfg &q = *smp->cfg;
+        if ((e = select_drawn(tokens, smp->u_keep, q.keep_prob, q.mask_id, smp->tokens_out, idx, count, (int)m.T, s)) != cudaSuccess) return cuda_fail(e, "select");
+        if ((e = gather_rows(u, idx, count, ug, dtype, (int)m.T, m.d, s)) != cudaSuccess) return cuda_fail(e, "gather");
+        for (int64_t t0 = 0; t0 < m.T; t0 += l.logits_rows) {
+            const int rows = (int)((m.T - t0) < l.logits_rows ? (m.T - t0) : l.logits_rows);
+            GemmArgs a{};
+            a.A = static_cast<char *>(ug) + (size_t)t0 * m.d * m.es; a.lda = m.d;
+            a.B = weights->w_vocab; a.ldb = m.d;
+            a.C = ws + l.logits; a.ldc = cfg->vocab;
+            a.in_dtype = dtype; a.c_dtype = dtype; a.M = rows; a.N = cfg->vocab; a.K = m.d;
+            a.m_dev = count; a.m_off = (int)t0;
+            if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "vocab projection");
+            if ((e = draw_rows(a.C, cfg->vocab, dtype, idx, count, (int)t0, rows, smp->u_cat, q.mask_id, q.vocab_real, smp->tokens_out, s)) != cudaSuccess)
+                return cuda_fail(e, "draw");
+        }
+        return DM_OK;
+    }
     const int64_t rows_per = logits ? m.T : l.logits_rows;
     for (int64_t t0 = 0; t0 < m.T; t0 += rows_per) {
         const int rows = (int)((m.T - t0) < rows_per ? (m.T - t0) : rows_per);
@@ -541,6 +582,24 @@ int dm_denoise_step_cond(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const
                          void *cuda_stream) {
     if (!blk) return fail(DM_ERR_INVALID_ARG, "block configuration is NULL");
     return denoise_impl(cfg, blk, weights, block_weights, tokens, tau, logits, argmax_out, states, workspace, workspace_bytes, cuda_stream);
+}
+
+int dm_denoise_sample_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes) {
+    Dims m;
+    if (!cfg || !bytes) return fail(DM_ERR_INVALID_ARG, "NULL argument");
+    int st = check_cfg(&cfg->mixer, &m);
+    if (st != DM_OK) return st;
+    if (cfg->vocab <= 0 || (blk && blk->d_ff <= 0)) return fail(DM_ERR_INVALID_ARG, "vocab and d_ff must be positive");
+    *bytes = stack_ws(cfg, m, blk, true).total;
+    return DM_OK;
+}
+
+int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights,
+                           const dm_block_weights *block_weights, const int32_t *tokens_in, const float *tau,
+                           const dm_sample_cfg *sample, const float *u_keep, const float *u_cat, int32_t *tokens_out,
+                           const dm_layer_state *states, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    const SampleArgs smp{sample, u_keep, u_cat, tokens_out};
+    return denoise_impl(cfg, blk, weights, block_weights, tokens_in, tau, nullptr, nullptr, states, workspace, workspace_bytes, cuda_stream, &smp);
 }
 
 int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype, int64_t rows, int32_t in_features,

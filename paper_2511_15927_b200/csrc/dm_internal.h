@@ -39,6 +39,8 @@ struct GemmArgs {
     const float *col_scale;  // [ceil(M / cs_rows), ld_cs] or NULL: one scale vector per group of cs_rows consecutive rows
     int cs_rows;
     int64_t ld_cs;           // row pitch of col_scale (0 = N)
+    const int *m_dev;        // device int or NULL: only rows [0, clamp(*m_dev - m_off, 0, M)) are computed (row count known on the device only)
+    int m_off;
 };
 cudaError_t gemm_simple(const GemmArgs &a, cudaStream_t s);
 // Tensor-core path (tcgen05 + TMEM + TMA).  Returns cudaErrorNotSupported for shapes it does not take.
@@ -85,6 +87,14 @@ cudaError_t adaln_rows(const float *r, const float *gamma, const float *beta, in
 // mod[b, :] = b_cond + W_cond tau[b, :]   (W_cond [n_out, d_c] dtype, b_cond [n_out] fp32 or NULL, tau [B, d_c] fp32)
 cudaError_t modulation_rows(const float *tau, const void *w_cond, const float *b_cond, float *mod, int dtype, int B, int n_out, int d_c,
                             cudaStream_t s);
+// Reverse step (Sec. 2, Eq. 3): tokens_out = tokens_in; idx[0..*count) = positions drawn this step (masked and u_keep >= keep_prob)
+cudaError_t select_drawn(const int32_t *tokens_in, const float *u_keep, float keep_prob, int mask_id, int32_t *tokens_out, int32_t *idx,
+                         int *count, int T, cudaStream_t s);
+// dst[j, :] = src[idx[j], :] for j < *count
+cudaError_t gather_rows(const void *src, const int32_t *idx, const int *count, void *dst, int dtype, int T, int d, cudaStream_t s);
+// tokens_out[idx[row0 + r]] = inverse-CDF draw at u_cat from softmax(logits[r, 0..vocab_real) without mask_id), r < rows, row0 + r < *count
+cudaError_t draw_rows(const void *logits, int64_t ld, int dtype, const int32_t *idx, const int *count, int row0, int rows,
+                      const float *u_cat, int mask_id, int vocab_real, int32_t *tokens_out, cudaStream_t s);
 // out[t] = argmax_v logits[t, v], lowest index on ties
 cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s);
 // conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])

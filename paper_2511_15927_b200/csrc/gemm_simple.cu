@@ -16,7 +16,8 @@ __global__ void __launch_bounds__(256)
 gemm_simple_kernel(const TIn *__restrict__ A, int64_t lda, const TIn *__restrict__ B, int64_t ldb,
                    TOut *C, int64_t ldc, int M, int N, int K,
                    const float *__restrict__ row_scale, const float *addend, int64_t ld_add, int silu_cols,
-                   const float *__restrict__ col_bias, int gelu, const float *__restrict__ col_scale, int cs_rows, int64_t ld_cs) {
+                   const float *__restrict__ col_bias, int gelu, const float *__restrict__ col_scale, int cs_rows, int64_t ld_cs, const int *__restrict__ m_dev, int m_off) {
+    if (m_dev) M = min(M, max(0, *m_dev - m_off));
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -74,7 +75,7 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     gemm_simple_kernel<TIn, TOut><<<grid, 256, 0, s>>>(
         static_cast<const TIn *>(a.A), a.lda, static_cast<const TIn *>(a.B), a.ldb,
         static_cast<TOut *>(a.C), a.ldc, a.M, a.N, a.K, a.row_scale, a.addend, a.ld_add, a.silu_cols,
-        a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : a.N);
+        a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : a.N, a.m_dev, a.m_off);
     count_launch();
     return cudaGetLastError();
 }

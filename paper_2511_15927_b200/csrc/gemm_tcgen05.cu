@@ -32,6 +32,7 @@ struct EpiArgs {
     int M, N, K;
     int silu_cols;   // SiLU on output columns below this one
     const float *col_bias; int gelu; const float *col_scale; int cs_rows; int64_t ld_cs;   // see GemmArgs
+    const int *m_dev; int m_off;
     int n_fast;      // tile order: consecutive tiles step along N (the A rows are streamed once, B stays in L2) or along M
 };
 
@@ -46,7 +47,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile int *abort_flag = &bars->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (ep.M + BM - 1) / BM, tiles_n = (ep.N + BN - 1) / BN;
+    // rows to compute: all of them, or the count another kernel left on the device (tiles beyond it are skipped)
+    const int M_eff = ep.m_dev ? min(ep.M, max(0, *ep.m_dev - ep.m_off)) : ep.M;
+    const int tiles_m = (M_eff + BM - 1) / BM, tiles_n = (ep.N + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_n;
     const int kblocks = (ep.K + BK - 1) / BK;
     constexpr uint32_t TMEM_COLS = 2 * BN;          // two accumulator buffers; 256 or 512 columns
@@ -131,7 +134,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!ok) break;
             fence_after();
             const int row = m0 + q * 32 + lane;
-            const bool row_ok = row < ep.M;
+            const bool row_ok = row < M_eff;
             const float sc = (ep.row_scale && row_ok) ? ep.row_scale[row] : 1.f;
             const float *add_row = ep.addend ? ep.addend + (int64_t)row * ep.ld_add : nullptr;
 #pragma unroll 1
@@ -274,7 +277,7 @@ cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
     const int grid = tiles < sm_count() ? tiles : sm_count();
     // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
     EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols,
-               a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.M > a.N ? 1 : 0};
+               a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.m_dev, a.m_off, a.M > a.N ? 1 : 0};
     gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma, mb, ep, status);
     count_launch();
     return cudaGetLastError();

@@ -121,3 +121,29 @@ def oracle_kwargs(shape, flags=dm.DM_FLAGS_DEFAULT, eps=1e-5):
     return dict(expand=shape.expand, d_state=shape.d_state, n_heads=shape.n_heads, n_groups=shape.n_groups,
                 gated_norm=bool(flags & dm.DM_FLAG_GATED_RMSNORM), conv_bias=bool(flags & dm.DM_FLAG_CONV_BIAS),
                 d_skip=bool(flags & dm.DM_FLAG_D_SKIP), norm_eps=eps)
+
+
+def run_sample_step(shape, dtype, sw, tokens, vocab, u_keep, u_cat, keep_prob, mask_id, vocab_real, tau=None, d_ff=0,
+                    rms_eps=1e-5, ln_eps=1e-5):
+    """dm_denoise_sample_step on host arrays; returns tokens_out [B, L] int32."""
+    n_layers = len(sw["layers"])
+    scfg = dm.dm_stack_cfg(cfg_of(shape, dtype), n_layers, vocab, rms_eps)
+    dsw = dev_stack_weights(sw, dtype)
+    csw, keep = dm.make_stack_weights(dsw)
+    blk = cbw = taud = None
+    if tau is not None:
+        blk = dm.dm_block_cfg(d_ff, tau.shape[1], ln_eps)
+        dbw = dev_block_weights(sw, dtype)
+        cbw = dm.make_block_weights(dbw)
+        taud = dev(np.asarray(tau, np.float32))
+    tok = dev(np.asarray(tokens, np.int32))
+    out = torch.full_like(tok, -7)
+    uk, uc = dev(np.asarray(u_keep, np.float32)), dev(np.asarray(u_cat, np.float32))
+    nb = dm.dm_denoise_sample_workspace_bytes(scfg, blk)
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_denoise_sample_step(scfg, blk, csw, cbw, tok.data_ptr(), taud.data_ptr() if taud is not None else 0,
+                              dm.dm_sample_cfg(mask_id, vocab_real, keep_prob), uk.data_ptr(), uc.data_ptr(), out.data_ptr(), None,
+                              ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    return out.cpu().numpy()
