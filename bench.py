@@ -166,6 +166,9 @@ STACKS = {
     "cfg2_stack_n128": dict(shape=I.MixerShape(4, 4096, 1024, 2, 128, 4, 32), layers=24, vocab=50304),
     "cfg4_decode": dict(shape=I.MixerShape(16, 32, 2048, 2, 128, 4, 64), layers=24, vocab=50304, prefix=2048),
     # the same stack with the timestep-conditioned block of App. A.1 in every layer (AdaLN, mixer, AdaLN, MLP with d_ff = 2 d)
+    # one reverse step of the masked diffusion (Sec. 2, Eq. 3) on the cfg 2 stack, mid-generation: half of the positions
+    # masked, p = 16 of them drawn per sequence and step (K = L / p steps per generation, Sec. 4.3)
+    "cfg2_sample": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, sample=dict(p=16)),
     "cfg2_stack_cond": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, cond=dict(d_ff=2048, d_cond=128)),
 }
 
@@ -231,11 +234,24 @@ def run_stack(args, rank, local_rank, world):
         cbw = dm.make_block_weights(w["blocks"])
         tau = torch.from_numpy(I.make_timestep_embedding(B, cond["d_cond"], seed=0)).cuda()
 
+    smp = spec.get("sample")
+    if smp:
+        masked_per_row = Lb // 2
+        scfg_s = dm.dm_sample_cfg(50257, 50258, 1.0 - smp["p"] / masked_per_row)
+        gen = torch.Generator(device="cuda").manual_seed(1)
+        u_keep = torch.rand(B, Lb, generator=gen, device="cuda")
+        u_cat = torch.rand(B, Lb, generator=gen, device="cuda")
+
     def ws_bytes(cfg):
+        if smp:
+            return dm.dm_denoise_sample_workspace_bytes(cfg, blk if cond else None)
         return dm.dm_denoise_cond_workspace_bytes(cfg, blk) if cond else dm.dm_denoise_workspace_bytes(cfg)
 
     def denoise(cfg, tok_ptr, amax_ptr, st):
-        if cond:
+        if smp:
+            dm.dm_denoise_sample_step(cfg, blk if cond else None, csw, cbw if cond else None, tok_ptr, tau.data_ptr() if cond else 0, scfg_s,
+                                      u_keep.data_ptr(), u_cat.data_ptr(), amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
+        elif cond:
             dm.dm_denoise_step_cond(cfg, blk, csw, cbw, tok_ptr, tau.data_ptr(), 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
         else:
             dm.dm_denoise_step(cfg, csw, tok_ptr, 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
@@ -245,6 +261,14 @@ def run_stack(args, rank, local_rank, world):
         return dm.dm_stack_cfg(G.cfg_of(sh, I.BF16), layers, vocab, 1e-5)
 
     def tokens(L, n):
+        if smp:                                   # mid-generation: every other position is [MASK]
+            out = []
+            for i in range(n):
+                t = I.make_tokens(B, L, 50257, 50257, seed=i)
+                t[:, (i % 2)::2] = 50257
+                t[:, (1 - i % 2)::2] = np.where(t[:, (1 - i % 2)::2] == 50257, 11, t[:, (1 - i % 2)::2])
+                out.append(torch.from_numpy(t).cuda())
+            return out
         return [torch.from_numpy(I.make_tokens(B, L, 50257, 50257, seed=i)).cuda() for i in range(n)]
 
     scfg = stack_cfg(Lb)
@@ -361,6 +385,8 @@ def run_stack(args, rank, local_rank, world):
                             "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T / (ms_step * 1e-3),
                             "parallelism": "replicas only" if world > 1 else "1 GPU",
                             "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
+                           **({"sample": "half of the positions masked, p = %d drawn per sequence and step" % smp["p"],
+                               "generated_tokens_per_s_at_K_eq_L_over_p": world * T / ((Lb // smp["p"]) * ms_step * 1e-3)} if smp else {}),
                            **extra),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels, "cpu_baseline": None}
     print(json.dumps(line), flush=True)
