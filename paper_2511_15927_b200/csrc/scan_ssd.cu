@@ -383,8 +383,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const int ch = min(h * Pr + cg * 4 + e, a.conv_ch - 1);      // padding columns read some valid weight: their results are unused
                 const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)ch * a.k;
 #pragma unroll
-                for (int m = 0; m < 4; ++m) wl[e][m] = m < a.k ? __bfloat162float(cw[a.k - 1 - m]) : 0.f;
-                cbias[e] = has_bias ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[ch]) : 0.f;
+                for (int m = 0; m < 4; ++m) wl[e][m] = m < a.k ? 0.5f * __bfloat162float(cw[a.k - 1 - m]) : 0.f;      // halved: the loop wants v/2
+                cbias[e] = has_bias ? 0.5f * __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[ch]) : 0.f;
             }
 #pragma unroll
             for (int e2 = 0; e2 < 2; ++e2) {
@@ -393,7 +393,6 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 for (int m = 0; m < 4; ++m) wl2[e2][m] = pk2(wl[2 * e2][m], wl[2 * e2 + 1][m]);
             }
         }
-        const f32x2 half2 = pk2(0.5f, 0.5f);
         const int first = rev ? rb * RB + RB - 1 : rb * RB, step = rev ? -1 : 1;   // first-in-time chunk row of the block
         const int toff = rev ? 0 : HALO;                                          // tile row = chunk row + toff
         const int srow = t & (WG - 1), sh = t >> 7;      // state row and column half of this thread
@@ -482,9 +481,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 uint32_t ox[2], os[2];
 #pragma unroll
                 for (int e2 = 0; e2 < 2; ++e2) {
-                    f32x2 v = fma2(wl2[e2][3], h3[e2], cb2[e2]);
-                    v = fma2(wl2[e2][2], h2[e2], v); v = fma2(wl2[e2][1], h1[e2], v); v = fma2(wl2[e2][0], cur[e2], v);
-                    const f32x2 hh = mul2(v, half2);             // SiLU(v) = v/2 + v/2 tanh(v/2)
+                    f32x2 hh = fma2(wl2[e2][3], h3[e2], cb2[e2]);          // half of the conv output (weights and bias are halved)
+                    hh = fma2(wl2[e2][2], h2[e2], hh); hh = fma2(wl2[e2][1], h1[e2], hh); hh = fma2(wl2[e2][0], cur[e2], hh);
+                    // SiLU(v) = v/2 + v/2 tanh(v/2)
                     float ha, hb;
                     upk2(hh, ha, hb);
                     const f32x2 o = fma2(hh, pk2(tanh_fast(ha), tanh_fast(hb)), hh);

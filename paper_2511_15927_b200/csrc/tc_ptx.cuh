@@ -40,18 +40,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one gave up); the first
 // wait to give up raises the CTA's abort flag and stores DM_ERR_TIMEOUT in the device status word.
+// Up to 64 probes back to back: a waiting warp competes for issue slots with the working ones, so the loop around the
+// probe is four instructions and nothing else.
+__device__ __forceinline__ bool mbar_probe64(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+        "mov.u32 n, 0;\n\t"
+        "MBAR_PROBE_%=:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra MBAR_DONE_%=;\n\t"
+        "add.u32 n, n, 1;\n\t"
+        "setp.lt.u32 q, n, 64;\n\t"
+        "@q bra MBAR_PROBE_%=;\n\t"
+        "MBAR_DONE_%=:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
-                atomicExch(status, (int)DM_ERR_TIMEOUT);
-                return false;
-            }
+    for (;;) {
+        if (mbar_probe64(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+            *abort_flag = 1;
+            atomicExch(status, (int)DM_ERR_TIMEOUT);
+            return false;
         }
     }
 }
