@@ -65,7 +65,7 @@ def test_cfg3_32k_prefix_and_suffix_independence(G):
 
 
 def test_cfg2_layer_sampled_row_against_the_oracle(G):
-    """d_state 16 (the CUDA-core scan) at B=4, L=4096, d_model 1024."""
+    """d_state 16 (zero-padded to 128 on the tensor-core scan) at B=4, L=4096, d_model 1024."""
     shape, dtype = I.CONFIGS["cfg2_layer"]
     wf, wr = I.make_mixer_weights(shape, 0, dtype)
     x = I.make_activations(shape, 0, dtype)
@@ -86,3 +86,28 @@ def test_cfg4_block_step_sampled_rows_against_the_oracle(G):
         assert G.rel_l2(y[b], y_o[0]) <= BF16_REL and G.max_abs(y[b], y_o[0]) <= BF16_ABS, (b, G.rel_l2(y[b], y_o[0]))
         assert G.rel_l2(ssm_out[b], s_o[0]) <= BF16_REL, (b, G.rel_l2(ssm_out[b], s_o[0]))
         assert G.rel_l2(conv_out[b], c_o[0]) <= BF16_REL, (b, G.rel_l2(conv_out[b], c_o[0]))      # the block's last pre-conv rows, stored in bf16
+
+
+def test_paper_shape_whole_sequence_against_the_oracle(G):
+    """The paper's 1.3B mixer shape (App. A.1 / App. C: d = 1920, 120 heads of 32, d_state 128) at L = 1024: heads of 32
+    channels on the tensor-core scan, every head against the oracle, the last one (whose tile reaches past the x columns)
+    included."""
+    shape, dtype = I.CONFIGS["paper_1p3b"]
+    assert shape.headdim == 32 and shape.n_heads == 120
+    wf, wr = I.make_mixer_weights(shape, 0, dtype)
+    x = I.make_activations(shape, 0, dtype)
+    got = G.run_forward(shape, dtype, wf, wr, x)
+    _check_rows(G, got, x, wf, wr, shape, rows=(0,))
+
+
+def test_cfg3_64k_runs_and_is_deterministic(G):
+    """The longest context of the paper's throughput sweep (Sec. 4.3): finite, run-to-run bit-identical, and the
+    left-to-right layer's first 1024 outputs equal those of the 1024-token call (prefix independence at full length)."""
+    shape, dtype = I.CONFIGS["cfg3_64k"]
+    wf, wr = I.make_mixer_weights(shape, 0, dtype)
+    x = I.make_activations(shape, 0, dtype)
+    a = G.run_forward(shape, dtype, wf, wr, x, dir_mask=1)
+    assert np.all(np.isfinite(a))
+    np.testing.assert_array_equal(a, G.run_forward(shape, dtype, wf, wr, x, dir_mask=1))
+    short = I.MixerShape(1, 1024, shape.d_model, shape.expand, shape.d_state, shape.d_conv, shape.n_heads)
+    np.testing.assert_array_equal(a[:, :1024], G.run_forward(short, dtype, wf, wr, np.ascontiguousarray(x[:, :1024]), dir_mask=1))
