@@ -1,6 +1,6 @@
 """GPU parity of dm_bimamba_forward / dm_bimamba_block_step against the CPU oracle, through the C ABI.
 
-Tolerances (stated by the benchmark spec for this path): fp32 I/O rel-L2 <= 1e-4; bf16 I/O with fp32 accumulation
+Tolerances: fp32 I/O rel-L2 <= 1e-4 (fp32 products and sums in another order than the oracle's fp64); bf16 I/O with fp32 accumulation
 rel-L2 <= 1e-2 and max-abs <= 5e-2; index work (state placement, carried conv rows) bit-exact.
 """
 import numpy as np
