@@ -443,3 +443,28 @@ def noise_schedule(K: int, eps: float = 1e-3):
     (the last step, to eps, still leaves s / t of the masked tokens to a final clean-up pass with keep 0)."""
     t = 1.0 - (1.0 - eps) * np.arange(K + 1) / K
     return t
+
+
+# --------------------------------------------------------------------------------------------
+# Bidirectional multi-head attention mixer of the hybrid variant (Sec. 3.3, App. C Transformer-layer table)
+# --------------------------------------------------------------------------------------------
+def attention_mixer(x, w_qkv, w_o, n_heads: int):
+    """The hybrid's attention mixer: full (non-causal) multi-head self-attention over each sequence, no position
+    encoding.  App. C counts it as QKV and output projections (8 d^2 FLOPs) plus QK^T and Attn.V (4 L d).
+    x [B, L, d]; w_qkv [3 d, d] with rows [Q | K | V], each split into n_heads blocks of d / n_heads;
+    w_o [d, d].  out = concat_h softmax(Q_h K_h^T / sqrt(d_h)) V_h  W_o^T."""
+    x = np.asarray(x, F64)
+    B, L, d = x.shape
+    dh = d // n_heads
+    qkv = x @ np.asarray(w_qkv, F64).T
+    q, k, v = qkv[..., :d], qkv[..., d:2 * d], qkv[..., 2 * d:]
+    out = np.zeros((B, L, d), F64)
+    for b in range(B):
+        for h in range(n_heads):
+            sl = slice(h * dh, (h + 1) * dh)
+            s = q[b, :, sl] @ k[b, :, sl].T / np.sqrt(dh)
+            s = s - s.max(axis=1, keepdims=True)
+            p = np.exp(s)
+            p /= p.sum(axis=1, keepdims=True)
+            out[b, :, sl] = p @ v[b, :, sl]
+    return out @ np.asarray(w_o, F64).T

@@ -580,3 +580,41 @@ def test_noise_schedule_endpoints_and_expected_unmasking():
     np.testing.assert_allclose(np.diff(t), np.diff(t)[0])                  # uniform spacing: K = L / p steps of equal size (Sec. 4.3)
     # the chance that a token is still masked after k steps telescopes to t_k (Eq. 1's marginal: masked w.p. t)
     np.testing.assert_allclose(np.cumprod(t[1:] / t[:-1]), t[1:], rtol=1e-12)
+
+
+# ------------------------------------------------------------------ attention mixer of the hybrid (Sec. 3.3)
+
+def test_attention_mixer_by_loops_and_its_invariances():
+    B, L, d, H = 2, 6, 8, 2
+    dh = d // H
+    x = rng.standard_normal((B, L, d)); wqkv = rng.standard_normal((3 * d, d)) * 0.5; wo = rng.standard_normal((d, d)) * 0.5
+    got = O.attention_mixer(x, wqkv, wo, H)
+    # scalar loops, straight from the definition
+    want = np.zeros((B, L, d))
+    for b in range(B):
+        q = [[sum(wqkv[j, c] * x[b, t, c] for c in range(d)) for j in range(d)] for t in range(L)]
+        k = [[sum(wqkv[d + j, c] * x[b, t, c] for c in range(d)) for j in range(d)] for t in range(L)]
+        v = [[sum(wqkv[2 * d + j, c] * x[b, t, c] for c in range(d)) for j in range(d)] for t in range(L)]
+        for t in range(L):
+            cat = [0.0] * d
+            for h in range(H):
+                sc = [sum(q[t][h * dh + e] * k[u][h * dh + e] for e in range(dh)) / dh ** 0.5 for u in range(L)]
+                m = max(sc); ex = [np.exp(a - m) for a in sc]; z = sum(ex)
+                for e in range(dh):
+                    cat[h * dh + e] = sum(ex[u] / z * v[u][h * dh + e] for u in range(L))
+            for j in range(d):
+                want[b, t, j] = sum(wo[j, c] * cat[c] for c in range(d))
+    np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-12)
+    # no position encoding and no causal mask: permuting the tokens permutes the outputs
+    perm = rng.permutation(L)
+    np.testing.assert_allclose(O.attention_mixer(x[:, perm], wqkv, wo, H), got[:, perm], rtol=1e-11, atol=1e-12)
+    # zero queries: uniform attention, every token receives the mean value vector
+    w0 = wqkv.copy(); w0[:d] = 0
+    vbar = (x @ w0[2 * d:].T).mean(axis=1, keepdims=True)
+    np.testing.assert_allclose(O.attention_mixer(x, w0, wo, H), np.broadcast_to(vbar @ wo.T, (B, L, d)), rtol=1e-11, atol=1e-12)
+    # sequences do not interact; a single token attends to itself: out = W_o V x
+    np.testing.assert_allclose(O.attention_mixer(x[:1], wqkv, wo, H), got[:1], rtol=1e-12)
+    one = x[:, :1]
+    np.testing.assert_allclose(O.attention_mixer(one, wqkv, wo, H), one @ wqkv[2 * d:].T @ wo.T, rtol=1e-11)
+    # the parameter-free part costs 4 L d FLOPs per token and the projections 8 d^2 (App. C, Transformer-layer table)
+    assert 2 * (3 * d) * d + 2 * d * d == 8 * d * d
