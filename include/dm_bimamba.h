@@ -213,6 +213,19 @@ int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
                            int32_t *tokens_out, const dm_layer_state *states,
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The attention mixer of the hybrid variant, Sec. 3.3 (one attention mixer every N mixer blocks): full
+ * (bidirectional, unmasked) multi-head self-attention over each sequence, no position encoding,
+ *     y = concat_h softmax(Q_h K_h^T / sqrt(d_h)) V_h  W_o^T,   [Q | K | V] = x W_qkv^T.
+ * x, y [B, L, d_model] dtype (y != x); w_qkv [3 * d_model, d_model] with rows [Q | K | V], each split into
+ * n_heads consecutive blocks of d_h = d_model / n_heads; w_o [d_model, d_model].  bf16 only, d_h = 64 only
+ * (DM_ERR_UNSUPPORTED otherwise).  The scores never leave the SM (running-maximum softmax over key tiles);
+ * P is rounded to bf16 before P V, accumulation is fp32.  The hybrid stack itself (which layers are attention)
+ * is not assembled by the library. */
+int dm_attention_workspace_bytes(int32_t batch, int32_t seqlen, int32_t d_model, int32_t dtype, size_t *bytes);
+int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t n_heads, int32_t dtype,
+                         const void *w_qkv, const void *w_o, const void *x, void *y,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* One dense projection as the mixer uses it (App. C counts 2mn FLOPs per token for a weight W in R^{m x n}):
  *     y[r, :] = row_scale[r] * (W x[r, :]) + addend[r, :]
  * x [rows, in_features] dtype; w [out_features, in_features] dtype; y [rows, out_features] of y_dtype

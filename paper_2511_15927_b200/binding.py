@@ -93,6 +93,10 @@ _lib.dm_denoise_sample_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_bl
                                         C.POINTER(dm_block_weights), _vp, _vp, C.POINTER(dm_sample_cfg), _vp, _vp, _vp,
                                         C.POINTER(dm_layer_state), _vp, _sz, _vp]
 _lib.dm_denoise_sample_step.restype = C.c_int
+_lib.dm_attention_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(_sz)]
+_lib.dm_attention_workspace_bytes.restype = C.c_int
+_lib.dm_attention_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.dm_attention_forward.restype = C.c_int
 _lib.dm_linear.argtypes = [C.c_int, _vp, _vp, _vp, C.c_int, C.c_int64, C.c_int32, C.c_int32, _vp, _vp, _vp]
 _lib.dm_linear.restype = C.c_int
 _lib.dm_profile_enable.argtypes = [C.c_int]
@@ -104,7 +108,8 @@ for _f in ("dm_profile_enable", "dm_profile_read", "dm_bimamba_workspace_bytes",
 EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count", "dm_bimamba_workspace_bytes",
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
            "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
-           "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step")
+           "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step",
+           "dm_attention_workspace_bytes", "dm_attention_forward")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -227,6 +232,18 @@ def dm_denoise_sample_step(cfg, blk, weights, block_weights, tokens_in: int, tau
     _ok(_lib.dm_denoise_sample_step(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(weights), block_weights,
                                     _vp(tokens_in), _vp(tau or None), C.byref(sample), _vp(u_keep), _vp(u_cat), _vp(tokens_out),
                                     states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_attention_workspace_bytes(batch: int, seqlen: int, d_model: int, dtype: int) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_attention_workspace_bytes(batch, seqlen, d_model, dtype, C.byref(n)))
+    return n.value
+
+
+def dm_attention_forward(batch: int, seqlen: int, d_model: int, n_heads: int, dtype: int, w_qkv: int, w_o: int, x: int, y: int,
+                         workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_attention_forward(batch, seqlen, d_model, n_heads, dtype, _vp(w_qkv), _vp(w_o), _vp(x), _vp(y), _vp(workspace),
+                                  _sz(workspace_bytes), _vp(cuda_stream)))
 
 
 # ------------------------------------------------------------------------------------------------

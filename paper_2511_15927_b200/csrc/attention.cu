@@ -1,0 +1,251 @@
+// Bidirectional multi-head attention for the hybrid variant (Sec. 3.3: one attention mixer every N mixer blocks):
+//     O_h = softmax(Q_h K_h^T / sqrt(d_h)) V_h        full (non-causal), no position encoding, d_h = 64.
+// One CTA per (128-query tile, head, sequence) walks the keys in tiles of 128 with the running-maximum form of the
+// softmax, so the L x L score matrix never leaves the SM:
+//     warp 0      TMA loads: the Q tile once, K and V tiles double-buffered
+//     warp 1      one thread issues  S = Q K^T  (both operands K-major in shared memory, fp32 accumulator in TMEM) and
+//                 O += P V  (A = P from TMEM as bf16, B = V [key][d_h] MN-major)
+//     warps 2-5   one query row per thread: S row -> running max m and sum l, P = 2^(s - m) as bf16 into TMEM, O scaled by
+//                 2^(m_old - m_new) in TMEM; at the end O / l -> bf16 -> global
+// S and P are double-buffered, so the scores of tile j+1 are computed while tile j goes through the softmax.
+// Every wait is bounded; on expiry the CTA stores DM_ERR_TIMEOUT in the device status word and leaves.
+#include "dm_internal.h"
+#include "tc_ptx.cuh"
+
+namespace dm {
+using namespace tc;
+namespace {
+
+constexpr int BQ = 128, BK = 128, DH = 64, NTHREADS = 192;
+constexpr uint32_t TILE = BQ * DH * 2;                      // 16 KB: 128 rows of 128 bytes
+constexpr uint32_t OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_BAR = 5 * TILE, SMEM_BYTES = 5 * TILE + 1024 + 1024;
+constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_P0 = 256, TM_P1 = 320, TM_O = 384, TM_COLS = 512;
+
+struct Bars {
+    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full[2], o_done;
+    uint32_t tmem_base;
+    int abort;
+};
+
+struct AttnArgs {
+    int B, L, d, H;
+    __nv_bfloat16 *out;          // [B*L, d]
+    float scale_log2;            // log2(e) / sqrt(d_h)
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    Bars *bars = reinterpret_cast<Bars *>(smem + OFF_BAR);
+    volatile int *abort_flag = &bars->abort;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int q0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z;
+    const int n_kv = (a.L + BK - 1) / BK;
+
+    if (tid == 0) {
+        mbar_init(&bars->q_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
+            mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
+            mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_empty[i], 128);
+            mbar_init(&bars->p_full[i], 128);
+        }
+        mbar_init(&bars->o_done, 1);
+        bars->abort = 0;
+        mbar_fence_init();
+    }
+    if (warp == 1) tmem_alloc(&bars->tmem_base, TM_COLS);
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    auto WAIT = [&](uint64_t *bar, uint32_t parity) { return mbar_wait(bar, parity, abort_flag, status); };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(&bars->q_full, TILE);
+            tma_load_3d(smem + OFF_Q, &map_qkv, h * DH, q0, b, &bars->q_full);
+            int issued_k = 0, issued_v = 0;
+            for (int j = 0; j < n_kv; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                if (!WAIT(&bars->k_empty[st], ph ^ 1)) break;
+                mbar_expect_tx(&bars->k_full[st], TILE);
+                tma_load_3d(smem + OFF_K + st * TILE, &map_qkv, a.d + h * DH, j * BK, b, &bars->k_full[st]);
+                issued_k = j + 1;
+                if (!WAIT(&bars->v_empty[st], ph ^ 1)) break;
+                mbar_expect_tx(&bars->v_full[st], TILE);
+                tma_load_3d(smem + OFF_V + st * TILE, &map_qkv, 2 * a.d + h * DH, j * BK, b, &bars->v_full[st]);
+                issued_v = j + 1;
+            }
+            if (*abort_flag) {             // aborting: bounded wait for the loads still in flight
+                mbar_wait_quiet(&bars->q_full, 0, 100000000ull);
+                for (int j = max(0, issued_k - 2); j < issued_k; ++j) mbar_wait_quiet(&bars->k_full[j & 1], (j >> 1) & 1, 100000000ull);
+                for (int j = max(0, issued_v - 2); j < issued_v; ++j) mbar_wait_quiet(&bars->v_full[j & 1], (j >> 1) & 1, 100000000ull);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t dQ = desc_lo_k(smem_u32(smem + OFF_Q));
+            constexpr uint32_t I_S = idesc_bf16(128, 128, 0, 0), I_O = idesc_bf16(128, 64, 0, 1);
+            auto issue_pv = [&](int j) -> bool {          // O (+)= P(j) V(j)
+                const int st = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                if (!WAIT(&bars->p_full[st], ph) || !WAIT(&bars->v_full[st], ph)) return false;
+                fence_after();
+                const uint32_t dV = desc_lo_mn(smem_u32(smem + OFF_V + st * TILE), TILE), tp = tmem + (st ? TM_P1 : TM_P0);
+                if (j == 0) umma_ts<0>(tmem + TM_O, tp, dV, I_O); else umma_ts<1>(tmem + TM_O, tp, dV, I_O);
+#pragma unroll
+                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_O, tp + 8 * kk, dV + kk * 128, I_O);
+                umma_commit(&bars->o_done);               // phase j: O holds tiles 0..j; P(j) and the V stage are free
+                umma_commit(&bars->v_empty[st]);
+                return true;
+            };
+            bool ok = WAIT(&bars->q_full, 0);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                if (!WAIT(&bars->k_full[st], ph) || !WAIT(&bars->s_empty[st], ph ^ 1)) { ok = false; break; }
+                fence_after();
+                const uint32_t dK = desc_lo_k(smem_u32(smem + OFF_K + st * TILE)), ts = tmem + (st ? TM_S1 : TM_S0);
+                umma_ss<0>(ts, dQ, dK, I_S);
+#pragma unroll
+                for (int kk = 1; kk < 4; ++kk) umma_ss<1>(ts, dQ + 2 * kk, dK + 2 * kk, I_S);
+                umma_commit(&bars->s_full[st]);
+                umma_commit(&bars->k_empty[st]);
+                if (j > 0) ok = issue_pv(j - 1);
+            }
+            if (ok) issue_pv(n_kv - 1);
+        }
+    } else {
+        // ------------------------------------------------------------ softmax, O scaling, output
+        const int q = warp & 3;                                   // TMEM lane quarter of this warp
+        const int row = q * 32 + lane;                            // query row of the tile
+        const uint32_t tlane = tmem + ((uint32_t)(q * 32) << 16);
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_kv; ++j) {
+            const int st = j & 1;
+            const uint32_t ph = (j >> 1) & 1;
+            ok = ok && WAIT(&bars->s_full[st], ph);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            fence_after();
+            const uint32_t ts = tlane + (st ? TM_S1 : TM_S0), tp = tlane + (st ? TM_P1 : TM_P0);
+            const int valid = min(BK, a.L - j * BK);              // keys of this tile inside the sequence
+            // pass 1: the row maximum of the scaled scores
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BK; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_x32(ts + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) if (c0 + i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
+            }
+            const float m_new = fmaxf(m, mx * a.scale_log2);
+            const float alpha = ex2f(m - m_new);                  // 0 on the first tile (m = -inf)
+            // pass 2: P = 2^(s - m_new) as bf16 into TMEM, and its row sum
+            float sum = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BK; c0 += 32) {
+                uint32_t r[32], pk[16];
+                tmem_ld_x32(ts + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float p0 = c0 + i < valid ? ex2f(fmaf(__uint_as_float(r[i]), a.scale_log2, -m_new)) : 0.f;
+                    const float p1 = c0 + i + 1 < valid ? ex2f(fmaf(__uint_as_float(r[i + 1]), a.scale_log2, -m_new)) : 0.f;
+                    const uint32_t w = pack_bf16(p0, p1);
+                    pk[i >> 1] = w;
+                    sum += bf16_lo(w) + bf16_hi(w);               // the sum of what the product will see
+                }
+                tmem_st_x16(tp + (c0 >> 1), pk);
+            }
+            l = fmaf(l, alpha, sum);
+            m = m_new;
+            fence_before();
+            mbar_arrive(&bars->s_empty[st]);                      // every read of S(j) has completed
+            // O holds tiles 0..j-1 once PV(j-1) has completed: scale it to the new maximum
+            if (j > 0) {
+                ok = WAIT(&bars->o_done, (uint32_t)((j - 1) & 1));
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                fence_after();
+#pragma unroll 1
+                for (int c0 = 0; c0 < DH; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_x32(tlane + TM_O + c0, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                    tmem_st_x32(tlane + TM_O + c0, r);
+                }
+            }
+            tmem_wait_st();
+            fence_before();
+            mbar_arrive(&bars->p_full[st]);
+        }
+        if (ok) {
+            ok = WAIT(&bars->o_done, (uint32_t)((n_kv - 1) & 1));
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            fence_after();
+            const float inv = 1.f / l;
+            const int t = q0 + row;
+#pragma unroll 1
+            for (int c0 = 0; c0 < DH; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_x32(tlane + TM_O + c0, r);
+                tmem_wait_ld();
+                if (t < a.L) {
+                    __nv_bfloat16 *dst = a.out + ((int64_t)b * a.L + t) * a.d + h * DH + c0;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8)
+                        *reinterpret_cast<uint4 *>(dst + i) =
+                            make_uint4(pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv),
+                                       pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv),
+                                       pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv),
+                                       pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv));
+                }
+            }
+        }
+    }
+    // ---------------------------------------------------------------- teardown
+    fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        fence_after();
+        tmem_dealloc(tmem, TM_COLS);
+    }
+}
+
+}  // namespace
+
+bool attention_supports(int dtype, int d, int n_heads) {
+    return dtype == DM_BF16 && n_heads > 0 && d == n_heads * DH && encode_fn() != nullptr;
+}
+
+// qkv [B*L, 3 d] bf16 (columns [Q | K | V], heads contiguous inside each), out [B*L, d] bf16
+cudaError_t attention_forward(const void *qkv, void *out, int B, int L, int d, int n_heads, cudaStream_t s) {
+    if (!attention_supports(DM_BF16, d, n_heads) || B <= 0 || L <= 0 || B > 65535 || n_heads > 65535) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const uint64_t dims[3] = {(uint64_t)3 * d, (uint64_t)L, (uint64_t)B};
+    const uint64_t str[2] = {(uint64_t)3 * d, (uint64_t)L * 3 * d};
+    const uint32_t box[3] = {(uint32_t)DH, (uint32_t)BQ, 1};
+    if (!make_map_bf16(&map, qkv, 3, dims, str, box)) return cudaErrorInvalidValue;
+    int *status = device_status_ptr();
+    if (!status) return cudaErrorUnknown;
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    AttnArgs a{B, L, d, n_heads, static_cast<__nv_bfloat16 *>(out), 1.4426950408889634f / sqrtf((float)DH)};
+    attention_kernel<<<dim3((L + BQ - 1) / BQ, n_heads, B), NTHREADS, SMEM_BYTES, s>>>(map, a, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace dm

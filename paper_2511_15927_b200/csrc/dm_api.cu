@@ -602,6 +602,42 @@ int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
     return denoise_impl(cfg, blk, weights, block_weights, tokens_in, tau, nullptr, nullptr, states, workspace, workspace_bytes, cuda_stream, &smp);
 }
 
+int dm_attention_workspace_bytes(int32_t batch, int32_t seqlen, int32_t d_model, int32_t dtype, size_t *bytes) {
+    if (!bytes || batch <= 0 || seqlen <= 0 || d_model <= 0) return fail(DM_ERR_INVALID_ARG, "sizes must be positive");
+    if (dtype != DM_BF16) return fail(DM_ERR_UNSUPPORTED, "the attention mixer takes bf16 only");
+    *bytes = align_up((size_t)batch * seqlen * 3 * d_model * 2) + align_up((size_t)batch * seqlen * d_model * 2);
+    return DM_OK;
+}
+
+int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t n_heads, int32_t dtype, const void *w_qkv,
+                         const void *w_o, const void *x, void *y, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    size_t need = 0;
+    int st = dm_attention_workspace_bytes(batch, seqlen, d_model, dtype, &need);
+    if (st != DM_OK) return st;
+    if (!w_qkv || !w_o || !x || !y) return fail(DM_ERR_INVALID_ARG, "NULL pointer");
+    if (x == y) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
+    if (!aligned16(w_qkv) || !aligned16(w_o) || !aligned16(x) || !aligned16(y)) return fail(DM_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if (n_heads <= 0 || d_model != n_heads * 64) return fail(DM_ERR_UNSUPPORTED, "the attention mixer needs heads of width 64 (d_model = 64 * n_heads)");
+    if (batch > 65535 || n_heads > 65535) return fail(DM_ERR_UNSUPPORTED, "batch and n_heads must be below 65536");
+    if (!attention_supports(dtype, d_model, n_heads)) return fail(DM_ERR_UNSUPPORTED, "the attention mixer is not available for this configuration");
+    if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t T = (int64_t)batch * seqlen;
+    char *ws = static_cast<char *>(workspace);
+    void *qkv = ws, *att = ws + align_up((size_t)T * 3 * d_model * 2);
+    GemmArgs a{};
+    a.A = x; a.lda = d_model; a.B = w_qkv; a.ldb = d_model; a.C = qkv; a.ldc = 3 * d_model;
+    a.in_dtype = dtype; a.c_dtype = dtype; a.M = (int)T; a.N = 3 * d_model; a.K = d_model;
+    cudaError_t e;
+    if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "qkv projection");
+    if ((e = attention_forward(qkv, att, batch, seqlen, d_model, n_heads, s)) != cudaSuccess) return cuda_fail(e, "attention");
+    GemmArgs o{};
+    o.A = att; o.lda = d_model; o.B = w_o; o.ldb = d_model; o.C = y; o.ldc = d_model;
+    o.in_dtype = dtype; o.c_dtype = dtype; o.M = (int)T; o.N = d_model; o.K = d_model;
+    if ((e = gemm(o, s)) != cudaSuccess) return cuda_fail(e, "attention output projection");
+    return DM_OK;
+}
+
 int dm_linear(int dtype, const void *x, const void *w, void *y, int y_dtype, int64_t rows, int32_t in_features,
               int32_t out_features, const float *row_scale, const float *addend, void *cuda_stream) {
     if ((dtype != DM_F32 && dtype != DM_BF16) || (y_dtype != DM_F32 && y_dtype != DM_BF16)) return fail(DM_ERR_INVALID_ARG, "bad dtype");

@@ -72,6 +72,11 @@ bool scan_ssd_supports(const ScanArgs &a);
 size_t scan_ssd_workspace_bytes(const ScanArgs &a);
 cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s);
 
+// Bidirectional multi-head attention over qkv [B*L, 3 d] (columns [Q | K | V], heads contiguous inside each) -> out [B*L, d];
+// bf16, head width 64.
+bool attention_supports(int dtype, int d, int n_heads);
+cudaError_t attention_forward(const void *qkv, void *out, int B, int L, int d, int n_heads, cudaStream_t s);
+
 // ---------------------------------------------------------------------------------------------
 // Small row-wise kernels
 // ---------------------------------------------------------------------------------------------
