@@ -468,3 +468,23 @@ def attention_mixer(x, w_qkv, w_o, n_heads: int):
             p /= p.sum(axis=1, keepdims=True)
             out[b, :, sl] = p @ v[b, :, sl]
     return out @ np.asarray(w_o, F64).T
+
+
+def denoise_step_hybrid(tokens, sw: dict, *, attn_period: int, attn_heads: int, tau=None, rms_eps: float = 1e-5,
+                        ln_eps: float = 1e-5, **kw):
+    """The hybrid stack (Sec. 3.3, App. A.3): the mixer of layer i is the attention mixer when i is a multiple of
+    attn_period (one attention mixer followed by attn_period - 1 bidirectional Mamba mixers; the paper uses 5), the
+    bidirectional Mamba mixer otherwise.  tau None: RMSNorm pre-norm + mixer + residual per layer; tau given: the
+    timestep-conditioned block around either mixer.  Attention layers carry "w_qkv" and "w_o"."""
+    r = np.asarray(sw["embed"], F64)[np.asarray(tokens)]
+    for i, layer in enumerate(sw["layers"]):
+        is_attn = attn_period > 0 and i % attn_period == 0
+        mix = (lambda u: attention_mixer(u, layer["w_qkv"], layer["w_o"], attn_heads)) if is_attn else \
+              (lambda u: bimamba_forward(u, layer["fwd"], layer["rev"], **kw))
+        if tau is None:
+            r = r + mix(rmsnorm(r, layer["norm_w"], rms_eps))
+        else:
+            b1, s1, g1, b2, s2, g2 = modulation(tau, layer["w_cond"], layer.get("b_cond"))
+            y = r + g1[:, None, :] * mix(adaln(r, s1, b1, ln_eps))
+            r = y + g2[:, None, :] * mlp(adaln(y, s2, b2, ln_eps), layer["w_up"], layer["w_down"], layer.get("b_up"), layer.get("b_down"))
+    return rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T

@@ -618,3 +618,29 @@ def test_attention_mixer_by_loops_and_its_invariances():
     np.testing.assert_allclose(O.attention_mixer(one, wqkv, wo, H), one @ wqkv[2 * d:].T @ wo.T, rtol=1e-11)
     # the parameter-free part costs 4 L d FLOPs per token and the projections 8 d^2 (App. C, Transformer-layer table)
     assert 2 * (3 * d) * d + 2 * d * d == 8 * d * d
+
+
+def test_hybrid_stack_places_attention_every_period_layers():
+    d, H_attn = 6, 2
+    sw, tau = _tiny_cond_stack(n_layers=6, d=d)
+    r = np.random.default_rng(77)
+    for l in sw["layers"]:
+        l["w_qkv"] = r.standard_normal((3 * d, d)) * 0.3; l["w_o"] = r.standard_normal((d, d)) * 0.3
+    tok = rng.integers(0, 11, (2, 5))
+    # period 0: no attention anywhere = the plain stacks
+    np.testing.assert_allclose(O.denoise_step_hybrid(tok, sw, attn_period=0, attn_heads=H_attn, **KW), O.denoise_step(tok, sw, **KW), rtol=1e-12)
+    np.testing.assert_allclose(O.denoise_step_hybrid(tok, sw, attn_period=0, attn_heads=H_attn, tau=tau, **KW),
+                               O.denoise_step_cond(tok, tau, sw, **KW), rtol=1e-12)
+    # period 5 on 6 layers: layers 0 and 5 are attention (1 attention + 4 Mamba, repeated); rebuilt layer by layer
+    x = sw["embed"][tok]
+    for i, l in enumerate(sw["layers"]):
+        u = O.rmsnorm(x, l["norm_w"])
+        x = x + (O.attention_mixer(u, l["w_qkv"], l["w_o"], H_attn) if i in (0, 5) else O.bimamba_forward(u, l["fwd"], l["rev"], **KW))
+    np.testing.assert_allclose(O.denoise_step_hybrid(tok, sw, attn_period=5, attn_heads=H_attn, **KW),
+                               O.rmsnorm(x, sw["final_norm_w"]) @ sw["w_vocab"].T, rtol=1e-11)
+    # Mamba weights of an attention layer are not used, and vice versa
+    sw2 = {**sw, "layers": [dict(l) for l in sw["layers"]]}
+    sw2["layers"][0]["fwd"] = {**sw2["layers"][0]["fwd"], "w_out": 0 * sw2["layers"][0]["fwd"]["w_out"]}
+    sw2["layers"][1]["w_o"] = 0 * sw2["layers"][1]["w_o"]
+    np.testing.assert_array_equal(O.denoise_step_hybrid(tok, sw2, attn_period=5, attn_heads=H_attn, tau=tau, **KW),
+                                  O.denoise_step_hybrid(tok, sw, attn_period=5, attn_heads=H_attn, tau=tau, **KW))
