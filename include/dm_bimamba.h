@@ -226,6 +226,28 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
                          const void *w_qkv, const void *w_o, const void *x, void *y,
                          void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The hybrid stack, Sec. 3.3 / App. A.3: layer l uses the attention mixer when l is a multiple of attn_period
+ * (one attention mixer followed by attn_period - 1 bidirectional Mamba mixers; the paper fixes 5) and the
+ * bidirectional Mamba mixer otherwise; attn_period = 0 means no attention layer.  Around either mixer the layer is
+ * the RMSNorm pre-norm + residual of dm_denoise_step (blk == NULL) or the timestep-conditioned block of
+ * dm_denoise_step_cond (blk, block_weights, tau given).  attn_weights: HOST array of cfg->n_layers entries, read
+ * only where the layer is attention (the Mamba weights of those layers are not read).  Full-sequence mode only:
+ * block mode would need a key/value cache for the attention layers.  bf16, attention heads of width 64. */
+typedef struct {
+    int32_t attn_period;   /* N: layers 0, N, 2N, ... are attention; 0 = none */
+    int32_t attn_heads;    /* d_model = 64 * attn_heads */
+} dm_hybrid_cfg;
+typedef struct {
+    const void *w_qkv;     /* [3 * d_model, d_model] dtype, rows [Q | K | V] */
+    const void *w_o;       /* [d_model, d_model] dtype */
+} dm_attn_weights;
+int dm_denoise_hybrid_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes);
+int dm_denoise_step_hybrid(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_hybrid_cfg *hybrid,
+                           const dm_stack_weights *weights, const dm_block_weights *block_weights,
+                           const dm_attn_weights *attn_weights, const int32_t *tokens, const float *tau,
+                           void *logits, int32_t *argmax_out,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* One dense projection as the mixer uses it (App. C counts 2mn FLOPs per token for a weight W in R^{m x n}):
  *     y[r, :] = row_scale[r] * (W x[r, :]) + addend[r, :]
  * x [rows, in_features] dtype; w [out_features, in_features] dtype; y [rows, out_features] of y_dtype

@@ -51,6 +51,14 @@ class dm_block_cfg(C.Structure):
     _fields_ = [("d_ff", C.c_int32), ("d_cond", C.c_int32), ("ln_eps", C.c_float)]
 
 
+class dm_hybrid_cfg(C.Structure):
+    _fields_ = [("attn_period", C.c_int32), ("attn_heads", C.c_int32)]
+
+
+class dm_attn_weights(C.Structure):
+    _fields_ = [("w_qkv", C.c_void_p), ("w_o", C.c_void_p)]
+
+
 class dm_sample_cfg(C.Structure):
     _fields_ = [("mask_id", C.c_int32), ("vocab_real", C.c_int32), ("keep_prob", C.c_float)]
 
@@ -93,6 +101,11 @@ _lib.dm_denoise_sample_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_bl
                                         C.POINTER(dm_block_weights), _vp, _vp, C.POINTER(dm_sample_cfg), _vp, _vp, _vp,
                                         C.POINTER(dm_layer_state), _vp, _sz, _vp]
 _lib.dm_denoise_sample_step.restype = C.c_int
+_lib.dm_denoise_hybrid_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(_sz)]
+_lib.dm_denoise_hybrid_workspace_bytes.restype = C.c_int
+_lib.dm_denoise_step_hybrid.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_hybrid_cfg), C.POINTER(dm_stack_weights),
+                                        C.POINTER(dm_block_weights), C.POINTER(dm_attn_weights), _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.dm_denoise_step_hybrid.restype = C.c_int
 _lib.dm_attention_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(_sz)]
 _lib.dm_attention_workspace_bytes.restype = C.c_int
 _lib.dm_attention_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -109,7 +122,7 @@ EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count"
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
            "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
            "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step",
-           "dm_attention_workspace_bytes", "dm_attention_forward")
+           "dm_attention_workspace_bytes", "dm_attention_forward", "dm_denoise_hybrid_workspace_bytes", "dm_denoise_step_hybrid")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -234,6 +247,20 @@ def dm_denoise_sample_step(cfg, blk, weights, block_weights, tokens_in: int, tau
                                     states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
 
 
+def dm_denoise_hybrid_workspace_bytes(cfg: dm_stack_cfg, blk=None) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_denoise_hybrid_workspace_bytes(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(n)))
+    return n.value
+
+
+def dm_denoise_step_hybrid(cfg, blk, hybrid: dm_hybrid_cfg, weights, block_weights, attn_weights, tokens: int, tau: int, logits: int,
+                           argmax_out: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    """attn_weights: ctypes array (dm_attn_weights * n_layers); blk / block_weights / tau: None (0) for the plain stack."""
+    _ok(_lib.dm_denoise_step_hybrid(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(hybrid), C.byref(weights),
+                                    block_weights, attn_weights, _vp(tokens), _vp(tau or None), _vp(logits or None),
+                                    _vp(argmax_out or None), _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
 def dm_attention_workspace_bytes(batch: int, seqlen: int, d_model: int, dtype: int) -> int:
     n = _sz(0)
     _ok(_lib.dm_attention_workspace_bytes(batch, seqlen, d_model, dtype, C.byref(n)))
@@ -283,4 +310,13 @@ def make_block_weights(layers):
     for i, l in enumerate(layers):
         arr[i] = dm_block_weights(*[(l[n].data_ptr() if l.get(n) is not None else None)
                                     for n in ("w_cond", "b_cond", "w_up", "b_up", "w_down", "b_down")])
+    return arr
+
+
+def make_attn_weights(layers):
+    """layers: list of {"w_qkv", "w_o"} of device tensors, or None for layers that are not attention."""
+    arr = (dm_attn_weights * len(layers))()
+    for i, l in enumerate(layers):
+        if l is not None:
+            arr[i] = dm_attn_weights(l["w_qkv"].data_ptr(), l["w_o"].data_ptr())
     return arr

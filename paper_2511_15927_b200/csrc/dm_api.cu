@@ -230,11 +230,11 @@ static int check_ws(const void *ws, size_t have, size_t need) {
 }
 
 struct StackWs {
-    size_t r, u, logits, mixer, mod, hmid, idx, count, ug, total;
+    size_t r, u, logits, mixer, mod, hmid, idx, count, ug, qkv, att, total;
     int logits_rows;
 };
 
-static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg *blk = nullptr, bool sampler = false) {
+static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg *blk = nullptr, bool sampler = false, bool hybrid = false) {
     StackWs w;
     size_t off = 0;
     w.r = off; off += align_up((size_t)m.T * m.d * sizeof(float));
@@ -252,6 +252,11 @@ static StackWs stack_ws(const dm_stack_cfg *c, const Dims &m, const dm_block_cfg
         w.idx = off; off += align_up((size_t)m.T * sizeof(int32_t));
         w.count = off; off += align_up(sizeof(int));
         w.ug = off; off += align_up((size_t)m.T * m.d * m.es);
+    }
+    w.qkv = w.att = off;
+    if (hybrid) {
+        w.qkv = off; off += align_up((size_t)m.T * 3 * m.d * m.es);
+        w.att = off; off += align_up((size_t)m.T * m.d * m.es);
     }
     w.total = off;
     return w;
@@ -426,11 +431,14 @@ int dm_bimamba_block_step(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], co
 struct SampleArgs {
     const dm_sample_cfg *cfg; const float *u_keep, *u_cat; int32_t *tokens_out;
 };
+struct HybridArgs {
+    const dm_hybrid_cfg *cfg; const dm_attn_weights *aw;      // aw: HOST array of n_layers entries (used where the layer is attention)
+};
 
 static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights, const dm_block_weights *bw,
                         const int32_t *tokens, const float *tau, void *logits,
                         int32_t *argmax_out, const dm_layer_state *states, void *workspace, size_t workspace_bytes,
-                        void *cuda_stream, const SampleArgs *smp = nullptr) {
+                        void *cuda_stream, const SampleArgs *smp = nullptr, const HybridArgs *hyb = nullptr) {
     Dims m;
     if (!cfg || !weights) return fail(DM_ERR_INVALID_ARG, "cfg or weights is NULL");
     int st = check_cfg(&cfg->mixer, &m);
@@ -465,8 +473,22 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
                 return fail(DM_ERR_INVALID_ARG, "layer %d: block weights must be 16-byte aligned", i);
         }
     }
+    const int period = hyb ? hyb->cfg->attn_period : 0;
+    if (hyb) {
+        if (!hyb->cfg || !hyb->aw) return fail(DM_ERR_INVALID_ARG, "hybrid configuration or attention weights are NULL");
+        if (period < 0) return fail(DM_ERR_INVALID_ARG, "attn_period must be >= 0");
+        if (period > 0) {
+            if (states) return fail(DM_ERR_UNSUPPORTED, "block mode needs a key/value cache for the attention layers, which is not built");
+            if (hyb->cfg->attn_heads <= 0 || m.d != 64 * hyb->cfg->attn_heads || !attention_supports(cfg->mixer.dtype, m.d, hyb->cfg->attn_heads))
+                return fail(DM_ERR_UNSUPPORTED, "attention layers need bf16 and heads of width 64 (d_model = 64 * attn_heads)");
+            for (int i = 0; i < cfg->n_layers; i += period)
+                if (!hyb->aw[i].w_qkv || !hyb->aw[i].w_o || !aligned16(hyb->aw[i].w_qkv) || !aligned16(hyb->aw[i].w_o))
+                    return fail(DM_ERR_INVALID_ARG, "layer %d: attention weights must be non-NULL and 16-byte aligned", i);
+        }
+    }
     for (int i = 0; i < cfg->n_layers; ++i) {
         if (!blk && !weights->layers[i].norm_w) return fail(DM_ERR_INVALID_ARG, "layer %d: norm_w is NULL", i);
+        if (period > 0 && i % period == 0) continue;          // an attention layer: its Mamba weights are not read
         if ((st = check_weights(&cfg->mixer, weights->layers[i].dir)) != DM_OK) return st;
         if (states) {
             const dm_layer_state &q = states[i];
@@ -478,7 +500,7 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
                 return fail(DM_ERR_INVALID_ARG, "state_out needs the left-to-right direction");
         }
     }
-    const StackWs l = stack_ws(cfg, m, blk, smp != nullptr);
+    const StackWs l = stack_ws(cfg, m, blk, smp != nullptr, period > 0);
     if ((st = check_ws(workspace, workspace_bytes, l.total)) != DM_OK) return st;
     char *ws = static_cast<char *>(workspace);
     float *r = reinterpret_cast<float *>(ws + l.r);
@@ -500,10 +522,25 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
         } else {
             if ((e = rmsnorm_rows(r, lw.norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "rmsnorm");
         }
-        const dm_layer_state *q = states ? &states[i] : nullptr;
-        st = run_mixer(&cfg->mixer, m, lw.dir, u, out, q ? q->ssm_in : nullptr, q ? q->conv_in : nullptr,
-                       q ? q->ssm_out : nullptr, q ? q->conv_out : nullptr, ws + l.mixer, s);
-        if (st != DM_OK) return st;
+        if (period > 0 && i % period == 0) {
+            // attention mixer (Sec. 3.3): r <- r + [gate *] Attn(u); gate and residual ride in the output projection's epilogue
+            void *qkv = ws + l.qkv, *att = ws + l.att;
+            GemmArgs a{};
+            a.A = u; a.lda = m.d; a.B = hyb->aw[i].w_qkv; a.ldb = m.d; a.C = qkv; a.ldc = 3 * m.d;
+            a.in_dtype = dtype; a.c_dtype = dtype; a.M = (int)m.T; a.N = 3 * m.d; a.K = m.d;
+            if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "qkv projection");
+            if ((e = attention_forward(qkv, att, m.B, m.L, m.d, hyb->cfg->attn_heads, s)) != cudaSuccess) return cuda_fail(e, "attention");
+            GemmArgs o{};
+            o.A = att; o.lda = m.d; o.B = hyb->aw[i].w_o; o.ldb = m.d; o.C = r; o.ldc = m.d;
+            o.in_dtype = dtype; o.c_dtype = DM_F32; o.M = (int)m.T; o.N = m.d; o.K = m.d;
+            o.addend = r; o.ld_add = m.d; o.col_scale = out.col_scale; o.cs_rows = out.cs_rows; o.ld_cs = out.ld_cs;
+            if ((e = gemm(o, s)) != cudaSuccess) return cuda_fail(e, "attention output projection");
+        } else {
+            const dm_layer_state *q = states ? &states[i] : nullptr;
+            st = run_mixer(&cfg->mixer, m, lw.dir, u, out, q ? q->ssm_in : nullptr, q ? q->conv_in : nullptr,
+                           q ? q->ssm_out : nullptr, q ? q->conv_out : nullptr, ws + l.mixer, s);
+            if (st != DM_OK) return st;
+        }
         if (blk) {
             // r <- r + gate2 * (W_down GELU(W_up AdaLN(r) + b_up) + b_down): activation, bias, gate and residual ride in the epilogues
             if ((e = adaln_rows(r, mod + 4 * m.d, mod + 3 * m.d, ldm, u, dtype, (int)m.T, m.L, m.d, blk->ln_eps, s)) != cudaSuccess) return cuda_fail(e, "adaln");
@@ -600,6 +637,26 @@ int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
                            const dm_layer_state *states, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     const SampleArgs smp{sample, u_keep, u_cat, tokens_out};
     return denoise_impl(cfg, blk, weights, block_weights, tokens_in, tau, nullptr, nullptr, states, workspace, workspace_bytes, cuda_stream, &smp);
+}
+
+int dm_denoise_hybrid_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes) {
+    Dims m;
+    if (!cfg || !bytes) return fail(DM_ERR_INVALID_ARG, "NULL argument");
+    int st = check_cfg(&cfg->mixer, &m);
+    if (st != DM_OK) return st;
+    if (cfg->vocab <= 0 || (blk && blk->d_ff <= 0)) return fail(DM_ERR_INVALID_ARG, "vocab and d_ff must be positive");
+    *bytes = stack_ws(cfg, m, blk, false, true).total;
+    return DM_OK;
+}
+
+int dm_denoise_step_hybrid(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_hybrid_cfg *hybrid,
+                           const dm_stack_weights *weights, const dm_block_weights *block_weights,
+                           const dm_attn_weights *attn_weights, const int32_t *tokens, const float *tau, void *logits,
+                           int32_t *argmax_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!hybrid) return fail(DM_ERR_INVALID_ARG, "hybrid configuration is NULL");
+    const HybridArgs hyb{hybrid, attn_weights};
+    return denoise_impl(cfg, blk, weights, block_weights, tokens, tau, logits, argmax_out, nullptr, workspace, workspace_bytes, cuda_stream,
+                        nullptr, &hyb);
 }
 
 int dm_attention_workspace_bytes(int32_t batch, int32_t seqlen, int32_t d_model, int32_t dtype, size_t *bytes) {

@@ -147,3 +147,28 @@ def run_sample_step(shape, dtype, sw, tokens, vocab, u_keep, u_cat, keep_prob, m
                               ws.data_ptr(), nb, st)
     dm.dm_check(st)
     return out.cpu().numpy()
+
+
+def run_denoise_hybrid(shape, dtype, sw, tokens, vocab, attn_period, attn_heads, tau=None, d_ff=0, rms_eps=1e-5, ln_eps=1e-5):
+    """dm_denoise_step_hybrid on host arrays; layers of sw that are attention carry "w_qkv" and "w_o".  Returns logits."""
+    n_layers = len(sw["layers"])
+    scfg = dm.dm_stack_cfg(cfg_of(shape, dtype), n_layers, vocab, rms_eps)
+    dsw = dev_stack_weights(sw, dtype)
+    csw, keep = dm.make_stack_weights(dsw)
+    blk = cbw = taud = None
+    if tau is not None:
+        blk = dm.dm_block_cfg(d_ff, tau.shape[1], ln_eps)
+        dbw = dev_block_weights(sw, dtype)
+        cbw = dm.make_block_weights(dbw)
+        taud = dev(np.asarray(tau, np.float32))
+    daw = [({"w_qkv": dev(l["w_qkv"], dtype), "w_o": dev(l["w_o"], dtype)} if "w_qkv" in l else None) for l in sw["layers"]]
+    caw = dm.make_attn_weights(daw)
+    tok = dev(np.asarray(tokens, np.int32))
+    logits = torch.empty((shape.batch, shape.seqlen, vocab), device="cuda", dtype=tdtype(dtype))
+    nb = dm.dm_denoise_hybrid_workspace_bytes(scfg, blk)
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_denoise_step_hybrid(scfg, blk, dm.dm_hybrid_cfg(attn_period, attn_heads), csw, cbw, caw, tok.data_ptr(),
+                              taud.data_ptr() if taud is not None else 0, logits.data_ptr(), 0, ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    return logits.float().cpu().numpy().astype(np.float64)

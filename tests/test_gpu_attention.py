@@ -82,3 +82,35 @@ def test_attention_argument_checks(G):
     with pytest.raises(dm.DmError):
         _run(G, x, wq, wo, 4)                                # heads of width 32: unsupported
     assert dm.dm_kernel_launch_count() == before
+
+
+def _hybrid_stack(shape, layers, V, seed, cond):
+    sw = I.make_stack_weights(shape, layers, V, seed=seed, dtype=I.BF16, perturb=True)
+    d = shape.d_model
+    r = np.random.default_rng(seed)
+    for i, l in enumerate(sw["layers"]):
+        l["w_qkv"] = I.round_to_bf16((1.0 / np.sqrt(d)) * r.standard_normal((3 * d, d), dtype=np.float32))
+        l["w_o"] = I.round_to_bf16((0.5 / np.sqrt(d)) * r.standard_normal((d, d), dtype=np.float32))
+    tau, d_ff = None, 0
+    if cond:
+        d_ff = 2 * d
+        I.add_block_weights(sw, shape, d_ff, 32, seed=seed, dtype=I.BF16)
+        tau = I.make_timestep_embedding(shape.batch, 32, seed=seed)
+    return sw, tau, d_ff
+
+
+@pytest.mark.parametrize("cond", [False, True])
+def test_hybrid_stack_against_the_oracle(G, cond):
+    """Attention mixer in layers 0 and 3 of a 5-layer stack (period 3), bidirectional Mamba elsewhere."""
+    shape = I.MixerShape(2, 150, 128, 2, 128, 4, 4)          # d_model 128 = 2 attention heads of 64
+    V = 504
+    sw, tau, d_ff = _hybrid_stack(shape, 5, V, 21, cond)
+    tok = I.make_tokens(2, 150, V - 1, V - 1, seed=21)
+    want = O.denoise_step_hybrid(tok, sw, attn_period=3, attn_heads=2, tau=tau, **G.oracle_kwargs(shape))
+    got = G.run_denoise_hybrid(shape, I.BF16, sw, tok, V, 3, 2, tau=tau, d_ff=d_ff)
+    assert np.all(np.isfinite(got))
+    assert G.rel_l2(got, want) <= 1e-2, G.rel_l2(got, want)
+    # period 0: no attention layer; identical to the stack without the hybrid entry point
+    plain, _, _ = G.run_denoise(shape, I.BF16, sw, tok, V, want_argmax=False, tau=tau, d_ff=d_ff)
+    np.testing.assert_array_equal(G.run_denoise_hybrid(shape, I.BF16, sw, tok, V, 0, 2, tau=tau, d_ff=d_ff), plain)
+    assert np.any(got != plain)
