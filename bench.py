@@ -169,11 +169,13 @@ STACKS = {
     # one reverse step of the masked diffusion (Sec. 2, Eq. 3) on the cfg 2 stack, mid-generation: half of the positions
     # masked, p = 16 of them drawn per sequence and step (K = L / p steps per generation, Sec. 4.3)
     "cfg2_sample": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, sample=dict(p=16)),
+    # the hybrid of Sec. 3.3 on the cfg 2 stack: attention mixer in layers 0, 5, 10, 15, 20 (16 heads of 64), Mamba elsewhere
+    "cfg2_stack_hybrid": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, hybrid=dict(period=5, heads=16)),
     "cfg2_stack_cond": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, cond=dict(d_ff=2048, d_cond=128)),
 }
 
 
-def device_stack_weights(torch, shape, layers, vocab, seed=0, cond=None):
+def device_stack_weights(torch, shape, layers, vocab, seed=0, cond=None, hybrid=None):
     """Random-init bf16 weights of a stack, drawn on the device with the distributions of inputs.py (the host
     generator would take minutes at these sizes).  Returns the dict layout make_stack_weights() of the binding takes."""
     g = torch.Generator(device="cuda").manual_seed(seed)
@@ -206,6 +208,11 @@ def device_stack_weights(torch, shape, layers, vocab, seed=0, cond=None):
                       for _ in range(layers)]}
     if cond:
         out["blocks"] = [block() for _ in range(layers)]
+    if hybrid:
+        d = s.d_model
+        out["attn"] = [({"w_qkv": (torch.randn(3 * d, d, generator=g, device="cuda") / d ** 0.5).to(bf),
+                         "w_o": (0.5 * torch.randn(d, d, generator=g, device="cuda") / d ** 0.5).to(bf)} if i % hybrid["period"] == 0 else None)
+                       for i in range(layers)]
     return out
 
 
@@ -226,7 +233,8 @@ def run_stack(args, rank, local_rank, world):
     shape, layers, vocab, prefix = spec["shape"], spec["layers"], spec["vocab"], spec.get("prefix")
     B, Lb = shape.batch, shape.seqlen
     cond = spec.get("cond")
-    w = device_stack_weights(torch, shape, layers, vocab, cond=cond)
+    hyb = spec.get("hybrid")
+    w = device_stack_weights(torch, shape, layers, vocab, cond=cond, hybrid=hyb)
     csw, keep = dm.make_stack_weights(w)
     stream = torch.cuda.current_stream().cuda_stream
     if cond:
@@ -242,13 +250,22 @@ def run_stack(args, rank, local_rank, world):
         u_keep = torch.rand(B, Lb, generator=gen, device="cuda")
         u_cat = torch.rand(B, Lb, generator=gen, device="cuda")
 
+    if hyb:
+        hcfg = dm.dm_hybrid_cfg(hyb["period"], hyb["heads"])
+        caw = dm.make_attn_weights(w["attn"])
+
     def ws_bytes(cfg):
+        if hyb:
+            return dm.dm_denoise_hybrid_workspace_bytes(cfg, blk if cond else None)
         if smp:
             return dm.dm_denoise_sample_workspace_bytes(cfg, blk if cond else None)
         return dm.dm_denoise_cond_workspace_bytes(cfg, blk) if cond else dm.dm_denoise_workspace_bytes(cfg)
 
     def denoise(cfg, tok_ptr, amax_ptr, st):
-        if smp:
+        if hyb:
+            dm.dm_denoise_step_hybrid(cfg, blk if cond else None, hcfg, csw, cbw if cond else None, caw, tok_ptr, tau.data_ptr() if cond else 0,
+                                      0, amax_ptr, ws.data_ptr(), ws.numel(), stream)
+        elif smp:
             dm.dm_denoise_sample_step(cfg, blk if cond else None, csw, cbw if cond else None, tok_ptr, tau.data_ptr() if cond else 0, scfg_s,
                                       u_keep.data_ptr(), u_cat.data_ptr(), amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
         elif cond:
@@ -361,6 +378,7 @@ def run_stack(args, rank, local_rank, world):
     inp = stage_ms[dm.DM_STAGE_IN_PROJ] / n_calls
     scn = stage_ms[dm.DM_STAGE_SCAN] / n_calls
     outp = stage_ms[dm.DM_STAGE_OUT_PROJ] / n_calls
+    n_mamba = layers - ((layers + hyb["period"] - 1) // hyb["period"] if hyb else 0)      # the other layers are attention
     f_in, f_out = gemm_flops_per_token(shape)
     in_tf, out_tf = f_in * T / (inp * 1e-3) / 1e12, f_out * T / (outp * 1e-3) / 1e12
     scan_bytes = scan_bytes_per_token(shape, 2) * T
@@ -369,7 +387,7 @@ def run_stack(args, rank, local_rank, world):
     scan_gbs = scan_bytes / (scn * 1e-3) / 1e9
     kernels = {"in_proj_per_layer": {"ms": inp, "tflops": in_tf}, "scan_per_layer": {"ms": scn, "gbs": scan_gbs},
                "out_proj_per_layer": {"ms": outp, "tflops": out_tf},
-               "rest_of_step_ms": ms_step - layers * (inp + scn + outp)}
+               "rest_of_step_ms": ms_step - n_mamba * (inp + scn + outp)}
     if scn >= max(inp, outp):
         roofline = {"kernel": "fused conv+scan+gate (per layer)", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": scan_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
@@ -385,6 +403,8 @@ def run_stack(args, rank, local_rank, world):
                             "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T / (ms_step * 1e-3),
                             "parallelism": "replicas only" if world > 1 else "1 GPU",
                             "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
+                           **({"hybrid": "attention mixer (%d heads of 64) in every %dth layer, %d Mamba layers; the attention layers are inside rest_of_step_ms"
+                                         % (hyb["heads"], hyb["period"], n_mamba)} if hyb else {}),
                            **({"sample": "half of the positions masked, p = %d drawn per sequence and step" % smp["p"],
                                "generated_tokens_per_s_at_K_eq_L_over_p": world * T / ((Lb // smp["p"]) * ms_step * 1e-3)} if smp else {}),
                            **extra),
