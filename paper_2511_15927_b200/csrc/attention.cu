@@ -7,7 +7,8 @@
 //                 O += P V  (A = P from TMEM as bf16, B = V [key][d_h] MN-major)
 //     warps 2-5   one query row per thread: S row -> running max m and sum l, P = 2^(s - m) as bf16 into TMEM, O scaled by
 //                 2^(m_old - m_new) in TMEM; at the end O / l -> bf16 -> global
-// S and P are double-buffered, so the scores of tile j+1 are computed while tile j goes through the softmax.
+// A CTA holds 256 TMEM columns (S 128, P 64, O 64) and 82 KB of shared memory, so two CTAs share an SM: while one is in
+// its softmax (latency bound: one warp per scheduler), the other one's products and softmax fill the gaps.
 // Every wait is bounded; on expiry the CTA stores DM_ERR_TIMEOUT in the device status word and leaves.
 #include "dm_internal.h"
 #include "tc_ptx.cuh"
@@ -19,10 +20,10 @@ namespace {
 constexpr int BQ = 128, BK = 128, DH = 64, NTHREADS = 192;
 constexpr uint32_t TILE = BQ * DH * 2;                      // 16 KB: 128 rows of 128 bytes
 constexpr uint32_t OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_BAR = 5 * TILE, SMEM_BYTES = 5 * TILE + 1024 + 1024;
-constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_P0 = 256, TM_P1 = 320, TM_O = 384, TM_COLS = 512;
+constexpr uint32_t TM_S = 0, TM_P = 128, TM_O = 192, TM_COLS = 256;      // S fp32 128 columns, P bf16 64, O fp32 64
 
 struct Bars {
-    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full[2], o_done;
+    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full, s_empty, p_full, o_done;
     uint32_t tmem_base;
     int abort;
 };
@@ -33,7 +34,7 @@ struct AttnArgs {
     float scale_log2;            // log2(e) / sqrt(d_h)
 };
 
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(NTHREADS, 2)
 attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -48,9 +49,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
             mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
-            mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_empty[i], 128);
-            mbar_init(&bars->p_full[i], 128);
         }
+        mbar_init(&bars->s_full, 1); mbar_init(&bars->s_empty, 128);
+        mbar_init(&bars->p_full, 128);
         mbar_init(&bars->o_done, 1);
         bars->abort = 0;
         mbar_fence_init();
@@ -94,9 +95,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
             auto issue_pv = [&](int j) -> bool {          // O (+)= P(j) V(j)
                 const int st = j & 1;
                 const uint32_t ph = (j >> 1) & 1;
-                if (!WAIT(&bars->p_full[st], ph) || !WAIT(&bars->v_full[st], ph)) return false;
+                if (!WAIT(&bars->p_full, (uint32_t)(j & 1)) || !WAIT(&bars->v_full[st], ph)) return false;
                 fence_after();
-                const uint32_t dV = desc_lo_mn(smem_u32(smem + OFF_V + st * TILE), TILE), tp = tmem + (st ? TM_P1 : TM_P0);
+                const uint32_t dV = desc_lo_mn(smem_u32(smem + OFF_V + st * TILE), TILE), tp = tmem + TM_P;
                 if (j == 0) umma_ts<0>(tmem + TM_O, tp, dV, I_O); else umma_ts<1>(tmem + TM_O, tp, dV, I_O);
 #pragma unroll
                 for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_O, tp + 8 * kk, dV + kk * 128, I_O);
@@ -108,13 +109,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int st = j & 1;
                 const uint32_t ph = (j >> 1) & 1;
-                if (!WAIT(&bars->k_full[st], ph) || !WAIT(&bars->s_empty[st], ph ^ 1)) { ok = false; break; }
+                if (!WAIT(&bars->k_full[st], ph) || !WAIT(&bars->s_empty, (uint32_t)((j & 1) ^ 1))) { ok = false; break; }
                 fence_after();
-                const uint32_t dK = desc_lo_k(smem_u32(smem + OFF_K + st * TILE)), ts = tmem + (st ? TM_S1 : TM_S0);
+                const uint32_t dK = desc_lo_k(smem_u32(smem + OFF_K + st * TILE)), ts = tmem + TM_S;
                 umma_ss<0>(ts, dQ, dK, I_S);
 #pragma unroll
                 for (int kk = 1; kk < 4; ++kk) umma_ss<1>(ts, dQ + 2 * kk, dK + 2 * kk, I_S);
-                umma_commit(&bars->s_full[st]);
+                umma_commit(&bars->s_full);
                 umma_commit(&bars->k_empty[st]);
                 if (j > 0) ok = issue_pv(j - 1);
             }
@@ -128,13 +129,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n_kv; ++j) {
-            const int st = j & 1;
-            const uint32_t ph = (j >> 1) & 1;
-            ok = ok && WAIT(&bars->s_full[st], ph);
+            ok = ok && WAIT(&bars->s_full, (uint32_t)(j & 1));
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             fence_after();
-            const uint32_t ts = tlane + (st ? TM_S1 : TM_S0), tp = tlane + (st ? TM_P1 : TM_P0);
+            const uint32_t ts = tlane + TM_S, tp = tlane + TM_P;
             const int valid = min(BK, a.L - j * BK);              // keys of this tile inside the sequence
             // pass 1: the row maximum of the scaled scores
             float mx = -INFINITY;
@@ -148,6 +147,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
             }
             const float m_new = fmaxf(m, mx * a.scale_log2);
             const float alpha = ex2f(m - m_new);                  // 0 on the first tile (m = -inf)
+            // P is single-buffered: P V of the previous tile must have read it (that product also completes O for the scaling below)
+            if (j > 0) {
+                ok = WAIT(&bars->o_done, (uint32_t)((j - 1) & 1));
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                fence_after();
+            }
             // pass 2: P = 2^(s - m_new) as bf16 into TMEM, and its row sum
             float sum = 0.f;
 #pragma unroll 1
@@ -159,22 +165,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
                 for (int i = 0; i < 32; i += 2) {
                     const float p0 = c0 + i < valid ? ex2f(fmaf(__uint_as_float(r[i]), a.scale_log2, -m_new)) : 0.f;
                     const float p1 = c0 + i + 1 < valid ? ex2f(fmaf(__uint_as_float(r[i + 1]), a.scale_log2, -m_new)) : 0.f;
-                    const uint32_t w = pack_bf16(p0, p1);
-                    pk[i >> 1] = w;
-                    sum += bf16_lo(w) + bf16_hi(w);               // the sum of what the product will see
+                    pk[i >> 1] = pack_bf16(p0, p1);
+                    sum += p0 + p1;
                 }
                 tmem_st_x16(tp + (c0 >> 1), pk);
             }
             l = fmaf(l, alpha, sum);
             m = m_new;
             fence_before();
-            mbar_arrive(&bars->s_empty[st]);                      // every read of S(j) has completed
+            mbar_arrive(&bars->s_empty);                          // every read of S(j) has completed
             // O holds tiles 0..j-1 once PV(j-1) has completed: scale it to the new maximum
             if (j > 0) {
-                ok = WAIT(&bars->o_done, (uint32_t)((j - 1) & 1));
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                fence_after();
 #pragma unroll 1
                 for (int c0 = 0; c0 < DH; c0 += 32) {
                     uint32_t r[32];
@@ -187,7 +188,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
             }
             tmem_wait_st();
             fence_before();
-            mbar_arrive(&bars->p_full[st]);
+            mbar_arrive(&bars->p_full);
         }
         if (ok) {
             ok = WAIT(&bars->o_done, (uint32_t)((n_kv - 1) & 1));
