@@ -171,6 +171,10 @@ STACKS = {
     "cfg2_sample": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, sample=dict(p=16)),
     # the hybrid of Sec. 3.3 on the cfg 2 stack: attention mixer in layers 0, 5, 10, 15, 20 (16 heads of 64), Mamba elsewhere
     "cfg2_stack_hybrid": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, hybrid=dict(period=5, heads=16)),
+    # the paper's 1.3B DiffuMamba (App. A.1: d = 1920, 24 timestep-conditioned blocks, 120 heads of 32, d_state 128, d_ff = 2 d) at its
+    # B = 8, L = 1024 throughput point (App. D): one reverse step with p = 16 tokens drawn per sequence, K = L / 16 steps per generation
+    "paper_b8_1k_sample": dict(shape=I.MixerShape(8, 1024, 1920, 2, 128, 4, 120), layers=24, vocab=50304,
+                               cond=dict(d_ff=3840, d_cond=128), sample=dict(p=16)),
     "cfg2_stack_cond": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, cond=dict(d_ff=2048, d_cond=128)),
 }
 
