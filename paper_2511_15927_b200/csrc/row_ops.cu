@@ -39,33 +39,97 @@ __global__ void embed_kernel(const T *__restrict__ embed, const int32_t *__restr
     for (int c = threadIdx.x; c < d; c += blockDim.x) r[t * d + c] = ldf(embed + (int64_t)id * d + c);
 }
 
+// The two row kernels below keep the token's channels in registers between the statistics and the output (one read
+// of r): thread i holds channels 4 (i + 256 k) .. +3 for k < ROW_K, which covers d <= 4096; wider rows are re-read.
+constexpr int ROW_THREADS = 256, ROW_K = 4;
+
+template <typename T> __device__ __forceinline__ void st4(T *p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void st4<float>(float *p, float a, float b, float c, float d) { *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d); }
+template <> __device__ __forceinline__ void st4<__nv_bfloat16>(__nv_bfloat16 *p, float a, float b, float c, float d) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+}
+
 template <typename T>
-__global__ void rmsnorm_kernel(const float *__restrict__ r, const T *__restrict__ w, T *__restrict__ u, int d, float eps) {
+__global__ void __launch_bounds__(ROW_THREADS)
+rmsnorm_kernel(const float *__restrict__ r, const T *__restrict__ w, T *__restrict__ u, int d, float eps) {
     __shared__ float red[32];
     const int64_t t = blockIdx.x;
+    const float *row = r + t * d;
+    const bool fast = (d & 3) == 0 && d <= 4 * ROW_THREADS * ROW_K;
+    float4 v[ROW_K];
     float s = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = r[t * d + c]; s = fmaf(v, v, s); }
+    if (fast) {
+#pragma unroll
+        for (int k = 0; k < ROW_K; ++k) {
+            const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+            v[k] = c < d ? *reinterpret_cast<const float4 *>(row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            s = fmaf(v[k].x, v[k].x, s); s = fmaf(v[k].y, v[k].y, s); s = fmaf(v[k].z, v[k].z, s); s = fmaf(v[k].w, v[k].w, s);
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) { const float x = row[c]; s = fmaf(x, x, s); }
+    }
     s = block_sum(s, red);
     const float rs = rsqrtf(s / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) stf(u + t * d + c, r[t * d + c] * rs * ldf(w + c));
+    if (fast) {
+#pragma unroll
+        for (int k = 0; k < ROW_K; ++k) {
+            const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+            if (c < d) st4(u + t * d + c, v[k].x * rs * ldf(w + c), v[k].y * rs * ldf(w + c + 1), v[k].z * rs * ldf(w + c + 2), v[k].w * rs * ldf(w + c + 3));
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) stf(u + t * d + c, row[c] * rs * ldf(w + c));
+    }
 }
 
 // u[t, :] = gamma[b, :] * (r[t, :] - mean) / sqrt(var + eps) + beta[b, :], b = t / L  (App. A.1, Eq. "AdaLN");
 // gamma and beta are rows of the per-sequence modulation table (row pitch ld_mod).
 template <typename T>
-__global__ void adaln_kernel(const float *__restrict__ r, const float *__restrict__ gamma, const float *__restrict__ beta, int64_t ld_mod,
-                             T *__restrict__ u, int L, int d, float eps) {
+__global__ void __launch_bounds__(ROW_THREADS)
+adaln_kernel(const float *__restrict__ r, const float *__restrict__ gamma, const float *__restrict__ beta, int64_t ld_mod,
+             T *__restrict__ u, int L, int d, float eps) {
     __shared__ float red[32];
     const int64_t t = blockIdx.x, b = t / L;
+    const float *row = r + t * d, *g = gamma + b * ld_mod, *be = beta + b * ld_mod;
+    const bool fast = (d & 3) == 0 && d <= 4 * ROW_THREADS * ROW_K;
+    float4 v[ROW_K];
     float s = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) s += r[t * d + c];
+    if (fast) {
+#pragma unroll
+        for (int k = 0; k < ROW_K; ++k) {
+            const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+            v[k] = c < d ? *reinterpret_cast<const float4 *>(row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            s += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) s += row[c];
+    }
     const float mu = block_sum(s, red) / (float)d;
-    __syncthreads();
     float q = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = r[t * d + c] - mu; q = fmaf(v, v, q); }
+    if (fast) {
+#pragma unroll
+        for (int k = 0; k < ROW_K; ++k) {
+            const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+            if (c < d) {
+                const float a0 = v[k].x - mu, a1 = v[k].y - mu, a2 = v[k].z - mu, a3 = v[k].w - mu;
+                q = fmaf(a0, a0, q); q = fmaf(a1, a1, q); q = fmaf(a2, a2, q); q = fmaf(a3, a3, q);
+            }
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) { const float x = row[c] - mu; q = fmaf(x, x, q); }
+    }
     const float rs = rsqrtf(block_sum(q, red) / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x)
-        stf(u + t * d + c, fmaf(gamma[b * ld_mod + c], (r[t * d + c] - mu) * rs, beta[b * ld_mod + c]));
+    if (fast) {
+#pragma unroll
+        for (int k = 0; k < ROW_K; ++k) {
+            const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+            if (c < d)
+                st4(u + t * d + c, fmaf(g[c], (v[k].x - mu) * rs, be[c]), fmaf(g[c + 1], (v[k].y - mu) * rs, be[c + 1]),
+                    fmaf(g[c + 2], (v[k].z - mu) * rs, be[c + 2]), fmaf(g[c + 3], (v[k].w - mu) * rs, be[c + 3]));
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) stf(u + t * d + c, fmaf(g[c], (row[c] - mu) * rs, be[c]));
+    }
 }
 
 // mod[b, j] = bias[j] + sum_c w[j, c] tau[b, c]: the modulation vectors of one layer (App. A.1: (gamma, beta) = W_cond tau).
