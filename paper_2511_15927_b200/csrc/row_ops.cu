@@ -151,9 +151,28 @@ __global__ void argmax_kernel(const T *__restrict__ logits, int32_t *__restrict_
     __shared__ int bi[32];
     const int64_t t = blockIdx.x;
     float best = -INFINITY; int idx = 0x7fffffff;
-    for (int v = threadIdx.x; v < V; v += blockDim.x) {
-        const float x = ldf(logits + t * V + v);
-        if (x > best || (x == best && v < idx)) { best = x; idx = v; }
+    const T *row = logits + t * V;
+    constexpr int PER = 16 / (int)sizeof(T);            // elements per 16-byte load
+    if ((reinterpret_cast<uintptr_t>(row) & 15u) == 0) {
+        const int nvec = V / PER;
+        for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+            const uint4 q = *reinterpret_cast<const uint4 *>(row + (int64_t)i * PER);
+            const T *e = reinterpret_cast<const T *>(&q);
+#pragma unroll
+            for (int j = 0; j < PER; ++j) {                 // increasing v inside the thread: strict > keeps the lowest index
+                const float x = ldf(e + j);
+                if (x > best) { best = x; idx = i * PER + j; }
+            }
+        }
+        for (int v = nvec * PER + threadIdx.x; v < V; v += blockDim.x) {
+            const float x = ldf(row + v);
+            if (x > best || (x == best && v < idx)) { best = x; idx = v; }
+        }
+    } else {
+        for (int v = threadIdx.x; v < V; v += blockDim.x) {
+            const float x = ldf(row + v);
+            if (x > best || (x == best && v < idx)) { best = x; idx = v; }
+        }
     }
     for (int off = 16; off > 0; off >>= 1) {
         const float ob = __shfl_xor_sync(0xffffffffu, best, off);
