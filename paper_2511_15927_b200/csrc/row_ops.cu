@@ -23,12 +23,14 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
     return t;
 }
 
+// One warp per row: the lanes read the row's per-head sums side by side, then reduce in a fixed order.
 __global__ void rstd_kernel(const float *__restrict__ ssq, float *__restrict__ rstd, int rows, int H, float inv_n, float eps) {
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (r >= rows) return;
     float s = 0.f;
-    for (int h = 0; h < H; ++h) s += ssq[(int64_t)r * H + h];
-    rstd[r] = rsqrtf(s * inv_n + eps);
+    for (int h = lane; h < H; h += 32) s += ssq[(int64_t)r * H + h];
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0) rstd[r] = rsqrtf(s * inv_n + eps);
 }
 
 template <typename T>
@@ -213,7 +215,7 @@ __global__ void cast_kernel(const float *__restrict__ src, T *__restrict__ dst, 
 }  // namespace
 
 cudaError_t rstd_from_ssq(const float *ssq, float *rstd, int rows, int H, int d_inner, float eps, cudaStream_t s) {
-    rstd_kernel<<<(rows + 255) / 256, 256, 0, s>>>(ssq, rstd, rows, H, 1.f / (float)d_inner, eps);
+    rstd_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ssq, rstd, rows, H, 1.f / (float)d_inner, eps);
     count_launch();
     return cudaGetLastError();
 }
