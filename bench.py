@@ -241,6 +241,7 @@ def run_stack(args, rank, local_rank, world):
     w = device_stack_weights(torch, shape, layers, vocab, cond=cond, hybrid=hyb)
     csw, keep = dm.make_stack_weights(w)
     stream = torch.cuda.current_stream().cuda_stream
+    stream_box = [stream]                      # the stream the library is given (the capture stream while a graph is recorded)
     if cond:
         blk = dm.dm_block_cfg(cond["d_ff"], cond["d_cond"], 1e-5)
         cbw = dm.make_block_weights(w["blocks"])
@@ -268,14 +269,14 @@ def run_stack(args, rank, local_rank, world):
     def denoise(cfg, tok_ptr, amax_ptr, st):
         if hyb:
             dm.dm_denoise_step_hybrid(cfg, blk if cond else None, hcfg, csw, cbw if cond else None, caw, tok_ptr, tau.data_ptr() if cond else 0,
-                                      0, amax_ptr, ws.data_ptr(), ws.numel(), stream)
+                                      0, amax_ptr, ws.data_ptr(), ws.numel(), stream_box[0])
         elif smp:
             dm.dm_denoise_sample_step(cfg, blk if cond else None, csw, cbw if cond else None, tok_ptr, tau.data_ptr() if cond else 0, scfg_s,
-                                      u_keep.data_ptr(), u_cat.data_ptr(), amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
+                                      u_keep.data_ptr(), u_cat.data_ptr(), amax_ptr, st, ws.data_ptr(), ws.numel(), stream_box[0])
         elif cond:
-            dm.dm_denoise_step_cond(cfg, blk, csw, cbw, tok_ptr, tau.data_ptr(), 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
+            dm.dm_denoise_step_cond(cfg, blk, csw, cbw, tok_ptr, tau.data_ptr(), 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream_box[0])
         else:
-            dm.dm_denoise_step(cfg, csw, tok_ptr, 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream)
+            dm.dm_denoise_step(cfg, csw, tok_ptr, 0, amax_ptr, st, ws.data_ptr(), ws.numel(), stream_box[0])
 
     def stack_cfg(L):
         sh = I.MixerShape(B, L, shape.d_model, shape.expand, shape.d_state, shape.d_conv, shape.n_heads)
@@ -348,13 +349,34 @@ def run_stack(args, rank, local_rank, world):
     dm.dm_check(stream)
     T = B * Lb
     ms_step = ms_total / args.steps
+    if args.graph:
+        # the same step recorded once per token buffer into a CUDA graph and replayed: no launch work on the host
+        graphs, cap = [], torch.cuda.Stream()
+        for i in range(4):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap):
+                stream_box[0] = torch.cuda.current_stream().cuda_stream
+                denoise(scfg, toks[i].data_ptr(), amax.data_ptr(), states)
+            stream_box[0] = stream
+            graphs.append(g)
+        denoise(scfg, toks[0].data_ptr(), amax.data_ptr(), states)
+        torch.cuda.synchronize()
+        eager = amax.clone()
+        amax.fill_(-1)
+        graphs[0].replay()
+        torch.cuda.synchronize()
+        if not torch.equal(eager, amax):
+            raise RuntimeError("the step replayed from the CUDA graph does not reproduce the eager step's token ids")
+        ms_graph = timed(lambda i: graphs[i % 4].replay(), args.steps) / args.steps
+        dm.dm_check(stream)
+        extra = dict(extra, cuda_graph_ms_per_step=ms_graph)
     if prefix:
         # the alternative without a cache: re-encode prefix + block
         fcfg = stack_cfg(prefix + Lb)
         ftok = tokens(prefix + Lb, 2)
         famax = torch.empty((B, prefix + Lb), device="cuda", dtype=torch.int32)
         ms_full = timed(lambda i: denoise(fcfg, ftok[i % 2].data_ptr(), famax.data_ptr(), None), max(2, args.steps // 4)) / max(2, args.steps // 4)
-        extra = {"prefix": prefix, "full_reencode_ms_per_step": ms_full, "state_carry_speedup": ms_full / ms_step}
+        extra = dict(extra, prefix=prefix, full_reencode_ms_per_step=ms_full, state_carry_speedup=ms_full / ms_step)
     # end to end: token ids from pinned host memory in, arg-max ids back, inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -428,6 +450,7 @@ def main():
     ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="stack workloads: also time the step replayed from a captured CUDA graph")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = max(args.warmup, 1) if args.impl == "reference" else 3
