@@ -130,3 +130,36 @@ def test_half_width_heads_run_with_padded_channels(G, N):
     _check(G, y_g, y_o)
     _check(G, s_g, s_o)
     _check(G, c_g, c_o)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_seeded_mix_of_shapes_and_options(G, seed):
+    """A seeded draw over what the kernel takes -- length, batch, headdim 64 or 32, d_state, conv width, flags,
+    direction mask, carried state or none -- against the oracle: combinations that the other tests visit one at a time."""
+    r = np.random.default_rng(1000 + seed)
+    P = int(r.choice([64, 32]))
+    H = int(r.choice([2, 4, 8])) * (2 if P == 32 else 1)
+    N = int(r.choice([128, 64, 32, 16]))
+    while (2 * N + H) % 8:                                   # 16-byte rows of the in_proj output
+        H += 2 if P == 32 else 1
+    d_inner = P * H
+    B, L, k = int(r.integers(1, 4)), int(r.integers(1, 700)), int(r.choice([4, 4, 3, 2]))
+    flags = int(r.choice([7, 7, 6, 5, 3]))
+    dir_mask = int(r.choice([3, 3, 1, 2]))
+    shape = I.MixerShape(B, L, d_inner // 2, 2, N, k, H)
+    assert shape.headdim == P and shape.d_in_proj % 8 == 0
+    wf, wr = I.make_mixer_weights(shape, seed, I.BF16, perturb=True)
+    x = I.make_activations(shape, seed, I.BF16)
+    kw = G.oracle_kwargs(shape, flags)
+    if r.random() < 0.5:
+        ssm_in, conv_in = I.make_states(shape, seed, I.BF16)
+        y_o, s_o, c_o = O.bimamba_block_step(x, wf, wr, ssm_state_in=ssm_in, conv_state_in=conv_in, dir_mask=dir_mask, **kw)
+        want_state = bool(dir_mask & 1)
+        y_g, s_g, c_g = G.run_block_step(shape, I.BF16, wf, wr, x, ssm_in, conv_in, want_state=want_state, flags=flags, dir_mask=dir_mask)
+        _check(G, y_g, y_o)
+        if want_state:
+            _check(G, s_g, s_o)
+            _check(G, c_g, c_o)
+    else:
+        _check(G, G.run_forward(shape, I.BF16, wf, wr, x, flags=flags, dir_mask=dir_mask),
+               O.bimamba_forward(x, wf, wr, dir_mask=dir_mask, **kw))
