@@ -488,3 +488,27 @@ def denoise_step_hybrid(tokens, sw: dict, *, attn_period: int, attn_heads: int, 
             y = r + g1[:, None, :] * mix(adaln(r, s1, b1, ln_eps))
             r = y + g2[:, None, :] * mlp(adaln(y, s2, b2, ln_eps), layer["w_up"], layer["w_down"], layer.get("b_up"), layer.get("b_down"))
     return rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T
+
+
+def attention_block_step(x_blk, w_qkv, w_o, n_heads: int, k_cache=None, v_cache=None):
+    """The attention mixer in block-autoregressive decoding (Sec. 4.3: the cache of a denoised block is kept and reused):
+    the block's queries attend to the cached keys and values of the committed prefix and, without a mask, to the block
+    itself.  k_cache, v_cache: [B, Lc, d] (None = empty prefix).  Returns (y_blk, k_all, v_all) with the block's keys and
+    values appended, i.e. the cache a commit of this block would leave."""
+    x = np.asarray(x_blk, F64)
+    B, G, d = x.shape
+    dh = d // n_heads
+    qkv = x @ np.asarray(w_qkv, F64).T
+    q, k, v = qkv[..., :d], qkv[..., d:2 * d], qkv[..., 2 * d:]
+    if k_cache is not None:
+        k = np.concatenate([np.asarray(k_cache, F64), k], axis=1)
+        v = np.concatenate([np.asarray(v_cache, F64), v], axis=1)
+    out = np.zeros((B, G, d), F64)
+    for b in range(B):
+        for h in range(n_heads):
+            sl = slice(h * dh, (h + 1) * dh)
+            s = q[b, :, sl] @ k[b, :, sl].T / np.sqrt(dh)
+            p = np.exp(s - s.max(axis=1, keepdims=True))
+            p /= p.sum(axis=1, keepdims=True)
+            out[b, :, sl] = p @ v[b, :, sl]
+    return out @ np.asarray(w_o, F64).T, k, v

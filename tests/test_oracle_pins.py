@@ -644,3 +644,21 @@ def test_hybrid_stack_places_attention_every_period_layers():
     sw2["layers"][1]["w_o"] = 0 * sw2["layers"][1]["w_o"]
     np.testing.assert_array_equal(O.denoise_step_hybrid(tok, sw2, attn_period=5, attn_heads=H_attn, tau=tau, **KW),
                                   O.denoise_step_hybrid(tok, sw, attn_period=5, attn_heads=H_attn, tau=tau, **KW))
+
+
+def test_attention_block_step_with_a_key_value_cache():
+    B, d, H = 2, 8, 2
+    x = rng.standard_normal((B, 9, d)); wqkv = rng.standard_normal((3 * d, d)) * 0.5; wo = rng.standard_normal((d, d)) * 0.5
+    # an empty cache: the block alone
+    y, k, v = O.attention_block_step(x, wqkv, wo, H)
+    np.testing.assert_allclose(y, O.attention_mixer(x, wqkv, wo, H), rtol=1e-12)
+    np.testing.assert_allclose(k, x @ wqkv[d:2 * d].T, rtol=1e-12); np.testing.assert_allclose(v, x @ wqkv[2 * d:].T, rtol=1e-12)
+    # prefix of 5 tokens cached, block of 4: the block's rows of full attention over all 9 tokens (the prefix rows of that
+    # full pass differ, since a committed prefix never saw the block -- only the block's rows are compared)
+    _, k5, v5 = O.attention_block_step(x[:, :5], wqkv, wo, H)
+    y_blk, k9, v9 = O.attention_block_step(x[:, 5:], wqkv, wo, H, k5, v5)
+    np.testing.assert_allclose(y_blk, O.attention_mixer(x, wqkv, wo, H)[:, 5:], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(k9, k, rtol=1e-12); np.testing.assert_allclose(v9, v, rtol=1e-12)
+    # the cache is read, not recomputed: scaling the cached values scales their contribution
+    y_zero, _, _ = O.attention_block_step(x[:, 5:], wqkv, wo, H, k5, 0 * v5)
+    assert np.abs(y_zero - y_blk).max() > 1e-3
