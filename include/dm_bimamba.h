@@ -231,8 +231,8 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
  * bidirectional Mamba mixer otherwise; attn_period = 0 means no attention layer.  Around either mixer the layer is
  * the RMSNorm pre-norm + residual of dm_denoise_step (blk == NULL) or the timestep-conditioned block of
  * dm_denoise_step_cond (blk, block_weights, tau given).  attn_weights: HOST array of cfg->n_layers entries, read
- * only where the layer is attention (the Mamba weights of those layers are not read).  Full-sequence mode only:
- * block mode would need a key/value cache for the attention layers.  bf16, attention heads of width 64. */
+ * only where the layer is attention (the Mamba weights of those layers are not read).  Full-sequence mode; block
+ * mode is dm_denoise_step_hybrid_block.  bf16, attention heads of width 64. */
 typedef struct {
     int32_t attn_period;   /* N: layers 0, N, 2N, ... are attention; 0 = none */
     int32_t attn_heads;    /* d_model = 64 * attn_heads */
@@ -241,12 +241,40 @@ typedef struct {
     const void *w_qkv;     /* [3 * d_model, d_model] dtype, rows [Q | K | V] */
     const void *w_o;       /* [d_model, d_model] dtype */
 } dm_attn_weights;
+/* Key/value cache of one attention layer in block mode (Sec. 4.3): rows [0, len) hold the committed prefix.  A step
+ * writes the block's keys and values to rows [len, len + G) -- whether or not the caller then commits them by
+ * advancing len -- and its queries attend to rows [0, len + G), unmasked. */
+typedef struct {
+    void   *k_cache;   /* [B, cap, d_model] dtype */
+    void   *v_cache;   /* [B, cap, d_model] dtype */
+    int32_t len;       /* committed rows */
+    int32_t cap;       /* rows allocated; len + G <= cap */
+} dm_attn_state;
 int dm_denoise_hybrid_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes);
 int dm_denoise_step_hybrid(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_hybrid_cfg *hybrid,
                            const dm_stack_weights *weights, const dm_block_weights *block_weights,
                            const dm_attn_weights *attn_weights, const int32_t *tokens, const float *tau,
                            void *logits, int32_t *argmax_out,
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* dm_denoise_step_hybrid in block mode (Sec. 4.3): cfg->mixer.seqlen = G tokens of the active block per sequence;
+ * `states` carries the Mamba layers' states as in dm_denoise_step, `attn_states` (HOST array of cfg->n_layers entries,
+ * read where the layer is attention) the attention layers' key/value caches. */
+int dm_denoise_step_hybrid_block(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_hybrid_cfg *hybrid,
+                                 const dm_stack_weights *weights, const dm_block_weights *block_weights,
+                                 const dm_attn_weights *attn_weights, const int32_t *tokens, const float *tau,
+                                 void *logits, int32_t *argmax_out, const dm_layer_state *states,
+                                 const dm_attn_state *attn_states,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* dm_attention_forward for the active block of block-autoregressive decoding, with a key/value cache (dm_attn_state's
+ * convention): the block's keys and values are written to rows [cache_len, cache_len + block_len) of the caches and
+ * the block's queries attend to rows [0, cache_len + block_len).  Workspace as dm_attention_workspace_bytes(batch,
+ * block_len, ...). */
+int dm_attention_block_step(int32_t batch, int32_t block_len, int32_t d_model, int32_t n_heads, int32_t dtype,
+                            const void *w_qkv, const void *w_o, const void *x_blk,
+                            void *k_cache, void *v_cache, int32_t cache_len, int32_t cache_cap, void *y_blk,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* One dense projection as the mixer uses it (App. C counts 2mn FLOPs per token for a weight W in R^{m x n}):
  *     y[r, :] = row_scale[r] * (W x[r, :]) + addend[r, :]

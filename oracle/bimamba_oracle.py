@@ -471,23 +471,44 @@ def attention_mixer(x, w_qkv, w_o, n_heads: int):
 
 
 def denoise_step_hybrid(tokens, sw: dict, *, attn_period: int, attn_heads: int, tau=None, rms_eps: float = 1e-5,
-                        ln_eps: float = 1e-5, **kw):
+                        ln_eps: float = 1e-5, states_in=None, return_states: bool = False, **kw):
     """The hybrid stack (Sec. 3.3, App. A.3): the mixer of layer i is the attention mixer when i is a multiple of
     attn_period (one attention mixer followed by attn_period - 1 bidirectional Mamba mixers; the paper uses 5), the
     bidirectional Mamba mixer otherwise.  tau None: RMSNorm pre-norm + mixer + residual per layer; tau given: the
-    timestep-conditioned block around either mixer.  Attention layers carry "w_qkv" and "w_o"."""
+    timestep-conditioned block around either mixer.  Attention layers carry "w_qkv" and "w_o".
+    Block mode (states_in given or return_states): every layer runs as a block step from its entry of states_in --
+    (ssm, conv) for a Mamba layer, (k_cache, v_cache) for an attention layer, None for an empty prefix -- and the
+    states after the block are returned in the same form."""
+    block_mode = states_in is not None or return_states
     r = np.asarray(sw["embed"], F64)[np.asarray(tokens)]
+    states_out = []
     for i, layer in enumerate(sw["layers"]):
         is_attn = attn_period > 0 and i % attn_period == 0
-        mix = (lambda u: attention_mixer(u, layer["w_qkv"], layer["w_o"], attn_heads)) if is_attn else \
-              (lambda u: bimamba_forward(u, layer["fwd"], layer["rev"], **kw))
+        st = None if states_in is None else states_in[i]
+
+        def mix(u, layer=layer, is_attn=is_attn, st=st):
+            if is_attn:
+                if not block_mode:
+                    return attention_mixer(u, layer["w_qkv"], layer["w_o"], attn_heads)
+                kc, vc = (None, None) if st is None else st
+                y, k_all, v_all = attention_block_step(u, layer["w_qkv"], layer["w_o"], attn_heads, kc, vc)
+                states_out.append((k_all, v_all))
+                return y
+            if not block_mode:
+                return bimamba_forward(u, layer["fwd"], layer["rev"], **kw)
+            s_in, c_in = (None, None) if st is None else st
+            y, s_out, c_out = bimamba_block_step(u, layer["fwd"], layer["rev"], ssm_state_in=s_in, conv_state_in=c_in, **kw)
+            states_out.append((s_out, c_out))
+            return y
+
         if tau is None:
             r = r + mix(rmsnorm(r, layer["norm_w"], rms_eps))
         else:
             b1, s1, g1, b2, s2, g2 = modulation(tau, layer["w_cond"], layer.get("b_cond"))
             y = r + g1[:, None, :] * mix(adaln(r, s1, b1, ln_eps))
             r = y + g2[:, None, :] * mlp(adaln(y, s2, b2, ln_eps), layer["w_up"], layer["w_down"], layer.get("b_up"), layer.get("b_down"))
-    return rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T
+    logits = rmsnorm(r, sw["final_norm_w"], rms_eps) @ np.asarray(sw["w_vocab"], F64).T
+    return (logits, states_out) if return_states else logits
 
 
 def attention_block_step(x_blk, w_qkv, w_o, n_heads: int, k_cache=None, v_cache=None):

@@ -29,20 +29,22 @@ struct Bars {
 };
 
 struct AttnArgs {
-    int B, L, d, H;
-    __nv_bfloat16 *out;          // [B*L, d]
+    int B, Lq, Lk, d, H;         // Lq queries per sequence attend to Lk keys
+    int kx0, vx0;                // column of head 0's keys / values in their tensor maps
+    __nv_bfloat16 *out;          // [B*Lq, d]
     float scale_log2;            // log2(e) / sqrt(d_h)
 };
 
 __global__ void __launch_bounds__(NTHREADS, 2)
-attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, int *status) {
+attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, const AttnArgs a, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     Bars *bars = reinterpret_cast<Bars *>(smem + OFF_BAR);
     volatile int *abort_flag = &bars->abort;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int q0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z;
-    const int n_kv = (a.L + BK - 1) / BK;
+    const int n_kv = (a.Lk + BK - 1) / BK;
 
     if (tid == 0) {
         mbar_init(&bars->q_full, 1);
@@ -67,18 +69,18 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             mbar_expect_tx(&bars->q_full, TILE);
-            tma_load_3d(smem + OFF_Q, &map_qkv, h * DH, q0, b, &bars->q_full);
+            tma_load_3d(smem + OFF_Q, &map_q, h * DH, q0, b, &bars->q_full);
             int issued_k = 0, issued_v = 0;
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j & 1;
                 const uint32_t ph = (j >> 1) & 1;
                 if (!WAIT(&bars->k_empty[st], ph ^ 1)) break;
                 mbar_expect_tx(&bars->k_full[st], TILE);
-                tma_load_3d(smem + OFF_K + st * TILE, &map_qkv, a.d + h * DH, j * BK, b, &bars->k_full[st]);
+                tma_load_3d(smem + OFF_K + st * TILE, &map_k, a.kx0 + h * DH, j * BK, b, &bars->k_full[st]);
                 issued_k = j + 1;
                 if (!WAIT(&bars->v_empty[st], ph ^ 1)) break;
                 mbar_expect_tx(&bars->v_full[st], TILE);
-                tma_load_3d(smem + OFF_V + st * TILE, &map_qkv, 2 * a.d + h * DH, j * BK, b, &bars->v_full[st]);
+                tma_load_3d(smem + OFF_V + st * TILE, &map_v, a.vx0 + h * DH, j * BK, b, &bars->v_full[st]);
                 issued_v = j + 1;
             }
             if (*abort_flag) {             // aborting: bounded wait for the loads still in flight
@@ -134,7 +136,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
             if (!ok) break;
             fence_after();
             const uint32_t ts = tlane + TM_S, tp = tlane + TM_P;
-            const int valid = min(BK, a.L - j * BK);              // keys of this tile inside the sequence
+            const int valid = min(BK, a.Lk - j * BK);             // keys of this tile inside the sequence
             // pass 1: the row maximum of the scaled scores
             float mx = -INFINITY;
 #pragma unroll 1
@@ -203,8 +205,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
                 uint32_t r[32];
                 tmem_ld_x32(tlane + TM_O + c0, r);
                 tmem_wait_ld();
-                if (t < a.L) {
-                    __nv_bfloat16 *dst = a.out + ((int64_t)b * a.L + t) * a.d + h * DH + c0;
+                if (t < a.Lq) {
+                    __nv_bfloat16 *dst = a.out + ((int64_t)b * a.Lq + t) * a.d + h * DH + c0;
 #pragma unroll
                     for (int i = 0; i < 32; i += 8)
                         *reinterpret_cast<uint4 *>(dst + i) =
@@ -225,26 +227,58 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qkv, const AttnArgs a, 
     }
 }
 
+// The block's keys and values (columns [d, 3 d) of qkv [B*G, 3 d]) go to rows [len, len + G) of the caches [B, cap, d].
+__global__ void kv_append_kernel(const __nv_bfloat16 *__restrict__ qkv, __nv_bfloat16 *__restrict__ kc, __nv_bfloat16 *__restrict__ vc,
+                                 int G, int d, int len, int cap) {
+    const int t = blockIdx.x, b = blockIdx.y;
+    const uint4 *src = reinterpret_cast<const uint4 *>(qkv + ((int64_t)b * G + t) * 3 * d + d);
+    uint4 *dk = reinterpret_cast<uint4 *>(kc + ((int64_t)b * cap + len + t) * d), *dv = reinterpret_cast<uint4 *>(vc + ((int64_t)b * cap + len + t) * d);
+    const int n = d / 8;                                   // 16-byte pieces per row (d is a multiple of 64)
+    for (int i = threadIdx.x; i < n; i += blockDim.x) { dk[i] = src[i]; dv[i] = src[n + i]; }
+}
+
 }  // namespace
 
 bool attention_supports(int dtype, int d, int n_heads) {
     return dtype == DM_BF16 && n_heads > 0 && d == n_heads * DH && encode_fn() != nullptr;
 }
 
-// qkv [B*L, 3 d] bf16 (columns [Q | K | V], heads contiguous inside each), out [B*L, d] bf16
-cudaError_t attention_forward(const void *qkv, void *out, int B, int L, int d, int n_heads, cudaStream_t s) {
-    if (!attention_supports(DM_BF16, d, n_heads) || B <= 0 || L <= 0 || B > 65535 || n_heads > 65535) return cudaErrorNotSupported;
-    CUtensorMap map;
-    const uint64_t dims[3] = {(uint64_t)3 * d, (uint64_t)L, (uint64_t)B};
-    const uint64_t str[2] = {(uint64_t)3 * d, (uint64_t)L * 3 * d};
+// qkv [B*Lq, 3 d] bf16 (columns [Q | K | V], heads contiguous inside each), out [B*Lq, d] bf16.
+// k_cache == NULL: keys and values are the K and V columns of qkv (Lk = Lq).  Otherwise the block's keys and values are
+// first appended at rows [cache_len, cache_len + Lq) of k_cache, v_cache [B, cache_cap, d], and the queries attend to the
+// first cache_len + Lq rows of the caches.
+cudaError_t attention_forward(const void *qkv, void *out, int B, int Lq, int d, int n_heads, void *k_cache, void *v_cache,
+                              int cache_len, int cache_cap, cudaStream_t s) {
+    if (!attention_supports(DM_BF16, d, n_heads) || B <= 0 || Lq <= 0 || B > 65535 || n_heads > 65535) return cudaErrorNotSupported;
+    const bool cached = k_cache != nullptr;
+    if (cached && (!v_cache || cache_len < 0 || cache_len + Lq > cache_cap)) return cudaErrorInvalidValue;
+    const int Lk = cached ? cache_len + Lq : Lq;
+    CUtensorMap mq, mk, mv;
     const uint32_t box[3] = {(uint32_t)DH, (uint32_t)BQ, 1};
-    if (!make_map_bf16(&map, qkv, 3, dims, str, box)) return cudaErrorInvalidValue;
+    {
+        const uint64_t dims[3] = {(uint64_t)3 * d, (uint64_t)Lq, (uint64_t)B};
+        const uint64_t str[2] = {(uint64_t)3 * d, (uint64_t)Lq * 3 * d};
+        if (!make_map_bf16(&mq, qkv, 3, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    if (cached) {
+        // the maps end at the last valid key: the rest of a tile is filled with zeros, whatever the cache holds there
+        const uint64_t dims[3] = {(uint64_t)d, (uint64_t)Lk, (uint64_t)B};
+        const uint64_t str[2] = {(uint64_t)d, (uint64_t)cache_cap * d};
+        if (!make_map_bf16(&mk, k_cache, 3, dims, str, box) || !make_map_bf16(&mv, v_cache, 3, dims, str, box)) return cudaErrorInvalidValue;
+        kv_append_kernel<<<dim3(Lq, B), 128, 0, s>>>(static_cast<const __nv_bfloat16 *>(qkv), static_cast<__nv_bfloat16 *>(k_cache),
+                                                      static_cast<__nv_bfloat16 *>(v_cache), Lq, d, cache_len, cache_cap);
+        count_launch();
+        cudaError_t e0 = cudaGetLastError();
+        if (e0 != cudaSuccess) return e0;
+    } else {
+        mk = mq; mv = mq;
+    }
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
     cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    AttnArgs a{B, L, d, n_heads, static_cast<__nv_bfloat16 *>(out), 1.4426950408889634f / sqrtf((float)DH)};
-    attention_kernel<<<dim3((L + BQ - 1) / BQ, n_heads, B), NTHREADS, SMEM_BYTES, s>>>(map, a, status);
+    AttnArgs a{B, Lq, Lk, d, n_heads, cached ? 0 : d, cached ? 0 : 2 * d, static_cast<__nv_bfloat16 *>(out), 1.4426950408889634f / sqrtf((float)DH)};
+    attention_kernel<<<dim3((Lq + BQ - 1) / BQ, n_heads, B), NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, a, status);
     count_launch();
     return cudaGetLastError();
 }

@@ -433,6 +433,7 @@ struct SampleArgs {
 };
 struct HybridArgs {
     const dm_hybrid_cfg *cfg; const dm_attn_weights *aw;      // aw: HOST array of n_layers entries (used where the layer is attention)
+    const dm_attn_state *ast = nullptr;                       // block mode: key/value caches of the attention layers (HOST array), or NULL
 };
 
 static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights, const dm_block_weights *bw,
@@ -478,7 +479,14 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
         if (!hyb->cfg || !hyb->aw) return fail(DM_ERR_INVALID_ARG, "hybrid configuration or attention weights are NULL");
         if (period < 0) return fail(DM_ERR_INVALID_ARG, "attn_period must be >= 0");
         if (period > 0) {
-            if (states) return fail(DM_ERR_UNSUPPORTED, "block mode needs a key/value cache for the attention layers, which is not built");
+            if (states && !hyb->ast) return fail(DM_ERR_INVALID_ARG, "block mode needs the key/value caches of the attention layers");
+            if (hyb->ast)
+                for (int i = 0; i < cfg->n_layers; i += period) {
+                    const dm_attn_state &q = hyb->ast[i];
+                    if (!q.k_cache || !q.v_cache || !aligned16(q.k_cache) || !aligned16(q.v_cache))
+                        return fail(DM_ERR_INVALID_ARG, "layer %d: key/value caches must be non-NULL and 16-byte aligned", i);
+                    if (q.len < 0 || q.len + m.L > q.cap) return fail(DM_ERR_INVALID_ARG, "layer %d: cache length + block length exceeds its capacity", i);
+                }
             if (hyb->cfg->attn_heads <= 0 || m.d != 64 * hyb->cfg->attn_heads || !attention_supports(cfg->mixer.dtype, m.d, hyb->cfg->attn_heads))
                 return fail(DM_ERR_UNSUPPORTED, "attention layers need bf16 and heads of width 64 (d_model = 64 * attn_heads)");
             for (int i = 0; i < cfg->n_layers; i += period)
@@ -529,7 +537,8 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
             a.A = u; a.lda = m.d; a.B = hyb->aw[i].w_qkv; a.ldb = m.d; a.C = qkv; a.ldc = 3 * m.d;
             a.in_dtype = dtype; a.c_dtype = dtype; a.M = (int)m.T; a.N = 3 * m.d; a.K = m.d;
             if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "qkv projection");
-            if ((e = attention_forward(qkv, att, m.B, m.L, m.d, hyb->cfg->attn_heads, s)) != cudaSuccess) return cuda_fail(e, "attention");
+            if ((e = attention_forward(qkv, att, m.B, m.L, m.d, hyb->cfg->attn_heads, hyb->ast ? hyb->ast[i].k_cache : nullptr,
+                                       hyb->ast ? hyb->ast[i].v_cache : nullptr, hyb->ast ? hyb->ast[i].len : 0, hyb->ast ? hyb->ast[i].cap : 0, s)) != cudaSuccess) return cuda_fail(e, "attention");
             GemmArgs o{};
             o.A = att; o.lda = m.d; o.B = hyb->aw[i].w_o; o.ldb = m.d; o.C = r; o.ldc = m.d;
             o.in_dtype = dtype; o.c_dtype = DM_F32; o.M = (int)m.T; o.N = m.d; o.K = m.d;
@@ -659,6 +668,51 @@ int dm_denoise_step_hybrid(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
                         nullptr, &hyb);
 }
 
+int dm_denoise_step_hybrid_block(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_hybrid_cfg *hybrid,
+                                 const dm_stack_weights *weights, const dm_block_weights *block_weights,
+                                 const dm_attn_weights *attn_weights, const int32_t *tokens, const float *tau, void *logits,
+                                 int32_t *argmax_out, const dm_layer_state *states, const dm_attn_state *attn_states,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!hybrid) return fail(DM_ERR_INVALID_ARG, "hybrid configuration is NULL");
+    HybridArgs hyb{hybrid, attn_weights};
+    hyb.ast = attn_states;
+    return denoise_impl(cfg, blk, weights, block_weights, tokens, tau, logits, argmax_out, states, workspace, workspace_bytes, cuda_stream,
+                        nullptr, &hyb);
+}
+
+int dm_attention_block_step(int32_t batch, int32_t block_len, int32_t d_model, int32_t n_heads, int32_t dtype, const void *w_qkv,
+                            const void *w_o, const void *x_blk, void *k_cache, void *v_cache, int32_t cache_len, int32_t cache_cap,
+                            void *y_blk, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    size_t need = 0;
+    int st = dm_attention_workspace_bytes(batch, block_len, d_model, dtype, &need);
+    if (st != DM_OK) return st;
+    if (!w_qkv || !w_o || !x_blk || !y_blk || !k_cache || !v_cache) return fail(DM_ERR_INVALID_ARG, "NULL pointer");
+    if (x_blk == y_blk) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
+    if (!aligned16(w_qkv) || !aligned16(w_o) || !aligned16(x_blk) || !aligned16(y_blk) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(DM_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if (n_heads <= 0 || d_model != n_heads * 64) return fail(DM_ERR_UNSUPPORTED, "the attention mixer needs heads of width 64 (d_model = 64 * n_heads)");
+    if (batch > 65535 || n_heads > 65535) return fail(DM_ERR_UNSUPPORTED, "batch and n_heads must be below 65536");
+    if (cache_len < 0 || cache_len + block_len > cache_cap) return fail(DM_ERR_INVALID_ARG, "cache length + block length exceeds the cache's capacity");
+    if (!attention_supports(dtype, d_model, n_heads)) return fail(DM_ERR_UNSUPPORTED, "the attention mixer is not available for this configuration");
+    if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t T = (int64_t)batch * block_len;
+    char *ws = static_cast<char *>(workspace);
+    void *qkv = ws, *att = ws + align_up((size_t)T * 3 * d_model * 2);
+    GemmArgs a{};
+    a.A = x_blk; a.lda = d_model; a.B = w_qkv; a.ldb = d_model; a.C = qkv; a.ldc = 3 * d_model;
+    a.in_dtype = dtype; a.c_dtype = dtype; a.M = (int)T; a.N = 3 * d_model; a.K = d_model;
+    cudaError_t e;
+    if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "qkv projection");
+    if ((e = attention_forward(qkv, att, batch, block_len, d_model, n_heads, k_cache, v_cache, cache_len, cache_cap, s)) != cudaSuccess)
+        return cuda_fail(e, "attention");
+    GemmArgs o{};
+    o.A = att; o.lda = d_model; o.B = w_o; o.ldb = d_model; o.C = y_blk; o.ldc = d_model;
+    o.in_dtype = dtype; o.c_dtype = dtype; o.M = (int)T; o.N = d_model; o.K = d_model;
+    if ((e = gemm(o, s)) != cudaSuccess) return cuda_fail(e, "attention output projection");
+    return DM_OK;
+}
+
 int dm_attention_workspace_bytes(int32_t batch, int32_t seqlen, int32_t d_model, int32_t dtype, size_t *bytes) {
     if (!bytes || batch <= 0 || seqlen <= 0 || d_model <= 0) return fail(DM_ERR_INVALID_ARG, "sizes must be positive");
     if (dtype != DM_BF16) return fail(DM_ERR_UNSUPPORTED, "the attention mixer takes bf16 only");
@@ -687,7 +741,7 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
     a.in_dtype = dtype; a.c_dtype = dtype; a.M = (int)T; a.N = 3 * d_model; a.K = d_model;
     cudaError_t e;
     if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "qkv projection");
-    if ((e = attention_forward(qkv, att, batch, seqlen, d_model, n_heads, s)) != cudaSuccess) return cuda_fail(e, "attention");
+    if ((e = attention_forward(qkv, att, batch, seqlen, d_model, n_heads, nullptr, nullptr, 0, 0, s)) != cudaSuccess) return cuda_fail(e, "attention");
     GemmArgs o{};
     o.A = att; o.lda = d_model; o.B = w_o; o.ldb = d_model; o.C = y; o.ldc = d_model;
     o.in_dtype = dtype; o.c_dtype = dtype; o.M = (int)T; o.N = d_model; o.K = d_model;

@@ -75,7 +75,10 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s);
 // Bidirectional multi-head attention over qkv [B*L, 3 d] (columns [Q | K | V], heads contiguous inside each) -> out [B*L, d];
 // bf16, head width 64.
 bool attention_supports(int dtype, int d, int n_heads);
-cudaError_t attention_forward(const void *qkv, void *out, int B, int L, int d, int n_heads, cudaStream_t s);
+// k_cache != NULL: block mode -- the block's K, V are appended at rows [cache_len, cache_len + L) of the caches [B, cache_cap, d]
+// and the queries attend to the first cache_len + L rows.
+cudaError_t attention_forward(const void *qkv, void *out, int B, int L, int d, int n_heads, void *k_cache, void *v_cache,
+                              int cache_len, int cache_cap, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // Small row-wise kernels

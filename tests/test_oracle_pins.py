@@ -662,3 +662,32 @@ def test_attention_block_step_with_a_key_value_cache():
     # the cache is read, not recomputed: scaling the cached values scales their contribution
     y_zero, _, _ = O.attention_block_step(x[:, 5:], wqkv, wo, H, k5, 0 * v5)
     assert np.abs(y_zero - y_blk).max() > 1e-3
+
+
+def test_hybrid_stack_block_mode_left_to_right_equals_one_pass_on_the_block_rows():
+    """Left-to-right Mamba direction only: two blocks through the carried states and key/value caches give, on the second
+    block's rows, the logits of ... a pass in which the first block never saw the second: rebuilt layer by layer."""
+    d, H_attn = 6, 2
+    sw, _ = _tiny_cond_stack(n_layers=3, d=d)
+    r = np.random.default_rng(78)
+    for l in sw["layers"]:
+        l["w_qkv"] = r.standard_normal((3 * d, d)) * 0.3; l["w_o"] = r.standard_normal((d, d)) * 0.3
+    tok = rng.integers(0, 11, (2, 9))
+    kw = dict(KW, dir_mask=O.DIR_FWD)
+    l1, st = O.denoise_step_hybrid(tok[:, :5], sw, attn_period=2, attn_heads=H_attn, return_states=True, **kw)
+    l2, st2 = O.denoise_step_hybrid(tok[:, 5:], sw, attn_period=2, attn_heads=H_attn, states_in=st, return_states=True, **kw)
+    assert len(st) == 3 and st[0][0].shape == (2, 5, d) and st2[0][0].shape == (2, 9, d) and st[1][0].ndim == 4
+    # layer by layer: the prefix rows evolve alone; the block rows see the prefix through the Mamba state (exactly, for the
+    # left-to-right direction) and through the cached keys and values
+    xa, xb = sw["embed"][tok[:, :5]], sw["embed"][tok[:, 5:]]
+    for i, l in enumerate(sw["layers"]):
+        ua, ub = O.rmsnorm(xa, l["norm_w"]), O.rmsnorm(xb, l["norm_w"])
+        if i % 2 == 0:
+            ya, ka, va = O.attention_block_step(ua, l["w_qkv"], l["w_o"], H_attn)
+            yb, _, _ = O.attention_block_step(ub, l["w_qkv"], l["w_o"], H_attn, ka, va)
+        else:
+            full = O.bimamba_forward(np.concatenate([ua, ub], 1), l["fwd"], l["rev"], **kw)     # causal: the prefix rows do not see the block
+            ya, yb = full[:, :5], full[:, 5:]
+        xa, xb = xa + ya, xb + yb
+    np.testing.assert_allclose(l1, O.rmsnorm(xa, sw["final_norm_w"]) @ sw["w_vocab"].T, rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(l2, O.rmsnorm(xb, sw["final_norm_w"]) @ sw["w_vocab"].T, rtol=1e-9, atol=1e-11)
