@@ -59,6 +59,10 @@ class dm_attn_weights(C.Structure):
     _fields_ = [("w_qkv", C.c_void_p), ("w_o", C.c_void_p)]
 
 
+class dm_attn_state(C.Structure):
+    _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("len", C.c_int32), ("cap", C.c_int32)]
+
+
 class dm_sample_cfg(C.Structure):
     _fields_ = [("mask_id", C.c_int32), ("vocab_real", C.c_int32), ("keep_prob", C.c_float)]
 
@@ -106,6 +110,13 @@ _lib.dm_denoise_hybrid_workspace_bytes.restype = C.c_int
 _lib.dm_denoise_step_hybrid.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_hybrid_cfg), C.POINTER(dm_stack_weights),
                                         C.POINTER(dm_block_weights), C.POINTER(dm_attn_weights), _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.dm_denoise_step_hybrid.restype = C.c_int
+_lib.dm_denoise_step_hybrid_block.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_hybrid_cfg), C.POINTER(dm_stack_weights),
+                                              C.POINTER(dm_block_weights), C.POINTER(dm_attn_weights), _vp, _vp, _vp, _vp,
+                                              C.POINTER(dm_layer_state), C.POINTER(dm_attn_state), _vp, _sz, _vp]
+_lib.dm_denoise_step_hybrid_block.restype = C.c_int
+_lib.dm_attention_block_step.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32,
+                                         _vp, _vp, _sz, _vp]
+_lib.dm_attention_block_step.restype = C.c_int
 _lib.dm_attention_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(_sz)]
 _lib.dm_attention_workspace_bytes.restype = C.c_int
 _lib.dm_attention_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -122,7 +133,8 @@ EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count"
            "dm_denoise_workspace_bytes", "dm_check", "dm_bimamba_forward", "dm_bimamba_forward_host",
            "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
            "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step",
-           "dm_attention_workspace_bytes", "dm_attention_forward", "dm_denoise_hybrid_workspace_bytes", "dm_denoise_step_hybrid")
+           "dm_attention_workspace_bytes", "dm_attention_forward", "dm_denoise_hybrid_workspace_bytes", "dm_denoise_step_hybrid",
+           "dm_denoise_step_hybrid_block", "dm_attention_block_step")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -259,6 +271,21 @@ def dm_denoise_step_hybrid(cfg, blk, hybrid: dm_hybrid_cfg, weights, block_weigh
     _ok(_lib.dm_denoise_step_hybrid(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(hybrid), C.byref(weights),
                                     block_weights, attn_weights, _vp(tokens), _vp(tau or None), _vp(logits or None),
                                     _vp(argmax_out or None), _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_denoise_step_hybrid_block(cfg, blk, hybrid: dm_hybrid_cfg, weights, block_weights, attn_weights, tokens: int, tau: int, logits: int,
+                                 argmax_out: int, states, attn_states, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    """states: (dm_layer_state * n_layers) or None; attn_states: (dm_attn_state * n_layers)."""
+    _ok(_lib.dm_denoise_step_hybrid_block(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(hybrid), C.byref(weights),
+                                          block_weights, attn_weights, _vp(tokens), _vp(tau or None), _vp(logits or None),
+                                          _vp(argmax_out or None), states, attn_states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_attention_block_step(batch: int, block_len: int, d_model: int, n_heads: int, dtype: int, w_qkv: int, w_o: int, x_blk: int,
+                            k_cache: int, v_cache: int, cache_len: int, cache_cap: int, y_blk: int, workspace: int,
+                            workspace_bytes: int, cuda_stream: int = 0) -> None:
+    _ok(_lib.dm_attention_block_step(batch, block_len, d_model, n_heads, dtype, _vp(w_qkv), _vp(w_o), _vp(x_blk), _vp(k_cache), _vp(v_cache),
+                                     cache_len, cache_cap, _vp(y_blk), _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
 
 
 def dm_attention_workspace_bytes(batch: int, seqlen: int, d_model: int, dtype: int) -> int:

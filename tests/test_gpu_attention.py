@@ -114,3 +114,97 @@ def test_hybrid_stack_against_the_oracle(G, cond):
     plain, _, _ = G.run_denoise(shape, I.BF16, sw, tok, V, want_argmax=False, tau=tau, d_ff=d_ff)
     np.testing.assert_array_equal(G.run_denoise_hybrid(shape, I.BF16, sw, tok, V, 0, 2, tau=tau, d_ff=d_ff), plain)
     assert np.any(got != plain)
+
+
+def test_attention_block_step_with_cache(G):
+    """Prefix of 200 tokens through the block entry point with an empty cache, then a block of 40 that attends to the cached
+    prefix and to itself: outputs and cache contents against the oracle; rows past the valid keys of the cache hold NaN on
+    purpose (the kernel must not let them in)."""
+    from paper_2511_15927_b200 import binding as dm
+    B, H, cap = 2, 2, 300
+    d = 64 * H
+    x, wq, wo = _case(B, 240, H, 31, 1.0)
+    wqd, wod = G.dev(wq, I.BF16), G.dev(wo, I.BF16)
+    kc = torch.full((B, cap, d), float("nan"), device="cuda", dtype=torch.bfloat16)
+    vc = torch.full((B, cap, d), float("nan"), device="cuda", dtype=torch.bfloat16)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def run(xb, cache_len):
+        xd = G.dev(xb, I.BF16)
+        yd = torch.empty_like(xd)
+        nb = dm.dm_attention_workspace_bytes(B, xb.shape[1], d, dm.DM_BF16)
+        ws = G.workspace(nb)
+        dm.dm_attention_block_step(B, xb.shape[1], d, H, dm.DM_BF16, wqd.data_ptr(), wod.data_ptr(), xd.data_ptr(), kc.data_ptr(), vc.data_ptr(),
+                                   cache_len, cap, yd.data_ptr(), ws.data_ptr(), nb, st)
+        dm.dm_check(st)
+        return yd.float().cpu().numpy().astype(np.float64)
+
+    y1 = run(np.ascontiguousarray(x[:, :200]), 0)
+    w1, k1, v1 = O.attention_block_step(x[:, :200], wq, wo, H)
+    assert np.all(np.isfinite(y1)) and G.rel_l2(y1, w1) <= BF16_REL
+    y2 = run(np.ascontiguousarray(x[:, 200:]), 200)
+    # the oracle continues from the cache as the library stores it (bf16)
+    k1r, v1r = kc[:, :200].float().cpu().numpy().astype(np.float64), vc[:, :200].float().cpu().numpy().astype(np.float64)
+    assert G.rel_l2(k1r, k1) <= 5e-3 and G.rel_l2(v1r, v1) <= 5e-3
+    w2, k2, v2 = O.attention_block_step(x[:, 200:], wq, wo, H, k1r, v1r)
+    assert np.all(np.isfinite(y2)) and G.rel_l2(y2, w2) <= BF16_REL and G.max_abs(y2, w2) <= BF16_ABS
+    assert G.rel_l2(kc[:, :240].float().cpu().numpy().astype(np.float64), k2) <= 5e-3
+    assert torch.isnan(kc[:, 240:]).all() and torch.isnan(vc[:, 240:]).all()          # nothing written past the block
+    before = dm.dm_kernel_launch_count()
+    with pytest.raises(dm.DmError):
+        run(np.ascontiguousarray(x[:, :100]), 250)                                     # 250 + 100 > cap
+    assert dm.dm_kernel_launch_count() == before
+
+
+def test_hybrid_stack_block_mode(G):
+    """Prefix pass commits Mamba states and key/value caches, the next block starts from them (Sec. 4.3)."""
+    from paper_2511_15927_b200 import binding as dm
+    import tests.gpu_util as U
+    B, G1, G2, V, layers, period, heads = 2, 96, 32, 504, 4, 2, 2
+    full = I.MixerShape(B, G1 + G2, 128, 2, 128, 4, 4)
+    sw, _, _ = _hybrid_stack(full, layers, V, 41, False)
+    tok = I.make_tokens(B, G1 + G2, V - 1, V - 1, seed=41)
+    kw = G.oracle_kwargs(full)
+    want1, st_o = O.denoise_step_hybrid(tok[:, :G1], sw, attn_period=period, attn_heads=heads, return_states=True, **kw)
+    d, cap = full.d_model, 160
+    dsw = U.dev_stack_weights(sw, I.BF16)
+    csw, keep = dm.make_stack_weights(dsw)
+    daw = [{"w_qkv": G.dev(l["w_qkv"], I.BF16), "w_o": G.dev(l["w_o"], I.BF16)} for l in sw["layers"]]
+    caw = dm.make_attn_weights(daw)
+    caches = [(torch.zeros((B, cap, d), device="cuda", dtype=torch.bfloat16), torch.zeros((B, cap, d), device="cuda", dtype=torch.bfloat16)) for _ in range(layers)]
+    ssm = [torch.zeros((B, full.n_heads, full.headdim, full.d_state), device="cuda") for _ in range(layers)]
+    conv = [torch.zeros((B, full.d_conv - 1, full.conv_ch), device="cuda", dtype=torch.bfloat16) for _ in range(layers)]
+    st = torch.cuda.current_stream().cuda_stream
+
+    def step(tokens, L, cache_len, first):
+        shape = I.MixerShape(B, L, full.d_model, 2, full.d_state, 4, full.n_heads)
+        scfg = dm.dm_stack_cfg(U.cfg_of(shape, I.BF16), layers, V, 1e-5)
+        states = (dm.dm_layer_state * layers)()
+        ast = (dm.dm_attn_state * layers)()
+        for i in range(layers):
+            if first:
+                states[i] = dm.dm_layer_state(None, None, ssm[i].data_ptr(), conv[i].data_ptr())       # commit
+            else:
+                states[i] = dm.dm_layer_state(ssm[i].data_ptr(), conv[i].data_ptr(), None, None)       # read only
+            ast[i] = dm.dm_attn_state(caches[i][0].data_ptr(), caches[i][1].data_ptr(), cache_len, cap)
+        td = G.dev(np.asarray(tokens, np.int32))
+        logits = torch.empty((B, L, V), device="cuda", dtype=torch.bfloat16)
+        nb = dm.dm_denoise_hybrid_workspace_bytes(scfg, None)
+        ws = G.workspace(nb)
+        dm.dm_denoise_step_hybrid_block(scfg, None, dm.dm_hybrid_cfg(period, heads), csw, None, caw, td.data_ptr(), 0, logits.data_ptr(), 0,
+                                        states, ast, ws.data_ptr(), nb, st)
+        dm.dm_check(st)
+        return logits.float().cpu().numpy().astype(np.float64)
+
+    got1 = step(tok[:, :G1], G1, 0, True)
+    assert G.rel_l2(got1, want1) <= 1e-2, G.rel_l2(got1, want1)
+    # the oracle continues from the states as the library holds them
+    st_in = []
+    for i in range(layers):
+        if i % period == 0:
+            st_in.append((caches[i][0][:, :G1].float().cpu().numpy().astype(np.float64), caches[i][1][:, :G1].float().cpu().numpy().astype(np.float64)))
+        else:
+            st_in.append((ssm[i].cpu().numpy().astype(np.float64), conv[i].float().cpu().numpy().astype(np.float64)))
+    want2, _ = O.denoise_step_hybrid(tok[:, G1:], sw, attn_period=period, attn_heads=heads, states_in=st_in, return_states=True, **kw)
+    got2 = step(tok[:, G1:], G2, G1, False)
+    assert G.rel_l2(got2, want2) <= 1e-2, G.rel_l2(got2, want2)
