@@ -202,6 +202,11 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
 // --------------------------------------------------------------------------------------------------
 // Launch 2: the chunked scan.
 // --------------------------------------------------------------------------------------------------
+// HALFP: the model's headdim is P / 2.  The CTA still moves 64-channel tiles (the second half is padding that never
+// leaves it), but the conv, the state hand-over and the epilogue work on the 32 real channels only, split over the
+// same threads; the padded halves of the w o x' tile and of the state copy are zeroed once, so the padded state
+// columns stay zero.
+template <bool HALFP>
 __global__ void __launch_bounds__(NTHREADS, 1)
 ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_z,
                 const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_c,
@@ -370,9 +375,10 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
     } else if (warp < 4 + 4 * NWG) {
         // ============================================================ state update; conv + SiLU of the x tile; w o x'
-        constexpr int RB = Q * 16 / ROLE;               // rows per thread
+        constexpr int CG = HALFP ? 8 : 16;              // 8-byte column groups (4 channels each) that carry real channels
+        constexpr int RB = Q * CG / ROLE;               // rows per thread
         const int t = tid - 4 * 32;                     // 0..ROLE-1
-        const int cg = t & 15, rb = t >> 4;             // 8-byte column group (4 channels) x block of RB rows
+        const int cg = t & (CG - 1), rb = t / CG;       // column group x block of RB rows
         const uint32_t colx = cg >> 1, sub = (cg & 1) * 8;
         f32x2 wl2[2][4], cb2[2];                        // per channel pair; wl2[.][m] multiplies the row m steps back in time
         {
@@ -396,6 +402,15 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int first = rev ? rb * RB + RB - 1 : rb * RB, step = rev ? -1 : 1;   // first-in-time chunk row of the block
         const int toff = rev ? 0 : HALO;                                          // tile row = chunk row + toff
         const int srow = t & (WG - 1), sh = t >> 7;      // state row and column half of this thread
+        constexpr int SC8 = HALFP ? 2 : 4;              // 8-column groups of the state per thread
+        if (HALFP) {                                     // padded halves of w o x' and of the bf16 state copy
+            for (int i = t; i < Q * 4; i += ROLE) {
+                const int r = i >> 2, c16 = 4 + (i & 3);
+                const uint32_t o = r * 128 + ((c16 ^ (r & 7)) << 4);
+                *reinterpret_cast<uint4 *>(smem + OFF_XS + o) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4 *>(smem + OFF_H + o) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
         // incoming state -> TMEM (fp32)
         {
             const float *h0 = (!rev && a.ssm_in && srow < a.Nr && sh * 32 < Pr) ? a.ssm_in + (((int64_t)b * a.H + h) * Pr) * a.Nr + srow : nullptr;
@@ -404,6 +419,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(sh * 32 + p) * a.Nr]) : 0u;
             tmem_st_x32(tlane + TM_HS + sh * 32, hs);
             tmem_wait_st();
+            fence_before();                              // the hand-over (after the group barrier) may read columns another warp stored
         }
         // The fp32 state lives in TMEM and St accumulates onto it: before chunk c's St is issued, the state entering the
         // chunk is copied to shared memory as bf16 (B operand of Yb) and scaled in place by the chunk's total decay, so
@@ -412,7 +428,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_after();
             const f32x2 dec2 = pk2(dec, dec);
 #pragma unroll 1
-            for (int c8 = sh * 4; c8 < sh * 4 + 4; ++c8) {   // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
+            for (int c8 = sh * SC8; c8 < sh * SC8 + SC8; ++c8) {   // 8 state columns (one 16-byte chunk of the bf16 copy) at a time
                 uint32_t hs[8];
                 tmem_ld_x8(tlane + TM_HS + c8 * 8, hs);
                 tmem_wait_ld();
@@ -467,9 +483,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             named_sync(1, ROLE);                           // halo rows are in registers; wbuf is visible
             // Row j of the block sits at j * 128 + ((colx ^ (j & 7)) << 4) in both tiles; with j & 7 = jx this is
             // ((9 jx) ^ colx) << 4, so one running counter k = 144 jx and one exclusive-or give the offset of every row.
-            uint8_t *bx = xt + (toff + rb * RB) * 128 + sub, *bs = smem + OFF_XS + rb * RB * 128 + sub;
+            constexpr int R8 = 8 / RB;                          // blocks per group of eight rows
+            const int r8 = (rb / R8) * 8, rlo = (rb % R8) * RB;  // the block starts rlo rows into the eight rows at r8
+            uint8_t *bx = xt + (toff + r8) * 128 + sub, *bs = smem + OFF_XS + r8 * 128 + sub;
             const uint8_t *wp = reinterpret_cast<const uint8_t *>(misc->wbuf + rb * RB + (rev ? RB - 1 : 0));
-            uint32_t k = rev ? (RB - 1) * 144u : 0u;
+            uint32_t k = (uint32_t)(rlo + (rev ? RB - 1 : 0)) * 144u;
 #pragma unroll 2
             for (int tau = 0; tau < RB; ++tau) {
                 const uint32_t off = k ^ (colx << 4);
@@ -602,6 +620,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ============================================================ epilogue
         const int eg = (warp - 4 - 8 * NWG) >> 2;       // group index: channels [eg, eg+1) * P / NWG
         const int row = (tid - (4 + 8 * NWG) * 32) & (WG - 1);
+        constexpr int EC8 = HALFP ? 2 : 4;              // 8-channel groups per thread
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
             const int sz = c % NZ, sd = c % NDL, pc = rev ? nch - 1 - c : c;
@@ -617,12 +636,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const f32x2 ei2 = pk2(ei, ei);
             f32x2 ss2 = pk2(0.f, 0.f);
 #pragma unroll 1
-            for (int c8 = eg * 4; c8 < eg * 4 + 4; ++c8) {   // 8 channels (one 16-byte chunk of z) at a time
+            for (int c8 = eg * EC8; c8 < eg * EC8 + EC8; ++c8) {   // 8 channels (one 16-byte chunk of z) at a time
                 uint32_t ya[8], yb[8];
                 tmem_ld_x8(tlane + TM_YA + c8 * 8, ya);
                 tmem_ld_x8(tlane + (par ? TM_YB1 : TM_YB0) + c8 * 8, yb);
                 tmem_wait_ld();
-                if (c8 == eg * 4 + 3) { fence_before(); mbar_arrive(&misc->ya_empty); mbar_arrive(&misc->yb_empty[par]); }
+                if (c8 == eg * EC8 + EC8 - 1) { fence_before(); mbar_arrive(&misc->ya_empty); mbar_arrive(&misc->yb_empty[par]); }
                 uint4 *zp = reinterpret_cast<uint4 *>(zt + row * 128 + ((c8 ^ (row & 7)) << 4));
                 const uint4 zv = *zp;
                 const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
@@ -637,8 +656,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     ss2 = fma2(g, g, ss2);
                     ow[e2] = f2_to_bf2(mul2(g, nw[e2]));
                 }
-                if (Pr == P) *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-                else if (eg == 0 && t < L)      // half-width head: its 32 channels go out with plain stores, 64 bytes per token
+                if (!HALFP) *zp = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                else if (t < L)                 // half-width head: its 32 channels go out with plain stores, 64 bytes per token
                     *reinterpret_cast<uint4 *>(a.g + ((int64_t)seq * L + t) * a.d_inner + h * Pr + c8 * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
             }
             float ss, ss_hi;
@@ -647,9 +666,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (eg == 1) misc->ssq_part[row] = ss;
             fence_proxy_async();
             named_sync(2, ROLE);
-            if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + (Pr == P ? misc->ssq_part[row] : 0.f);
+            if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + misc->ssq_part[row];
             if (eg == 0 && row == 0) {
-                if (Pr == P) {
+                if (!HALFP) {
                     tma_store_3d(&map_g, zt, h * P, pc * Q, seq);    // rows past the end of the sequence are clipped
                     bulk_commit();
                     bulk_wait_read0();
@@ -741,9 +760,10 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(ssd_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    auto kern = a.P == P ? ssd_scan_kernel<false> : ssd_scan_kernel<true>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    ssd_scan_kernel<<<dim3(a.H, ndir, a.B), NTHREADS, SMEM_BYTES, s>>>(mx, mz, mb, mc, mg, k, dir0, status);
+    kern<<<dim3(a.H, ndir, a.B), NTHREADS, SMEM_BYTES, s>>>(mx, mz, mb, mc, mg, k, dir0, status);
     count_launch();
     return cudaGetLastError();
 }
