@@ -317,7 +317,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // Order per iteration: S(c), Yb(c), Ya(c-1), St(c).  S(c) goes out as soon as the mask of chunk c-1 has read
         // S(c-1); Yb(c) follows at once (its accumulator is double-buffered, so it does not wait for the epilogue of
         // chunk c-1), which frees the single C' buffer early enough for the next chunk's load.
-        if (lane == 0) {
+        // Half-width heads: the whole warp walks the loop and waits, one elected lane issues the products and their
+        // commits (the operand descriptors then live in uniform registers and a product takes a third of the time to
+        // issue), and Ya(c-1) goes out before Yb(c) so that the mask of chunk c starts earlier.  With full-width heads
+        // the conv groups are the longer chain and both changes only take issue slots from them at the wrong time
+        // (measured 5 % slower), so there one lane runs the loop and Ya(c-1) follows Yb(c).
+        auto mma_role = [&](const bool leader) {
             // low halves of the operand descriptors; a K step of 16 advances a K-major operand by 32 bytes inside its
             // 64-wide tile (+2) or to the next tile (+T16/16), an MN-major operand by 16 rows (+2048/16)
             const uint32_t dH = desc_lo_mn(smem_u32(smem + OFF_H), T16), dXs = desc_lo_mn(smem_u32(smem + OFF_XS), T16);
@@ -330,11 +335,11 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!WAIT2(&misc->w_full, c & 1, &misc->ya_empty, (c & 1) ^ 1)) return false;
                 fence_after();
                 const uint32_t dX = dX0 + (uint32_t)sx * (XTILE >> 4);
-                umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
+                if (leader) umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
 #pragma unroll
-                for (int kk = 1; kk < 8; ++kk) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
-                umma_commit(&misc->y_full);              // Yb of the same chunk was issued earlier: it has completed as well; also frees W
-                umma_commit(&misc->empty_x[sx]);
+                for (int kk = 1; kk < 8; ++kk) if (leader) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
+                if (leader) umma_commit(&misc->y_full);              // Yb of the same chunk was issued earlier: it has completed as well; also frees W
+                if (leader) umma_commit(&misc->empty_x[sx]);
                 return true;
             };
             bool ok = true;
@@ -345,34 +350,37 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 // S = C' B'^T  (both K-major in shared memory)
                 if (!WAIT3(&misc->full_c, par, &misc->full_b[sb], (c / NB) & 1, &misc->s_empty, par ^ 1)) break;
                 fence_after();
-                umma_ss<0>(tmem + TM_S, dC, dBk, I128);
+                if (leader) umma_ss<0>(tmem + TM_S, dC, dBk, I128);
 #pragma unroll
                 for (int kk = 1; kk < 8; ++kk) {
                     const uint32_t o = (kk >> 2) * (T16 >> 4) + 2 * (kk & 3);
-                    umma_ss<1>(tmem + TM_S, dC + o, dBk + o, I128);
+                    if (leader) umma_ss<1>(tmem + TM_S, dC + o, dBk + o, I128);
                 }
-                umma_commit(&misc->s_full);
+                if (leader) umma_commit(&misc->s_full);
+                if constexpr (HALFP) { if (c > 0 && !issue_ya(c - 1)) break; }
                 // Yb = C' h_in  (A = C' K-major, B = bf16 state [n][p] MN-major) into the buffer the epilogue of chunk c-2 has drained;
                 // its completion releases C' (S was issued before it) and the state copy
                 const uint32_t tyb = tmem + (par ? TM_YB1 : TM_YB0);
                 if (!WAIT2(&misc->h_full, par, &misc->yb_empty[par], ((c >> 1) & 1) ^ 1)) break;
                 fence_after();
-                umma_ss<0>(tyb, dC, dH, I64);
+                if (leader) umma_ss<0>(tyb, dC, dH, I64);
 #pragma unroll
-                for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tyb, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), dH + kk * 128, I64);
-                umma_commit(&misc->empty_c);             // also releases the bf16 state copy
-                if (c > 0 && !issue_ya(c - 1)) break;
+                for (int kk = 1; kk < 8; ++kk) if (leader) umma_ss<1>(tyb, dC + (kk >> 2) * (T16 >> 4) + 2 * (kk & 3), dH + kk * 128, I64);
+                if (leader) umma_commit(&misc->empty_c);             // also releases the bf16 state copy
+                if constexpr (!HALFP) { if (c > 0 && !issue_ya(c - 1)) break; }
                 // h += B'^T (w o x')  (A = B' [j][n] MN-major, B = w o x' [j][p] MN-major), onto the state the conv groups have scaled
                 if (!WAIT2(&misc->xs_full, par, &misc->hs_ready, par)) break;
                 fence_after();
-                umma_ss<1>(tmem + TM_HS, dBm, dXs, I64T);
+                if (leader) umma_ss<1>(tmem + TM_HS, dBm, dXs, I64T);
 #pragma unroll
-                for (int kk = 1; kk < 8; ++kk) umma_ss<1>(tmem + TM_HS, dBm + kk * 128, dXs + kk * 128, I64T);
-                umma_commit(&misc->st_full);             // also frees the w o x' buffer
-                umma_commit(&misc->empty_b[sb]);
+                for (int kk = 1; kk < 8; ++kk) if (leader) umma_ss<1>(tmem + TM_HS, dBm + kk * 128, dXs + kk * 128, I64T);
+                if (leader) umma_commit(&misc->st_full);             // also frees the w o x' buffer
+                if (leader) umma_commit(&misc->empty_b[sb]);
                 if (c == nch - 1) ok = issue_ya(c);
             }
-        }
+        };
+        if constexpr (HALFP) mma_role(elect_one());
+        else if (lane == 0) mma_role(true);
     } else if (warp < 4 + 4 * NWG) {
         // ============================================================ state update; conv + SiLU of the x tile; w o x'
         constexpr int CG = HALFP ? 8 : 16;              // 8-byte column groups (4 channels each) that carry real channels
