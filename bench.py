@@ -31,7 +31,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (taken on
 # cfg3_8k = 8192 tokens; traffic of both kernels grows in proportion to the token count, so other single-layer bf16
 # workloads of the same widths scale it by their tokens; None = no capture applies).
-NCU_TRAFFIC_PER_TOKEN = {"scan": (286.4246e6 + 109.3309e6) / 8192,      # ssd_scan_kernel, profiles/ssd_scan_cfg3_8k.txt
+NCU_TRAFFIC_PER_TOKEN = {"scan": (286.4230e6 + 108.9836e6) / 8192,      # ssd_scan_kernel, profiles/ssd_scan_cfg3_8k.txt
                          "in_proj": (72.3308e6 + 112.3448e6) / 8192}    # gemm_tc_kernel<256>, one direction, profiles/gemm_tc_cfg3_8k.txt
 NCU_WIDTHS = (2048, 128, 64)                                             # d_model, d_state, heads the captures were taken at
 
