@@ -61,7 +61,12 @@ typedef struct {
     int32_t flags;      /* DM_FLAG_* */
     int32_t dir_mask;   /* DM_DIR_BOTH; one direction alone is meant for invariant tests */
     int32_t chunk;      /* tokens per scan chunk; 0 = library default.  Results do not depend on it
-                           beyond rounding order. */
+                           beyond rounding order.  bf16 with d_state <= 128 runs the chunked form of the
+                           recurrence and takes 0, 128 (tensor-core kernel; the default above 64 tokens)
+                           or 32 (CUDA-core kernel; the default up to 64 tokens, i.e. for the blocks of
+                           block-autoregressive decoding) -- other values: DM_ERR_UNSUPPORTED.  fp32, and
+                           d_state 256, run the sequential form, where any chunk > 0 only sizes the
+                           staging buffers. */
     float   norm_eps;   /* epsilon of the gated RMS norm */
 } dm_mixer_cfg;
 
@@ -219,8 +224,8 @@ int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
  * x, y [B, L, d_model] dtype (y != x); w_qkv [3 * d_model, d_model] with rows [Q | K | V], each split into
  * n_heads consecutive blocks of d_h = d_model / n_heads; w_o [d_model, d_model].  bf16 only, d_h = 64 only
  * (DM_ERR_UNSUPPORTED otherwise).  The scores never leave the SM (running-maximum softmax over key tiles);
- * P is rounded to bf16 before P V, accumulation is fp32.  The hybrid stack itself (which layers are attention)
- * is not assembled by the library. */
+ * P is rounded to bf16 before P V, accumulation is fp32.  The hybrid stack (which layers are attention) is
+ * dm_denoise_step_hybrid below. */
 int dm_attention_workspace_bytes(int32_t batch, int32_t seqlen, int32_t d_model, int32_t dtype, size_t *bytes);
 int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t n_heads, int32_t dtype,
                          const void *w_qkv, const void *w_o, const void *x, void *y,

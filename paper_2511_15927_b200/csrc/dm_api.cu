@@ -66,6 +66,7 @@ static int cuda_fail(cudaError_t e, const char *what) {
 
 struct Dims {
     int B, L, d, d_inner, H, P, N, k, G, conv_ch, d_in_proj;
+    int ldz;          // row pitch of the in_proj output in the workspace: d_in_proj rounded up to 8 elements (16-byte rows for TMA and vector loads)
     int64_t T;
     size_t es;
 };
@@ -91,10 +92,13 @@ static int check_cfg(const dm_mixer_cfg *c, Dims *o) {
     if (N != 16 && N != 32 && N != 64 && N != 128 && N != 256) return fail(DM_ERR_UNSUPPORTED, "d_state must be 16, 32, 64, 128 or 256");
     if ((int64_t)P * (N / 16) > 1024) return fail(DM_ERR_UNSUPPORTED, "headdim * d_state / 16 must not exceed 1024");
     if ((int64_t)c->batch * c->seqlen > (int64_t)1 << 30) return fail(DM_ERR_UNSUPPORTED, "batch*seqlen too large");
+    if (!scan_ssd_chunk_ok(c->dtype, N, c->chunk))
+        return fail(DM_ERR_UNSUPPORTED, "bf16 with d_state <= 128 runs the chunked scan: chunk must be 0, 32 or 128 (got %d)", c->chunk);
     o->B = c->batch; o->L = c->seqlen; o->d = c->d_model; o->d_inner = (int)d_inner; o->H = c->n_heads; o->P = P;
     o->N = N; o->k = c->d_conv; o->G = 1;
     o->conv_ch = o->d_inner + 2 * N;
     o->d_in_proj = 2 * o->d_inner + 2 * N + o->H;
+    o->ldz = (o->d_in_proj + 7) / 8 * 8;
     o->T = (int64_t)c->batch * c->seqlen;
     o->es = dtype_size(c->dtype);
     return DM_OK;
@@ -122,14 +126,14 @@ struct MixerWs {
 static MixerWs mixer_ws(const dm_mixer_cfg *c, const Dims &m) {
     MixerWs w;
     size_t off = 0;
-    w.zx = off;   off += align_up((size_t)2 * m.T * m.d_in_proj * m.es);
+    w.zx = off;   off += align_up((size_t)2 * m.T * m.ldz * m.es);
     w.g = off;    off += align_up((size_t)2 * m.T * m.d_inner * m.es);
     w.ssq = off;  off += align_up((size_t)2 * m.T * m.H * sizeof(float));
     w.rstd = off; off += align_up((size_t)2 * m.T * sizeof(float));
     w.ytmp = off; off += align_up((size_t)m.T * m.d * sizeof(float));
     ScanArgs sa{};
     sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
-    sa.d_in_proj = m.d_in_proj; sa.conv_ch = m.conv_ch; sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask;
+    sa.d_in_proj = m.ldz; sa.conv_ch = m.conv_ch; sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask; sa.chunk = c->chunk;
     {
         const size_t a_ssd = scan_ssd_workspace_bytes(sa), a_seq = scan_seq_workspace_bytes(sa);
         w.scan = off; off += align_up(a_ssd > a_seq ? a_ssd : a_seq);
@@ -161,7 +165,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
 
     ScanArgs sa{};
     sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
-    sa.d_in_proj = m.d_in_proj; sa.conv_ch = m.conv_ch;
+    sa.d_in_proj = m.ldz; sa.conv_ch = m.conv_ch;          // the kernels use it as the row pitch only
     sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask; sa.chunk = c->chunk;
     sa.zx = zx; sa.g = g; sa.ssq = norm_on ? ssq : nullptr;
     for (int dir = 0; dir < 2; ++dir) {
@@ -180,7 +184,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         StageTimer tm(DM_STAGE_IN_PROJ, s);
         GemmArgs a{};
         a.A = x; a.lda = m.d; a.B = w[dir].w_in; a.ldb = m.d;
-        a.C = zx + (size_t)dir * m.T * m.d_in_proj * m.es; a.ldc = m.d_in_proj;
+        a.C = zx + (size_t)dir * m.T * m.ldz * m.es; a.ldc = m.ldz;
         a.in_dtype = c->dtype; a.c_dtype = c->dtype; a.M = (int)m.T; a.N = m.d_in_proj; a.K = m.d;
         a.silu_cols = ssd ? m.d_inner : 0;
         if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "in_proj");
@@ -193,7 +197,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
     if (e != cudaSuccess) return cuda_fail(e, "scan");
 
     if (conv_out && (c->dir_mask & DM_DIR_FWD)) {
-        e = conv_state_update(zx, conv_in, conv_out, c->dtype, m.B, m.L, m.k, m.d_inner, m.conv_ch, m.d_in_proj, s);
+        e = conv_state_update(zx, conv_in, conv_out, c->dtype, m.B, m.L, m.k, m.d_inner, m.conv_ch, m.ldz, s);
         if (e != cudaSuccess) return cuda_fail(e, "conv_state_update");
     }
     if (norm_on) {
@@ -799,7 +803,9 @@ int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], 
     Dims m;
     int st = check_cfg(cfg, &m);
     if (st != DM_OK) return st;
+    if ((st = check_weights(cfg, w)) != DM_OK) return st;        // everything the per-piece calls would reject is rejected here, before the first copy
     if (!x_host || !y_host) return fail(DM_ERR_INVALID_ARG, "x_host or y_host is NULL");
+    if (x_host == y_host) return fail(DM_ERR_INVALID_ARG, "y_host must not alias x_host");
     const size_t act = align_up((size_t)m.T * m.d * m.es);
     const size_t need = mixer_ws(cfg, m).total + 2 * act;
     if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;
@@ -822,24 +828,32 @@ int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2], 
     if ((e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess) return cuda_fail(e, "wait");      // after the caller's earlier work
     if ((e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess) return cuda_fail(e, "wait");
     dm_mixer_cfg piece_cfg = *cfg;
+    // A failure after the first copy was enqueued: let the copy streams drain (their copies still read and write the
+    // caller's buffers) and rejoin the caller's stream before reporting it.
+    auto bail = [&](int status) {
+        cudaStreamSynchronize(hp->in);
+        cudaStreamSynchronize(hp->out);
+        cudaStreamSynchronize(s);
+        return status;
+    };
     for (int i = 0; i < pieces; ++i) {
         const int r0 = i * rows, nr = (r0 + rows <= m.B) ? rows : m.B - r0;
         const size_t off = (size_t)r0 * row_bytes, bytes = (size_t)nr * row_bytes;
         if ((e = cudaMemcpyAsync(xd + off, static_cast<const char *>(x_host) + off, bytes, cudaMemcpyHostToDevice, hp->in)) != cudaSuccess)
-            return cuda_fail(e, "copy x to the device");
-        if ((e = cudaEventRecord(hp->copied[i], hp->in)) != cudaSuccess) return cuda_fail(e, "record");
-        if ((e = cudaStreamWaitEvent(s, hp->copied[i], 0)) != cudaSuccess) return cuda_fail(e, "wait");
+            return bail(cuda_fail(e, "copy x to the device"));
+        if ((e = cudaEventRecord(hp->copied[i], hp->in)) != cudaSuccess) return bail(cuda_fail(e, "record"));
+        if ((e = cudaStreamWaitEvent(s, hp->copied[i], 0)) != cudaSuccess) return bail(cuda_fail(e, "wait"));
         piece_cfg.batch = nr;
         st = dm_bimamba_forward(&piece_cfg, w, xd + off, yd + off, ws + 2 * act, workspace_bytes - 2 * act, cuda_stream);
-        if (st != DM_OK) return st;
-        if ((e = cudaEventRecord(hp->computed[i], s)) != cudaSuccess) return cuda_fail(e, "record");
-        if ((e = cudaStreamWaitEvent(hp->out, hp->computed[i], 0)) != cudaSuccess) return cuda_fail(e, "wait");
+        if (st != DM_OK) return bail(st);
+        if ((e = cudaEventRecord(hp->computed[i], s)) != cudaSuccess) return bail(cuda_fail(e, "record"));
+        if ((e = cudaStreamWaitEvent(hp->out, hp->computed[i], 0)) != cudaSuccess) return bail(cuda_fail(e, "wait"));
         if ((e = cudaMemcpyAsync(static_cast<char *>(y_host) + off, yd + off, bytes, cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
-            return cuda_fail(e, "copy y to the host");
+            return bail(cuda_fail(e, "copy y to the host"));
     }
-    if ((e = cudaEventRecord(hp->done, hp->out)) != cudaSuccess) return cuda_fail(e, "record");
-    if ((e = cudaStreamWaitEvent(s, hp->done, 0)) != cudaSuccess) return cuda_fail(e, "wait");
-    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e, "synchronize");
+    if ((e = cudaEventRecord(hp->done, hp->out)) != cudaSuccess) return bail(cuda_fail(e, "record"));
+    if ((e = cudaStreamWaitEvent(s, hp->done, 0)) != cudaSuccess) return bail(cuda_fail(e, "wait"));
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return bail(cuda_fail(e, "synchronize"));
     return DM_OK;
 }
 

@@ -55,7 +55,9 @@ struct ScanDir {
     const float *dt_bias, *A_log, *D;
 };
 struct ScanArgs {
-    int B, L, d_inner, H, P, N, k, d_in_proj, conv_ch;
+    int B, L, d_inner, H, P, N, k;
+    int d_in_proj;           // row pitch of zx in elements (>= 2 d_inner + 2 N + H; the columns beyond are padding)
+    int conv_ch;
     int dtype, flags, dir_mask, chunk;
     const void *zx;          // [2][B*L][d_in_proj] dtype: in_proj output of each direction
     int z_gated;             // the z columns of zx already hold SiLU(z) (applied by the in_proj epilogue); the tensor-core scan requires it
@@ -69,6 +71,8 @@ struct ScanArgs {
 size_t scan_seq_workspace_bytes(const ScanArgs &a);
 cudaError_t scan_sequential(const ScanArgs &a, void *ws, cudaStream_t s);
 bool scan_ssd_supports(const ScanArgs &a);
+// chunk values the chunked bf16 path takes (0 = default, 32 = CUDA-core kernel, 128 = tensor-core kernel); other paths take any chunk > 0
+bool scan_ssd_chunk_ok(int dtype, int d_state, int chunk);
 size_t scan_ssd_workspace_bytes(const ScanArgs &a);
 cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s);
 
@@ -108,7 +112,5 @@ cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int 
 // conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])
 cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *conv_out, int dtype, int B, int L,
                               int k, int d_inner, int conv_ch, int d_in_proj, cudaStream_t s);
-// y[i] = (dtype) src[i]
-cudaError_t cast_f32_rows(const float *src, void *dst, int dtype, size_t n, cudaStream_t s);
 
 }  // namespace dm

@@ -207,11 +207,6 @@ __global__ void conv_state_kernel(const T *__restrict__ zx, const T *__restrict_
     conv_out[((int64_t)b * (k - 1) + r) * conv_ch + c] = v;
 }
 
-template <typename T>
-__global__ void cast_kernel(const float *__restrict__ src, T *__restrict__ dst, size_t n) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) stf(dst + i, src[i]);
-}
-
 }  // namespace
 
 cudaError_t rstd_from_ssq(const float *ssq, float *rstd, int rows, int H, int d_inner, float eps, cudaStream_t s) {
@@ -267,14 +262,6 @@ cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *con
     else
         conv_state_kernel<<<grid, 256, 0, s>>>(static_cast<const float *>(zx_fwd), static_cast<const float *>(conv_in),
                                                static_cast<float *>(conv_out), L, k, d_inner, conv_ch, d_in_proj);
-    count_launch();
-    return cudaGetLastError();
-}
-
-cudaError_t cast_f32_rows(const float *src, void *dst, int dtype, size_t n, cudaStream_t s) {
-    const int blocks = (int)((n + 255) / 256 > 148 * 16 ? 148 * 16 : (n + 255) / 256);
-    if (dtype == DM_BF16) cast_kernel<<<blocks, 256, 0, s>>>(src, static_cast<__nv_bfloat16 *>(dst), n);
-    else cast_kernel<<<blocks, 256, 0, s>>>(src, static_cast<float *>(dst), n);
     count_launch();
     return cudaGetLastError();
 }

@@ -13,8 +13,9 @@
 // One __syncthreads per chunk hands the buffers over.  The first chunk is prepared, and the last one finished, by all
 // threads.  B' and C' (conv + SiLU of the B and C columns, shared by all heads) come from a small launch of their own.
 //
-// This is the exact (fp32) form of the recurrence; it is the kernel for fp32 I/O, for d_state other than 128 or
-// headdim other than 64, and for blocks with a carried conv state (block-autoregressive decoding).
+// This is the exact (fp32) form of the recurrence: the kernel for fp32 I/O (whose 1e-4 tolerance rules out bf16
+// products) and for d_state above 128; bf16 I/O with d_state <= 128 runs the chunked kernels of scan_ssd.cu, block
+// decoding with carried state included.
 #include "dm_internal.h"
 
 namespace dm {

@@ -1,7 +1,7 @@
-// Fused conv + selective scan + gate for bf16 I/O with d_state = 128 and headdim = 64, in the chunked
-// (state-space-duality) form of the same recurrence, with the chunk products on the tensor cores.
+// Fused conv + selective scan + gate for bf16 I/O with d_state <= 128 (zero-padded to 128) and headdim 64 or 32, in
+// the chunked (state-space-duality) form of the same recurrence.
 //
-// Unrolling h_t = a_t h_{t-1} + Delta_t x_t (x) B_t over one chunk of Q = 128 tokens, with
+// Unrolling h_t = a_t h_{t-1} + Delta_t x_t (x) B_t over one chunk of Q tokens, with
 // Lambda_i = sum_{r <= i} Delta_r A (inclusive, in the direction's own time order) gives
 //     y_i   = sum_{j <= i} exp(Lambda_i - Lambda_j) (C_i . B_j) Delta_j x_j  +  exp(Lambda_i) C_i . h_in  +  D x_i
 //     h_out = exp(Lambda_last) h_in + sum_j exp(Lambda_last - Lambda_j) Delta_j x_j (x) B_j
@@ -11,9 +11,10 @@
 //
 // Launch 1 (ssd_prep): per (direction, batch row, chunk): conv + SiLU of the B and C columns (shared by
 // all heads) to bf16, and Lambda, Lambda' of every head (in log2 units), into scratch.
-// Launch 2 (ssd_scan): one CTA per (batch row, direction, head) walks the chunks in the direction's time
-// order.  Both directions use the same physical chunk grid [c*Q, (c+1)*Q); the reverse direction visits
-// the chunks in descending order and uses the transposed causal mask, so nothing is ever flipped in memory.
+// Launch 2, long sequences (ssd_scan, Q = 128, chunk products on the tcgen05 tensor cores): one CTA per (batch row,
+// direction, head) walks the chunks in the direction's time order.  Both directions use the same physical chunk grid
+// [c*Q, (c+1)*Q); the reverse direction visits the chunks in descending order and uses the transposed causal mask, so
+// nothing is ever flipped in memory.
 // The CTA is a pipeline of specialised warps that work on different chunks at the same time:
 //     warp 0      TMA loads of the x tile (+ conv halo) and of Lambda, Lambda'
 //     warp 1      issues the four tcgen05 products of a chunk:  S = C B^T,  Yb = C h_in,  Ya = W x',  St = B^T (w o x')
@@ -27,6 +28,11 @@
 // Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
 // device status word, all roles leave their loops, outstanding TMA traffic is waited for (bounded), TMEM is
 // freed and the CTA returns.
+// Launch 2, short blocks (ssd_block, Q = 32, fp32 on the CUDA cores): the active block of block-autoregressive decoding
+// is 32 tokens, a quarter of one tensor-core tile, and a call has thousands of (batch row, head) items of that size; for
+// them the pipeline above is all set-up and tear-down.  ssd_block keeps the state of a head in registers, takes the
+// 32 x 32 matrix S of each sub-chunk from the prep launch (which computes it once per (batch row, direction) with
+// mma.sync) and does the rest of the identities above in fp32.  It is also what `chunk = 32` selects at any length.
 #include <cstddef>
 
 #include "dm_internal.h"
@@ -99,9 +105,28 @@ __device__ __forceinline__ float silu_fast(float v) { return v / (1.f + __expf(-
 // chain of dependent memory round trips, so many small CTAs per SM hide it better than few large ones.
 // --------------------------------------------------------------------------------------------------
 constexpr int PREP_PARTS = 4, PREP_THREADS = 128, PREP_HEADS = 64 / PREP_PARTS;
+constexpr int QB = Q / PREP_PARTS;          // tokens per sub-chunk of the short-block kernel = rows of one prep CTA
+constexpr int BCT_LD = N / 2 + 4;           // row pitch (32-bit words) of the prep CTA's B' / C' tile: 16-byte rows, conflict-free ldmatrix
+static_assert(QB == 32, "one prep CTA covers exactly one sub-chunk");
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t &r0, uint32_t &r1, const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(smem_u32(p)));
+}
+// D (16 x 8, fp32) += A (16 x 16, row-major) B (16 x 8, column-major), bf16 operands
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Sb != NULL (short-block mode): the CTA also writes S[i][j] = C'_i . B'_j over its own 32 rows, fp32, to Sb[seq][pc * 4 + part][32][32].
 __global__ void __launch_bounds__(PREP_THREADS)
-ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, int dir0) {
+ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, float *__restrict__ Sb,
+                int dir0) {
     __shared__ float dsm[Q][PREP_HEADS + 1];
+    __shared__ __align__(16) uint32_t bct[2][QB][BCT_LD];     // short-block mode: this CTA's rows of B' ([0]) and C' ([1]) as bf16 pairs
     const int pc = blockIdx.x / PREP_PARTS, part = blockIdx.x % PREP_PARTS, b = blockIdx.y, dir = dir0 + blockIdx.z;
     const bool rev = dir == 1;
     const int L = a.L, k = a.k, tid = threadIdx.x;
@@ -150,7 +175,35 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
                 v0 = fmaf(wl[0][m], bf16_lo(raw[i + 3 - m]), v0);
                 v1 = fmaf(wl[1][m], bf16_hi(raw[i + 3 - m]), v1);
             }
-            if (t < L) *reinterpret_cast<uint32_t *>(dst + (int64_t)t * N) = pack_bf16(silu_fast(v0), silu_fast(v1));
+            const uint32_t pk = pack_bf16(silu_fast(v0), silu_fast(v1));
+            if (t < L) *reinterpret_cast<uint32_t *>(dst + (int64_t)t * N) = pk;
+            if (Sb) bct[isC ? 1 : 0][rev ? QB - 1 - i : i][pi] = pk;          // row of the tile = physical row inside the block
+        }
+    }
+    if (Sb) {
+        // S = C' B'^T of this block's 32 rows on the legacy tensor path: warp = 16 rows i x 16 columns j, K = d_state
+        __syncthreads();
+        const int warp = tid >> 5, lane = tid & 31;
+        const int mt = warp & 1, nh = warp >> 1;
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+        for (int k0 = 0; k0 < N; k0 += 16) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(a0, a1, a2, a3, &bct[1][16 * mt + (lane & 15)][(k0 + (lane >> 4) * 8) / 2]);
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                uint32_t b0, b1;
+                ldmatrix_x2(b0, b1, &bct[0][16 * nh + 8 * nt + (lane & 7)][(k0 + ((lane >> 3) & 1) * 8) / 2]);
+                mma_bf16_16816(acc[nt], a0, a1, a2, a3, b0, b1);
+            }
+        }
+        float *S = Sb + (seq * (a.nch * PREP_PARTS) + pc * PREP_PARTS + part) * (QB * QB);
+        const int gr = lane >> 2, qc = lane & 3;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const int col = 16 * nh + 8 * nt + 2 * qc, row = 16 * mt + gr;
+            *reinterpret_cast<float2 *>(S + row * QB + col) = make_float2(acc[nt][0], acc[nt][1]);
+            *reinterpret_cast<float2 *>(S + (row + 8) * QB + col) = make_float2(acc[nt][2], acc[nt][3]);
         }
     }
     // ---- Delta, then the inclusive cumulative log-decay of every head in the direction's time order
@@ -696,8 +749,239 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
 }
 
+// --------------------------------------------------------------------------------------------------
+// Launch 2 for short blocks: sub-chunks of QB = 32 tokens, fp32 on the CUDA cores.
+// One CTA of 4 * PP threads per (batch row, direction, head of PP channels).  Thread (p, s4) = (tid / 4, tid % 4) keeps the 32
+// state entries h[p][n], n = 4 (4 k + s4) + e (k < 8, e < 4), in registers across the sub-chunks; per sub-chunk:
+//   load    x rows (+3 rows of conv history), B', C' (bf16 -> fp32), S (from the prep launch), Lambda, Lambda'
+//   conv    x' = SiLU(conv(x));   W_ij = S_ij 2^(Lambda_i - Lambda'_j) [+ D on the diagonal] for j not after i, else 0
+//   y       Yb: each thread's partial C'_i . h[p] over its 32 states for all 32 tokens, then a transposing reduction over
+//           the four lanes of p that leaves tokens i = 4 m + s4 with lane s4;  y_i = 2^(Lambda_i - Lambda_0) Yb_i + sum_j W_ij x'_j[p]
+//   gate    through shared memory to a (token, 8 channels) layout: g = y SiLU(z), sum of squares, * norm_w, 16-byte stores
+//   state   h <- 2^(Lambda_last - Lambda_0) h + sum_j 2^(Lambda_last - Lambda'_j) x'_j[p] B'_j   (only if someone will read it)
+// Lambda_0 is Lambda of the token before the sub-chunk inside the same 128-token chunk of the prep launch (0 at its start).
+// --------------------------------------------------------------------------------------------------
+constexpr int CLD = N + 4;             // row pitch of the fp32 B' / C' tiles
+constexpr int WLD = QB + 4;            // row pitch of W: 16-byte rows, conflict-free float4 reads by four different rows
+template <int PP> constexpr size_t block_smem_bytes() { return sizeof(float) * (2 * QB * CLD + (QB + 3) * PP + QB * PP + QB * WLD + 3 * QB + 4); }
+
+template <int PP>
+__global__ void __launch_bounds__(4 * PP, PP == 64 ? 2 : 4)
+ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __nv_bfloat16 *__restrict__ Cp, const float *__restrict__ Sb, int dir0) {
+    constexpr int NT = 4 * PP, U8 = PP / 8;
+    extern __shared__ __align__(16) float bsm[];
+    float (*Cs)[CLD] = reinterpret_cast<float (*)[CLD]>(bsm);
+    float (*Bs)[CLD] = reinterpret_cast<float (*)[CLD]>(bsm + QB * CLD);
+    float (*xr)[PP] = reinterpret_cast<float (*)[PP]>(bsm + 2 * QB * CLD);                   // raw x rows of the sub-chunk and its conv history; later its y
+    float (*xs)[PP] = reinterpret_cast<float (*)[PP]>(bsm + 2 * QB * CLD + (QB + 3) * PP);   // x'
+    float (*Ws)[WLD] = reinterpret_cast<float (*)[WLD]>(bsm + 2 * QB * CLD + (QB + 3) * PP + QB * PP);
+    float *lam = bsm + 2 * QB * CLD + (QB + 3) * PP + QB * PP + QB * WLD, *lamp = lam + QB, *wjs = lamp + QB, *sc = wjs + QB;
+
+    const int tid = threadIdx.x, p = tid >> 2, s4 = tid & 3;
+    const int h = blockIdx.x, b = blockIdx.z, dir = dir0 + blockIdx.y;
+    const bool rev = dir == 1;
+    const int L = a.L, k = a.k;
+    const int64_t seq = (int64_t)dir * a.B + b;
+    const ScanDir &w = a.dir[dir];
+    const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
+    const float *dA_head = a.dA + ((seq * a.H + h) * 2) * a.Lp;
+    const int nsub = (L + QB - 1) / QB, nsub_all = a.nch * PREP_PARTS;
+    const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
+    const bool norm_on = (a.flags & DM_FLAG_GATED_RMSNORM) != 0;
+
+    // per-thread constants: conv taps of channel tid % PP (wl[m] multiplies the row m steps back in time), norm weights of the epilogue's 8 channels
+    const int cch = tid % PP, crg = tid / PP;
+    float wl[4], cbias;
+    {
+        const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)(h * PP + cch) * k;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) wl[m] = m < k ? __bfloat162float(cw[k - 1 - m]) : 0.f;
+        cbias = ((a.flags & DM_FLAG_CONV_BIAS) && w.conv_b) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[h * PP + cch]) : 0.f;
+    }
+    const int ei = tid / U8, ec = (tid % U8) * 8;      // epilogue: token row of the sub-chunk, first of 8 channels
+    float nw[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        nw[e] = (norm_on && w.norm_w) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * PP + ec + e]) : 1.f;
+
+    float hst[32];
+    {
+        const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * PP + p) * a.Nr : nullptr;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            const int n0 = 4 * (4 * kk + s4);
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (h0 && n0 < a.Nr) v = *reinterpret_cast<const float4 *>(h0 + n0);      // rows beyond the model's d_state are padding
+            hst[4 * kk] = v.x; hst[4 * kk + 1] = v.y; hst[4 * kk + 2] = v.z; hst[4 * kk + 3] = v.w;
+        }
+    }
+
+    for (int si = 0; si < nsub; ++si) {
+        const int sub = rev ? nsub - 1 - si : si, r0 = sub * QB;
+        const bool have_state = si > 0 || (!rev && a.ssm_in != nullptr);
+        const bool need_update = si + 1 < nsub || (!rev && a.ssm_out != nullptr);
+        __syncthreads();                                   // the previous sub-chunk's readers are done with the tiles
+        // ---- load
+        if (tid < QB) {
+            lam[tid] = dA_head[r0 + tid];
+            lamp[tid] = dA_head[a.Lp + r0 + tid];
+        } else if (tid == QB) {
+            const int rb = rev ? r0 + QB : r0 - 1;         // the token before the sub-chunk in time
+            sc[0] = (rev ? (r0 + QB) % Q != 0 : r0 % Q != 0) ? dA_head[rb] : 0.f;
+        }
+        for (int u = tid; u < (QB + 3) * U8; u += NT) {
+            const int rr = u / U8, c = (u % U8) * 8;
+            const int pr = rev ? r0 + rr : r0 - 3 + rr;    // physical row; the history sits before the chunk (->) or after it (<-)
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (pr >= 0 && pr < L) v = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)pr * a.d_in_proj + a.d_inner + h * PP + c));
+            else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0)            // rows before the sequence: the carried conv state
+                v = __ldg(reinterpret_cast<const uint4 *>(a.conv_in + ((int64_t)b * (k - 1) + (k - 1 + pr)) * a.conv_ch + h * PP + c));
+            const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { xr[rr][c + 2 * e] = bf16_lo(wv[e]); xr[rr][c + 2 * e + 1] = bf16_hi(wv[e]); }
+        }
+        for (int u = tid; u < QB * (N / 8); u += NT) {
+            const int i = u / (N / 8), c = (u % (N / 8)) * 8;
+            const int64_t off = (seq * L + r0 + i) * N + c;
+            const bool ok = r0 + i < L;
+            if (have_state) {
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (ok) v = __ldg(reinterpret_cast<const uint4 *>(Cp + off));
+                *reinterpret_cast<float4 *>(&Cs[i][c]) = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+                *reinterpret_cast<float4 *>(&Cs[i][c + 4]) = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
+            }
+            if (need_update) {
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (ok) v = __ldg(reinterpret_cast<const uint4 *>(Bp + off));
+                *reinterpret_cast<float4 *>(&Bs[i][c]) = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+                *reinterpret_cast<float4 *>(&Bs[i][c + 4]) = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
+            }
+        }
+        {
+            const float *S = Sb + (seq * nsub_all + sub) * (QB * QB);
+            for (int e = tid; e < QB * QB; e += NT) Ws[e / QB][e % QB] = S[e];
+        }
+        __syncthreads();
+        // ---- conv + SiLU: thread = channel cch, rows 8 crg .. 8 crg + 7;  mask: W in place of S;  state weights w_j
+#pragma unroll
+        for (int ii = 0; ii < QB * PP / NT; ++ii) {
+            const int i = crg * (QB * PP / NT) + ii;
+            float v = cbias;
+#pragma unroll
+            for (int m = 0; m < 4; ++m) v = fmaf(wl[m], xr[rev ? i + m : i + 3 - m][cch], v);
+            xs[i][cch] = v / (1.f + __expf(-v));
+        }
+        for (int e = tid; e < QB * QB; e += NT) {
+            const int i = e / QB, j = e % QB;
+            const bool ok = (rev ? j >= i : j <= i) && r0 + i < L && r0 + j < L;
+            Ws[i][j] = ok ? fmaf(Ws[i][j], ex2f(lam[i] - lamp[j]), i == j ? Dh : 0.f) : 0.f;
+        }
+        const float lam_last = lam[rev ? 0 : QB - 1], lam0 = sc[0];      // rows past the end of the sequence have Delta = 0: Lambda stays put there
+        if (tid < QB) wjs[tid] = r0 + tid < L ? ex2f(lam_last - lamp[tid]) : 0.f;
+        __syncthreads();
+        // ---- y of tokens i = 4 m + s4, channel p
+        float y8[8];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) y8[m] = 0.f;
+        if (have_state) {
+            float acc[QB];
+#pragma unroll
+            for (int i = 0; i < QB; ++i) {
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const float4 c4 = *reinterpret_cast<const float4 *>(&Cs[i][4 * (4 * kk + s4)]);
+                    s0 = fmaf(hst[4 * kk], c4.x, s0); s1 = fmaf(hst[4 * kk + 1], c4.y, s1);
+                    s0 = fmaf(hst[4 * kk + 2], c4.z, s0); s1 = fmaf(hst[4 * kk + 3], c4.w, s1);
+                }
+                acc[i] = s0 + s1;
+            }
+            // transposing reduction over the four lanes of p: lane s4 ends with the full sums of tokens i = 4 m + s4
+            float r16[16];
+            const bool hi2 = (s4 & 2) != 0;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int ilo = (q >> 1) * 4 + (q & 1), ihi = ilo + 2;       // tokens with bit 1 clear / set
+                const float send = hi2 ? acc[ilo] : acc[ihi], keep = hi2 ? acc[ihi] : acc[ilo];
+                r16[q] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+            }
+            const bool hi1 = (s4 & 1) != 0;
+#pragma unroll
+            for (int m = 0; m < 8; ++m) {
+                const float send = hi1 ? r16[2 * m] : r16[2 * m + 1], keep = hi1 ? r16[2 * m + 1] : r16[2 * m];
+                y8[m] = (keep + __shfl_xor_sync(0xffffffffu, send, 1)) * ex2f(lam[4 * m + s4] - lam0);
+            }
+        }
+        float xv[QB];
+#pragma unroll
+        for (int j = 0; j < QB; ++j) xv[j] = xs[j][p];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int jq = 0; jq < 8; ++jq) {
+                if (rev ? jq >= m : jq <= m) {             // the other 4-column groups of rows 4 m .. 4 m + 3 are all zero
+                    const float4 w4 = *reinterpret_cast<const float4 *>(&Ws[4 * m + s4][4 * jq]);
+                    s0 = fmaf(w4.x, xv[4 * jq], s0); s1 = fmaf(w4.y, xv[4 * jq + 1], s1);
+                    s0 = fmaf(w4.z, xv[4 * jq + 2], s0); s1 = fmaf(w4.w, xv[4 * jq + 3], s1);
+                }
+            }
+            y8[m] += s0 + s1;
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) xr[4 * m + s4][p] = y8[m];          // the raw rows were last read before the previous barrier
+        __syncthreads();
+        // ---- gate: thread = (token ei, channels ec .. ec + 7)
+        {
+            const int row = r0 + ei;
+            const bool ok = row < L;
+            uint4 zv = make_uint4(0u, 0u, 0u, 0u);
+            if (ok) zv = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)row * a.d_in_proj + h * PP + ec));      // holds SiLU(z): the in_proj epilogue applied it
+            const float zf[8] = {bf16_lo(zv.x), bf16_hi(zv.x), bf16_lo(zv.y), bf16_hi(zv.y), bf16_lo(zv.z), bf16_hi(zv.z), bf16_lo(zv.w), bf16_hi(zv.w)};
+            float g[8], ss = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { g[e] = xr[ei][ec + e] * zf[e]; ss = fmaf(g[e], g[e], ss); g[e] *= nw[e]; }
+#pragma unroll
+            for (int off = 1; off < U8; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+            if (ok) {
+                *reinterpret_cast<uint4 *>(a.g + (seq * L + row) * a.d_inner + h * PP + ec) =
+                    make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]), pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
+                if (a.ssq && ec == 0) a.ssq[(seq * L + row) * a.H + h] = ss;
+            }
+        }
+        // ---- state after the sub-chunk
+        if (need_update) {
+            const float dec = ex2f(lam_last - lam0);
+#pragma unroll
+            for (int q = 0; q < 32; ++q) hst[q] *= dec;
+#pragma unroll 4
+            for (int j = 0; j < QB; ++j) {
+                const float wx = wjs[j] * xs[j][p];
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[j][4 * (4 * kk + s4)]);
+                    hst[4 * kk] = fmaf(wx, b4.x, hst[4 * kk]); hst[4 * kk + 1] = fmaf(wx, b4.y, hst[4 * kk + 1]);
+                    hst[4 * kk + 2] = fmaf(wx, b4.z, hst[4 * kk + 2]); hst[4 * kk + 3] = fmaf(wx, b4.w, hst[4 * kk + 3]);
+                }
+            }
+        }
+    }
+    if (!rev && a.ssm_out) {
+        float *ho = a.ssm_out + (((int64_t)b * a.H + h) * PP + p) * a.Nr;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            const int n0 = 4 * (4 * kk + s4);
+            if (n0 < a.Nr) *reinterpret_cast<float4 *>(ho + n0) = make_float4(hst[4 * kk], hst[4 * kk + 1], hst[4 * kk + 2], hst[4 * kk + 3]);
+        }
+    }
+}
+
+constexpr int BLOCK_MAX_L = 2 * QB;       // sequences up to this length take the short-block kernel by default
+
+bool block_mode(const ScanArgs &a) { return a.chunk == QB || (a.chunk == 0 && a.L <= BLOCK_MAX_L); }
+
 struct Scratch {
-    size_t bp, cp, da, total;
+    size_t bp, cp, da, sb, total;
     int nch, Lp;
 };
 Scratch scratch_layout(const ScanArgs &a) {
@@ -708,23 +992,35 @@ Scratch scratch_layout(const ScanArgs &a) {
     s.bp = off; off += align_up((size_t)2 * a.B * a.L * N * 2);
     s.cp = off; off += align_up((size_t)2 * a.B * a.L * N * 2);
     s.da = off; off += align_up((size_t)2 * a.B * a.H * 2 * s.Lp * 4);
+    s.sb = off;
+    if (block_mode(a)) off += align_up((size_t)2 * a.B * s.nch * PREP_PARTS * QB * QB * 4);
     s.total = off;
     return s;
 }
 
+bool shape_ok(const ScanArgs &a) {
+    if (a.dtype != DM_BF16 || a.N < 4 || a.N > N || a.N % 4 || (a.P != P && a.P != P / 2)) return false;
+    if (a.chunk != 0 && a.chunk != QB && a.chunk != Q) return false;
+    return true;
+}
+
 }  // namespace
 
+bool scan_ssd_chunk_ok(int dtype, int d_state, int chunk) {
+    return !(dtype == DM_BF16 && d_state <= N) || chunk == 0 || chunk == QB || chunk == Q;
+}
+
 bool scan_ssd_supports(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || (a.P != P && a.P != P / 2) || a.k < 2 || a.k > 4) return false;
+    if (!shape_ok(a) || a.k < 2 || a.k > 4) return false;
     if (a.P != P && 2 * a.N < P / 2) return false;                        // a half-width head's tile reaches P/2 columns past the last head: they must exist in the row
-    if (!a.z_gated) return false;                                         // the gate's SiLU is the in_proj epilogue's job on this path   // smaller d_state: zero-padded to N
-    if (a.d_in_proj % 8 || a.d_inner % 8) return false;                  // 16-byte rows for TMA and vector access
+    if (!a.z_gated) return false;                                         // the gate's SiLU is the in_proj epilogue's job on this path
+    if (a.d_in_proj % 8 || a.d_inner % 8 || a.conv_ch % 8) return false;  // 16-byte rows for TMA and vector access
     if (a.H > 65535 || a.B > 65535) return false;
     return encode_fn() != nullptr;
 }
 
 size_t scan_ssd_workspace_bytes(const ScanArgs &a) {
-    if (a.dtype != DM_BF16 || a.N < 2 || a.N > N || a.N % 2 || (a.P != P && a.P != P / 2)) return 0;
+    if (!shape_ok(a)) return 0;
     return scratch_layout(a).total;
 }
 
@@ -741,6 +1037,22 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out; k.conv_in = static_cast<const __nv_bfloat16 *>(a.conv_in);
     k.dir[0] = a.dir[0]; k.dir[1] = a.dir[1];
     const int ndir = a.dir_mask == DM_DIR_BOTH ? 2 : 1, dir0 = a.dir_mask == DM_DIR_REV ? 1 : 0;
+    const bool blk = block_mode(a);
+    float *Sb = blk ? reinterpret_cast<float *>(base + l.sb) : nullptr;
+
+    ssd_prep_kernel<<<dim3(l.nch * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (blk) {
+        auto kern = a.P == P ? ssd_block_kernel<P> : ssd_block_kernel<P / 2>;
+        const size_t smem = a.P == P ? block_smem_bytes<P>() : block_smem_bytes<P / 2>();
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<dim3(a.H, ndir, a.B), 4 * a.P, smem, s>>>(k, Bp, Cp, Sb, dir0);
+        count_launch();
+        return cudaGetLastError();
+    }
 
     CUtensorMap mx, mz, mb, mc, mg;
     {
@@ -763,11 +1075,6 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     }
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
-
-    ssd_prep_kernel<<<dim3(l.nch * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, dir0);
-    count_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     auto kern = a.P == P ? ssd_scan_kernel<false> : ssd_scan_kernel<true>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;

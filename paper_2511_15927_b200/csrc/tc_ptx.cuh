@@ -124,12 +124,6 @@ __device__ __forceinline__ uint64_t desc_k_sw128(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
            ((uint64_t)2 << 61);
 }
-// MN-major operand: each K index is one 128-byte row holding 64 contiguous M/N elements; groups of 8 K
-// rows are `sbo` bytes apart; the next 64 M/N elements start `lbo` bytes further.
-__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | ((uint64_t)1 << 46) |
-           ((uint64_t)2 << 61);
-}
 // Instruction descriptor: D fp32, A and B bf16; *_mn = 1 selects the MN-major form of that operand.
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n, int a_mn, int b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) |
@@ -187,18 +181,6 @@ __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t *r) {
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// MMA whose A operand (M rows x K, bf16 pairs packed along K, row m in TMEM lane m) is read from TMEM.
-__device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Copy of one K = 16 slice (128 rows x 32 bytes) of a K-major shared-memory operand into TMEM, in the layout the
-// MMA expects for an A operand held in TMEM (row m in lane m, 8 columns of bf16 pairs).
-__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t s_desc) {
-    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
-}
 // The same descriptors split in two 32-bit halves, for loops that step through an operand: only the low half (start
 // address, leading byte offset) changes, by +bytes/16 per step, so that a step costs one integer add.
 constexpr uint32_t DESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (2u << 29);          // stride 1024 B between 8-row groups, 128-byte swizzle
@@ -220,10 +202,6 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32
         "mov.b64 db, {%2, %4};\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI_SW128), "n"(ACC) : "memory");
-}
-__device__ __forceinline__ void tmem_cp_128x256b_lo(uint32_t taddr, uint32_t s_lo) {
-    asm volatile("{\n\t.reg .b64 ds;\n\tmov.b64 ds, {%1, %2};\n\ttcgen05.cp.cta_group::1.128x256b [%0], ds;\n\t}"
-                 ::"r"(taddr), "r"(s_lo), "r"(DESC_HI_SW128) : "memory");
 }
 // TMA store of a shared-memory tile (bulk async-group completion).
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, const void *smem_src, int x, int y, int z) {
@@ -277,7 +255,6 @@ __device__ __forceinline__ f32x2 pk2(float lo, float hi) { f32x2 r; asm("mov.b64
 __device__ __forceinline__ void upk2(f32x2 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 // two bf16 in one word -> two floats (exact)
 __device__ __forceinline__ f32x2 bf2_to_f2(uint32_t w) { return pk2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)); }
 __device__ __forceinline__ uint32_t f2_to_bf2(f32x2 v) {
@@ -285,15 +262,6 @@ __device__ __forceinline__ uint32_t f2_to_bf2(f32x2 v) {
     upk2(v, lo, hi);
     __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&b);
-}
-
-// Compiler-level ordering for pipelined TMEM loads: placed after tmem_wait_ld(), it makes every later use of the
-// loaded registers depend on a point after the wait (volatile asm statements keep their order).
-__device__ __forceinline__ void reg_fence8(uint32_t *r) {
-    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]));
-}
-__device__ __forceinline__ void reg_fence32(uint32_t *r) {
-    reg_fence8(r); reg_fence8(r + 8); reg_fence8(r + 16); reg_fence8(r + 24);
 }
 
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }

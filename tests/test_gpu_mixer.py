@@ -100,15 +100,38 @@ def test_causality_on_gpu(G):
     assert np.all(dr[0, 41:] == 0) and np.any(dr[0, :41] != 0)
 
 
-@pytest.mark.parametrize("dtype,N", [(I.F32, 16), (I.BF16, 128)])
-def test_chunk_size_invariance(G, dtype, N):
-    shape = I.MixerShape(1, 300, 128, 2, N, 4, 4)
-    wf, wr, x = _case(shape, dtype, seed=7)
+def test_chunk_size_invariance_fp32(G):
+    """Sequential (exact) kernel: any chunk length gives the same result up to fp32 rounding order."""
+    shape = I.MixerShape(1, 300, 128, 2, 16, 4, 4)
+    wf, wr, x = _case(shape, I.F32, seed=7)
     want = O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape))
-    outs = [G.run_forward(shape, dtype, wf, wr, x, chunk=c) for c in (32, 64, 128, 256)]
+    outs = [G.run_forward(shape, I.F32, wf, wr, x, chunk=c) for c in (32, 64, 128, 256)]
     for o in outs:
-        _check(o, want, dtype)
-        np.testing.assert_allclose(o, outs[0], rtol=2e-2 if dtype == I.BF16 else 1e-4, atol=2e-2 if dtype == I.BF16 else 1e-5)
+        _check(o, want, I.F32)
+        np.testing.assert_allclose(o, outs[0], rtol=1e-4, atol=1e-5)
+
+
+@pytest.mark.parametrize("L", [300, 127, 128, 129, 257, 40])
+@pytest.mark.parametrize("P", [64, 32])
+def test_chunk_size_invariance_bf16(G, L, P):
+    """Chunked bf16 path: chunk = 128 is the tensor-core kernel, chunk = 32 the CUDA-core kernel with a quarter of the
+    chunk length (a different kernel with its own arithmetic: fp32 products, state in registers).  Both must match the
+    oracle and each other on lengths around the chunk boundaries; other chunk values are refused."""
+    from paper_2511_15927_b200 import binding as dm
+    H = 4 if P == 64 else 8
+    shape = I.MixerShape(2, L, 128, 2, 128, 4, H)
+    wf, wr, x = _case(shape, I.BF16, seed=7 + L)
+    want = O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape))
+    o32 = G.run_forward(shape, I.BF16, wf, wr, x, chunk=32)
+    o128 = G.run_forward(shape, I.BF16, wf, wr, x, chunk=128)
+    _check(o32, want, I.BF16)
+    _check(o128, want, I.BF16)
+    assert G.rel_l2(o32, o128) <= BF16_REL and G.max_abs(o32, o128) <= BF16_ABS
+    assert not np.array_equal(o32, o128)                      # two kernels, not one launched twice
+    for bad in (64, 256, 16):
+        with pytest.raises(dm.DmError) as e:
+            G.run_forward(shape, I.BF16, wf, wr, x, chunk=bad)
+        assert e.value.status == dm.DM_ERR_UNSUPPORTED
 
 
 def test_run_to_run_determinism(G):

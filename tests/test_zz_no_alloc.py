@@ -3,9 +3,11 @@ cudaMalloc allowed where they run, or all memory already handed to their own poo
 intermediates in a fixed array inside the library instead of a caller workspace.
 
 Checked here through the C ABI: two calls in a row (different inputs, so that anything left behind by the
-first call would show in the second) must match dm_bimamba_forward on the same inputs within the bf16
-tolerance of the other parity tests, and a configuration too large for the built-in array must be refused
-before any kernel is launched.  This file sorts last so that a run stopping at the first failure has already
+first call would show in the second) must equal dm_bimamba_forward on the same inputs bit for bit -- both run
+the same kernels in the same order, only the scratch address differs, so even a partly overlapping or
+misplaced scratch region would show -- and stay inside the tolerance of the other parity tests; the second
+call must leave the device's free memory unchanged (it allocates nothing); and a configuration too large for
+the built-in array must be refused before any kernel is launched.  This file sorts last so that a run stopping at the first failure has already
 run every other test; it also passes when run alone in a fresh process.
 """
 import numpy as np
@@ -51,6 +53,28 @@ def test_two_calls_match_the_workspace_entry_point(G, dtype, N, H):
         assert np.all(np.isfinite(got))
         assert G.rel_l2(got, want) <= (BF16_REL if dtype == I.BF16 else 1e-4), G.rel_l2(got, want)
         assert G.max_abs(got, want) <= BF16_ABS, G.max_abs(got, want)
+        np.testing.assert_array_equal(got, want)            # same kernels, same inputs: identical bits
+
+
+def test_second_call_allocates_nothing(G):
+    """Device memory in use does not move across a call (after a first call has looked the array's address up)."""
+    import torch
+    from paper_2511_15927_b200 import binding as dm
+    shape, dtype = I.MixerShape(2, 300, 256, 2, 128, 4, 8), I.BF16
+    wf, wr = I.make_mixer_weights(shape, 23, dtype)
+    cfg = G.cfg_of(shape, dtype)
+    dwf, dwr = G.dev_dir_weights(wf, dtype), G.dev_dir_weights(wr, dtype)
+    xd = G.dev(I.make_activations(shape, 23, dtype), dtype)
+    yd = torch.empty_like(xd)
+    st = torch.cuda.current_stream().cuda_stream
+    cw = (dm.make_dir_weights(dwf), dm.make_dir_weights(dwr))
+    dm.dm_bimamba_forward_static(cfg, cw, xd.data_ptr(), yd.data_ptr(), st)
+    dm.dm_check(st)
+    free0, _ = torch.cuda.mem_get_info()
+    dm.dm_bimamba_forward_static(cfg, cw, xd.data_ptr(), yd.data_ptr(), st)
+    dm.dm_check(st)
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
 
 
 def test_oversized_configuration_is_refused_without_a_launch(G):
