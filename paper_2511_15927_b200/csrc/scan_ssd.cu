@@ -28,11 +28,12 @@
 // Every hand-off is an mbarrier; every wait is bounded.  On expiry the CTA stores DM_ERR_TIMEOUT in the
 // device status word, all roles leave their loops, outstanding TMA traffic is waited for (bounded), TMEM is
 // freed and the CTA returns.
-// Launch 2, short blocks (ssd_block, Q = 32, fp32 on the CUDA cores): the active block of block-autoregressive decoding
-// is 32 tokens, a quarter of one tensor-core tile, and a call has thousands of (batch row, head) items of that size; for
-// them the pipeline above is all set-up and tear-down.  ssd_block keeps the state of a head in registers, takes the
-// 32 x 32 matrix S of each sub-chunk from the prep launch (which computes it once per (batch row, direction) with
-// mma.sync) and does the rest of the identities above in fp32.  It is also what `chunk = 32` selects at any length.
+// Launch 2, short blocks (ssd_block, Q = 32, products with mma.sync from registers): the active block of block-autoregressive
+// decoding is 32 tokens, a quarter of one tcgen05 tile, and a call has thousands of (batch row, head) items of that size;
+// for them the pipeline above is all set-up and tear-down.  ssd_block is a plain CTA of 256 threads per item: it takes the
+// 32 x 32 matrix S of each sub-chunk from the prep launch (which computes it once per (batch row, direction)), builds W
+// and runs the other three products of the identities above on 16 x 8 x 16 tiles; a state that has to outlive the
+// sub-chunk stays in its fp32 accumulators.  It is also what `chunk = 32` selects at any length.
 #include <cstddef>
 
 #include "dm_internal.h"
@@ -77,6 +78,7 @@ struct Misc {
     uint64_t xs_full, s_full, s_empty, w_full, st_full, hs_ready, h_full, y_full, ya_empty, yb_empty[2];
     uint32_t tmem_base;
     int abort;
+    int ticket;                   // order in which this CTA started (fused prep: the first ones take the prep role)
     alignas(16) float norm_w[P];  // the three arrays below are read as float4
     alignas(16) float wbuf[Q];
     alignas(16) float cbuf[NWG][4][Q]; // per mask warp: column factors of the off-diagonal blocks
@@ -99,6 +101,50 @@ struct SsdArgs {
 };
 
 __device__ __forceinline__ float silu_fast(float v) { return v / (1.f + __expf(-v)); }
+// Arithmetic shared by the two forms of the prep work (the launch of its own below and the prep role inside the scan
+// launch), so that both give the same bits.
+// conv + SiLU of one bf16 channel pair: r[m] = the pre-conv pair m steps back in time, wl[e][m] its weight
+__device__ __forceinline__ uint32_t prep_conv_pair(const float (&wl)[2][4], const float (&bias)[2], const uint32_t (&r)[4]) {
+    float v0 = bias[0], v1 = bias[1];
+#pragma unroll
+    for (int m = 3; m >= 0; --m) {
+        v0 = fmaf(wl[0][m], bf16_lo(r[m]), v0);
+        v1 = fmaf(wl[1][m], bf16_hi(r[m]), v1);
+    }
+    return pack_bf16(silu_fast(v0), silu_fast(v1));
+}
+__device__ __forceinline__ float prep_delta(__nv_bfloat16 dt, float dt_bias) {
+    const float v = __bfloat162float(dt) + dt_bias;
+    return fmaxf(v, 0.f) + log1pf(expf(-fabsf(v)));
+}
+// One warp, one head, one 128-token chunk: d[r * ld] = Delta of physical chunk row r.  Writes Lambda (inclusive cumulative
+// Delta A in the direction's time order, log2 units) to dl[0..Q) and Lambda' = Lambda - log2 Delta to dl[Lp..Lp + Q).
+__device__ __forceinline__ void prep_lambda_head(const float *d_col, int ld, float A_log, bool rev, int lane, float *dl, int Lp) {
+    const float Ah = -expf(A_log) * 1.4426950408889634f;
+    float d[4], cum[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int tau = 4 * lane + e, r = rev ? Q - 1 - tau : tau;
+        d[e] = d_col[r * ld];
+    }
+    cum[0] = d[0] * Ah; cum[1] = fmaf(d[1], Ah, cum[0]); cum[2] = fmaf(d[2], Ah, cum[1]); cum[3] = fmaf(d[3], Ah, cum[2]);
+    float run = cum[3];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float up = __shfl_up_sync(0xffffffffu, run, off);
+        if (lane >= off) run += up;
+    }
+    const float base = run - cum[3];                             // sum over the lanes before this one
+    float lam[4], lamp[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { lam[e] = base + cum[e]; lamp[e] = lam[e] - log2f(d[e]); }    // Delta = 0 (padding): Lambda' = +inf
+    const int rlo = rev ? Q - 4 - 4 * lane : 4 * lane;           // lowest physical row of this lane's four
+    const float4 v0 = rev ? make_float4(lam[3], lam[2], lam[1], lam[0]) : make_float4(lam[0], lam[1], lam[2], lam[3]);
+    const float4 v1 = rev ? make_float4(lamp[3], lamp[2], lamp[1], lamp[0]) : make_float4(lamp[0], lamp[1], lamp[2], lamp[3]);
+    *reinterpret_cast<float4 *>(dl + rlo) = v0;
+    *reinterpret_cast<float4 *>(dl + Lp + rlo) = v1;
+}
+
 // --------------------------------------------------------------------------------------------------
 // Launch 1: B', C' (bf16) and Lambda, Lambda' (fp32, log2 units).  A CTA takes one quarter of one physical chunk of one
 // (direction, batch row): 32 of its rows for B' and C', 16 of every 64 heads for the decays.  The work per CTA is a
@@ -169,13 +215,8 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             const int t = first + i * step;
-            float v0 = bias[0], v1 = bias[1];
-#pragma unroll
-            for (int m = 3; m >= 0; --m) {
-                v0 = fmaf(wl[0][m], bf16_lo(raw[i + 3 - m]), v0);
-                v1 = fmaf(wl[1][m], bf16_hi(raw[i + 3 - m]), v1);
-            }
-            const uint32_t pk = pack_bf16(silu_fast(v0), silu_fast(v1));
+            const uint32_t win[4] = {raw[i + 3], raw[i + 2], raw[i + 1], raw[i]};
+            const uint32_t pk = prep_conv_pair(wl, bias, win);
             if (t < L) *reinterpret_cast<uint32_t *>(dst + (int64_t)t * N) = pk;
             if (Sb) bct[isC ? 1 : 0][rev ? QB - 1 - i : i][pi] = pk;          // row of the tile = physical row inside the block
         }
@@ -207,48 +248,111 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
         }
     }
     // ---- Delta, then the inclusive cumulative log-decay of every head in the direction's time order
-    const float LOG2E = 1.4426950408889634f;
     for (int h0 = 0; h0 < a.H; h0 += 64) {
         __syncthreads();
 #pragma unroll 4
         for (int i = 0; i < Q * PREP_HEADS / PREP_THREADS; ++i) {
             const int idx = tid + PREP_THREADS * i, hh = idx % PREP_HEADS, r = idx / PREP_HEADS, t = r0 + r, h = h0 + part * PREP_HEADS + hh;
-            float d = 0.f;
-            if (t < L && h < a.H) {
-                const float v = __bfloat162float(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h]) + w.dt_bias[h];
-                d = fmaxf(v, 0.f) + log1pf(expf(-fabsf(v)));
-            }
-            dsm[r][hh] = d;
+            dsm[r][hh] = (t < L && h < a.H) ? prep_delta(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h], w.dt_bias[h]) : 0.f;
         }
         __syncthreads();
         const int warp = tid >> 5, lane = tid & 31;
         for (int hh = warp; hh < PREP_HEADS && h0 + part * PREP_HEADS + hh < a.H; hh += PREP_THREADS / 32) {
             const int h = h0 + part * PREP_HEADS + hh;
-            const float Ah = -expf(w.A_log[h]) * LOG2E;
-            float d[4], cum[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int tau = 4 * lane + e, r = rev ? Q - 1 - tau : tau;
-                d[e] = dsm[r][hh];
-            }
-            cum[0] = d[0] * Ah; cum[1] = fmaf(d[1], Ah, cum[0]); cum[2] = fmaf(d[2], Ah, cum[1]); cum[3] = fmaf(d[3], Ah, cum[2]);
-            float run = cum[3];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const float up = __shfl_up_sync(0xffffffffu, run, off);
-                if (lane >= off) run += up;
-            }
-            const float base = run - cum[3];                             // sum over the lanes before this one
-            float lam[4], lamp[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { lam[e] = base + cum[e]; lamp[e] = lam[e] - log2f(d[e]); }    // Delta = 0 (padding): Lambda' = +inf
-            float *dl = dA + ((seq * a.H + h) * 2) * a.Lp + r0;
-            const int rlo = rev ? Q - 4 - 4 * lane : 4 * lane;           // lowest physical row of this lane's four
-            const float4 v0 = rev ? make_float4(lam[3], lam[2], lam[1], lam[0]) : make_float4(lam[0], lam[1], lam[2], lam[3]);
-            const float4 v1 = rev ? make_float4(lamp[3], lamp[2], lamp[1], lamp[0]) : make_float4(lamp[0], lamp[1], lamp[2], lamp[3]);
-            *reinterpret_cast<float4 *>(dl + rlo) = v0;
-            *reinterpret_cast<float4 *>(dl + a.Lp + rlo) = v1;
+            prep_lambda_head(&dsm[0][hh], PREP_HEADS + 1, w.A_log[h], rev, lane, dA + ((seq * a.H + h) * 2) * a.Lp + r0, a.Lp);
         }
+    }
+}
+
+// --------------------------------------------------------------------------------------------------
+// The same prep work as a role inside the scan launch.  When the scan has fewer CTAs than the GPU has SMs (one long
+// sequence: 2 H CTAs), the launch is widened by `nprep` CTAs; the CTAs that start first take the prep role (a ticket
+// from an atomic counter decides, so the role never waits for a CTA that has not been scheduled), work through the
+// (batch row, chunk, direction) items in the order the scan consumes them and release one flag per item; the scan CTAs'
+// load warps acquire the flag of a chunk before they fetch its B', C', Lambda.  The whole CTA works on one item: 131 rows
+// of the B and C columns and the dt columns are staged in shared memory with 16-byte loads, then every thread filters
+// one channel pair over a run of rows and every warp scans heads.
+// --------------------------------------------------------------------------------------------------
+struct PrepJob {
+    __nv_bfloat16 *Bp, *Cp;
+    float *dA;
+    int *sync;          // [0]: ticket counter, [1 + seq * nch + pc]: item flags; zeroed before the launch.  NULL: no fused prep
+    int nprep, ndir;
+};
+constexpr int PREP_SEG = 7, PREP_SEG_ROWS = (Q + PREP_SEG - 1) / PREP_SEG;     // row runs per channel pair
+constexpr uint32_t PREP_RAW_BYTES = (Q + 3) * N * 4, PREP_SMEM = PREP_RAW_BYTES + Q * 65 * 4;
+
+__device__ __forceinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, int first, int dir0, uint8_t *smem) {
+    static_assert(PREP_SEG * 128 == NTHREADS && PREP_SMEM <= OFF_MISC, "prep role: thread and shared-memory layout");
+    uint32_t *rawt = reinterpret_cast<uint32_t *>(smem);                       // [Q + 3][N] words: pre-conv rows, B pairs 0..63 | C pairs 64..127
+    float *dsm = reinterpret_cast<float *>(smem + PREP_RAW_BYTES);              // [Q][65] Delta of one tile of 64 heads
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int L = a.L, k = a.k, n_items = pj.ndir * a.B * a.nch;
+    for (int it = first; it < n_items; it += pj.nprep) {
+        const int dir = dir0 + it % pj.ndir, c = (it / pj.ndir) % a.nch, b = it / (pj.ndir * a.nch);
+        const bool rev = dir == 1;
+        const int pc = rev ? a.nch - 1 - c : c, r0 = pc * Q;
+        const ScanDir &w = a.dir[dir];
+        const int64_t seq = (int64_t)dir * a.B + b;
+        const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
+        const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
+        __syncthreads();                                                       // the previous item's readers are done with the tiles
+        // ---- stage the rows: tile row rr = physical row r0 - 3 + rr (->: history first) or r0 + rr (<-: history last)
+        for (int u = tid; u < (Q + 3) * 32; u += NTHREADS) {
+            const int rr = u >> 5, c16 = u & 31, ch = (c16 & 15) * 8;
+            const int pr = rev ? r0 + rr : r0 - 3 + rr;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (ch < a.Nr) {                                                   // beyond the model's d_state: zero padding
+                const int cc = a.d_inner + ((c16 >> 4) ? a.Nr : 0) + ch;       // conv channel
+                if (pr >= 0 && pr < L) v = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)pr * a.d_in_proj + a.d_inner + cc));
+                else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0)       // rows before the sequence: the carried conv state
+                    v = __ldg(reinterpret_cast<const uint4 *>(a.conv_in + ((int64_t)b * (k - 1) + (k - 1 + pr)) * a.conv_ch + cc));
+            }
+            *reinterpret_cast<uint4 *>(rawt + rr * N + c16 * 4) = v;
+        }
+        __syncthreads();
+        // ---- conv + SiLU: thread = (channel pair, run of rows)
+        {
+            const int pi = tid & 127, seg = tid >> 7, pp = pi & 63;
+            const bool isC = pi >= 64, valid = 2 * pp < a.Nr;
+            const int cc = a.d_inner + (isC ? a.Nr : 0) + (valid ? 2 * pp : 0);
+            const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)cc * k;
+            float wl[2][4], bias[2] = {0.f, 0.f};
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+#pragma unroll
+                for (int m = 0; m < 4; ++m) wl[e][m] = (m < k && valid) ? __bfloat162float(cw[e * k + k - 1 - m]) : 0.f;
+            if (has_bias && valid) {
+                bias[0] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc]);
+                bias[1] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc + 1]);
+            }
+            __nv_bfloat16 *dst = (isC ? pj.Cp : pj.Bp) + 2 * pp + seq * L * N;
+            const int i0 = seg * PREP_SEG_ROWS, i1 = min(Q, i0 + PREP_SEG_ROWS);
+            for (int i = i0; i < i1; ++i) {
+                const uint32_t *col = rawt + pi + (rev ? i : i + 3) * N;           // the row itself; m steps back in time = m rows further (<-) or back (->)
+                const int st = rev ? N : -N;
+                const uint32_t win[4] = {col[0], col[st], col[2 * st], col[3 * st]};
+                const uint32_t pk = prep_conv_pair(wl, bias, win);
+                if (r0 + i < L) *reinterpret_cast<uint32_t *>(dst + (int64_t)(r0 + i) * N) = pk;
+            }
+        }
+        // ---- Delta and the cumulative log-decay, 64 heads at a time
+        for (int h0 = 0; h0 < a.H; h0 += 64) {
+            __syncthreads();
+            for (int idx = tid; idx < Q * 64; idx += NTHREADS) {
+                const int hh = idx & 63, r = idx >> 6, t = r0 + r, h = h0 + hh;
+                dsm[r * 65 + hh] = (t < L && h < a.H) ? prep_delta(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h], w.dt_bias[h]) : 0.f;
+            }
+            __syncthreads();
+            for (int hh = warp; hh < 64 && h0 + hh < a.H; hh += NTHREADS / 32) {
+                const int h = h0 + hh;
+                prep_lambda_head(dsm + hh, 65, w.A_log[h], rev, lane, pj.dA + ((seq * a.H + h) * 2) * a.Lp + r0, a.Lp);
+            }
+        }
+        // ---- publish the item
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) st_release_gpu(pj.sync + 1 + seq * a.nch + pc, 1);
     }
 }
 
@@ -263,7 +367,7 @@ template <bool HALFP>
 __global__ void __launch_bounds__(NTHREADS, 1)
 ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_z,
                 const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_c,
-                const __grid_constant__ CUtensorMap map_g, const SsdArgs a, int dir0, int *status) {
+                const __grid_constant__ CUtensorMap map_g, const SsdArgs a, const PrepJob pj, int dir0, int *status) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -271,8 +375,17 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     volatile int *abort_flag = &misc->abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int h = blockIdx.x, b = blockIdx.z, dir = dir0 + blockIdx.y;
+    int item = blockIdx.x;                     // (batch row, direction, head), heads fastest
+    if (pj.sync) {
+        if (tid == 0) misc->ticket = atomicAdd(pj.sync, 1);
+        __syncthreads();
+        const int ticket = misc->ticket;
+        if (ticket < pj.nprep) { prep_role(a, pj, ticket, dir0, smem); return; }
+        item = ticket - pj.nprep;
+    }
+    const int h = item % a.H, b = item / (a.H * pj.ndir), dir = dir0 + (item / a.H) % pj.ndir;
     const bool rev = dir == 1;
+    const int *ready = pj.sync ? pj.sync + 1 + ((int64_t)dir * a.B + b) * a.nch : nullptr;     // per chunk: its B', C', Lambda are in memory
     const int L = a.L, nch = a.nch;
     const int seq = dir * a.B + b;
     const ScanDir &w = a.dir[dir];
@@ -316,6 +429,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int c = 0; c < nch; ++c) {
                 const int sx = c % NX, sd = c % NDL, pc = rev ? nch - 1 - c : c;
                 if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
+                if (ready && !flag_wait(ready + pc, abort_flag, status)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
                 tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
                 mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
@@ -350,6 +464,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int c = 0; c < nch; ++c) {
                 const int sb = c % NB, pc = rev ? nch - 1 - c : c;
                 if (!WAIT(&misc->empty_b[sb], ((c / NB) & 1) ^ 1)) break;
+                if (ready && !flag_wait(ready + pc, abort_flag, status)) break;
                 mbar_expect_tx(&misc->full_b[sb], 2 * T16);
                 tma_load_3d(smem + OFF_B + sb * 2 * T16, &map_b, 0, pc * Q, seq, &misc->full_b[sb]);
                 tma_load_3d(smem + OFF_B + sb * 2 * T16 + T16, &map_b, 64, pc * Q, seq, &misc->full_b[sb]);
@@ -750,34 +865,52 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 }
 
 // --------------------------------------------------------------------------------------------------
-// Launch 2 for short blocks: sub-chunks of QB = 32 tokens, fp32 on the CUDA cores.
-// One CTA of 4 * PP threads per (batch row, direction, head of PP channels).  Thread (p, s4) = (tid / 4, tid % 4) keeps the 32
-// state entries h[p][n], n = 4 (4 k + s4) + e (k < 8, e < 4), in registers across the sub-chunks; per sub-chunk:
-//   load    x rows (+3 rows of conv history), B', C' (bf16 -> fp32), S (from the prep launch), Lambda, Lambda'
-//   conv    x' = SiLU(conv(x));   W_ij = S_ij 2^(Lambda_i - Lambda'_j) [+ D on the diagonal] for j not after i, else 0
-//   y       Yb: each thread's partial C'_i . h[p] over its 32 states for all 32 tokens, then a transposing reduction over
-//           the four lanes of p that leaves tokens i = 4 m + s4 with lane s4;  y_i = 2^(Lambda_i - Lambda_0) Yb_i + sum_j W_ij x'_j[p]
+// Launch 2 for short blocks: sub-chunks of QB = 32 tokens; the four products of a sub-chunk on the legacy tensor path
+// (mma.sync m16n8k16, bf16 operands from shared memory through ldmatrix, fp32 accumulators in registers).
+// One CTA of 4 * PP threads per (batch row, direction, head of PP channels); per sub-chunk:
+//   load    x rows (+3 rows of conv history), C' and B' rows as they are (bf16), S (fp32, from the prep launch), Lambda, Lambda';
+//           the incoming state as a bf16 copy [p][n] (from ssm_in, or from the accumulators of the previous sub-chunk)
+//   conv    x' = SiLU(conv(x)) and w_j x'_j as bf16 [j][p];   W_ij = S_ij 2^(Lambda_i - Lambda'_j) [+ D on the diagonal] for j not after i, else 0
+//   y       Yb = C' h^T (K = d_state), rows scaled by 2^(Lambda_i - Lambda_0), then += W x' (K = 32) into the same accumulators:
+//           warp = 16 tokens x 16 channels
 //   gate    through shared memory to a (token, 8 channels) layout: g = y SiLU(z), sum of squares, * norm_w, 16-byte stores
-//   state   h <- 2^(Lambda_last - Lambda_0) h + sum_j 2^(Lambda_last - Lambda'_j) x'_j[p] B'_j   (only if someone will read it)
+//   state   (only if someone will read it) h <- 2^(Lambda_last - Lambda_0) h + (w o x')^T B': warp = 16 channels x 64 states, the
+//           fp32 state stays in the accumulators from one sub-chunk to the next
 // Lambda_0 is Lambda of the token before the sub-chunk inside the same 128-token chunk of the prep launch (0 at its start).
 // --------------------------------------------------------------------------------------------------
-constexpr int CLD = N + 4;             // row pitch of the fp32 B' / C' tiles
-constexpr int WLD = QB + 4;            // row pitch of W: 16-byte rows, conflict-free float4 reads by four different rows
-template <int PP> constexpr size_t block_smem_bytes() { return sizeof(float) * (2 * QB * CLD + (QB + 3) * PP + QB * PP + QB * WLD + 3 * QB + 4); }
+constexpr int NLD = N + 8;             // row pitch (bf16) of the C', B' and state tiles: 16-byte rows, conflict-free ldmatrix
+constexpr int SLD = QB + 4;            // row pitch (fp32) of S
+constexpr int WTL = QB + 8;            // row pitch (bf16) of W
+template <int PP> struct BlockSmem {
+    static constexpr int XLD = PP + 8;             // row pitch (bf16) of x' and w o x'
+    static constexpr size_t ct = 0, bt = ct + QB * NLD * 2, ht = bt + QB * NLD * 2, xt = ht + PP * NLD * 2, wxt = xt + QB * XLD * 2,
+                            wt = wxt + QB * XLD * 2, xr = wt + QB * WTL * 2, ss = xr + (QB + 3) * PP * 4, lam = ss + QB * SLD * 4,
+                            total = lam + (2 * QB + 4) * 4;
+    static_assert(ht % 16 == 0 && xt % 16 == 0 && wxt % 16 == 0 && wt % 16 == 0 && xr % 16 == 0 && ss % 16 == 0 && lam % 16 == 0, "16-byte tiles");
+};
+__device__ __forceinline__ void ldmatrix_x4_t(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ void ldmatrix_x2_t(uint32_t &r0, uint32_t &r1, const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(smem_u32(p)));
+}
 
 template <int PP>
-__global__ void __launch_bounds__(4 * PP, PP == 64 ? 2 : 4)
+__global__ void __launch_bounds__(4 * PP, 3)
 ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __nv_bfloat16 *__restrict__ Cp, const float *__restrict__ Sb, int dir0) {
-    constexpr int NT = 4 * PP, U8 = PP / 8;
-    extern __shared__ __align__(16) float bsm[];
-    float (*Cs)[CLD] = reinterpret_cast<float (*)[CLD]>(bsm);
-    float (*Bs)[CLD] = reinterpret_cast<float (*)[CLD]>(bsm + QB * CLD);
-    float (*xr)[PP] = reinterpret_cast<float (*)[PP]>(bsm + 2 * QB * CLD);                   // raw x rows of the sub-chunk and its conv history; later its y
-    float (*xs)[PP] = reinterpret_cast<float (*)[PP]>(bsm + 2 * QB * CLD + (QB + 3) * PP);   // x'
-    float (*Ws)[WLD] = reinterpret_cast<float (*)[WLD]>(bsm + 2 * QB * CLD + (QB + 3) * PP + QB * PP);
-    float *lam = bsm + 2 * QB * CLD + (QB + 3) * PP + QB * PP + QB * WLD, *lamp = lam + QB, *wjs = lamp + QB, *sc = wjs + QB;
+    constexpr int NT = 4 * PP, U8 = PP / 8, MT = PP / 16, XLD = BlockSmem<PP>::XLD;
+    extern __shared__ __align__(16) uint8_t bsm[];
+    __nv_bfloat16 (*Ct)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::ct);      // C' rows [i][n]
+    __nv_bfloat16 (*Bt)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::bt);      // B' rows [j][n]
+    __nv_bfloat16 (*Ht)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::ht);      // incoming state [p][n]
+    __nv_bfloat16 (*Xt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::xt);      // x' [j][p]
+    __nv_bfloat16 (*WXt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::wxt);    // w_j x'_j [j][p]
+    __nv_bfloat16 (*Wt)[WTL] = reinterpret_cast<__nv_bfloat16 (*)[WTL]>(bsm + BlockSmem<PP>::wt);      // W [i][j]
+    float (*xr)[PP] = reinterpret_cast<float (*)[PP]>(bsm + BlockSmem<PP>::xr);                        // raw x rows and conv history; later the sub-chunk's y
+    float (*Ss)[SLD] = reinterpret_cast<float (*)[SLD]>(bsm + BlockSmem<PP>::ss);
+    float *lam = reinterpret_cast<float *>(bsm + BlockSmem<PP>::lam), *lamp = lam + QB, *sc = lamp + QB;
 
-    const int tid = threadIdx.x, p = tid >> 2, s4 = tid & 3;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gr = lane >> 2, qc = lane & 3;
     const int h = blockIdx.x, b = blockIdx.z, dir = dir0 + blockIdx.y;
     const bool rev = dir == 1;
     const int L = a.L, k = a.k;
@@ -788,6 +921,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
     const int nsub = (L + QB - 1) / QB, nsub_all = a.nch * PREP_PARTS;
     const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
     const bool norm_on = (a.flags & DM_FLAG_GATED_RMSNORM) != 0;
+    const bool keep_state = nsub > 1 || (!rev && a.ssm_out != nullptr);        // the fp32 state is carried in the accumulators
 
     // per-thread constants: conv taps of channel tid % PP (wl[m] multiplies the row m steps back in time), norm weights of the epilogue's 8 channels
     const int cch = tid % PP, crg = tid / PP;
@@ -799,26 +933,34 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
         cbias = ((a.flags & DM_FLAG_CONV_BIAS) && w.conv_b) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[h * PP + cch]) : 0.f;
     }
     const int ei = tid / U8, ec = (tid % U8) * 8;      // epilogue: token row of the sub-chunk, first of 8 channels
-    float nw[8];
+    uint32_t nwp[4];                                   // norm weights of those channels as bf16 pairs (ones when the norm is off)
 #pragma unroll
-    for (int e = 0; e < 8; ++e)
-        nw[e] = (norm_on && w.norm_w) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * PP + ec + e]) : 1.f;
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 *nwq = static_cast<const __nv_bfloat16 *>(w.norm_w) + h * PP + ec + 2 * e;
+        nwp[e] = (norm_on && w.norm_w) ? pack_bf16(__bfloat162float(nwq[0]), __bfloat162float(nwq[1])) : 0x3F803F80u;
+    }
 
-    float hst[32];
-    {
-        const float *h0 = (!rev && a.ssm_in) ? a.ssm_in + (((int64_t)b * a.H + h) * PP + p) * a.Nr : nullptr;
+    // state accumulators: warp = channels [16 smt, +16) x states [64 snh, +64): tile t covers states 64 snh + 8 t .. + 7;
+    // a thread holds rows p = 16 smt + gr (+8), columns n = 64 snh + 8 t + 2 qc (+1)
+    const int smt = warp % MT, snh = warp / MT;
+    float hacc[8][4];
+    const float *h_in = (!rev && a.ssm_in) ? a.ssm_in + ((int64_t)b * a.H + h) * PP * a.Nr : nullptr;
+    if (keep_state) {
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-            const int n0 = 4 * (4 * kk + s4);
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (h0 && n0 < a.Nr) v = *reinterpret_cast<const float4 *>(h0 + n0);      // rows beyond the model's d_state are padding
-            hst[4 * kk] = v.x; hst[4 * kk + 1] = v.y; hst[4 * kk + 2] = v.z; hst[4 * kk + 3] = v.w;
+        for (int t = 0; t < 8; ++t) {
+            const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
+            float2 v0 = make_float2(0.f, 0.f), v1 = v0;
+            if (h_in && n < a.Nr) {                        // columns beyond the model's d_state are padding
+                v0 = *reinterpret_cast<const float2 *>(h_in + (int64_t)p0 * a.Nr + n);
+                v1 = *reinterpret_cast<const float2 *>(h_in + (int64_t)(p0 + 8) * a.Nr + n);
+            }
+            hacc[t][0] = v0.x; hacc[t][1] = v0.y; hacc[t][2] = v1.x; hacc[t][3] = v1.y;
         }
     }
 
     for (int si = 0; si < nsub; ++si) {
         const int sub = rev ? nsub - 1 - si : si, r0 = sub * QB;
-        const bool have_state = si > 0 || (!rev && a.ssm_in != nullptr);
+        const bool have_state = si > 0 || h_in != nullptr;
         const bool need_update = si + 1 < nsub || (!rev && a.ssm_out != nullptr);
         __syncthreads();                                   // the previous sub-chunk's readers are done with the tiles
         // ---- load
@@ -836,142 +978,155 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             if (pr >= 0 && pr < L) v = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)pr * a.d_in_proj + a.d_inner + h * PP + c));
             else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0)            // rows before the sequence: the carried conv state
                 v = __ldg(reinterpret_cast<const uint4 *>(a.conv_in + ((int64_t)b * (k - 1) + (k - 1 + pr)) * a.conv_ch + h * PP + c));
-            const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { xr[rr][c + 2 * e] = bf16_lo(wv[e]); xr[rr][c + 2 * e + 1] = bf16_hi(wv[e]); }
+            *reinterpret_cast<float4 *>(&xr[rr][c]) = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+            *reinterpret_cast<float4 *>(&xr[rr][c + 4]) = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
         }
         for (int u = tid; u < QB * (N / 8); u += NT) {
             const int i = u / (N / 8), c = (u % (N / 8)) * 8;
             const int64_t off = (seq * L + r0 + i) * N + c;
             const bool ok = r0 + i < L;
-            if (have_state) {
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (ok) v = __ldg(reinterpret_cast<const uint4 *>(Cp + off));
-                *reinterpret_cast<float4 *>(&Cs[i][c]) = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
-                *reinterpret_cast<float4 *>(&Cs[i][c + 4]) = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
-            }
-            if (need_update) {
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (ok) v = __ldg(reinterpret_cast<const uint4 *>(Bp + off));
-                *reinterpret_cast<float4 *>(&Bs[i][c]) = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
-                *reinterpret_cast<float4 *>(&Bs[i][c + 4]) = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
-            }
+            if (have_state) *reinterpret_cast<uint4 *>(&Ct[i][c]) = ok ? __ldg(reinterpret_cast<const uint4 *>(Cp + off)) : make_uint4(0u, 0u, 0u, 0u);
+            if (need_update) *reinterpret_cast<uint4 *>(&Bt[i][c]) = ok ? __ldg(reinterpret_cast<const uint4 *>(Bp + off)) : make_uint4(0u, 0u, 0u, 0u);
         }
         {
             const float *S = Sb + (seq * nsub_all + sub) * (QB * QB);
-            for (int e = tid; e < QB * QB; e += NT) Ws[e / QB][e % QB] = S[e];
+            for (int e = tid; e < QB * QB; e += NT) Ss[e / QB][e % QB] = S[e];
         }
+        if (have_state) {
+            if (si == 0) {
+                // bf16 copy of the carried state: thread = (channel, 32 of its states in four runs of 8)
+                const int p = tid >> 2, s4 = tid & 3;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const int n0 = 8 * (4 * kk + s4);
+                    float4 v0 = make_float4(0.f, 0.f, 0.f, 0.f), v1 = v0;
+                    if (n0 < a.Nr) {
+                        v0 = *reinterpret_cast<const float4 *>(h_in + (int64_t)p * a.Nr + n0);
+                        v1 = *reinterpret_cast<const float4 *>(h_in + (int64_t)p * a.Nr + n0 + 4);
+                    }
+                    *reinterpret_cast<uint4 *>(&Ht[p][n0]) = make_uint4(pack_bf16(v0.x, v0.y), pack_bf16(v0.z, v0.w), pack_bf16(v1.x, v1.y), pack_bf16(v1.z, v1.w));
+                }
+            } else {
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {              // from the accumulators of the previous sub-chunk
+                    const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
+                    *reinterpret_cast<uint32_t *>(&Ht[p0][n]) = pack_bf16(hacc[t][0], hacc[t][1]);
+                    *reinterpret_cast<uint32_t *>(&Ht[p0 + 8][n]) = pack_bf16(hacc[t][2], hacc[t][3]);
+                }
+            }
+        }
+        // the gate's z (it holds SiLU(z): the in_proj epilogue applied it), fetched now so that its latency hides behind the products
+        uint4 zv = make_uint4(0u, 0u, 0u, 0u);
+        if (r0 + ei < L) zv = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)(r0 + ei) * a.d_in_proj + h * PP + ec));
         __syncthreads();
-        // ---- conv + SiLU: thread = channel cch, rows 8 crg .. 8 crg + 7;  mask: W in place of S;  state weights w_j
+        // ---- conv + SiLU: thread = channel cch, rows 8 crg .. 8 crg + 7;  mask: W from S
+        const float lam_last = lam[rev ? 0 : QB - 1], lam0 = sc[0];      // rows past the end of the sequence have Delta = 0: Lambda stays put there
 #pragma unroll
         for (int ii = 0; ii < QB * PP / NT; ++ii) {
             const int i = crg * (QB * PP / NT) + ii;
             float v = cbias;
 #pragma unroll
             for (int m = 0; m < 4; ++m) v = fmaf(wl[m], xr[rev ? i + m : i + 3 - m][cch], v);
-            xs[i][cch] = v / (1.f + __expf(-v));
+            const float xv = v / (1.f + __expf(-v));
+            Xt[i][cch] = __float2bfloat16_rn(xv);
+            WXt[i][cch] = __float2bfloat16_rn(r0 + i < L ? ex2f(lam_last - lamp[i]) * xv : 0.f);
         }
-        for (int e = tid; e < QB * QB; e += NT) {
-            const int i = e / QB, j = e % QB;
-            const bool ok = (rev ? j >= i : j <= i) && r0 + i < L && r0 + j < L;
-            Ws[i][j] = ok ? fmaf(Ws[i][j], ex2f(lam[i] - lamp[j]), i == j ? Dh : 0.f) : 0.f;
+        for (int e = tid; e < QB * QB / 2; e += NT) {
+            const int i = e / (QB / 2), j = (e % (QB / 2)) * 2;
+            float wv[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int jj = j + q;
+                const bool ok = (rev ? jj >= i : jj <= i) && r0 + i < L && r0 + jj < L;
+                wv[q] = ok ? fmaf(Ss[i][jj], ex2f(lam[i] - lamp[jj]), i == jj ? Dh : 0.f) : 0.f;
+            }
+            *reinterpret_cast<uint32_t *>(&Wt[i][j]) = pack_bf16(wv[0], wv[1]);
         }
-        const float lam_last = lam[rev ? 0 : QB - 1], lam0 = sc[0];      // rows past the end of the sequence have Delta = 0: Lambda stays put there
-        if (tid < QB) wjs[tid] = r0 + tid < L ? ex2f(lam_last - lamp[tid]) : 0.f;
         __syncthreads();
-        // ---- y of tokens i = 4 m + s4, channel p
-        float y8[8];
+        // ---- y: warp = tokens [16 ymt, +16) x channels [16 ynh, +16)
+        {
+            const int ymt = warp & 1, ynh = warp >> 1;
+            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            if (have_state) {
 #pragma unroll
-        for (int m = 0; m < 8; ++m) y8[m] = 0.f;
-        if (have_state) {
-            float acc[QB];
+                for (int k0 = 0; k0 < N; k0 += 16) {
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4(a0, a1, a2, a3, &Ct[16 * ymt + (lane & 15)][k0 + (lane >> 4) * 8]);
 #pragma unroll
-            for (int i = 0; i < QB; ++i) {
-                float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const float4 c4 = *reinterpret_cast<const float4 *>(&Cs[i][4 * (4 * kk + s4)]);
-                    s0 = fmaf(hst[4 * kk], c4.x, s0); s1 = fmaf(hst[4 * kk + 1], c4.y, s1);
-                    s0 = fmaf(hst[4 * kk + 2], c4.z, s0); s1 = fmaf(hst[4 * kk + 3], c4.w, s1);
+                    for (int nt = 0; nt < 2; ++nt) {
+                        uint32_t b0, b1;
+                        ldmatrix_x2(b0, b1, &Ht[16 * ynh + 8 * nt + (lane & 7)][k0 + ((lane >> 3) & 1) * 8]);
+                        mma_bf16_16816(acc[nt], a0, a1, a2, a3, b0, b1);
+                    }
                 }
-                acc[i] = s0 + s1;
+                const float e0 = ex2f(lam[16 * ymt + gr] - lam0), e1 = ex2f(lam[16 * ymt + gr + 8] - lam0);
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) { acc[nt][0] *= e0; acc[nt][1] *= e0; acc[nt][2] *= e1; acc[nt][3] *= e1; }
             }
-            // transposing reduction over the four lanes of p: lane s4 ends with the full sums of tokens i = 4 m + s4
-            float r16[16];
-            const bool hi2 = (s4 & 2) != 0;
 #pragma unroll
-            for (int q = 0; q < 16; ++q) {
-                const int ilo = (q >> 1) * 4 + (q & 1), ihi = ilo + 2;       // tokens with bit 1 clear / set
-                const float send = hi2 ? acc[ilo] : acc[ihi], keep = hi2 ? acc[ihi] : acc[ilo];
-                r16[q] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-            }
-            const bool hi1 = (s4 & 1) != 0;
+            for (int k0 = 0; k0 < QB; k0 += 16) {
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4(a0, a1, a2, a3, &Wt[16 * ymt + (lane & 15)][k0 + (lane >> 4) * 8]);
 #pragma unroll
-            for (int m = 0; m < 8; ++m) {
-                const float send = hi1 ? r16[2 * m] : r16[2 * m + 1], keep = hi1 ? r16[2 * m + 1] : r16[2 * m];
-                y8[m] = (keep + __shfl_xor_sync(0xffffffffu, send, 1)) * ex2f(lam[4 * m + s4] - lam0);
-            }
-        }
-        float xv[QB];
-#pragma unroll
-        for (int j = 0; j < QB; ++j) xv[j] = xs[j][p];
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int jq = 0; jq < 8; ++jq) {
-                if (rev ? jq >= m : jq <= m) {             // the other 4-column groups of rows 4 m .. 4 m + 3 are all zero
-                    const float4 w4 = *reinterpret_cast<const float4 *>(&Ws[4 * m + s4][4 * jq]);
-                    s0 = fmaf(w4.x, xv[4 * jq], s0); s1 = fmaf(w4.y, xv[4 * jq + 1], s1);
-                    s0 = fmaf(w4.z, xv[4 * jq + 2], s0); s1 = fmaf(w4.w, xv[4 * jq + 3], s1);
+                for (int nt = 0; nt < 2; ++nt) {
+                    uint32_t b0, b1;
+                    ldmatrix_x2_t(b0, b1, &Xt[k0 + (lane & 15)][16 * ynh + 8 * nt]);
+                    mma_bf16_16816(acc[nt], a0, a1, a2, a3, b0, b1);
                 }
             }
-            y8[m] += s0 + s1;
-        }
 #pragma unroll
-        for (int m = 0; m < 8; ++m) xr[4 * m + s4][p] = y8[m];          // the raw rows were last read before the previous barrier
+            for (int nt = 0; nt < 2; ++nt) {               // the raw rows were last read before the previous barrier
+                const int col = 16 * ynh + 8 * nt + 2 * qc, row = 16 * ymt + gr;
+                *reinterpret_cast<float2 *>(&xr[row][col]) = make_float2(acc[nt][0], acc[nt][1]);
+                *reinterpret_cast<float2 *>(&xr[row + 8][col]) = make_float2(acc[nt][2], acc[nt][3]);
+            }
+        }
+        // ---- state after the sub-chunk: h <- dec h + (w o x')^T B'
+        if (need_update) {
+            const float dec = ex2f(lam_last - lam0);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) { hacc[t][0] *= dec; hacc[t][1] *= dec; hacc[t][2] *= dec; hacc[t][3] *= dec; }
+#pragma unroll
+            for (int k0 = 0; k0 < QB; k0 += 16) {
+                uint32_t a0, a1, a2, a3;                    // A = (w o x')^T [p][j] read transposed from [j][p]
+                ldmatrix_x4_t(a0, a1, a2, a3, &WXt[k0 + (lane & 7) + ((lane >> 4) & 1) * 8][16 * smt + ((lane >> 3) & 1) * 8]);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    uint32_t b0, b1;                        // B = B' [j][n] read transposed
+                    ldmatrix_x2_t(b0, b1, &Bt[k0 + (lane & 15)][64 * snh + 8 * t]);
+                    mma_bf16_16816(hacc[t], a0, a1, a2, a3, b0, b1);
+                }
+            }
+        }
         __syncthreads();
         // ---- gate: thread = (token ei, channels ec .. ec + 7)
         {
             const int row = r0 + ei;
-            const bool ok = row < L;
-            uint4 zv = make_uint4(0u, 0u, 0u, 0u);
-            if (ok) zv = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)row * a.d_in_proj + h * PP + ec));      // holds SiLU(z): the in_proj epilogue applied it
             const float zf[8] = {bf16_lo(zv.x), bf16_hi(zv.x), bf16_lo(zv.y), bf16_hi(zv.y), bf16_lo(zv.z), bf16_hi(zv.z), bf16_lo(zv.w), bf16_hi(zv.w)};
+            const float nw[8] = {bf16_lo(nwp[0]), bf16_hi(nwp[0]), bf16_lo(nwp[1]), bf16_hi(nwp[1]), bf16_lo(nwp[2]), bf16_hi(nwp[2]), bf16_lo(nwp[3]), bf16_hi(nwp[3])};
+            const float4 y0 = *reinterpret_cast<const float4 *>(&xr[ei][ec]), y1 = *reinterpret_cast<const float4 *>(&xr[ei][ec + 4]);
+            const float yv[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
             float g[8], ss = 0.f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { g[e] = xr[ei][ec + e] * zf[e]; ss = fmaf(g[e], g[e], ss); g[e] *= nw[e]; }
+            for (int e = 0; e < 8; ++e) { g[e] = yv[e] * zf[e]; ss = fmaf(g[e], g[e], ss); g[e] *= nw[e]; }
 #pragma unroll
             for (int off = 1; off < U8; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-            if (ok) {
+            if (row < L) {
                 *reinterpret_cast<uint4 *>(a.g + (seq * L + row) * a.d_inner + h * PP + ec) =
                     make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]), pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
                 if (a.ssq && ec == 0) a.ssq[(seq * L + row) * a.H + h] = ss;
             }
         }
-        // ---- state after the sub-chunk
-        if (need_update) {
-            const float dec = ex2f(lam_last - lam0);
-#pragma unroll
-            for (int q = 0; q < 32; ++q) hst[q] *= dec;
-#pragma unroll 4
-            for (int j = 0; j < QB; ++j) {
-                const float wx = wjs[j] * xs[j][p];
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[j][4 * (4 * kk + s4)]);
-                    hst[4 * kk] = fmaf(wx, b4.x, hst[4 * kk]); hst[4 * kk + 1] = fmaf(wx, b4.y, hst[4 * kk + 1]);
-                    hst[4 * kk + 2] = fmaf(wx, b4.z, hst[4 * kk + 2]); hst[4 * kk + 3] = fmaf(wx, b4.w, hst[4 * kk + 3]);
-                }
-            }
-        }
     }
     if (!rev && a.ssm_out) {
-        float *ho = a.ssm_out + (((int64_t)b * a.H + h) * PP + p) * a.Nr;
+        float *ho = a.ssm_out + ((int64_t)b * a.H + h) * PP * a.Nr;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-            const int n0 = 4 * (4 * kk + s4);
-            if (n0 < a.Nr) *reinterpret_cast<float4 *>(ho + n0) = make_float4(hst[4 * kk], hst[4 * kk + 1], hst[4 * kk + 2], hst[4 * kk + 3]);
+        for (int t = 0; t < 8; ++t) {
+            const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
+            if (n < a.Nr) {
+                *reinterpret_cast<float2 *>(ho + (int64_t)p0 * a.Nr + n) = make_float2(hacc[t][0], hacc[t][1]);
+                *reinterpret_cast<float2 *>(ho + (int64_t)(p0 + 8) * a.Nr + n) = make_float2(hacc[t][2], hacc[t][3]);
+            }
         }
     }
 }
@@ -981,7 +1136,7 @@ constexpr int BLOCK_MAX_L = 2 * QB;       // sequences up to this length take th
 bool block_mode(const ScanArgs &a) { return a.chunk == QB || (a.chunk == 0 && a.L <= BLOCK_MAX_L); }
 
 struct Scratch {
-    size_t bp, cp, da, sb, total;
+    size_t bp, cp, da, sb, sy, total;
     int nch, Lp;
 };
 Scratch scratch_layout(const ScanArgs &a) {
@@ -994,6 +1149,7 @@ Scratch scratch_layout(const ScanArgs &a) {
     s.da = off; off += align_up((size_t)2 * a.B * a.H * 2 * s.Lp * 4);
     s.sb = off;
     if (block_mode(a)) off += align_up((size_t)2 * a.B * s.nch * PREP_PARTS * QB * QB * 4);
+    s.sy = off; off += align_up(((size_t)2 * a.B * s.nch + 1) * sizeof(int));      // ticket counter and item flags of the fused prep
     s.total = off;
     return s;
 }
@@ -1040,13 +1196,24 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     const bool blk = block_mode(a);
     float *Sb = blk ? reinterpret_cast<float *>(base + l.sb) : nullptr;
 
-    ssd_prep_kernel<<<dim3(l.nch * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);
-    count_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    // One long sequence leaves SMs without a scan CTA: they take the prep work inside the scan launch (see prep_role).
+    const int nscan = a.H * ndir * a.B, n_items = ndir * a.B * l.nch;
+    PrepJob pj{Bp, Cp, dA, nullptr, 0, ndir};
+    if (!blk && nscan < sm_count() && a.N % 8 == 0) {
+        pj.sync = reinterpret_cast<int *>(base + l.sy);
+        pj.nprep = n_items < sm_count() - nscan ? n_items : sm_count() - nscan;
+    }
+    cudaError_t e;
+    if (pj.sync) {
+        if ((e = cudaMemsetAsync(pj.sync, 0, ((size_t)2 * a.B * l.nch + 1) * sizeof(int), s)) != cudaSuccess) return e;
+    } else {
+        ssd_prep_kernel<<<dim3(l.nch * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     if (blk) {
         auto kern = a.P == P ? ssd_block_kernel<P> : ssd_block_kernel<P / 2>;
-        const size_t smem = a.P == P ? block_smem_bytes<P>() : block_smem_bytes<P / 2>();
+        const size_t smem = a.P == P ? BlockSmem<P>::total : BlockSmem<P / 2>::total;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<dim3(a.H, ndir, a.B), 4 * a.P, smem, s>>>(k, Bp, Cp, Sb, dir0);
@@ -1078,7 +1245,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     auto kern = a.P == P ? ssd_scan_kernel<false> : ssd_scan_kernel<true>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    kern<<<dim3(a.H, ndir, a.B), NTHREADS, SMEM_BYTES, s>>>(mx, mz, mb, mc, mg, k, dir0, status);
+    kern<<<nscan + pj.nprep, NTHREADS, SMEM_BYTES, s>>>(mx, mz, mb, mc, mg, k, pj, dir0, status);
     count_launch();
     return cudaGetLastError();
 }

@@ -100,6 +100,31 @@ __device__ __forceinline__ void ld_global_256(const void *p, uint32_t (&v)[8]) {
 }
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Orders this thread's earlier generic-proxy view of memory (e.g. after an acquire load of a flag another CTA released)
+// before its later async-proxy operations (TMA and bulk loads) on any state space.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire_gpu(const int *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int *p, int v) { asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory"); }
+// Bounded wait for a flag in global memory that another CTA of the same launch sets once (same abort protocol as mbar_wait).
+__device__ __forceinline__ bool flag_wait(const int *flag, volatile int *abort_flag, int *status) {
+    if (ld_acquire_gpu(flag) != 0) { fence_proxy_async_all(); return true; }
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i)
+            if (ld_acquire_gpu(flag) != 0) { fence_proxy_async_all(); return true; }
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+            *abort_flag = 1;
+            atomicExch(status, (int)DM_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
 
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
     asm volatile(
