@@ -28,18 +28,39 @@ from paper_2511_15927_b200 import inputs as I  # noqa: E402
 METRIC = "denoised tokens/s per bidirectional Mamba layer"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (taken on
-# cfg3_8k = 8192 tokens; traffic of both kernels grows in proportion to the token count, so other single-layer bf16
+# dram__bytes_read.sum + dram__bytes_write.sum per launch come from the ncu summaries committed under profiles/ (captured on
+# cfg3_8k = 8192 tokens; the traffic of both kernels grows in proportion to the token count, so other single-layer bf16
 # workloads of the same widths scale it by their tokens; None = no capture applies).
-NCU_TRAFFIC_PER_TOKEN = {"scan": (286.4230e6 + 108.9836e6) / 8192,      # ssd_scan_kernel, profiles/ssd_scan_cfg3_8k.txt
-                         "in_proj": (72.3308e6 + 112.3448e6) / 8192}    # gemm_tc_kernel<256>, one direction, profiles/gemm_tc_cfg3_8k.txt
+NCU_PROFILES = {"scan": "ssd_scan_cfg3_8k.txt", "in_proj": "gemm_tc_cfg3_8k.txt"}
+NCU_TOKENS = 8192
 NCU_WIDTHS = (2048, 128, 64)                                             # d_model, d_state, heads the captures were taken at
 
 
-def ncu_traffic(kind, shape, dtype, tokens):
-    if dtype != I.BF16 or (shape.d_model, shape.d_state, shape.n_heads) != NCU_WIDTHS or kind not in NCU_TRAFFIC_PER_TOKEN:
+def profile_traffic(kind):
+    """Bytes per launch (DRAM read + write) of the first captured launch in the kernel's profile summary, or None."""
+    import re
+    path = os.path.join(ROOT, "profiles", NCU_PROFILES.get(kind, ""))
+    if not os.path.isfile(path):
         return None
-    return NCU_TRAFFIC_PER_TOKEN[kind] * tokens
+    rd = wr = None
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    with open(path) as f:
+        for line in f:
+            m = re.match(r"\s*dram__bytes_(read|write)\.sum\s+(\w+)\s+([0-9.eE+-]+)", line)
+            if m and m.group(2) in scale:
+                v = float(m.group(3)) * scale[m.group(2)]
+                if m.group(1) == "read" and rd is None:
+                    rd = v
+                elif m.group(1) == "write" and wr is None:
+                    wr = v
+    return rd + wr if rd is not None and wr is not None else None
+
+
+def ncu_traffic(kind, shape, dtype, tokens):
+    if dtype != I.BF16 or (shape.d_model, shape.d_state, shape.n_heads) != NCU_WIDTHS:
+        return None
+    per_launch = profile_traffic(kind)
+    return per_launch / NCU_TOKENS * tokens if per_launch else None
 
 
 def load_peaks():
@@ -130,6 +151,32 @@ def oracle_sample_seconds(shape: I.MixerShape, dtype: str, sample_len: int, seed
     return time.perf_counter() - t0
 
 
+def oracle_stack_sample_seconds(spec, n_tok: int, n_layers: int = 2, seed: int = 0):
+    """Time the fp64 oracle, as it stands, on a bounded sample of a stack workload: batch row 0, the first n_tok tokens, the
+    first n_layers layers at full widths plus the output head.  The metric is per layer, so fewer layers do not change what
+    is measured.  Returns (seconds, layers run)."""
+    from oracle import bimamba_oracle as O
+    sh = spec["shape"]
+    s1 = I.MixerShape(1, n_tok, sh.d_model, sh.expand, sh.d_state, sh.d_conv, sh.n_heads, sh.n_groups)
+    sw = I.make_stack_weights(s1, n_layers, spec["vocab"], seed=seed, dtype=I.BF16)
+    tok = I.make_tokens(1, n_tok, 50257, 50257, seed=seed)
+    kw = dict(expand=sh.expand, d_state=sh.d_state, n_heads=sh.n_heads, n_groups=sh.n_groups)
+    cond = spec.get("cond")
+    if cond:
+        I.add_block_weights(sw, s1, cond["d_ff"], cond["d_cond"], seed=seed, dtype=I.BF16)
+        tau = I.make_timestep_embedding(1, cond["d_cond"], seed=seed)
+    t0 = time.perf_counter()
+    if cond:
+        O.denoise_step_cond(tok, tau, sw, **kw)
+    else:
+        O.denoise_step(tok, sw, **kw)
+    return time.perf_counter() - t0, n_layers
+
+
+def host_cores() -> int:
+    return int(os.cpu_count() or 1)
+
+
 def blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -154,9 +201,33 @@ def run_reference(args, shape, dtype, rank):
             "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": args.workload, "sample": desc},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "threads_used": blas_threads(), "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_reference_stack(args):
+    """The reference arm on a stack workload: the CPU oracle on a bounded sample (see oracle_stack_sample_seconds)."""
+    spec = STACKS[args.workload]
+    if spec.get("hybrid"):
+        print(json.dumps({"impl": "reference", "unavailable": "the oracle sample covers the Mamba stacks; the hybrid's attention layers are not sampled"}), flush=True)
+        return
+    n_tok = min(spec["shape"].seqlen, args.ref_tokens)
+    for _ in range(min(args.warmup, 1)):
+        oracle_stack_sample_seconds(spec, n_tok)
+    secs, nl = [], 2
+    for _ in range(args.steps):
+        sec, nl = oracle_stack_sample_seconds(spec, n_tok)
+        secs.append(sec)
+    sec = float(np.sum(secs))
+    value = n_tok * nl * args.steps / sec
+    desc = f"batch row 0, first {n_tok} tokens, first {nl} layers + output head of {args.workload} per step (full widths)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": args.workload, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "threads_used": blas_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
@@ -176,6 +247,13 @@ STACKS = {
     "paper_b8_1k_sample": dict(shape=I.MixerShape(8, 1024, 1920, 2, 128, 4, 120), layers=24, vocab=50304,
                                cond=dict(d_ff=3840, d_cond=128), sample=dict(p=16)),
     "cfg2_stack_cond": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, cond=dict(d_ff=2048, d_cond=128)),
+    # block-autoregressive decoding as stated: a 2048-token prefix committed once, then 64 blocks of 32 tokens, each with 8 denoising
+    # passes that read the carried state and one commit pass that writes the next block's state (ping-pong); step = one block
+    "cfg4_loop": dict(shape=I.MixerShape(16, 32, 2048, 2, 128, 4, 64), layers=24, vocab=50304, prefix=2048, loop=dict(blocks=64, passes=8)),
+    # whole generations with dm_generate: K = L / p reverse steps of Eq. 3 plus the clean-up pass, from an all-mask start; step = one generation
+    "paper_b8_1k_generate": dict(shape=I.MixerShape(8, 1024, 1920, 2, 128, 4, 120), layers=24, vocab=50304,
+                                 cond=dict(d_ff=3840, d_cond=128), generate=dict(p=16)),
+    "cfg2_generate_1k": dict(shape=I.MixerShape(4, 1024, 1024, 2, 16, 4, 32), layers=24, vocab=50304, generate=dict(p=16)),
 }
 
 
@@ -318,9 +396,45 @@ def run_stack(args, rank, local_rank, world):
         ws = G.workspace(nb)
     toks = tokens(Lb, 4)
     amax = torch.empty((B, Lb), device="cuda", dtype=torch.int32)
+    loop, gen = spec.get("loop"), spec.get("generate")
+    passes_per_step = 1                                   # denoiser evaluations in one step
 
     def step(i):
         denoise(scfg, toks[i % 4].data_ptr(), amax.data_ptr(), states)
+
+    if loop:
+        # second set of state buffers; block i reads set i % 2 in its denoising passes and commits into the other one
+        st_bufs2 = [(torch.empty_like(sb), torch.empty_like(cb)) for sb, cb in st_bufs]
+        sets = (st_bufs, st_bufs2)
+        read_st, commit_st = [], []
+        for par in range(2):
+            rd, cm = (dm.dm_layer_state * layers)(), (dm.dm_layer_state * layers)()
+            for i in range(layers):
+                (si, ci), (so, co) = sets[par][i], sets[1 - par][i]
+                rd[i] = dm.dm_layer_state(si.data_ptr(), ci.data_ptr(), None, None)
+                cm[i] = dm.dm_layer_state(si.data_ptr(), ci.data_ptr(), so.data_ptr(), co.data_ptr())
+            read_st.append(rd); commit_st.append(cm)
+        passes_per_step = loop["passes"] + 1
+
+        def step(i):                                      # one block: its denoising passes, then the commit pass over its final tokens
+            for p in range(loop["passes"]):
+                denoise(scfg, toks[(i + p) % 4].data_ptr(), amax.data_ptr(), read_st[i % 2])
+            denoise(scfg, toks[(i + 3) % 4].data_ptr(), amax.data_ptr(), commit_st[i % 2])
+    if gen:
+        K = Lb // gen["p"]
+        gcfg = dm.dm_generate_cfg(K, 1e-3, 50257, 50258)
+        g2 = torch.Generator(device="cuda").manual_seed(2)
+        gu_keep = torch.rand(K + 1, B, Lb, generator=g2, device="cuda")
+        gu_cat = torch.rand(K + 1, B, Lb, generator=g2, device="cuda")
+        gtau = torch.from_numpy(np.stack([I.make_timestep_embedding(B, cond["d_cond"], seed=k) for k in range(K + 1)])).cuda() if cond else None
+        gstart = torch.full((B, Lb), 50257, device="cuda", dtype=torch.int32)
+        nbg = dm.dm_generate_workspace_bytes(scfg, blk if cond else None)
+        ws = G.workspace(max(nb, nbg))
+        passes_per_step = K + 1
+
+        def step(i):                                      # one generation from an all-mask start: K reverse steps + the clean-up pass
+            dm.dm_generate(scfg, blk if cond else None, csw, cbw if cond else None, gcfg, gstart.data_ptr(), gtau.data_ptr() if cond else 0,
+                           gu_keep.data_ptr(), gu_cat.data_ptr(), amax.data_ptr(), 0, ws.data_ptr(), ws.numel(), stream_box[0])
 
     def timed(fn, n):
         for i in range(args.warmup):
@@ -356,13 +470,18 @@ def run_stack(args, rank, local_rank, world):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=cap):
                 stream_box[0] = torch.cuda.current_stream().cuda_stream
-                denoise(scfg, toks[i].data_ptr(), amax.data_ptr(), states)
+                step(i)
             stream_box[0] = stream
             graphs.append(g)
-        denoise(scfg, toks[0].data_ptr(), amax.data_ptr(), states)
+        if loop:                                          # same starting state for the eager block and the replayed one
+            saved = [(sb.clone(), cb.clone()) for sb, cb in st_bufs]
+        step(0)
         torch.cuda.synchronize()
         eager = amax.clone()
         amax.fill_(-1)
+        if loop:
+            for (sb, cb), (s0, c0) in zip(st_bufs, saved):
+                sb.copy_(s0); cb.copy_(c0)
         graphs[0].replay()
         torch.cuda.synchronize()
         if not torch.equal(eager, amax):
@@ -376,7 +495,7 @@ def run_stack(args, rank, local_rank, world):
         ftok = tokens(prefix + Lb, 2)
         famax = torch.empty((B, prefix + Lb), device="cuda", dtype=torch.int32)
         ms_full = timed(lambda i: denoise(fcfg, ftok[i % 2].data_ptr(), famax.data_ptr(), None), max(2, args.steps // 4)) / max(2, args.steps // 4)
-        extra = dict(extra, prefix=prefix, full_reencode_ms_per_step=ms_full, state_carry_speedup=ms_full / ms_step)
+        extra = dict(extra, prefix=prefix, full_reencode_ms_per_pass=ms_full, state_carry_speedup=ms_full / (ms_step / passes_per_step))
     # end to end: token ids from pinned host memory in, arg-max ids back, inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -386,7 +505,11 @@ def run_stack(args, rank, local_rank, world):
 
         def host_step(i):
             td.copy_(th, non_blocking=True)
-            denoise(scfg, td.data_ptr(), amax.data_ptr(), states)
+            if loop or gen:                               # the block's / the generation's start tokens in, its final ids out
+                (gstart if gen else toks[i % 4]).copy_(td, non_blocking=True)
+                step(i)
+            else:
+                denoise(scfg, td.data_ptr(), amax.data_ptr(), states)
             ah.copy_(amax, non_blocking=True)
             torch.cuda.synchronize()
         for i in range(2):
@@ -395,7 +518,7 @@ def run_stack(args, rank, local_rank, world):
         for i in range(args.steps):
             host_step(i)
         sec = time.perf_counter() - t0
-        e2e = {"value": world * T * layers * args.steps / sec, "unit": UNIT, "h2d_bytes_per_step": T * 4, "d2h_bytes_per_step": T * 4}
+        e2e = {"value": world * T * passes_per_step * layers * args.steps / sec, "unit": UNIT, "h2d_bytes_per_step": T * 4, "d2h_bytes_per_step": T * 4}
     if rank != 0:
         D.shutdown()
         return
@@ -413,28 +536,140 @@ def run_stack(args, rank, local_rank, world):
     scan_gbs = scan_bytes / (scn * 1e-3) / 1e9
     kernels = {"in_proj_per_layer": {"ms": inp, "tflops": in_tf}, "scan_per_layer": {"ms": scn, "gbs": scan_gbs},
                "out_proj_per_layer": {"ms": outp, "tflops": out_tf},
-               "rest_of_step_ms": ms_step - n_mamba * (inp + scn + outp)}
+               "rest_of_step_ms": ms_step - passes_per_step * n_mamba * (inp + scn + outp)}
+    burst = ms_total < 1000.0
+    tpk = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    tsrc = peaks["source"] + (" (burst bf16: timed region under 1 s)" if burst else " (sustained bf16: timed region over 1 s)")
+    scan_entry = {"kernel": "fused conv+scan+gate (per layer)", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                  "frac": scan_gbs / peaks["hbm_gbs"], "frac_of_8tbs": scan_gbs / 8000.0, "ms": scn, "algorithmic_bytes": scan_bytes,
+                  "traffic": None, "peak_source": peaks["source"] + " (copy bandwidth)"}
     if scn >= max(inp, outp):
-        roofline = {"kernel": "fused conv+scan+gate (per layer)", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": scan_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+        roofline = dict(scan_entry)
     else:
         tf = in_tf if inp >= outp else out_tf
         roofline = {"kernel": ("in_proj" if inp >= outp else "out_proj") + " GEMM (per layer)", "bound": "tensor", "achieved": tf,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops_sustained"],
-                    "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)"}
-    line = {"metric": METRIC, "value": world * T * layers / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                    "peak": tpk, "unit": "TFLOP/s", "frac": tf / tpk, "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                    "traffic": None, "peak_source": tsrc}
+    roofline["scan"] = scan_entry
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline and not hyb:
+        n_tok = min(Lb, 128)
+        sec, nl = oracle_stack_sample_seconds(spec, n_tok)
+        cpu_baseline = {"value": n_tok * nl / sec, "unit": UNIT, "cores": host_cores(), "threads_used": blas_threads(), "kind": "oracle",
+                        "sample": f"batch row 0, first {n_tok} tokens, first {nl} layers + output head of {args.workload} (full widths), {sec:.1f} s; "
+                                  "the metric is per layer"}
+    npass = passes_per_step
+    line = {"metric": METRIC, "value": world * T * npass * layers / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": dict({"workload": args.workload, "batch": B, "seq_len": Lb, "d_model": shape.d_model, "d_state": shape.d_state,
-                            "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T / (ms_step * 1e-3),
+                            "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T * npass / (ms_step * 1e-3),
                             "parallelism": "replicas only" if world > 1 else "1 GPU",
                             "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
                            **({"hybrid": "attention mixer (%d heads of 64) in every %dth layer, %d Mamba layers; the attention layers are inside rest_of_step_ms"
                                          % (hyb["heads"], hyb["period"], n_mamba)} if hyb else {}),
                            **({"sample": "half of the positions masked, p = %d drawn per sequence and step" % smp["p"],
                                "generated_tokens_per_s_at_K_eq_L_over_p": world * T / ((Lb // smp["p"]) * ms_step * 1e-3)} if smp else {}),
+                           **({"loop": "step = one block of %d tokens per sequence: %d denoising passes reading the carried state + 1 commit pass; "
+                                       "%d blocks after a %d-token prefix" % (Lb, loop["passes"], loop["blocks"], prefix),
+                               "generated_tokens_per_s": world * T / (ms_step * 1e-3), "ms_per_pass": ms_step / npass} if loop else {}),
+                           **({"generate": "step = one generation of %d tokens per sequence from an all-mask start: K = L / %d = %d reverse steps "
+                                           "(Eq. 3) + the clean-up pass, one dm_generate call" % (Lb, gen["p"], Lb // gen["p"]),
+                               "generated_tokens_per_s": world * T / (ms_step * 1e-3), "ms_per_pass": ms_step / npass} if gen else {}),
                            **extra),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels, "cpu_baseline": None}
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline}
+    print(json.dumps(line), flush=True)
+    D.shutdown()
+
+
+def fit_latency(lengths, ms):
+    """Non-negative least-squares fit of the per-step latency t(L) = a L^2 + b L + c (Sec. 4.3, latency decomposition: the
+    quadratic term is what attention adds; a linear-time mixer should give a ~ 0).  L is scaled to units of 1024 tokens so
+    that the three columns have comparable size.  Returns a, b, c in ms per (1024 tokens)^2, ms per 1024 tokens, ms."""
+    from scipy.optimize import nnls
+    x = np.asarray(lengths, np.float64) / 1024.0
+    A = np.stack([x * x, x, np.ones_like(x)], axis=1)
+    coef, resid = nnls(A, np.asarray(ms, np.float64))
+    return [float(v) for v in coef], float(resid)
+
+
+def run_lsweep(args, rank, local_rank, world):
+    """cfg 3's sweep over L at batch 1 (the paper's throughput axis, Sec. 4.3, up to its longest context 65 536) with the
+    fit of fit_latency() over the whole mixer step and over the fused scan alone."""
+    import torch
+    from paper_2511_15927_b200 import build
+    if rank == 0 or world == 1:
+        build.build()
+    from paper_2511_15927_b200 import dist_util as D
+    D.init("nccl", local_rank)
+    from paper_2511_15927_b200 import binding as dm
+    torch.cuda.set_device(local_rank)
+    from paper_2511_15927_b200 import torch_io as G
+    lengths = [2048, 4096, 8192, 16384, 32768, 65536]
+    base, dtype = I.CONFIGS["cfg3_8k"]
+    wf, wr = I.make_mixer_weights(base, 0, dtype)
+    cw = (dm.make_dir_weights(G.dev_dir_weights(wf, dtype)), dm.make_dir_weights(G.dev_dir_weights(wr, dtype)))
+    keep = cw
+    stream = torch.cuda.current_stream().cuda_stream
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    rows, launches = [], 0
+    for L in lengths:
+        shape = I.MixerShape(1, L, base.d_model, base.expand, base.d_state, base.d_conv, base.n_heads)
+        cfg = G.cfg_of(shape, dtype)
+        g = torch.Generator(device="cuda").manual_seed(L)
+        xs = [torch.randn(1, L, shape.d_model, generator=g, device="cuda").to(torch.bfloat16) for _ in range(4)]
+        y = torch.empty_like(xs[0])
+        nb = dm.dm_bimamba_workspace_bytes(cfg)
+        ws = G.workspace(nb)
+        for i in range(args.warmup):
+            dm.dm_bimamba_forward(cfg, cw, xs[i % 4].data_ptr(), y.data_ptr(), ws.data_ptr(), nb, stream)
+        dm.dm_check(stream)
+        D.barrier(); torch.cuda.synchronize()
+        dm.dm_profile_enable(True); dm.dm_profile_read()
+        l0 = dm.dm_kernel_launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            dm.dm_bimamba_forward(cfg, cw, xs[i % 4].data_ptr(), y.data_ptr(), ws.data_ptr(), nb, stream)
+        e1.record()
+        D.barrier(); torch.cuda.synchronize()
+        launches += dm.dm_kernel_launch_count() - l0
+        stage_ms, stage_n = dm.dm_profile_read()
+        dm.dm_profile_enable(False)
+        dm.dm_check(stream)
+        ms = D.max_over_ranks(e0.elapsed_time(e1), "cuda") / args.steps
+        rows.append({"L": L, "ms_per_step": ms, "scan_ms": stage_ms[dm.DM_STAGE_SCAN] / max(stage_n[dm.DM_STAGE_SCAN], 1),
+                     "tokens_per_s": world * L / (ms * 1e-3)})
+        del xs, y, ws
+    clocks = sampler.stop() if sampler else None
+    if rank != 0:
+        D.shutdown()
+        return
+    (a, b, c), resid = fit_latency([r["L"] for r in rows], [r["ms_per_step"] for r in rows])
+    (sa, sb, sc), sresid = fit_latency([r["L"] for r in rows], [r["scan_ms"] for r in rows])
+    last = rows[-1]
+    peaks = load_peaks()
+    es = 2
+    shape = I.MixerShape(1, last["L"], base.d_model, base.expand, base.d_state, base.d_conv, base.n_heads)
+    scan_bytes = scan_bytes_per_token(shape, es) * last["L"]
+    scan_gbs = scan_bytes / (last["scan_ms"] * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": last["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": last["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": "lsweep_fit", "batch": 1, "seq_len": last["L"], "d_model": base.d_model, "d_state": base.d_state,
+                       "heads": base.n_heads, "sweep": rows,
+                       "latency_fit": {"model": "t(L) = a (L/1024)^2 + b (L/1024) + c, non-negative least squares, ms",
+                                       "mixer_step": {"a": a, "b": b, "c": c, "residual_ms": resid,
+                                                      "quadratic_share_at_65536": a * 64 * 64 / max(a * 64 * 64 + b * 64 + c, 1e-30)},
+                                       "fused_scan": {"a": sa, "b": sb, "c": sc, "residual_ms": sresid}},
+                       "l2": "inputs rotate over 4 buffers; every length's working set exceeds the 126 MB L2 from L = 4096 up",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+            "roofline": {"kernel": "fused conv+scan+gate at the longest length", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": scan_gbs / peaks["hbm_gbs"], "frac_of_8tbs": scan_gbs / 8000.0, "ms": last["scan_ms"],
+                         "algorithmic_bytes": scan_bytes, "traffic": ncu_traffic("scan", shape, I.BF16, last["L"]),
+                         "peak_source": peaks["source"] + " (copy bandwidth)"},
+            "cpu_baseline": None}
     print(json.dumps(line), flush=True)
     D.shutdown()
 
@@ -442,9 +677,9 @@ def run_stack(args, rank, local_rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 10; 64 blocks for cfg4_loop; 3 generations for the *_generate workloads)")
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS) + sorted(STACKS))
+    ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS) + sorted(STACKS) + ["lsweep_fit"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference arm's sample")
     ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
@@ -452,16 +687,26 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true", help="stack workloads: also time the step replayed from a captured CUDA graph")
     args = ap.parse_args()
+    if args.steps is None:
+        spec = STACKS.get(args.workload, {})
+        args.steps = spec["loop"]["blocks"] if spec.get("loop") else 3 if spec.get("generate") else 10
     if args.warmup < 3:
         args.warmup = max(args.warmup, 1) if args.impl == "reference" else 3
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.workload == "lsweep_fit":
+        if args.impl == "reference":
+            if rank == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the sweep is a post-processing workload of cfg3; run the reference arm on cfg3_8k"}), flush=True)
+            return
+        run_lsweep(args, rank, local_rank, world)
+        return
     if args.workload in STACKS:
         if args.impl == "reference":
             if rank == 0:
-                print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the oracle on single-layer workloads only"}), flush=True)
+                run_reference_stack(args)
             return
         run_stack(args, rank, local_rank, world)
         return
@@ -557,30 +802,46 @@ def main():
     scan_gbs = scan_bytes / (scan_ms * 1e-3) / 1e9
     in_tf = f_in * T / (inp_ms * 1e-3) / 1e12
     out_tf = f_out * T / (outp_ms * 1e-3) / 1e12
-    tensor_peak = peaks["bf16_tflops_sustained"]
+    def tfrac(tf):
+        return {"frac_of_%s_burst_tensor_peak" % peaks["source"]: tf / peaks["bf16_tflops"] if dtype == I.BF16 else None,
+                "frac_of_%s_sustained_tensor_peak" % peaks["source"]: tf / peaks["bf16_tflops_sustained"] if dtype == I.BF16 else None}
     kernels = {
-        "in_proj": {"ms": inp_ms, "tflops": in_tf, "frac_of_%s_tensor_peak" % peaks["source"]: in_tf / tensor_peak if dtype == I.BF16 else None},
+        "in_proj": dict({"ms": inp_ms, "tflops": in_tf}, **tfrac(in_tf)),
         "scan": {"ms": scan_ms, "gbs": scan_gbs, "frac_of_%s_hbm_peak" % peaks["source"]: scan_gbs / peaks["hbm_gbs"],
                  "frac_of_nominal_8tbs": scan_gbs / 8000.0, "algorithmic_bytes": scan_bytes},
-        "out_proj": {"ms": outp_ms, "tflops": out_tf, "frac_of_%s_tensor_peak" % peaks["source"]: out_tf / tensor_peak if dtype == I.BF16 else None},
+        "out_proj": dict({"ms": outp_ms, "tflops": out_tf}, **tfrac(out_tf)),
     }
+    # Tensor peak for the GEMMs: the timed region is tens of milliseconds at full clocks, i.e. the burst figure's regime;
+    # the sustained figure (a seconds-long loop under the power cap) is printed beside it.
+    burst = ms_total < 1000.0
+    tpk = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    tsrc = peaks["source"] + (" (burst bf16: timed region under 1 s)" if burst else " (sustained bf16)")
+    scan_entry = {"kernel": "fused conv+scan+gate", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                  "frac": scan_gbs / peaks["hbm_gbs"], "frac_of_8tbs": scan_gbs / 8000.0, "ms": scan_ms, "algorithmic_bytes": scan_bytes,
+                  "traffic": ncu_traffic("scan", shape, dtype, T), "peak_source": peaks["source"] + " (copy bandwidth)"}
+
+    def gemm_entry(name, tf, ms):
+        return {"kernel": name + " GEMM (one launch per direction)", "bound": "tensor", "achieved": tf, "peak": tpk, "unit": "TFLOP/s",
+                "frac": tf / tpk, "frac_of_sustained": tf / peaks["bf16_tflops_sustained"], "ms": ms,
+                "traffic": ncu_traffic(name, shape, dtype, T), "peak_source": tsrc}
     dominant = max(("in_proj", inp_ms), ("scan", scan_ms), ("out_proj", outp_ms), key=lambda kv: kv[1])[0]
     if dominant == "scan" or dtype != I.BF16:
-        roofline = {"kernel": "fused conv+scan+gate", "bound": "hbm", "achieved": scan_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": scan_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic("scan", shape, dtype, T),
-                    "peak_source": peaks["source"] + " (sustained copy)"}
+        roofline = dict(scan_entry)
     else:
-        tf = in_tf if dominant == "in_proj" else out_tf
-        roofline = {"kernel": dominant + " GEMM (one launch per direction)", "bound": "tensor", "achieved": tf, "peak": tensor_peak,
-                    "unit": "TFLOP/s", "frac": tf / tensor_peak, "traffic": ncu_traffic(dominant, shape, dtype, T),
-                    "peak_source": peaks["source"] + " (sustained bf16)"}
+        roofline = gemm_entry(dominant, in_tf if dominant == "in_proj" else out_tf, inp_ms if dominant == "in_proj" else outp_ms)
+    # the dominant kernel above; the kernel the metric names (the fused scan) and the other GEMM always ride along
+    roofline["scan"] = scan_entry
+    if dtype == I.BF16:
+        roofline["in_proj"] = gemm_entry("in_proj", in_tf, inp_ms)
+        roofline["out_proj"] = gemm_entry("out_proj", out_tf, outp_ms)
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         n_tok = min(shape.seqlen, args.cpu_baseline_tokens)
         sec = oracle_sample_seconds(shape, dtype, n_tok)
-        cpu_baseline = {"value": n_tok / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                        "sample": f"batch row 0, first {n_tok} tokens of {args.workload} (full widths, both directions), {sec:.1f} s"}
+        cpu_baseline = {"value": n_tok / sec, "unit": UNIT, "cores": host_cores(), "threads_used": blas_threads(), "kind": "oracle",
+                        "sample": f"batch row 0, first {n_tok} tokens of {args.workload} (full widths, both directions), {sec:.1f} s; "
+                                  "the token loop of the oracle is one Python thread, its matrix products use the BLAS threads"}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -218,6 +218,31 @@ int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
                            int32_t *tokens_out, const dm_layer_state *states,
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* A whole generation, Sec. 2 Eq. 3 with Sec. 4.3's step count (K = L / p denoising steps for p tokens per step): K
+ * reverse steps along the noise levels t_k = 1 - (1 - t_eps) k / K (k = 0..K; App. A.1's sampling eps is 1e-3), step k
+ * being dm_denoise_sample_step with keep_prob = (float)(t_{k+1} / t_k) computed in double, followed by one clean-up
+ * pass with keep_prob = 0 that draws every position still masked at noise level t_eps: K + 1 denoiser evaluations, all
+ * enqueued on `cuda_stream` by this one call, nothing read back to the host in between (the number of positions a
+ * step draws stays on the device), so the call can be recorded into a CUDA graph and replayed.
+ *   tokens_in  [B, L] int32: the start (all mask_id for unconditional generation; unmasked positions are a prompt and
+ *              are never changed).   tokens_out [B, L] int32, a different buffer: the result, free of mask_id.
+ *   u_keep, u_cat [K + 1, B, L] fp32 in [0, 1): the uniforms of every step (the caller's generator), see
+ *              dm_denoise_sample_step.   tau [K + 1, B, d_cond] fp32: the timestep embedding of every step's t_k, only
+ *              with blk != NULL (the timestep MLP is the caller's), else NULL.
+ *   trace      [K + 1, B, L] int32 or NULL: when given, the tokens after every step (trace[K] equals tokens_out).
+ * Workspace: dm_generate_workspace_bytes. */
+typedef struct {
+    int32_t steps;        /* K >= 1 */
+    float   t_eps;        /* in (0, 1) */
+    int32_t mask_id;      /* as dm_sample_cfg */
+    int32_t vocab_real;
+} dm_generate_cfg;
+int dm_generate_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes);
+int dm_generate(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights,
+                const dm_block_weights *block_weights, const dm_generate_cfg *gen, const int32_t *tokens_in,
+                const float *tau, const float *u_keep, const float *u_cat, int32_t *tokens_out, int32_t *trace,
+                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* The attention mixer of the hybrid variant, Sec. 3.3 (one attention mixer every N mixer blocks): full
  * (bidirectional, unmasked) multi-head self-attention over each sequence, no position encoding,
  *     y = concat_h softmax(Q_h K_h^T / sqrt(d_h)) V_h  W_o^T,   [Q | K | V] = x W_qkv^T.
@@ -319,6 +344,16 @@ int dm_bimamba_forward_host(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
 #define DM_STATIC_WORKSPACE_BYTES ((size_t)32 << 20)
 int dm_bimamba_forward_static(const dm_mixer_cfg *cfg, const dm_dir_weights w[2],
                               const void *x, void *y, void *cuda_stream);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper).  Every hand-off inside the pipelined kernels
+ * is a wait with a time limit; when one runs out, the CTA stores DM_ERR_TIMEOUT in the device status word, its other
+ * roles leave through an abort flag, and TMEM is freed before the CTA returns.  This call launches one small CTA that
+ * goes through exactly that sequence on purpose: one warp waits, for limit_us microseconds, on a barrier nothing arrives
+ * at; a second warp, holding TMEM columns, waits on another such barrier and must be released by the first one's abort.
+ * Nothing faults or hangs.  Afterwards dm_check(cuda_stream) returns DM_ERR_TIMEOUT once (and clears it), and
+ * out[0..2] (DEVICE, 3 x uint64) hold: 1 if the first wait gave up, 1 if the second was released by the abort flag,
+ * and the nanoseconds the second one waited. */
+int dm_selftest_wait_timeout(uint32_t limit_us, uint64_t *out, void *cuda_stream);
 
 /* Number of kernels this library has launched from this process since load (for benchmarks). */
 uint64_t dm_kernel_launch_count(void);

@@ -446,6 +446,32 @@ def noise_schedule(K: int, eps: float = 1e-3):
 
 
 # --------------------------------------------------------------------------------------------
+# The K-step generation loop around the reverse step (Sec. 2 Eq. 3, Sec. 4.3: K = L / p denoising steps)
+# --------------------------------------------------------------------------------------------
+def generation_keep_probs(K: int, eps: float = 1e-3):
+    """keep probability s / t of each of the K scheduled steps (t_k -> t_{k+1} of noise_schedule), as the
+    float32 values the decision `u_keep < s/t` is taken with, followed by 0 for the final clean-up pass
+    that unmasks whatever is still masked at noise level eps."""
+    t = noise_schedule(K, eps)
+    return [np.float32(t[k + 1] / t[k]) for k in range(K)] + [np.float32(0.0)]
+
+
+def generate(tokens, sw: dict, u_keep, u_cat, K: int, mask_id: int, vocab_real: int, *, eps: float = 1e-3, tau=None,
+             return_trace: bool = False, **kw):
+    """K reverse steps of Eq. 3 along noise_schedule(K, eps) plus the clean-up pass: step k runs the denoiser on
+    the current tokens (denoise_step, or denoise_step_cond with tau[k] when tau [K+1, B, d_c] is given), then
+    reverse_step with keep probability generation_keep_probs(K)[k] and the uniforms u_keep[k], u_cat[k]
+    ([K+1, B, L] each).  Returns the final tokens (and the tokens after every step when return_trace)."""
+    x = np.asarray(tokens).copy()
+    trace = []
+    for k, keep in enumerate(generation_keep_probs(K, eps)):
+        logits = denoise_step(x, sw, **kw) if tau is None else denoise_step_cond(x, tau[k], sw, **kw)
+        x = reverse_step(x, logits[..., :vocab_real], u_keep[k], u_cat[k], float(keep), mask_id)
+        trace.append(x.copy())
+    return (x, trace) if return_trace else x
+
+
+# --------------------------------------------------------------------------------------------
 # Bidirectional multi-head attention mixer of the hybrid variant (Sec. 3.3, App. C Transformer-layer table)
 # --------------------------------------------------------------------------------------------
 def attention_mixer(x, w_qkv, w_o, n_heads: int):

@@ -67,6 +67,10 @@ class dm_sample_cfg(C.Structure):
     _fields_ = [("mask_id", C.c_int32), ("vocab_real", C.c_int32), ("keep_prob", C.c_float)]
 
 
+class dm_generate_cfg(C.Structure):
+    _fields_ = [("steps", C.c_int32), ("t_eps", C.c_float), ("mask_id", C.c_int32), ("vocab_real", C.c_int32)]
+
+
 class dm_block_weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_cond", "b_cond", "w_up", "b_up", "w_down", "b_down")]
 
@@ -105,6 +109,11 @@ _lib.dm_denoise_sample_step.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_bl
                                         C.POINTER(dm_block_weights), _vp, _vp, C.POINTER(dm_sample_cfg), _vp, _vp, _vp,
                                         C.POINTER(dm_layer_state), _vp, _sz, _vp]
 _lib.dm_denoise_sample_step.restype = C.c_int
+_lib.dm_generate_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(_sz)]
+_lib.dm_generate_workspace_bytes.restype = C.c_int
+_lib.dm_generate.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_stack_weights), C.POINTER(dm_block_weights),
+                             C.POINTER(dm_generate_cfg), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.dm_generate.restype = C.c_int
 _lib.dm_denoise_hybrid_workspace_bytes.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(_sz)]
 _lib.dm_denoise_hybrid_workspace_bytes.restype = C.c_int
 _lib.dm_denoise_step_hybrid.argtypes = [C.POINTER(dm_stack_cfg), C.POINTER(dm_block_cfg), C.POINTER(dm_hybrid_cfg), C.POINTER(dm_stack_weights),
@@ -121,6 +130,8 @@ _lib.dm_attention_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C
 _lib.dm_attention_workspace_bytes.restype = C.c_int
 _lib.dm_attention_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.dm_attention_forward.restype = C.c_int
+_lib.dm_selftest_wait_timeout.argtypes = [C.c_uint32, _vp, _vp]
+_lib.dm_selftest_wait_timeout.restype = C.c_int
 _lib.dm_linear.argtypes = [C.c_int, _vp, _vp, _vp, C.c_int, C.c_int64, C.c_int32, C.c_int32, _vp, _vp, _vp]
 _lib.dm_linear.restype = C.c_int
 _lib.dm_profile_enable.argtypes = [C.c_int]
@@ -134,7 +145,7 @@ EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count"
            "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
            "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step",
            "dm_attention_workspace_bytes", "dm_attention_forward", "dm_denoise_hybrid_workspace_bytes", "dm_denoise_step_hybrid",
-           "dm_denoise_step_hybrid_block", "dm_attention_block_step")
+           "dm_denoise_step_hybrid_block", "dm_attention_block_step", "dm_generate_workspace_bytes", "dm_generate", "dm_selftest_wait_timeout")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -257,6 +268,25 @@ def dm_denoise_sample_step(cfg, blk, weights, block_weights, tokens_in: int, tau
     _ok(_lib.dm_denoise_sample_step(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(weights), block_weights,
                                     _vp(tokens_in), _vp(tau or None), C.byref(sample), _vp(u_keep), _vp(u_cat), _vp(tokens_out),
                                     states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_selftest_wait_timeout(limit_us: int, out: int, cuda_stream: int = 0) -> None:
+    """out: device pointer to 3 uint64."""
+    _ok(_lib.dm_selftest_wait_timeout(int(limit_us), _vp(out), _vp(cuda_stream)))
+
+
+def dm_generate_workspace_bytes(cfg: dm_stack_cfg, blk=None) -> int:
+    n = _sz(0)
+    _ok(_lib.dm_generate_workspace_bytes(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(n)))
+    return n.value
+
+
+def dm_generate(cfg, blk, weights, block_weights, gen: dm_generate_cfg, tokens_in: int, tau: int, u_keep: int, u_cat: int,
+                tokens_out: int, trace: int, workspace: int, workspace_bytes: int, cuda_stream: int = 0) -> None:
+    """u_keep, u_cat: [steps + 1, B, L]; tau: [steps + 1, B, d_cond] or 0; trace: [steps + 1, B, L] or 0."""
+    _ok(_lib.dm_generate(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(weights), block_weights, C.byref(gen),
+                         _vp(tokens_in), _vp(tau or None), _vp(u_keep), _vp(u_cat), _vp(tokens_out), _vp(trace or None),
+                         _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
 
 
 def dm_denoise_hybrid_workspace_bytes(cfg: dm_stack_cfg, blk=None) -> int:

@@ -652,6 +652,51 @@ int dm_denoise_sample_step(const dm_stack_cfg *cfg, const dm_block_cfg *blk, con
     return denoise_impl(cfg, blk, weights, block_weights, tokens_in, tau, nullptr, nullptr, states, workspace, workspace_bytes, cuda_stream, &smp);
 }
 
+int dm_generate_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes) {
+    size_t n = 0;
+    if (!bytes) return fail(DM_ERR_INVALID_ARG, "NULL argument");
+    int st = dm_denoise_sample_workspace_bytes(cfg, blk, &n);
+    if (st != DM_OK) return st;
+    *bytes = n + align_up((size_t)cfg->mixer.batch * cfg->mixer.seqlen * sizeof(int32_t));       // + the second token buffer of the ping-pong
+    return DM_OK;
+}
+
+int dm_generate(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack_weights *weights,
+                const dm_block_weights *block_weights, const dm_generate_cfg *gen, const int32_t *tokens_in,
+                const float *tau, const float *u_keep, const float *u_cat, int32_t *tokens_out, int32_t *trace,
+                void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!cfg || !gen) return fail(DM_ERR_INVALID_ARG, "cfg or gen is NULL");
+    if (gen->steps < 1 || !(gen->t_eps > 0.f && gen->t_eps < 1.f)) return fail(DM_ERR_INVALID_ARG, "steps must be >= 1 and t_eps in (0, 1)");
+    if (!tokens_in || !tokens_out || !u_keep || !u_cat) return fail(DM_ERR_INVALID_ARG, "NULL pointer in the generation arguments");
+    if (tokens_in == tokens_out) return fail(DM_ERR_INVALID_ARG, "tokens_out must not be tokens_in");
+    size_t need = 0, step_ws = 0;
+    int st = dm_generate_workspace_bytes(cfg, blk, &need);
+    if (st != DM_OK) return st;
+    if ((st = dm_denoise_sample_workspace_bytes(cfg, blk, &step_ws)) != DM_OK) return st;
+    if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;
+    const int64_t T = (int64_t)cfg->mixer.batch * cfg->mixer.seqlen;
+    int32_t *spare = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + step_ws);
+    const int K = gen->steps, n_calls = K + 1;
+    const int32_t *cur = tokens_in;
+    for (int k = 0; k < n_calls; ++k) {
+        // noise levels in double, the ratio rounded once to the float the decision u_keep < s/t is taken with
+        const double tk = 1.0 - (1.0 - (double)gen->t_eps) * k / K, tk1 = 1.0 - (1.0 - (double)gen->t_eps) * (k + 1) / K;
+        const dm_sample_cfg sc{gen->mask_id, gen->vocab_real, k < K ? (float)(tk1 / tk) : 0.f};
+        // destinations alternate so that the last step writes tokens_out (or follow the trace, copied out at the end)
+        int32_t *dst = trace ? trace + (int64_t)k * T : (((n_calls - 1 - k) & 1) ? spare : tokens_out);
+        const SampleArgs smp{&sc, u_keep + (int64_t)k * T, u_cat + (int64_t)k * T, dst};
+        st = denoise_impl(cfg, blk, weights, block_weights, cur, (blk && tau) ? tau + (int64_t)k * cfg->mixer.batch * blk->d_cond : tau,
+                          nullptr, nullptr, nullptr, workspace, step_ws, cuda_stream, &smp);
+        if (st != DM_OK) return st;
+        cur = dst;
+    }
+    if (trace) {
+        cudaError_t e = cudaMemcpyAsync(tokens_out, cur, (size_t)T * sizeof(int32_t), cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream));
+        if (e != cudaSuccess) return cuda_fail(e, "dm_generate: copy of the result");
+    }
+    return DM_OK;
+}
+
 int dm_denoise_hybrid_workspace_bytes(const dm_stack_cfg *cfg, const dm_block_cfg *blk, size_t *bytes) {
     Dims m;
     if (!cfg || !bytes) return fail(DM_ERR_INVALID_ARG, "NULL argument");
@@ -750,6 +795,16 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
     o.A = att; o.lda = d_model; o.B = w_o; o.ldb = d_model; o.C = y; o.ldc = d_model;
     o.in_dtype = dtype; o.c_dtype = dtype; o.M = (int)T; o.N = d_model; o.K = d_model;
     if ((e = gemm(o, s)) != cudaSuccess) return cuda_fail(e, "attention output projection");
+    return DM_OK;
+}
+
+int dm_selftest_wait_timeout(uint32_t limit_us, uint64_t *out, void *cuda_stream) {
+    if (!out) return fail(DM_ERR_INVALID_ARG, "out is NULL");
+    if (limit_us == 0 || limit_us > 1000000u) return fail(DM_ERR_INVALID_ARG, "limit_us must be in [1, 1000000]");
+    if (reinterpret_cast<uintptr_t>(out) & 7u) return fail(DM_ERR_INVALID_ARG, "out must be 8-byte aligned");
+    cudaError_t e = selftest_wait_timeout((unsigned long long)limit_us * 1000ull, reinterpret_cast<unsigned long long *>(out),
+                                          static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "dm_selftest_wait_timeout");
     return DM_OK;
 }
 

@@ -113,4 +113,7 @@ cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int 
 cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *conv_out, int dtype, int B, int L,
                               int k, int d_inner, int conv_ch, int d_in_proj, cudaStream_t s);
 
+// One CTA whose waits run out by design (see selftest.cu); out: 3 x uint64 on the device
+cudaError_t selftest_wait_timeout(unsigned long long limit_ns, unsigned long long *out, cudaStream_t s);
+
 }  // namespace dm

@@ -100,7 +100,7 @@ struct SsdArgs {
     ScanDir dir[2];
 };
 
-__device__ __forceinline__ float silu_fast(float v) { return v / (1.f + __expf(-v)); }
+__device__ __forceinline__ float silu_fast(float v) { const float hv = 0.5f * v; return fmaf(hv, tanh_fast(hv), hv); }     // SiLU(v) = v/2 + v/2 tanh(v/2)
 // Arithmetic shared by the two forms of the prep work (the launch of its own below and the prep role inside the scan
 // launch), so that both give the same bits.
 // conv + SiLU of one bf16 channel pair: r[m] = the pre-conv pair m steps back in time, wl[e][m] its weight
@@ -167,22 +167,22 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Sb != NULL (short-block mode): the CTA also writes S[i][j] = C'_i . B'_j over its own 32 rows, fp32, to Sb[seq][pc * 4 + part][32][32].
-__global__ void __launch_bounds__(PREP_THREADS)
-ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, float *__restrict__ Sb,
-                int dir0) {
-    __shared__ float dsm[Q][PREP_HEADS + 1];
-    __shared__ __align__(16) uint32_t bct[2][QB][BCT_LD];     // short-block mode: this CTA's rows of B' ([0]) and C' ([1]) as bf16 pairs
-    const int pc = blockIdx.x / PREP_PARTS, part = blockIdx.x % PREP_PARTS, b = blockIdx.y, dir = dir0 + blockIdx.z;
+// One unit of prep work, by a group of PREP_THREADS threads (tid = index in the group; `bar` = the group's named barrier): part
+// `part` of chunk pc of (direction, batch row): QB rows of B' and C', PREP_HEADS of every 64 heads for the decays.
+// dsm: the group's [Q][PREP_HEADS + 1] floats.  Sb != NULL (short-block mode, with bct = the group's [2][QB][BCT_LD] words): the unit
+// also writes S[i][j] = C'_i . B'_j over its rows, fp32, to Sb[seq][pc * PREP_PARTS + part][QB][QB].
+__device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA,
+                                          float *__restrict__ Sb, int dir, int b, int pc, int part, int tid, int bar, float *dsm,
+                                          uint32_t (*bct)[QB][BCT_LD]) {
     const bool rev = dir == 1;
-    const int L = a.L, k = a.k, tid = threadIdx.x;
+    const int L = a.L, k = a.k;
     const ScanDir &w = a.dir[dir];
     const int64_t seq = (int64_t)dir * a.B + b;
     const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
     const int r0 = pc * Q;
     const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
 
-    // ---- B and C channels: thread = channel pair, over this CTA's block of 32 rows; the 35-row window is loaded up front
+    // ---- B and C channels: thread = channel pair, over this unit's block of 32 rows; the 35-row window is loaded up front
     {
         const int cp = tid, rg = part;
         const bool isC = cp >= N / 2;
@@ -223,7 +223,7 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
     }
     if (Sb) {
         // S = C' B'^T of this block's 32 rows on the legacy tensor path: warp = 16 rows i x 16 columns j, K = d_state
-        __syncthreads();
+        named_sync(bar, PREP_THREADS);
         const int warp = tid >> 5, lane = tid & 31;
         const int mt = warp & 1, nh = warp >> 1;
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -249,19 +249,27 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
     }
     // ---- Delta, then the inclusive cumulative log-decay of every head in the direction's time order
     for (int h0 = 0; h0 < a.H; h0 += 64) {
-        __syncthreads();
+        named_sync(bar, PREP_THREADS);
 #pragma unroll 4
         for (int i = 0; i < Q * PREP_HEADS / PREP_THREADS; ++i) {
             const int idx = tid + PREP_THREADS * i, hh = idx % PREP_HEADS, r = idx / PREP_HEADS, t = r0 + r, h = h0 + part * PREP_HEADS + hh;
-            dsm[r][hh] = (t < L && h < a.H) ? prep_delta(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h], w.dt_bias[h]) : 0.f;
+            dsm[r * (PREP_HEADS + 1) + hh] = (t < L && h < a.H) ? prep_delta(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h], w.dt_bias[h]) : 0.f;
         }
-        __syncthreads();
+        named_sync(bar, PREP_THREADS);
         const int warp = tid >> 5, lane = tid & 31;
         for (int hh = warp; hh < PREP_HEADS && h0 + part * PREP_HEADS + hh < a.H; hh += PREP_THREADS / 32) {
             const int h = h0 + part * PREP_HEADS + hh;
-            prep_lambda_head(&dsm[0][hh], PREP_HEADS + 1, w.A_log[h], rev, lane, dA + ((seq * a.H + h) * 2) * a.Lp + r0, a.Lp);
+            prep_lambda_head(dsm + hh, PREP_HEADS + 1, w.A_log[h], rev, lane, dA + ((seq * a.H + h) * 2) * a.Lp + r0, a.Lp);
         }
     }
+}
+
+__global__ void __launch_bounds__(PREP_THREADS)
+ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, float *__restrict__ Sb,
+                int dir0) {
+    __shared__ float dsm[Q * (PREP_HEADS + 1)];
+    __shared__ __align__(16) uint32_t bct[2][QB][BCT_LD];     // short-block mode: this CTA's rows of B' ([0]) and C' ([1]) as bf16 pairs
+    prep_unit(a, Bp, Cp, dA, Sb, dir0 + blockIdx.z, blockIdx.y, blockIdx.x / PREP_PARTS, blockIdx.x % PREP_PARTS, threadIdx.x, 0, dsm, bct);
 }
 
 // --------------------------------------------------------------------------------------------------
@@ -269,9 +277,12 @@ ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *
 // sequence: 2 H CTAs), the launch is widened by `nprep` CTAs; the CTAs that start first take the prep role (a ticket
 // from an atomic counter decides, so the role never waits for a CTA that has not been scheduled), work through the
 // (batch row, chunk, direction) items in the order the scan consumes them and release one flag per item; the scan CTAs'
-// load warps acquire the flag of a chunk before they fetch its B', C', Lambda.  The whole CTA works on one item: 131 rows
-// of the B and C columns and the dt columns are staged in shared memory with 16-byte loads, then every thread filters
-// one channel pair over a run of rows and every warp scans heads.
+// load warps acquire the flag of a chunk before they fetch its B', C', Lambda through TMA (followed by a proxy fence: the
+// data were written through the generic proxy).  All threads of a prep CTA work on one item: its 131 rows of the B and C
+// columns and its dt columns are fetched with every load in flight at once -- the next item's while the current one is
+// computed -- and staged in shared memory; then every thread filters one channel pair over a run of rows and every warp
+// scans heads.  With two directions nprep is even, so that a CTA's items all belong to one direction and its conv
+// weights are read once.
 // --------------------------------------------------------------------------------------------------
 struct PrepJob {
     __nv_bfloat16 *Bp, *Cp;
@@ -279,53 +290,95 @@ struct PrepJob {
     int *sync;          // [0]: ticket counter, [1 + seq * nch + pc]: item flags; zeroed before the launch.  NULL: no fused prep
     int nprep, ndir;
 };
-constexpr int PREP_SEG = 7, PREP_SEG_ROWS = (Q + PREP_SEG - 1) / PREP_SEG;     // row runs per channel pair
-constexpr uint32_t PREP_RAW_BYTES = (Q + 3) * N * 4, PREP_SMEM = PREP_RAW_BYTES + Q * 65 * 4;
+// 16-byte asynchronous copy global -> shared; src_bytes = 16, or 0 to fill the destination with zeros (src must still be a valid address)
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-__device__ __forceinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, int first, int dir0, uint8_t *smem) {
+constexpr int PREP_SEG = 7, PREP_SEG_ROWS = (Q + PREP_SEG - 1) / PREP_SEG;     // row runs per channel pair
+// shared memory of a prep CTA: two stages of { rows [Q + 3][N] words, dt [Q][64] bf16 }, then Delta [Q][65] floats
+constexpr uint32_t PREP_RAW_BYTES = (Q + 3) * N * 4, PREP_DT_BYTES = Q * 64 * 2, PREP_STAGE = PREP_RAW_BYTES + PREP_DT_BYTES;
+constexpr uint32_t PREP_SMEM = 2 * PREP_STAGE + Q * 65 * 4;
+
+struct PrepItem { int dir, b, pc; };
+__device__ __forceinline__ PrepItem prep_item(const SsdArgs &a, const PrepJob &pj, int it, int dir0) {
+    PrepItem r;
+    r.dir = dir0 + it % pj.ndir;
+    const int c = (it / pj.ndir) % a.nch;
+    r.b = it / (pj.ndir * a.nch);
+    r.pc = r.dir == 1 ? a.nch - 1 - c : c;
+    return r;
+}
+// Asynchronous copies of the item's rows (tile row rr = physical row r0 - 3 + rr for ->, history first; r0 + rr for <-,
+// history last; rows and columns that do not exist are filled with zeros) and of the dt columns of the first 64 heads.
+__device__ __forceinline__ void prep_fetch(const SsdArgs &a, const PrepItem &q, uint8_t *stage, bool dt_vec) {
+    const int tid = threadIdx.x, L = a.L, k = a.k, r0 = q.pc * Q;
+    const bool rev = q.dir == 1;
+    const __nv_bfloat16 *zx = a.zx + ((int64_t)q.dir * a.B + q.b) * L * a.d_in_proj;
+    for (int u = tid; u < (Q + 3) * 32; u += NTHREADS) {
+        const int rr = u >> 5, c16 = u & 31, ch = (c16 & 15) * 8;
+        const int pr = rev ? r0 + rr : r0 - 3 + rr;
+        const __nv_bfloat16 *src = zx;
+        uint32_t nb = 0;
+        if (ch < a.Nr) {                                                       // beyond the model's d_state: zero padding
+            const int cc = a.d_inner + ((c16 >> 4) ? a.Nr : 0) + ch;           // conv channel
+            if (pr >= 0 && pr < L) { src = zx + (int64_t)pr * a.d_in_proj + a.d_inner + cc; nb = 16; }
+            else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0) {         // rows before the sequence: the carried conv state
+                src = a.conv_in + ((int64_t)q.b * (k - 1) + (k - 1 + pr)) * a.conv_ch + cc; nb = 16;
+            }
+        }
+        cp_async16(stage + rr * (N * 4) + c16 * 16, src, nb);
+    }
+    if (dt_vec)
+        for (int u = tid; u < Q * 8; u += NTHREADS) {
+            const int r = u >> 3, h8 = (u & 7) * 8;
+            const bool ok = r0 + r < L && h8 < a.H;
+            cp_async16(stage + PREP_RAW_BYTES + u * 16, ok ? zx + (int64_t)(r0 + r) * a.d_in_proj + a.d_inner + a.conv_ch + h8 : zx, ok ? 16 : 0);
+        }
+}
+
+__device__ __noinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, int first, int dir0, uint8_t *smem) {
     static_assert(PREP_SEG * 128 == NTHREADS && PREP_SMEM <= OFF_MISC, "prep role: thread and shared-memory layout");
-    uint32_t *rawt = reinterpret_cast<uint32_t *>(smem);                       // [Q + 3][N] words: pre-conv rows, B pairs 0..63 | C pairs 64..127
-    float *dsm = reinterpret_cast<float *>(smem + PREP_RAW_BYTES);              // [Q][65] Delta of one tile of 64 heads
+    float *dsm = reinterpret_cast<float *>(smem + 2 * PREP_STAGE);              // [Q][65] Delta of one tile of 64 heads
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L = a.L, k = a.k, n_items = pj.ndir * a.B * a.nch;
-    for (int it = first; it < n_items; it += pj.nprep) {
-        const int dir = dir0 + it % pj.ndir, c = (it / pj.ndir) % a.nch, b = it / (pj.ndir * a.nch);
-        const bool rev = dir == 1;
-        const int pc = rev ? a.nch - 1 - c : c, r0 = pc * Q;
-        const ScanDir &w = a.dir[dir];
-        const int64_t seq = (int64_t)dir * a.B + b;
-        const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
-        const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
-        __syncthreads();                                                       // the previous item's readers are done with the tiles
-        // ---- stage the rows: tile row rr = physical row r0 - 3 + rr (->: history first) or r0 + rr (<-: history last)
-        for (int u = tid; u < (Q + 3) * 32; u += NTHREADS) {
-            const int rr = u >> 5, c16 = u & 31, ch = (c16 & 15) * 8;
-            const int pr = rev ? r0 + rr : r0 - 3 + rr;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (ch < a.Nr) {                                                   // beyond the model's d_state: zero padding
-                const int cc = a.d_inner + ((c16 >> 4) ? a.Nr : 0) + ch;       // conv channel
-                if (pr >= 0 && pr < L) v = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)pr * a.d_in_proj + a.d_inner + cc));
-                else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0)       // rows before the sequence: the carried conv state
-                    v = __ldg(reinterpret_cast<const uint4 *>(a.conv_in + ((int64_t)b * (k - 1) + (k - 1 + pr)) * a.conv_ch + cc));
-            }
-            *reinterpret_cast<uint4 *>(rawt + rr * N + c16 * 4) = v;
+    if (first >= n_items) return;
+    // 16-byte copies of eight heads' dt: the dt columns start on a 16-byte boundary and the head count is a multiple of 8
+    const bool dt_vec = (a.d_inner + a.conv_ch) % 8 == 0 && a.H % 8 == 0;
+    prep_fetch(a, prep_item(a, pj, first, dir0), smem, dt_vec);
+    // conv weights of this thread's channel pair: every item of this CTA has the direction of the first one
+    const int dirc = dir0 + first % pj.ndir;
+    const ScanDir &w = a.dir[dirc];
+    const bool rev = dirc == 1;
+    const int pi = tid & 127, seg = tid >> 7, pp = pi & 63;
+    const bool isC = pi >= 64, valid = 2 * pp < a.Nr;
+    float wl[2][4], bias[2] = {0.f, 0.f};
+    {
+        const int cc = a.d_inner + (isC ? a.Nr : 0) + (valid ? 2 * pp : 0);
+        const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)cc * k;
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+            for (int m = 0; m < 4; ++m) wl[e][m] = (m < k && valid) ? __bfloat162float(cw[e * k + k - 1 - m]) : 0.f;
+        if ((a.flags & DM_FLAG_CONV_BIAS) && w.conv_b && valid) {
+            bias[0] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc]);
+            bias[1] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc + 1]);
         }
-        __syncthreads();
+    }
+    int stg = 0;
+    for (int it = first; it < n_items; it += pj.nprep, stg ^= 1) {
+        const PrepItem q = prep_item(a, pj, it, dir0);
+        const int r0 = q.pc * Q;
+        const int64_t seq = (int64_t)q.dir * a.B + q.b;
+        const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
+        const uint32_t *rawt = reinterpret_cast<const uint32_t *>(smem + stg * PREP_STAGE);
+        const __nv_bfloat16 *dtt = reinterpret_cast<const __nv_bfloat16 *>(smem + stg * PREP_STAGE + PREP_RAW_BYTES);
+        cp_async_wait_all();
+        __syncthreads();                           // this item's tiles have landed; the previous item's readers are done with the other stage and with dsm
+        if (it + pj.nprep < n_items) prep_fetch(a, prep_item(a, pj, it + pj.nprep, dir0), smem + (stg ^ 1) * PREP_STAGE, dt_vec);      // in flight while this item is computed
         // ---- conv + SiLU: thread = (channel pair, run of rows)
         {
-            const int pi = tid & 127, seg = tid >> 7, pp = pi & 63;
-            const bool isC = pi >= 64, valid = 2 * pp < a.Nr;
-            const int cc = a.d_inner + (isC ? a.Nr : 0) + (valid ? 2 * pp : 0);
-            const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)cc * k;
-            float wl[2][4], bias[2] = {0.f, 0.f};
-#pragma unroll
-            for (int e = 0; e < 2; ++e)
-#pragma unroll
-                for (int m = 0; m < 4; ++m) wl[e][m] = (m < k && valid) ? __bfloat162float(cw[e * k + k - 1 - m]) : 0.f;
-            if (has_bias && valid) {
-                bias[0] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc]);
-                bias[1] = __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[cc + 1]);
-            }
             __nv_bfloat16 *dst = (isC ? pj.Cp : pj.Bp) + 2 * pp + seq * L * N;
             const int i0 = seg * PREP_SEG_ROWS, i1 = min(Q, i0 + PREP_SEG_ROWS);
             for (int i = i0; i < i1; ++i) {
@@ -338,10 +391,13 @@ __device__ __forceinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, i
         }
         // ---- Delta and the cumulative log-decay, 64 heads at a time
         for (int h0 = 0; h0 < a.H; h0 += 64) {
-            __syncthreads();
+            if (h0 > 0) __syncthreads();                                       // the previous head tile's scans are done with dsm
             for (int idx = tid; idx < Q * 64; idx += NTHREADS) {
                 const int hh = idx & 63, r = idx >> 6, t = r0 + r, h = h0 + hh;
-                dsm[r * 65 + hh] = (t < L && h < a.H) ? prep_delta(zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h], w.dt_bias[h]) : 0.f;
+                float d = 0.f;
+                if (t < L && h < a.H)
+                    d = prep_delta((h0 == 0 && dt_vec) ? dtt[idx] : zx[(int64_t)t * a.d_in_proj + a.d_inner + a.conv_ch + h], w.dt_bias[h]);
+                dsm[r * 65 + hh] = d;
             }
             __syncthreads();
             for (int hh = warp; hh < 64 && h0 + hh < a.H; hh += NTHREADS / 32) {
@@ -352,7 +408,7 @@ __device__ __forceinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, i
         // ---- publish the item
         __threadfence();
         __syncthreads();
-        if (tid == 0) st_release_gpu(pj.sync + 1 + seq * a.nch + pc, 1);
+        if (tid == 0) atomicExch(pj.sync + 1 + seq * a.nch + q.pc, PREP_PARTS);
     }
 }
 
@@ -367,7 +423,7 @@ template <bool HALFP>
 __global__ void __launch_bounds__(NTHREADS, 1)
 ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_z,
                 const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_c,
-                const __grid_constant__ CUtensorMap map_g, const SsdArgs a, const PrepJob pj, int dir0, int *status) {
+                const __grid_constant__ CUtensorMap map_g, const __grid_constant__ SsdArgs a, const __grid_constant__ PrepJob pj, int dir0, int *status) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -385,7 +441,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
     const int h = item % a.H, b = item / (a.H * pj.ndir), dir = dir0 + (item / a.H) % pj.ndir;
     const bool rev = dir == 1;
-    const int *ready = pj.sync ? pj.sync + 1 + ((int64_t)dir * a.B + b) * a.nch : nullptr;     // per chunk: its B', C', Lambda are in memory
+    const int *ready = pj.sync ? pj.sync + 1 + ((int64_t)dir * a.B + b) * a.nch : nullptr;     // per chunk: units of its B', C', Lambda that are in memory
     const int L = a.L, nch = a.nch;
     const int seq = dir * a.B + b;
     const ScanDir &w = a.dir[dir];
@@ -428,8 +484,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             int issued = 0;
             for (int c = 0; c < nch; ++c) {
                 const int sx = c % NX, sd = c % NDL, pc = rev ? nch - 1 - c : c;
+                // the chunk's Lambda are in memory (fused prep): asked first, so that the flag's round trip to L2 hides behind the wait for a free stage
+                if (ready && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;
                 if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
-                if (ready && !flag_wait(ready + pc, abort_flag, status)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
                 tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
                 mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
@@ -463,8 +520,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             int issued_b = 0, issued_c = 0;
             for (int c = 0; c < nch; ++c) {
                 const int sb = c % NB, pc = rev ? nch - 1 - c : c;
+                if (ready && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;          // the chunk's B', C' are in memory
                 if (!WAIT(&misc->empty_b[sb], ((c / NB) & 1) ^ 1)) break;
-                if (ready && !flag_wait(ready + pc, abort_flag, status)) break;
                 mbar_expect_tx(&misc->full_b[sb], 2 * T16);
                 tma_load_3d(smem + OFF_B + sb * 2 * T16, &map_b, 0, pc * Q, seq, &misc->full_b[sb]);
                 tma_load_3d(smem + OFF_B + sb * 2 * T16 + T16, &map_b, 64, pc * Q, seq, &misc->full_b[sb]);
@@ -868,7 +925,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 // Launch 2 for short blocks: sub-chunks of QB = 32 tokens; the four products of a sub-chunk on the legacy tensor path
 // (mma.sync m16n8k16, bf16 operands from shared memory through ldmatrix, fp32 accumulators in registers).
 // One CTA of 4 * PP threads per (batch row, direction, head of PP channels); per sub-chunk:
-//   load    x rows (+3 rows of conv history), C' and B' rows as they are (bf16), S (fp32, from the prep launch), Lambda, Lambda';
+//   load    x rows (+3 rows of conv history), C' and B' rows as they are (bf16), S (fp32, from the prep launch): asynchronous
+//           16-byte copies, all in flight together; Lambda, Lambda';
 //           the incoming state as a bf16 copy [p][n] (from ssm_in, or from the accumulators of the previous sub-chunk)
 //   conv    x' = SiLU(conv(x)) and w_j x'_j as bf16 [j][p];   W_ij = S_ij 2^(Lambda_i - Lambda'_j) [+ D on the diagonal] for j not after i, else 0
 //   y       Yb = C' h^T (K = d_state), rows scaled by 2^(Lambda_i - Lambda_0), then += W x' (K = 32) into the same accumulators:
@@ -884,9 +942,9 @@ constexpr int WTL = QB + 8;            // row pitch (bf16) of W
 template <int PP> struct BlockSmem {
     static constexpr int XLD = PP + 8;             // row pitch (bf16) of x' and w o x'
     static constexpr size_t ct = 0, bt = ct + QB * NLD * 2, ht = bt + QB * NLD * 2, xt = ht + PP * NLD * 2, wxt = xt + QB * XLD * 2,
-                            wt = wxt + QB * XLD * 2, xr = wt + QB * WTL * 2, ss = xr + (QB + 3) * PP * 4, lam = ss + QB * SLD * 4,
-                            total = lam + (2 * QB + 4) * 4;
-    static_assert(ht % 16 == 0 && xt % 16 == 0 && wxt % 16 == 0 && wt % 16 == 0 && xr % 16 == 0 && ss % 16 == 0 && lam % 16 == 0, "16-byte tiles");
+                            wt = wxt + QB * XLD * 2, xr = wt + QB * WTL * 2, ys = xr + (QB + 4) * PP * 2, ss = ys + QB * PP * 4,
+                            lam = ss + QB * SLD * 4, total = lam + (2 * QB + 4) * 4;
+    static_assert(ht % 16 == 0 && xt % 16 == 0 && wxt % 16 == 0 && wt % 16 == 0 && xr % 16 == 0 && ys % 16 == 0 && ss % 16 == 0 && lam % 16 == 0, "16-byte tiles");
 };
 __device__ __forceinline__ void ldmatrix_x4_t(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, const void *p) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(smem_u32(p)));
@@ -906,7 +964,8 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
     __nv_bfloat16 (*Xt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::xt);      // x' [j][p]
     __nv_bfloat16 (*WXt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::wxt);    // w_j x'_j [j][p]
     __nv_bfloat16 (*Wt)[WTL] = reinterpret_cast<__nv_bfloat16 (*)[WTL]>(bsm + BlockSmem<PP>::wt);      // W [i][j]
-    float (*xr)[PP] = reinterpret_cast<float (*)[PP]>(bsm + BlockSmem<PP>::xr);                        // raw x rows and conv history; later the sub-chunk's y
+    __nv_bfloat16 (*xr)[PP] = reinterpret_cast<__nv_bfloat16 (*)[PP]>(bsm + BlockSmem<PP>::xr);        // raw x rows and conv history
+    float (*ys)[PP] = reinterpret_cast<float (*)[PP]>(bsm + BlockSmem<PP>::ys);                        // the sub-chunk's y
     float (*Ss)[SLD] = reinterpret_cast<float (*)[SLD]>(bsm + BlockSmem<PP>::ss);
     float *lam = reinterpret_cast<float *>(bsm + BlockSmem<PP>::lam), *lamp = lam + QB, *sc = lamp + QB;
 
@@ -971,26 +1030,29 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             const int rb = rev ? r0 + QB : r0 - 1;         // the token before the sub-chunk in time
             sc[0] = (rev ? (r0 + QB) % Q != 0 : r0 % Q != 0) ? dA_head[rb] : 0.f;
         }
+        // tiles that need no conversion go straight to shared memory with 16-byte asynchronous copies, all in flight at once
+        // (a copy of zero source bytes fills its 16 bytes with zeros: rows outside the sequence)
         for (int u = tid; u < (QB + 3) * U8; u += NT) {
             const int rr = u / U8, c = (u % U8) * 8;
             const int pr = rev ? r0 + rr : r0 - 3 + rr;    // physical row; the history sits before the chunk (->) or after it (<-)
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (pr >= 0 && pr < L) v = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)pr * a.d_in_proj + a.d_inner + h * PP + c));
-            else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0)            // rows before the sequence: the carried conv state
-                v = __ldg(reinterpret_cast<const uint4 *>(a.conv_in + ((int64_t)b * (k - 1) + (k - 1 + pr)) * a.conv_ch + h * PP + c));
-            *reinterpret_cast<float4 *>(&xr[rr][c]) = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
-            *reinterpret_cast<float4 *>(&xr[rr][c + 4]) = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
+            const __nv_bfloat16 *src = zx;
+            uint32_t nb = 0;
+            if (pr >= 0 && pr < L) { src = zx + (int64_t)pr * a.d_in_proj + a.d_inner + h * PP + c; nb = 16; }
+            else if (pr < 0 && !rev && a.conv_in && k - 1 + pr >= 0) {            // rows before the sequence: the carried conv state
+                src = a.conv_in + ((int64_t)b * (k - 1) + (k - 1 + pr)) * a.conv_ch + h * PP + c; nb = 16;
+            }
+            cp_async16(&xr[rr][c], src, nb);
         }
         for (int u = tid; u < QB * (N / 8); u += NT) {
             const int i = u / (N / 8), c = (u % (N / 8)) * 8;
-            const int64_t off = (seq * L + r0 + i) * N + c;
-            const bool ok = r0 + i < L;
-            if (have_state) *reinterpret_cast<uint4 *>(&Ct[i][c]) = ok ? __ldg(reinterpret_cast<const uint4 *>(Cp + off)) : make_uint4(0u, 0u, 0u, 0u);
-            if (need_update) *reinterpret_cast<uint4 *>(&Bt[i][c]) = ok ? __ldg(reinterpret_cast<const uint4 *>(Bp + off)) : make_uint4(0u, 0u, 0u, 0u);
+            const int64_t off = (seq * L + min(r0 + i, L - 1)) * N + c;
+            const uint32_t nb = r0 + i < L ? 16 : 0;
+            if (have_state) cp_async16(&Ct[i][c], Cp + off, nb);
+            if (need_update) cp_async16(&Bt[i][c], Bp + off, nb);
         }
         {
             const float *S = Sb + (seq * nsub_all + sub) * (QB * QB);
-            for (int e = tid; e < QB * QB; e += NT) Ss[e / QB][e % QB] = S[e];
+            for (int e = tid; e < QB * QB / 4; e += NT) cp_async16(&Ss[e / (QB / 4)][(e % (QB / 4)) * 4], S + 4 * e, 16);
         }
         if (have_state) {
             if (si == 0) {
@@ -1018,6 +1080,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
         // the gate's z (it holds SiLU(z): the in_proj epilogue applied it), fetched now so that its latency hides behind the products
         uint4 zv = make_uint4(0u, 0u, 0u, 0u);
         if (r0 + ei < L) zv = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)(r0 + ei) * a.d_in_proj + h * PP + ec));
+        cp_async_wait_all();
         __syncthreads();
         // ---- conv + SiLU: thread = channel cch, rows 8 crg .. 8 crg + 7;  mask: W from S
         const float lam_last = lam[rev ? 0 : QB - 1], lam0 = sc[0];      // rows past the end of the sequence have Delta = 0: Lambda stays put there
@@ -1026,7 +1089,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             const int i = crg * (QB * PP / NT) + ii;
             float v = cbias;
 #pragma unroll
-            for (int m = 0; m < 4; ++m) v = fmaf(wl[m], xr[rev ? i + m : i + 3 - m][cch], v);
+            for (int m = 0; m < 4; ++m) v = fmaf(wl[m], __bfloat162float(xr[rev ? i + m : i + 3 - m][cch]), v);
             const float xv = v / (1.f + __expf(-v));
             Xt[i][cch] = __float2bfloat16_rn(xv);
             WXt[i][cch] = __float2bfloat16_rn(r0 + i < L ? ex2f(lam_last - lamp[i]) * xv : 0.f);
@@ -1075,10 +1138,10 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
                 }
             }
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {               // the raw rows were last read before the previous barrier
+            for (int nt = 0; nt < 2; ++nt) {
                 const int col = 16 * ynh + 8 * nt + 2 * qc, row = 16 * ymt + gr;
-                *reinterpret_cast<float2 *>(&xr[row][col]) = make_float2(acc[nt][0], acc[nt][1]);
-                *reinterpret_cast<float2 *>(&xr[row + 8][col]) = make_float2(acc[nt][2], acc[nt][3]);
+                *reinterpret_cast<float2 *>(&ys[row][col]) = make_float2(acc[nt][0], acc[nt][1]);
+                *reinterpret_cast<float2 *>(&ys[row + 8][col]) = make_float2(acc[nt][2], acc[nt][3]);
             }
         }
         // ---- state after the sub-chunk: h <- dec h + (w o x')^T B'
@@ -1104,7 +1167,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             const int row = r0 + ei;
             const float zf[8] = {bf16_lo(zv.x), bf16_hi(zv.x), bf16_lo(zv.y), bf16_hi(zv.y), bf16_lo(zv.z), bf16_hi(zv.z), bf16_lo(zv.w), bf16_hi(zv.w)};
             const float nw[8] = {bf16_lo(nwp[0]), bf16_hi(nwp[0]), bf16_lo(nwp[1]), bf16_hi(nwp[1]), bf16_lo(nwp[2]), bf16_hi(nwp[2]), bf16_lo(nwp[3]), bf16_hi(nwp[3])};
-            const float4 y0 = *reinterpret_cast<const float4 *>(&xr[ei][ec]), y1 = *reinterpret_cast<const float4 *>(&xr[ei][ec + 4]);
+            const float4 y0 = *reinterpret_cast<const float4 *>(&ys[ei][ec]), y1 = *reinterpret_cast<const float4 *>(&ys[ei][ec + 4]);
             const float yv[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
             float g[8], ss = 0.f;
 #pragma unroll
@@ -1202,6 +1265,8 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     if (!blk && nscan < sm_count() && a.N % 8 == 0) {
         pj.sync = reinterpret_cast<int *>(base + l.sy);
         pj.nprep = n_items < sm_count() - nscan ? n_items : sm_count() - nscan;
+        if (ndir == 2) pj.nprep &= ~1;                             // even: every prep CTA then stays with one direction
+        if (pj.nprep == 0) pj.sync = nullptr;
     }
     cudaError_t e;
     if (pj.sync) {

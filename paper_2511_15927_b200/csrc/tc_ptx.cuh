@@ -58,18 +58,21 @@ __device__ __forceinline__ bool mbar_probe64(uint64_t *bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
         if (mbar_probe64(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+        if (globaltimer_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             atomicExch(status, (int)DM_ERR_TIMEOUT);
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    return mbar_wait_limit(bar, parity, abort_flag, status, WAIT_LIMIT_NS);
 }
 // Waits on two or three barriers at once: the first probes are issued back to back so that their latencies overlap
 // (a probe of a completed phase costs about a hundred clocks); whatever is not complete yet is then waited for in turn.
@@ -108,15 +111,16 @@ __device__ __forceinline__ int ld_acquire_gpu(const int *p) {
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release_gpu(int *p, int v) { asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory"); }
-// Bounded wait for a flag in global memory that another CTA of the same launch sets once (same abort protocol as mbar_wait).
+// Bounded wait until a counter in global memory, raised by other CTAs of the same launch with release semantics, has
+// reached TARGET (same abort protocol as mbar_wait).
+template <int TARGET>
 __device__ __forceinline__ bool flag_wait(const int *flag, volatile int *abort_flag, int *status) {
-    if (ld_acquire_gpu(flag) != 0) { fence_proxy_async_all(); return true; }
+    if (ld_acquire_gpu(flag) >= TARGET) { fence_proxy_async_all(); return true; }
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 16; ++i)
-            if (ld_acquire_gpu(flag) != 0) { fence_proxy_async_all(); return true; }
+            if (ld_acquire_gpu(flag) >= TARGET) { fence_proxy_async_all(); return true; }
         if (*abort_flag) return false;
         if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
             *abort_flag = 1;

@@ -172,3 +172,30 @@ def run_denoise_hybrid(shape, dtype, sw, tokens, vocab, attn_period, attn_heads,
                               taud.data_ptr() if taud is not None else 0, logits.data_ptr(), 0, ws.data_ptr(), nb, st)
     dm.dm_check(st)
     return logits.float().cpu().numpy().astype(np.float64)
+
+
+def run_generate(shape, dtype, sw, tokens, vocab, u_keep, u_cat, steps, mask_id, vocab_real, t_eps=1e-3, tau=None, d_ff=0,
+                 want_trace=True, rms_eps=1e-5, ln_eps=1e-5):
+    """dm_generate on host arrays: u_keep, u_cat [steps + 1, B, L]; tau [steps + 1, B, d_c] or None.  Returns (tokens_out, trace)."""
+    n_layers = len(sw["layers"])
+    scfg = dm.dm_stack_cfg(cfg_of(shape, dtype), n_layers, vocab, rms_eps)
+    dsw = dev_stack_weights(sw, dtype)
+    csw, keep = dm.make_stack_weights(dsw)
+    blk = cbw = taud = None
+    if tau is not None:
+        blk = dm.dm_block_cfg(d_ff, tau.shape[-1], ln_eps)
+        dbw = dev_block_weights(sw, dtype)
+        cbw = dm.make_block_weights(dbw)
+        taud = dev(np.asarray(tau, np.float32))
+    tok = dev(np.asarray(tokens, np.int32))
+    out = torch.full_like(tok, -7)
+    trace = torch.full((steps + 1,) + tuple(tok.shape), -7, device="cuda", dtype=torch.int32) if want_trace else None
+    uk, uc = dev(np.asarray(u_keep, np.float32)), dev(np.asarray(u_cat, np.float32))
+    nb = dm.dm_generate_workspace_bytes(scfg, blk)
+    ws = workspace(nb)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_generate(scfg, blk, csw, cbw, dm.dm_generate_cfg(steps, t_eps, mask_id, vocab_real), tok.data_ptr(),
+                   taud.data_ptr() if taud is not None else 0, uk.data_ptr(), uc.data_ptr(), out.data_ptr(),
+                   trace.data_ptr() if want_trace else 0, ws.data_ptr(), nb, st)
+    dm.dm_check(st)
+    return out.cpu().numpy(), (trace.cpu().numpy() if want_trace else None)

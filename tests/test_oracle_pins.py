@@ -691,3 +691,54 @@ def test_hybrid_stack_block_mode_left_to_right_equals_one_pass_on_the_block_rows
         xa, xb = xa + ya, xb + yb
     np.testing.assert_allclose(l1, O.rmsnorm(xa, sw["final_norm_w"]) @ sw["w_vocab"].T, rtol=1e-9, atol=1e-11)
     np.testing.assert_allclose(l2, O.rmsnorm(xb, sw["final_norm_w"]) @ sw["w_vocab"].T, rtol=1e-9, atol=1e-11)
+
+
+# ------------------------------------------------------------------------------------------------
+# The generation loop (Sec. 2 Eq. 3 applied K = L / p times, Sec. 4.3): pins that do not re-run the loop's own code
+# ------------------------------------------------------------------------------------------------
+def test_generation_survivors_follow_the_uniforms_in_closed_form():
+    """Which positions are still masked after step k depends on the uniforms alone: position j survives steps 0..k iff
+    u_keep[i, j] < s_i / t_i for every i <= k (and nothing survives the clean-up pass).  The survivor sets computed from
+    that closed form -- without the denoiser -- must be the mask pattern of every entry of the loop's trace."""
+    K, V, mask_id = 5, 40, 39
+    sw, kw = _tiny_stack(n_layers=1, V=V, seed=31), KW
+    r = np.random.default_rng(3)
+    uk, uc = r.random((K + 1, 2, 12), dtype=np.float32), r.random((K + 1, 2, 12), dtype=np.float32)
+    start = np.full((2, 12), mask_id, np.int32)
+    start[0, 3], start[1, 7] = 5, 11                                   # a two-token prompt
+    out, trace = O.generate(start, sw, uk, uc, K, mask_id, V, return_trace=True, **kw)
+    t = O.noise_schedule(K)
+    alive = start == mask_id
+    for k in range(K):
+        alive = alive & (uk[k] < np.float32(t[k + 1] / t[k]))
+        np.testing.assert_array_equal(trace[k] == mask_id, alive)
+    assert not np.any(trace[K] == mask_id) and np.array_equal(trace[K], out)
+    assert out[0, 3] == 5 and out[1, 7] == 11                          # the prompt is carried through every step
+    for k in range(1, K + 1):                                          # once drawn, a token never changes again
+        fixed = trace[k - 1] != mask_id
+        np.testing.assert_array_equal(trace[k][fixed], trace[k - 1][fixed])
+
+
+def test_generation_keep_probabilities_telescope_to_the_noise_levels():
+    """prod_{i <= k} s_i / t_i = t_{k+1} / t_0: the chance of still being masked after step k is the noise level itself
+    (the marginal of the forward process, Eq. 1); the list ends with the clean-up pass's 0."""
+    for K in (1, 4, 64):
+        kp = O.generation_keep_probs(K, 1e-3)
+        assert len(kp) == K + 1 and kp[-1] == 0.0
+        t = 1.0 - (1.0 - 1e-3) * np.arange(K + 1) / K                  # App. A.1: from 1 to the sampling eps
+        np.testing.assert_allclose(np.cumprod(np.asarray(kp[:-1], np.float64)), t[1:], rtol=1e-6)
+        assert all(0.0 < p < 1.0 for p in kp[:-1])
+
+
+def test_generation_with_one_step_is_two_reverse_steps():
+    """K = 1: one scheduled step (keep probability eps / 1) and the clean-up pass -- written out with reverse_step."""
+    V, mask_id = 40, 39
+    sw, kw = _tiny_stack(n_layers=1, V=V, seed=32), KW
+    r = np.random.default_rng(4)
+    uk, uc = r.random((2, 2, 12), dtype=np.float32), r.random((2, 2, 12), dtype=np.float32)
+    uk[0, 0, :3] = 0.0                                                 # below eps: these three stay masked in the scheduled step
+    start = np.full((2, 12), mask_id, np.int32)
+    x1 = O.reverse_step(start, O.denoise_step(start, sw, **kw), uk[0], uc[0], 1e-3, mask_id)
+    assert np.all(x1[0, :3] == mask_id) and np.all(x1[1] != mask_id)
+    x2 = O.reverse_step(x1, O.denoise_step(x1, sw, **kw), uk[1], uc[1], 0.0, mask_id)
+    np.testing.assert_array_equal(O.generate(start, sw, uk, uc, 1, mask_id, V, **kw), x2)
