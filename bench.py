@@ -679,7 +679,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None, help="timed steps (default 10; 64 blocks for cfg4_loop; 3 generations for the *_generate workloads)")
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS) + sorted(STACKS) + ["lsweep_fit"])
+    ap.add_argument("--workload", default="cfg1", choices=sorted(I.CONFIGS) + sorted(STACKS) + ["lsweep_fit", "cfg1_tied", "cfg3_8k_tied"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128, help="tokens per step of the reference arm's sample")
     ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
@@ -710,7 +710,9 @@ def main():
             return
         run_stack(args, rank, local_rank, world)
         return
-    shape, dtype = I.CONFIGS[args.workload]
+    # *_tied: the same shape with the directions sharing in_proj and out_proj (App. A.1 "bidirectional weight tie")
+    tied = args.workload.endswith("_tied")
+    shape, dtype = I.CONFIGS[args.workload[:-5] if tied else args.workload]
 
     if args.impl == "reference":
         run_reference(args, shape, dtype, rank)
@@ -728,7 +730,7 @@ def main():
 
     es = 2 if dtype == I.BF16 else 4
     T = shape.batch * shape.seqlen
-    cfg = G.cfg_of(shape, dtype)
+    cfg = G.cfg_of(shape, dtype, flags=dm.DM_FLAGS_DEFAULT | (dm.DM_FLAG_TIED_PROJ if tied else 0))
     wf, wr = I.make_mixer_weights(shape, 0, dtype)
     dwf, dwr = G.dev_dir_weights(wf, dtype), G.dev_dir_weights(wr, dtype)
     cw = (dm.make_dir_weights(dwf), dm.make_dir_weights(dwr))
@@ -799,6 +801,8 @@ def main():
     outp_ms = stage_ms[dm.DM_STAGE_OUT_PROJ] / args.steps
     scan_bytes = scan_bytes_per_token(shape, es) * T
     f_in, f_out = gemm_flops_per_token(shape)
+    if tied:                                               # one shared in_proj and one out_proj over the summed directions
+        f_in, f_out = f_in // 2, f_out // 2
     scan_gbs = scan_bytes / (scan_ms * 1e-3) / 1e9
     in_tf = f_in * T / (inp_ms * 1e-3) / 1e12
     out_tf = f_out * T / (outp_ms * 1e-3) / 1e12

@@ -40,7 +40,12 @@ typedef enum {
 } dm_status;
 
 enum { DM_F32 = 0, DM_BF16 = 1 };
-enum { DM_FLAG_GATED_RMSNORM = 1, DM_FLAG_CONV_BIAS = 2, DM_FLAG_D_SKIP = 4 };
+enum { DM_FLAG_GATED_RMSNORM = 1, DM_FLAG_CONV_BIAS = 2, DM_FLAG_D_SKIP = 4,
+       /* App. A.1 hyper-parameter "bidirectional weight tie" (False in the paper's runs): the two directions share in_proj and
+          out_proj (w[0].w_in, w[0].w_out; the ones of w[1] are not read) and keep their own conv, step-size, decay, skip and norm
+          parameters.  The shared in_proj is then computed once and the sum of the directions is taken before the one out_proj:
+          Mamba(x) = W_out (g-> + g<-), with each direction's gated-norm scale applied to its g first. */
+       DM_FLAG_TIED_PROJ = 8 };
 enum { DM_DIR_FWD = 1, DM_DIR_REV = 2, DM_DIR_BOTH = 3 };
 
 /* Sizes of one mixer call, in the paper's notation (Sec. 3.2: x in R^{B x L x d}; App. A.1

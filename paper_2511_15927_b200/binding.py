@@ -16,7 +16,7 @@ LIB_PATH = os.environ.get("DM_BIMAMBA_LIB") or os.path.join(_HERE, "libdm_bimamb
 
 DM_OK, DM_ERR_INVALID_ARG, DM_ERR_UNSUPPORTED, DM_ERR_WORKSPACE, DM_ERR_CUDA, DM_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 DM_F32, DM_BF16 = 0, 1
-DM_FLAG_GATED_RMSNORM, DM_FLAG_CONV_BIAS, DM_FLAG_D_SKIP = 1, 2, 4
+DM_FLAG_GATED_RMSNORM, DM_FLAG_CONV_BIAS, DM_FLAG_D_SKIP, DM_FLAG_TIED_PROJ = 1, 2, 4, 8
 DM_DIR_FWD, DM_DIR_REV, DM_DIR_BOTH = 1, 2, 3
 DM_FLAGS_DEFAULT = DM_FLAG_GATED_RMSNORM | DM_FLAG_CONV_BIAS | DM_FLAG_D_SKIP
 

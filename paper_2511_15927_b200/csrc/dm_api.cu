@@ -79,7 +79,7 @@ static int check_cfg(const dm_mixer_cfg *c, Dims *o) {
         return fail(DM_ERR_INVALID_ARG, "batch, seqlen, d_model, expand, d_state and n_heads must be positive");
     if (c->dtype != DM_F32 && c->dtype != DM_BF16) return fail(DM_ERR_INVALID_ARG, "dtype must be DM_F32 or DM_BF16");
     if (c->dir_mask < DM_DIR_FWD || c->dir_mask > DM_DIR_BOTH) return fail(DM_ERR_INVALID_ARG, "dir_mask must be 1, 2 or 3");
-    if (c->flags & ~(DM_FLAG_GATED_RMSNORM | DM_FLAG_CONV_BIAS | DM_FLAG_D_SKIP)) return fail(DM_ERR_INVALID_ARG, "unknown flag bits");
+    if (c->flags & ~(DM_FLAG_GATED_RMSNORM | DM_FLAG_CONV_BIAS | DM_FLAG_D_SKIP | DM_FLAG_TIED_PROJ)) return fail(DM_ERR_INVALID_ARG, "unknown flag bits");
     if (c->chunk < 0) return fail(DM_ERR_INVALID_ARG, "chunk must be >= 0");
     if (!(c->norm_eps >= 0.f)) return fail(DM_ERR_INVALID_ARG, "norm_eps must be >= 0");
     if (c->n_groups != 1) return fail(DM_ERR_UNSUPPORTED, "n_groups must be 1");
@@ -109,11 +109,12 @@ static int check_weights(const dm_mixer_cfg *c, const dm_dir_weights w[2]) {
     for (int dir = 0; dir < 2; ++dir) {
         if (!(c->dir_mask & (1 << dir))) continue;
         const dm_dir_weights &q = w[dir];
-        if (!q.w_in || !q.conv_w || !q.dt_bias || !q.A_log || !q.w_out) return fail(DM_ERR_INVALID_ARG, "direction %d: NULL weight pointer", dir);
+        const dm_dir_weights &pw = w[(c->flags & DM_FLAG_TIED_PROJ) ? 0 : dir];       // whose projections this direction uses
+        if (!pw.w_in || !q.conv_w || !q.dt_bias || !q.A_log || !pw.w_out) return fail(DM_ERR_INVALID_ARG, "direction %d: NULL weight pointer", dir);
         if ((c->flags & DM_FLAG_CONV_BIAS) && !q.conv_b) return fail(DM_ERR_INVALID_ARG, "direction %d: conv_b is NULL but DM_FLAG_CONV_BIAS is set", dir);
         if ((c->flags & DM_FLAG_D_SKIP) && !q.D) return fail(DM_ERR_INVALID_ARG, "direction %d: D is NULL but DM_FLAG_D_SKIP is set", dir);
         if ((c->flags & DM_FLAG_GATED_RMSNORM) && !q.norm_w) return fail(DM_ERR_INVALID_ARG, "direction %d: norm_w is NULL but DM_FLAG_GATED_RMSNORM is set", dir);
-        if (!aligned16(q.w_in) || !aligned16(q.w_out)) return fail(DM_ERR_INVALID_ARG, "direction %d: matrices must be 16-byte aligned", dir);
+        if (!aligned16(pw.w_in) || !aligned16(pw.w_out)) return fail(DM_ERR_INVALID_ARG, "direction %d: matrices must be 16-byte aligned", dir);
     }
     return DM_OK;
 }
@@ -173,6 +174,8 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         sa.dir[dir].dt_bias = w[dir].dt_bias; sa.dir[dir].A_log = w[dir].A_log; sa.dir[dir].D = w[dir].D;
     }
     sa.ssm_in = ssm_in; sa.conv_in = conv_in; sa.ssm_out = ssm_out;
+    const bool tied = (c->flags & DM_FLAG_TIED_PROJ) != 0;
+    sa.zx_tied = tied ? 1 : 0;
     // The tensor-core scan is bound by instruction issue while the GEMM's epilogue warps mostly wait: on that path the
     // gate's SiLU(z) (Sec. 3.2) is applied to the z columns by the in_proj epilogue.
     sa.z_gated = 1;
@@ -181,10 +184,11 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
 
     for (int dir = 0; dir < 2; ++dir) {
         if (!(c->dir_mask & (1 << dir))) continue;
+        if (tied && dir == 1 && (c->dir_mask & DM_DIR_FWD)) continue;         // tied projections: one in_proj serves both directions
         StageTimer tm(DM_STAGE_IN_PROJ, s);
         GemmArgs a{};
-        a.A = x; a.lda = m.d; a.B = w[dir].w_in; a.ldb = m.d;
-        a.C = zx + (size_t)dir * m.T * m.ldz * m.es; a.ldc = m.ldz;
+        a.A = x; a.lda = m.d; a.B = w[tied ? 0 : dir].w_in; a.ldb = m.d;
+        a.C = zx + (size_t)(tied ? 0 : dir) * m.T * m.ldz * m.es; a.ldc = m.ldz;
         a.in_dtype = c->dtype; a.c_dtype = c->dtype; a.M = (int)m.T; a.N = m.d_in_proj; a.K = m.d;
         a.silu_cols = ssd ? m.d_inner : 0;
         if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "in_proj");
@@ -204,6 +208,21 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         e = rstd_from_ssq(ssq, rstd, (int)(2 * m.T), m.H, m.d_inner, c->norm_eps, s);
         if (e != cudaSuccess) return cuda_fail(e, "rstd");
     }
+    if (tied && c->dir_mask == DM_DIR_BOTH) {
+        // shared out_proj: W_out (s-> g-> + s<- g<-) with s the gated-norm scale of each direction (1 without the norm); one GEMM
+        e = combine_directions(g, g + (size_t)m.T * m.d_inner * m.es, norm_on ? rstd : nullptr, norm_on ? rstd + m.T : nullptr, c->dtype, m.T,
+                               m.d_inner, s);
+        if (e != cudaSuccess) return cuda_fail(e, "combine_directions");
+        StageTimer tm(DM_STAGE_OUT_PROJ, s);
+        GemmArgs a{};
+        a.A = g; a.lda = m.d_inner; a.B = w[0].w_out; a.ldb = m.d_inner;
+        a.in_dtype = c->dtype; a.M = (int)m.T; a.N = m.d; a.K = m.d_inner;
+        a.addend = out.addend; a.ld_add = out.ld_add;
+        a.col_scale = out.col_scale; a.cs_rows = out.cs_rows; a.ld_cs = out.ld_cs;
+        a.C = out.y; a.ldc = m.d; a.c_dtype = out.y_dtype;
+        if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "out_proj");
+        return DM_OK;
+    }
     // out_proj of each direction; the second one adds the first (Mamba(x) = h-> + h<-)
     const float *carry = out.addend;
     int64_t ld_carry = out.ld_add;
@@ -214,7 +233,7 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         StageTimer tm(DM_STAGE_OUT_PROJ, s);
         GemmArgs a{};
         a.A = g + (size_t)dir * m.T * m.d_inner * m.es; a.lda = m.d_inner;
-        a.B = w[dir].w_out; a.ldb = m.d_inner;
+        a.B = w[tied ? 0 : dir].w_out; a.ldb = m.d_inner;
         a.in_dtype = c->dtype; a.M = (int)m.T; a.N = m.d; a.K = m.d_inner;
         a.row_scale = norm_on ? rstd + (size_t)dir * m.T : nullptr;
         a.addend = carry; a.ld_add = ld_carry;

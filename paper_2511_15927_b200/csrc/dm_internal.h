@@ -60,6 +60,7 @@ struct ScanArgs {
     int conv_ch;
     int dtype, flags, dir_mask, chunk;
     const void *zx;          // [2][B*L][d_in_proj] dtype: in_proj output of each direction
+    int zx_tied;             // both directions read zx[0] (shared in_proj, DM_FLAG_TIED_PROJ)
     int z_gated;             // the z columns of zx already hold SiLU(z) (applied by the in_proj epilogue); the tensor-core scan requires it
     void *g;                 // [2][B*L][d_inner]   dtype: gated output (times norm_w when the norm is on)
     float *ssq;              // [2][B*L][H] per-head sum of squares of the gated output (norm on), or NULL
@@ -109,6 +110,8 @@ cudaError_t draw_rows(const void *logits, int64_t ld, int dtype, const int32_t *
                       const float *u_cat, int mask_id, int vocab_real, int32_t *tokens_out, cudaStream_t s);
 // out[t] = argmax_v logits[t, v], lowest index on ties
 cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s);
+// Tied projections: g0[t, :] = s0[t] * g0[t, :] + s1[t] * g1[t, :]  (s = rstd of each direction, or 1 when rstd is NULL), in place over g0
+cudaError_t combine_directions(void *g0, const void *g1, const float *rstd0, const float *rstd1, int dtype, int64_t T, int d_inner, cudaStream_t s);
 // conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])
 cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *conv_out, int dtype, int B, int L,
                               int k, int d_inner, int conv_ch, int d_in_proj, cudaStream_t s);

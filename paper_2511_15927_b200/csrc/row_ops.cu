@@ -207,6 +207,40 @@ __global__ void conv_state_kernel(const T *__restrict__ zx, const T *__restrict_
     conv_out[((int64_t)b * (k - 1) + r) * conv_ch + c] = v;
 }
 
+// g0 <- s0 g0 + s1 g1, one block of threads per row (tied projections: the sum of the directions before the shared out_proj);
+// 16-byte accesses when the rows allow it (VEC = elements per 16 bytes, or 1)
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) combine_kernel(T *__restrict__ g0, const T *__restrict__ g1, const float *__restrict__ r0,
+                                                       const float *__restrict__ r1, int64_t rows, int d_inner) {
+    for (int64_t t = blockIdx.x; t < rows; t += gridDim.x) {
+        const float s0 = r0 ? r0[t] : 1.f, s1 = r1 ? r1[t] : 1.f;
+        T *a = g0 + t * d_inner;
+        const T *b = g1 + t * d_inner;
+        for (int c = threadIdx.x * VEC; c < d_inner; c += blockDim.x * VEC) {
+            if constexpr (VEC == 1) {
+                stf(a + c, fmaf(s0, ldf(a + c), s1 * ldf(b + c)));
+            } else {
+                uint4 va = *reinterpret_cast<const uint4 *>(a + c);
+                const uint4 vb = __ldg(reinterpret_cast<const uint4 *>(b + c));
+                uint32_t *wa = reinterpret_cast<uint32_t *>(&va);
+                const uint32_t *wb = reinterpret_cast<const uint32_t *>(&vb);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if constexpr (sizeof(T) == 2) {
+                        const float lo = fmaf(s0, __uint_as_float(wa[e] << 16), s1 * __uint_as_float(wb[e] << 16));
+                        const float hi = fmaf(s0, __uint_as_float(wa[e] & 0xFFFF0000u), s1 * __uint_as_float(wb[e] & 0xFFFF0000u));
+                        const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+                        wa[e] = *reinterpret_cast<const uint32_t *>(&pk);
+                    } else {
+                        wa[e] = __float_as_uint(fmaf(s0, __uint_as_float(wa[e]), s1 * __uint_as_float(wb[e])));
+                    }
+                }
+                *reinterpret_cast<uint4 *>(a + c) = va;
+            }
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t rstd_from_ssq(const float *ssq, float *rstd, int rows, int H, int d_inner, float eps, cudaStream_t s) {
@@ -262,6 +296,25 @@ cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *con
     else
         conv_state_kernel<<<grid, 256, 0, s>>>(static_cast<const float *>(zx_fwd), static_cast<const float *>(conv_in),
                                                static_cast<float *>(conv_out), L, k, d_inner, conv_ch, d_in_proj);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t combine_directions(void *g0, const void *g1, const float *rstd0, const float *rstd1, int dtype, int64_t T, int d_inner, cudaStream_t s) {
+    const int blocks = (int)(T < 148 * 8 ? T : 148 * 8);
+    const size_t es = dtype_size(dtype);
+    const bool vec = ((size_t)d_inner * es) % 16 == 0 && ((reinterpret_cast<uintptr_t>(g0) | reinterpret_cast<uintptr_t>(g1)) & 15u) == 0;
+    if (dtype == DM_BF16) {
+        auto *a = static_cast<__nv_bfloat16 *>(g0);
+        auto *b = static_cast<const __nv_bfloat16 *>(g1);
+        if (vec) combine_kernel<__nv_bfloat16, 8><<<blocks, 256, 0, s>>>(a, b, rstd0, rstd1, T, d_inner);
+        else combine_kernel<__nv_bfloat16, 1><<<blocks, 256, 0, s>>>(a, b, rstd0, rstd1, T, d_inner);
+    } else {
+        auto *a = static_cast<float *>(g0);
+        auto *b = static_cast<const float *>(g1);
+        if (vec) combine_kernel<float, 4><<<blocks, 256, 0, s>>>(a, b, rstd0, rstd1, T, d_inner);
+        else combine_kernel<float, 1><<<blocks, 256, 0, s>>>(a, b, rstd0, rstd1, T, d_inner);
+    }
     count_launch();
     return cudaGetLastError();
 }

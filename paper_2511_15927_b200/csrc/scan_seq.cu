@@ -65,7 +65,7 @@ bc_prep_kernel(const ScanArgs a, const int dir0, float *__restrict__ bc, const i
     const bool rev = dir == 1;
     const ScanDir &w = a.dir[dir];
     const int64_t T_all = (int64_t)a.B * L;
-    const T *zx = static_cast<const T *>(a.zx) + ((int64_t)dir * T_all + (int64_t)b * L) * a.d_in_proj;
+    const T *zx = static_cast<const T *>(a.zx) + ((int64_t)(a.zx_tied ? 0 : dir) * T_all + (int64_t)b * L) * a.d_in_proj;
     const T *conv_in = (!rev && a.conv_in) ? static_cast<const T *>(a.conv_in) + (int64_t)b * (k - 1) * a.conv_ch : nullptr;
     float *out = bc + ((int64_t)dir * T_all + (int64_t)b * L) * N2;
     const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b != nullptr;
@@ -126,7 +126,7 @@ scan_seq_kernel(const ScanArgs a, const int dir0, const int TC, const int LPC, c
     const bool norm_on = (a.flags & DM_FLAG_GATED_RMSNORM) != 0;
 
     const int64_t T_all = (int64_t)a.B * L;
-    const T *zx = static_cast<const T *>(a.zx) + ((int64_t)dir * T_all + (int64_t)b * L) * a.d_in_proj;
+    const T *zx = static_cast<const T *>(a.zx) + ((int64_t)(a.zx_tied ? 0 : dir) * T_all + (int64_t)b * L) * a.d_in_proj;
     T *gout = static_cast<T *>(a.g) + ((int64_t)dir * T_all + (int64_t)b * L) * a.d_inner;
     float *ssq = a.ssq ? a.ssq + ((int64_t)dir * T_all + (int64_t)b * L) * a.H : nullptr;
     const T *conv_in = (!rev && a.conv_in) ? static_cast<const T *>(a.conv_in) + (int64_t)b * (k - 1) * a.conv_ch : nullptr;

@@ -91,6 +91,7 @@ struct SsdArgs {
     int B, L, H, d_inner, d_in_proj, conv_ch, k, flags, nch, Lp;
     int Nr;                      // d_state of the model (<= N); B', C' and the state are zero-padded to N
     int Pr;                      // headdim of the model: P, or P / 2 (the CTA then carries the next head's channels as unused padding)
+    int zx_tied;                 // both directions read the in_proj output of direction 0 (shared projections)
     __nv_bfloat16 *g;            // [2][B*L][d_inner] gated output (written with plain stores when Pr < P, else through map_g)
     const __nv_bfloat16 *zx;
     float *ssq;
@@ -178,7 +179,7 @@ __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__res
     const int L = a.L, k = a.k;
     const ScanDir &w = a.dir[dir];
     const int64_t seq = (int64_t)dir * a.B + b;
-    const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
+    const __nv_bfloat16 *zx = a.zx + ((int64_t)(a.zx_tied ? 0 : dir) * a.B + b) * L * a.d_in_proj;
     const int r0 = pc * Q;
     const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
 
@@ -315,7 +316,7 @@ __device__ __forceinline__ PrepItem prep_item(const SsdArgs &a, const PrepJob &p
 __device__ __forceinline__ void prep_fetch(const SsdArgs &a, const PrepItem &q, uint8_t *stage, bool dt_vec) {
     const int tid = threadIdx.x, L = a.L, k = a.k, r0 = q.pc * Q;
     const bool rev = q.dir == 1;
-    const __nv_bfloat16 *zx = a.zx + ((int64_t)q.dir * a.B + q.b) * L * a.d_in_proj;
+    const __nv_bfloat16 *zx = a.zx + ((int64_t)(a.zx_tied ? 0 : q.dir) * a.B + q.b) * L * a.d_in_proj;
     for (int u = tid; u < (Q + 3) * 32; u += NTHREADS) {
         const int rr = u >> 5, c16 = u & 31, ch = (c16 & 15) * 8;
         const int pr = rev ? r0 + rr : r0 - 3 + rr;
@@ -371,7 +372,7 @@ __device__ __noinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, int 
         const PrepItem q = prep_item(a, pj, it, dir0);
         const int r0 = q.pc * Q;
         const int64_t seq = (int64_t)q.dir * a.B + q.b;
-        const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
+        const __nv_bfloat16 *zx = a.zx + ((int64_t)(a.zx_tied ? 0 : q.dir) * a.B + q.b) * L * a.d_in_proj;
         const uint32_t *rawt = reinterpret_cast<const uint32_t *>(smem + stg * PREP_STAGE);
         const __nv_bfloat16 *dtt = reinterpret_cast<const __nv_bfloat16 *>(smem + stg * PREP_STAGE + PREP_RAW_BYTES);
         cp_async_wait_all();
@@ -444,6 +445,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const int *ready = pj.sync ? pj.sync + 1 + ((int64_t)dir * a.B + b) * a.nch : nullptr;     // per chunk: units of its B', C', Lambda that are in memory
     const int L = a.L, nch = a.nch;
     const int seq = dir * a.B + b;
+    const int zseq = a.zx_tied ? b : seq;          // the sequence's rows in the in_proj output (shared by the directions when the projections are tied)
     const ScanDir &w = a.dir[dir];
     const bool norm_on = (a.flags & DM_FLAG_GATED_RMSNORM) != 0;
 
@@ -488,7 +490,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (ready && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;
                 if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
-                tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, seq, &misc->full_x[sx]);
+                tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, zseq, &misc->full_x[sx]);
                 mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
                 bulk_load(smem + OFF_DL + sd * 2 * Q * 4, dA_head + pc * Q, Q * 4, &misc->full_dl[sd]);
                 bulk_load(smem + OFF_DL + sd * 2 * Q * 4 + Q * 4, dA_head + a.Lp + pc * Q, Q * 4, &misc->full_dl[sd]);
@@ -508,7 +510,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const int sz = c % NZ, pc = rev ? nch - 1 - c : c;
                 if (!WAIT(&misc->empty_z[sz], ((c / NZ) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_z[sz], T16);
-                tma_load_3d(smem + OFF_Z + sz * T16, &map_z, h * Pr, pc * Q, seq, &misc->full_z[sz]);
+                tma_load_3d(smem + OFF_Z + sz * T16, &map_z, h * Pr, pc * Q, zseq, &misc->full_z[sz]);
                 issued = c + 1;
             }
             if (*abort_flag)
@@ -975,7 +977,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
     const int L = a.L, k = a.k;
     const int64_t seq = (int64_t)dir * a.B + b;
     const ScanDir &w = a.dir[dir];
-    const __nv_bfloat16 *zx = a.zx + seq * L * a.d_in_proj;
+    const __nv_bfloat16 *zx = a.zx + ((int64_t)(a.zx_tied ? 0 : dir) * a.B + b) * L * a.d_in_proj;
     const float *dA_head = a.dA + ((seq * a.H + h) * 2) * a.Lp;
     const int nsub = (L + QB - 1) / QB, nsub_all = a.nch * PREP_PARTS;
     const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
@@ -1251,7 +1253,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     float *dA = reinterpret_cast<float *>(base + l.da);
     SsdArgs k{};
     k.B = a.B; k.L = a.L; k.H = a.H; k.d_inner = a.d_inner; k.d_in_proj = a.d_in_proj; k.conv_ch = a.conv_ch; k.k = a.k;
-    k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp; k.Nr = a.N; k.Pr = a.P; k.g = static_cast<__nv_bfloat16 *>(a.g);
+    k.flags = a.flags; k.nch = l.nch; k.Lp = l.Lp; k.Nr = a.N; k.Pr = a.P; k.zx_tied = a.zx_tied; k.g = static_cast<__nv_bfloat16 *>(a.g);
     k.zx = static_cast<const __nv_bfloat16 *>(a.zx); k.ssq = a.ssq; k.dA = dA;
     k.ssm_in = a.ssm_in; k.ssm_out = a.ssm_out; k.conv_in = static_cast<const __nv_bfloat16 *>(a.conv_in);
     k.dir[0] = a.dir[0]; k.dir[1] = a.dir[1];

@@ -27,7 +27,7 @@ def dev(a, dtype=None):
 
 
 def dev_dir_weights(w: dict, dtype) -> dict:
-    return {k: dev(v, dtype if k in TYPED else None) for k, v in w.items()}
+    return {k: (dev(v, dtype if k in TYPED else None) if v is not None else None) for k, v in w.items()}
 
 
 def cfg_of(shape: I.MixerShape, dtype, flags=dm.DM_FLAGS_DEFAULT, dir_mask=dm.DM_DIR_BOTH, chunk=0, eps=1e-5):

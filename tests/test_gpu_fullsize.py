@@ -1,6 +1,7 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times (dm_bimamba_forward, bf16,
 d_model 2048, 64 heads x 64, d_state 128): batch rows of the B=8 / L=2048 workload and the whole L=8192 sequence
-against the CPU oracle, and at L=32768 -- where the oracle would take minutes -- a property that holds at any
+against the CPU oracle, the left-to-right layer over the whole L=16384 sequence, and at L=32768 -- where the oracle would take
+minutes -- a property that holds at any
 length: the left-to-right layer's outputs on a prefix do not depend on what follows it, and the right-to-left
 layer's outputs on a suffix do not depend on what precedes it."""
 import numpy as np
@@ -44,6 +45,22 @@ def test_cfg3_8k_whole_sequence_against_the_oracle(G):
     x = I.make_activations(shape, 0, dtype)
     got = G.run_forward(shape, dtype, wf, wr, x)
     _check_rows(G, got, x, wf, wr, shape, rows=(0,))
+
+
+def test_cfg3_16k_left_to_right_layer_against_the_oracle(G):
+    """The middle length of the scan-scaling sweep, element by element against the oracle: the whole 16 384-token sequence through
+    the left-to-right layer alone (one direction keeps the oracle's token loop under half a minute; the right-to-left layer
+    runs the same kernel with mirrored indices and is compared at 8192 above)."""
+    shape, dtype = I.CONFIGS["cfg3_16k"]
+    wf, wr = I.make_mixer_weights(shape, 0, dtype)
+    x = I.make_activations(shape, 0, dtype)
+    got = G.run_forward(shape, dtype, wf, wr, x, dir_mask=1)
+    want = O.bimamba_forward(x, wf, wr, dir_mask=O.DIR_FWD, **G.oracle_kwargs(shape))
+    assert np.all(np.isfinite(got))
+    assert G.rel_l2(got, want) <= BF16_REL, G.rel_l2(got, want)
+    assert G.max_abs(got, want) <= BF16_ABS, G.max_abs(got, want)
+    # the last 2048 tokens on their own: errors do not grow along the sequence
+    assert G.rel_l2(got[:, -2048:], want[:, -2048:]) <= BF16_REL
 
 
 def test_cfg3_32k_prefix_and_suffix_independence(G):
