@@ -46,6 +46,10 @@ cudaError_t gemm_simple(const GemmArgs &a, cudaStream_t s);
 // Tensor-core path (tcgen05 + TMEM + TMA).  Returns cudaErrorNotSupported for shapes it does not take.
 cudaError_t gemm_tcgen05(const GemmArgs &a, cudaStream_t s);
 bool gemm_tcgen05_supports(const GemmArgs &a);
+// Two problems of equal M, N, K and output type in one launch (same tile loop, one tail round).  The problems must be independent
+// of each other: neither reads what the other writes.
+bool gemm_tcgen05_pair_supports(const GemmArgs &a, const GemmArgs &b);
+cudaError_t gemm_tcgen05_pair(const GemmArgs &a, const GemmArgs &b, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // Fused conv + SiLU + discretisation + selective scan + gate, both directions in one launch.
@@ -110,6 +114,8 @@ cudaError_t draw_rows(const void *logits, int64_t ld, int dtype, const int32_t *
                       const float *u_cat, int mask_id, int vocab_real, int32_t *tokens_out, cudaStream_t s);
 // out[t] = argmax_v logits[t, v], lowest index on ties
 cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s);
+// y[i] = (dtype) (a[i] + b[i])
+cudaError_t add_partials(const float *a, const float *b, void *y, int dtype, size_t n, cudaStream_t s);
 // Tied projections: g0[t, :] = s0[t] * g0[t, :] + s1[t] * g1[t, :]  (s = rstd of each direction, or 1 when rstd is NULL), in place over g0
 cudaError_t combine_directions(void *g0, const void *g1, const float *rstd0, const float *rstd1, int dtype, int64_t T, int d_inner, cudaStream_t s);
 // conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])

@@ -36,9 +36,16 @@ struct EpiArgs {
     int n_fast;      // tile order: consecutive tiles step along N (the A rows are streamed once, B stays in L2) or along M
 };
 
+// Up to two problems of the same M, N, K in one launch (the two directions' in_proj, or their out_proj on short inputs): the tile
+// loop runs over both, so that they share one tail round and -- for in_proj, whose A operand is the same x -- the rows of A in L2.
+struct EpiPair { EpiArgs p[2]; int nprob; };
+
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const EpiArgs ep, int *status) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_b0,
+               const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
+               const __grid_constant__ EpiPair epp, int *status) {
+    const EpiArgs &ep = epp.p[0];              // sizes and tile order are common to both problems
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -50,7 +57,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // rows to compute: all of them, or the count another kernel left on the device (tiles beyond it are skipped)
     const int M_eff = ep.m_dev ? min(ep.M, max(0, *ep.m_dev - ep.m_off)) : ep.M;
     const int tiles_m = (M_eff + BM - 1) / BM, tiles_n = (ep.N + BN - 1) / BN;
-    const int num_tiles = tiles_m * tiles_n;
+    const int np = epp.nprob, tiles_np = tiles_n * np;         // the problems sit side by side along N
+    const int num_tiles = tiles_m * tiles_np;
+    // tile -> (row block, column block over both problems); the column block's problem is cb / tiles_n
+    auto tile_mb = [&](int tile) { return ep.n_fast ? tile / tiles_np : tile % tiles_m; };
+    auto tile_cb = [&](int tile) { return ep.n_fast ? tile % tiles_np : tile / tiles_m; };
     const int kblocks = (ep.K + BK - 1) / BK;
     constexpr uint32_t TMEM_COLS = 2 * BN;          // two accumulator buffers; 256 or 512 columns
 
@@ -74,14 +85,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (ep.n_fast ? tile / tiles_n : tile % tiles_m) * BM, n0 = (ep.n_fast ? tile % tiles_n : tile / tiles_m) * BN;
+                const int cb = tile_cb(tile), prob = cb / tiles_n;
+                const int m0 = tile_mb(tile) * BM, n0 = (cb - prob * tiles_n) * BN;
+                const CUtensorMap *ma = prob ? &map_a1 : &map_a0, *mb = prob ? &map_b1 : &map_b0;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!(ok = mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, status))) break;
                     uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_BYTES;
                     mbar_expect_tx(&bars->full[s], STAGE_BYTES);
-                    tma_load_2d(sa, &map_a, kb * BK, m0, &bars->full[s]);
-                    tma_load_2d(sb, &map_b, kb * BK, n0, &bars->full[s]);
+                    tma_load_2d(sa, ma, kb * BK, m0, &bars->full[s]);
+                    tma_load_2d(sb, mb, kb * BK, n0, &bars->full[s]);
                 }
             }
             if (!ok) {
@@ -122,13 +135,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int q = warp & 3;                            // warps 2,3,4,5 -> quarters 2,3,0,1
         // 32-byte stores and loads (one full sector per thread) when every row of C / of the addend starts on a 32-byte boundary
         const int c_es = ep.c_is_f32 ? 4 : 2;
-        const bool wide_c = (reinterpret_cast<uintptr_t>(ep.C) & 31u) == 0 && ((ep.ldc * c_es) & 31) == 0;
-        const bool wide_add = ep.addend && (reinterpret_cast<uintptr_t>(ep.addend) & 31u) == 0 && ((ep.ld_add * 4) & 31) == 0;
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
             const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
-            const int m0 = (ep.n_fast ? tile / tiles_n : tile % tiles_m) * BM, n0 = (ep.n_fast ? tile % tiles_n : tile / tiles_m) * BN;
+            const int cb = tile_cb(tile), prob = cb / tiles_n;
+            const int m0 = tile_mb(tile) * BM, n0 = (cb - prob * tiles_n) * BN;
+            const EpiArgs &ep = epp.p[prob];               // this tile's problem: its output, scales and addend
+            const bool wide_c = (reinterpret_cast<uintptr_t>(ep.C) & 31u) == 0 && ((ep.ldc * c_es) & 31) == 0;
+            const bool wide_add = ep.addend && (reinterpret_cast<uintptr_t>(ep.addend) & 31u) == 0 && ((ep.ld_add * 4) & 31) == 0;
             ok = mbar_wait(&bars->tmem_full[buf], bph, abort_flag, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -264,23 +279,41 @@ bool make_map(CUtensorMap *m, const void *base, int64_t rows, int64_t cols, int6
     return make_map_bf16(m, base, 2, dims, strides, box);
 }
 
+EpiArgs epi_of(const GemmArgs &a) {
+    // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
+    return EpiArgs{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols,
+                   a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.m_dev, a.m_off, a.M > a.N ? 1 : 0};
+}
+
+// b == NULL: one problem
 template <int BN>
-cudaError_t launch(const GemmArgs &a, cudaStream_t s) {
-    CUtensorMap ma, mb;
-    if (!make_map(&ma, a.A, a.M, a.K, a.lda, BM) || !make_map(&mb, a.B, a.N, a.K, a.ldb, BN)) return cudaErrorInvalidValue;
+cudaError_t launch(const GemmArgs &a, const GemmArgs *b, cudaStream_t s) {
+    CUtensorMap ma[2], mb[2];
+    if (!make_map(&ma[0], a.A, a.M, a.K, a.lda, BM) || !make_map(&mb[0], a.B, a.N, a.K, a.ldb, BN)) return cudaErrorInvalidValue;
+    ma[1] = ma[0]; mb[1] = mb[0];
+    if (b && (!make_map(&ma[1], b->A, b->M, b->K, b->lda, BM) || !make_map(&mb[1], b->B, b->N, b->K, b->ldb, BN))) return cudaErrorInvalidValue;
     constexpr size_t smem = STAGES * (size_t)(BM * BK * 2 + BN * BK * 2) + sizeof(PipeBars) + 1024;
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
-    const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
+    EpiPair epp{};
+    epp.p[0] = epi_of(a);
+    epp.p[1] = b ? epi_of(*b) : epp.p[0];
+    epp.nprob = b ? 2 : 1;
+    const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * epp.nprob;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
-    EpiArgs ep{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols,
-               a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.m_dev, a.m_off, a.M > a.N ? 1 : 0};
-    gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma, mb, ep, status);
+    gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma[0], mb[0], ma[1], mb[1], epp, status);
     count_launch();
     return cudaGetLastError();
+}
+
+// Tile width by rounds of CTAs: a 128 x 256 tile costs about 1.6 times a 128 x 128 one (it fetches 1.5 times the operands for
+// twice the products), so the wide tile wins whenever it saves a round -- also when it leaves a single round partly empty.
+bool wide_tile(const GemmArgs &a, int nprob) {
+    const int tm = (a.M + BM - 1) / BM, sms = sm_count();
+    const int rounds128 = (tm * ((a.N + 127) / 128) * nprob + sms - 1) / sms, rounds256 = (tm * ((a.N + 255) / 256) * nprob + sms - 1) / sms;
+    return !(a.N <= 128 || 10 * rounds128 <= 16 * rounds256);
 }
 
 }  // namespace
@@ -299,12 +332,17 @@ bool gemm_tcgen05_supports(const GemmArgs &a) {
 
 cudaError_t gemm_tcgen05(const GemmArgs &a, cudaStream_t s) {
     if (!gemm_tcgen05_supports(a)) return cudaErrorNotSupported;
-    // Tile width by rounds of CTAs: a 128 x 256 tile costs about 1.6 times a 128 x 128 one (it fetches 1.5 times the operands for
-    // twice the products), so the wide tile wins whenever it saves a round -- also when it leaves a single round partly empty.
-    const int tm = (a.M + BM - 1) / BM, sms = sm_count();
-    const int rounds128 = (tm * ((a.N + 127) / 128) + sms - 1) / sms, rounds256 = (tm * ((a.N + 255) / 256) + sms - 1) / sms;
-    if (a.N <= 128 || 10 * rounds128 <= 16 * rounds256) return launch<128>(a, s);
-    return launch<256>(a, s);
+    return wide_tile(a, 1) ? launch<256>(a, nullptr, s) : launch<128>(a, nullptr, s);
+}
+
+bool gemm_tcgen05_pair_supports(const GemmArgs &a, const GemmArgs &b) {
+    return gemm_tcgen05_supports(a) && gemm_tcgen05_supports(b) && a.M == b.M && a.N == b.N && a.K == b.K && !a.m_dev && !b.m_dev &&
+           a.c_dtype == b.c_dtype;
+}
+
+cudaError_t gemm_tcgen05_pair(const GemmArgs &a, const GemmArgs &b, cudaStream_t s) {
+    if (!gemm_tcgen05_pair_supports(a, b)) return cudaErrorNotSupported;
+    return wide_tile(a, 2) ? launch<256>(a, &b, s) : launch<128>(a, &b, s);
 }
 
 }  // namespace dm

@@ -207,6 +207,14 @@ __global__ void conv_state_kernel(const T *__restrict__ zx, const T *__restrict_
     conv_out[((int64_t)b * (k - 1) + r) * conv_ch + c] = v;
 }
 
+template <typename T>
+__global__ void __launch_bounds__(256) add_partials_kernel(const float *__restrict__ a, const float *__restrict__ b, T *__restrict__ y, size_t n4) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const float4 u = __ldg(reinterpret_cast<const float4 *>(a) + i), v = __ldg(reinterpret_cast<const float4 *>(b) + i);
+        st4(y + 4 * i, u.x + v.x, u.y + v.y, u.z + v.z, u.w + v.w);
+    }
+}
+
 // g0 <- s0 g0 + s1 g1, one block of threads per row (tied projections: the sum of the directions before the shared out_proj);
 // 16-byte accesses when the rows allow it (VEC = elements per 16 bytes, or 1)
 template <typename T, int VEC>
@@ -296,6 +304,16 @@ cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *con
     else
         conv_state_kernel<<<grid, 256, 0, s>>>(static_cast<const float *>(zx_fwd), static_cast<const float *>(conv_in),
                                                static_cast<float *>(conv_out), L, k, d_inner, conv_ch, d_in_proj);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t add_partials(const float *a, const float *b, void *y, int dtype, size_t n, cudaStream_t s) {
+    if (n % 4) return cudaErrorInvalidValue;
+    const size_t n4 = n / 4;
+    const int blocks = (int)((n4 + 255) / 256 > 148 * 8 ? 148 * 8 : (n4 + 255) / 256);
+    if (dtype == DM_BF16) add_partials_kernel<<<blocks, 256, 0, s>>>(a, b, static_cast<__nv_bfloat16 *>(y), n4);
+    else add_partials_kernel<<<blocks, 256, 0, s>>>(a, b, static_cast<float *>(y), n4);
     count_launch();
     return cudaGetLastError();
 }

@@ -114,9 +114,14 @@ __device__ __forceinline__ uint32_t prep_conv_pair(const float (&wl)[2][4], cons
     }
     return pack_bf16(silu_fast(v0), silu_fast(v1));
 }
+// softplus(dt + bias) = max(v, 0) + log1p(exp(-|v|)) with the fast exponential and logarithm: log1p by its series where 1 + e
+// would round e away (e < 2^-7: error below e^4 / 4), by log(1 + e) elsewhere.  Relative error of Delta about 1e-6, far inside
+// what the bf16 path needs.
 __device__ __forceinline__ float prep_delta(__nv_bfloat16 dt, float dt_bias) {
     const float v = __bfloat162float(dt) + dt_bias;
-    return fmaxf(v, 0.f) + log1pf(expf(-fabsf(v)));
+    const float e = __expf(-fabsf(v));
+    const float l = e < 0.0078125f ? e * fmaf(e, fmaf(e, 0.33333334f, -0.5f), 1.f) : __logf(1.f + e);
+    return fmaxf(v, 0.f) + l;
 }
 // One warp, one head, one 128-token chunk: d[r * ld] = Delta of physical chunk row r.  Writes Lambda (inclusive cumulative
 // Delta A in the direction's time order, log2 units) to dl[0..Q) and Lambda' = Lambda - log2 Delta to dl[Lp..Lp + Q).
@@ -138,7 +143,7 @@ __device__ __forceinline__ void prep_lambda_head(const float *d_col, int ld, flo
     const float base = run - cum[3];                             // sum over the lanes before this one
     float lam[4], lamp[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) { lam[e] = base + cum[e]; lamp[e] = lam[e] - log2f(d[e]); }    // Delta = 0 (padding): Lambda' = +inf
+    for (int e = 0; e < 4; ++e) { lam[e] = base + cum[e]; lamp[e] = lam[e] - __log2f(d[e]); }    // Delta = 0 (padding): Lambda' = +inf
     const int rlo = rev ? Q - 4 - 4 * lane : 4 * lane;           // lowest physical row of this lane's four
     const float4 v0 = rev ? make_float4(lam[3], lam[2], lam[1], lam[0]) : make_float4(lam[0], lam[1], lam[2], lam[3]);
     const float4 v1 = rev ? make_float4(lamp[3], lamp[2], lamp[1], lamp[0]) : make_float4(lamp[0], lamp[1], lamp[2], lamp[3]);
@@ -265,12 +270,14 @@ __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__res
     }
 }
 
+// grid.x covers the chunks the direction visits first: blockIdx.x / PREP_PARTS is the chunk's index in time order
 __global__ void __launch_bounds__(PREP_THREADS)
 ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, float *__restrict__ Sb,
                 int dir0) {
     __shared__ float dsm[Q * (PREP_HEADS + 1)];
     __shared__ __align__(16) uint32_t bct[2][QB][BCT_LD];     // short-block mode: this CTA's rows of B' ([0]) and C' ([1]) as bf16 pairs
-    prep_unit(a, Bp, Cp, dA, Sb, dir0 + blockIdx.z, blockIdx.y, blockIdx.x / PREP_PARTS, blockIdx.x % PREP_PARTS, threadIdx.x, 0, dsm, bct);
+    const int dir = dir0 + blockIdx.z, c = blockIdx.x / PREP_PARTS;
+    prep_unit(a, Bp, Cp, dA, Sb, dir, blockIdx.y, dir == 1 ? a.nch - 1 - c : c, blockIdx.x % PREP_PARTS, threadIdx.x, 0, dsm, bct);
 }
 
 // --------------------------------------------------------------------------------------------------
@@ -290,6 +297,7 @@ struct PrepJob {
     float *dA;
     int *sync;          // [0]: ticket counter, [1 + seq * nch + pc]: item flags; zeroed before the launch.  NULL: no fused prep
     int nprep, ndir;
+    int c0;             // chunks before this one (in time order) come from a prep launch of their own that ran before the scan launch
 };
 // 16-byte asynchronous copy global -> shared; src_bytes = 16, or 0 to fill the destination with zeros (src must still be a valid address)
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, uint32_t src_bytes) {
@@ -306,8 +314,8 @@ struct PrepItem { int dir, b, pc; };
 __device__ __forceinline__ PrepItem prep_item(const SsdArgs &a, const PrepJob &pj, int it, int dir0) {
     PrepItem r;
     r.dir = dir0 + it % pj.ndir;
-    const int c = (it / pj.ndir) % a.nch;
-    r.b = it / (pj.ndir * a.nch);
+    const int nc = a.nch - pj.c0, c = pj.c0 + (it / pj.ndir) % nc;
+    r.b = it / (pj.ndir * nc);
     r.pc = r.dir == 1 ? a.nch - 1 - c : c;
     return r;
 }
@@ -343,7 +351,7 @@ __device__ __noinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, int 
     static_assert(PREP_SEG * 128 == NTHREADS && PREP_SMEM <= OFF_MISC, "prep role: thread and shared-memory layout");
     float *dsm = reinterpret_cast<float *>(smem + 2 * PREP_STAGE);              // [Q][65] Delta of one tile of 64 heads
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int L = a.L, k = a.k, n_items = pj.ndir * a.B * a.nch;
+    const int L = a.L, k = a.k, n_items = pj.ndir * a.B * (a.nch - pj.c0);
     if (first >= n_items) return;
     // 16-byte copies of eight heads' dt: the dt columns start on a 16-byte boundary and the head count is a multiple of 8
     const bool dt_vec = (a.d_inner + a.conv_ch) % 8 == 0 && a.H % 8 == 0;
@@ -487,7 +495,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int c = 0; c < nch; ++c) {
                 const int sx = c % NX, sd = c % NDL, pc = rev ? nch - 1 - c : c;
                 // the chunk's Lambda are in memory (fused prep): asked first, so that the flag's round trip to L2 hides behind the wait for a free stage
-                if (ready && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;
+                if (ready && c >= pj.c0 && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;
                 if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
                 tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, zseq, &misc->full_x[sx]);
@@ -522,7 +530,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             int issued_b = 0, issued_c = 0;
             for (int c = 0; c < nch; ++c) {
                 const int sb = c % NB, pc = rev ? nch - 1 - c : c;
-                if (ready && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;          // the chunk's B', C' are in memory
+                if (ready && c >= pj.c0 && !flag_wait<PREP_PARTS>(ready + pc, abort_flag, status)) break;          // the chunk's B', C' are in memory
                 if (!WAIT(&misc->empty_b[sb], ((c / NB) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_b[sb], 2 * T16);
                 tma_load_3d(smem + OFF_B + sb * 2 * T16, &map_b, 0, pc * Q, seq, &misc->full_b[sb]);
@@ -1261,23 +1269,27 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     const bool blk = block_mode(a);
     float *Sb = blk ? reinterpret_cast<float *>(base + l.sb) : nullptr;
 
-    // One long sequence leaves SMs without a scan CTA: they take the prep work inside the scan launch (see prep_role).
-    const int nscan = a.H * ndir * a.B, n_items = ndir * a.B * l.nch;
-    PrepJob pj{Bp, Cp, dA, nullptr, 0, ndir};
-    if (!blk && nscan < sm_count() && a.N % 8 == 0) {
-        pj.sync = reinterpret_cast<int *>(base + l.sy);
+    // One long sequence leaves SMs without a scan CTA: they take the prep work inside the scan launch (see prep_role), except for
+    // the first PRE_CHUNKS chunks of every sequence and direction, which a small prep launch of their own has ready by the time the
+    // scan starts (a prep CTA inside the scan launch needs about 20 us for its first chunk; the scan would stand idle that long).
+    constexpr int PRE_CHUNKS = 8;
+    const int nscan = a.H * ndir * a.B;
+    PrepJob pj{Bp, Cp, dA, nullptr, 0, ndir, 0};
+    int n_pre = l.nch;                              // chunks (in time order) done by the prep launch
+    if (!blk && nscan < sm_count() && a.N % 8 == 0 && l.nch > PRE_CHUNKS) {
+        const int n_items = ndir * a.B * (l.nch - PRE_CHUNKS);
         pj.nprep = n_items < sm_count() - nscan ? n_items : sm_count() - nscan;
         if (ndir == 2) pj.nprep &= ~1;                             // even: every prep CTA then stays with one direction
-        if (pj.nprep == 0) pj.sync = nullptr;
+        if (pj.nprep > 0) {
+            pj.sync = reinterpret_cast<int *>(base + l.sy);
+            pj.c0 = n_pre = PRE_CHUNKS;
+        }
     }
     cudaError_t e;
-    if (pj.sync) {
-        if ((e = cudaMemsetAsync(pj.sync, 0, ((size_t)2 * a.B * l.nch + 1) * sizeof(int), s)) != cudaSuccess) return e;
-    } else {
-        ssd_prep_kernel<<<dim3(l.nch * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);
-        count_launch();
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    }
+    if (pj.sync && (e = cudaMemsetAsync(pj.sync, 0, ((size_t)2 * a.B * l.nch + 1) * sizeof(int), s)) != cudaSuccess) return e;
+    ssd_prep_kernel<<<dim3(n_pre * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (blk) {
         auto kern = a.P == P ? ssd_block_kernel<P> : ssd_block_kernel<P / 2>;
         const size_t smem = a.P == P ? BlockSmem<P>::total : BlockSmem<P / 2>::total;
