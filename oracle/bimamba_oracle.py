@@ -34,6 +34,13 @@ the two equations after it) is `diffusion_block` / `denoise_step_cond`.  Its ari
 leaves open there -- the third modulation vector per sublayer that App. C's 6*d count implies and the
 equation does not show (read as a gate on the sublayer's output), the MLP's activation (GELU, tanh
 form) and the epsilon of the normalisation -- is parity unpinned (by the paper) as well.
+
+The generation loop `generate` (K reverse steps of Eq. 3 along `noise_schedule`, then one pass with keep probability 0) has
+its arithmetic pinned (the survivor sets follow from the uniforms in closed form, the keep probabilities telescope to the
+noise levels).  That the tokens still masked at the last noise level are drawn in one extra pass is this build's reading of
+a point the paper leaves open: parity unpinned (by the paper).  The weight-tied variant needs no function of its own (it is
+`bimamba_forward` called with the shared matrices in both directions' parameter sets); which parameters the paper's
+"bidirectional weight tie" would cover is not stated: parity unpinned (by the paper).
 """
 from __future__ import annotations
 

@@ -65,13 +65,15 @@ constexpr uint32_t OFF_C = OFF_B + NB * 2 * T16;        // C' in transit to TMEM
 constexpr uint32_t OFF_XS = OFF_C + 2 * T16;            // w_j x'_j
 constexpr uint32_t OFF_H = OFF_XS + T16;                // bf16 copy of the incoming state [d_state rows][headdim]
 constexpr uint32_t OFF_DL = OFF_H + T16;                // NDL stages x (Lambda[Q], Lambda'[Q]) fp32
-constexpr uint32_t OFF_MISC = OFF_DL + NDL * 2 * Q * 4;
+constexpr uint32_t DL_HEAD = 2 * Q * 4;                  // one head's (Lambda, Lambda') of a chunk
+constexpr uint32_t OFF_MISC = OFF_DL + NDL * DL_HEAD;    // one head per CTA; two heads per CTA: OFF_MISC + NDL * DL_HEAD
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 7168 + 1024;  // + barriers/scalars + alignment slack
+constexpr uint32_t SMEM_BYTES_PAIR = SMEM_BYTES + NDL * DL_HEAD;
 static_assert(OFF_Z % 1024 == 0 && OFF_B % 1024 == 0 && OFF_C % 1024 == 0 && OFF_XS % 1024 == 0 && OFF_H % 1024 == 0, "tile alignment");
-static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+static_assert(SMEM_BYTES_PAIR <= 232448, "shared memory budget");
 
 // TMEM columns (all 512 are allocated)
-constexpr uint32_t TM_S = 0, TM_W = 128, TM_YB1 = 192, TM_YA = 256, TM_YB0 = 320, TM_HS = 448, TM_COLS = 512;    // Yb is double-buffered; columns 384..447 are unused
+constexpr uint32_t TM_S = 0, TM_W = 128, TM_YB1 = 192, TM_YA = 256, TM_YB0 = 320, TM_W1 = 384, TM_HS = 448, TM_COLS = 512;    // Yb is double-buffered; W1: the second head's W when a CTA carries two heads
 
 struct Misc {
     uint64_t full_x[NX], empty_x[NX], full_z[NZ], empty_z[NZ], full_b[NB], empty_b[NB], full_c, empty_c, full_dl[NDL], empty_dl[NDL];
@@ -80,7 +82,7 @@ struct Misc {
     int abort;
     int ticket;                   // order in which this CTA started (fused prep: the first ones take the prep role)
     alignas(16) float norm_w[P];  // the three arrays below are read as float4
-    alignas(16) float wbuf[Q];
+    alignas(16) float wbuf[2][Q];  // [1] only with two heads per CTA
     alignas(16) float cbuf[NWG][4][Q]; // per mask warp: column factors of the off-diagonal blocks
     float ssq_part[Q];            // sum of squares of the second epilogue group's channels
 };
@@ -424,11 +426,15 @@ __device__ __noinline__ void prep_role(const SsdArgs &a, const PrepJob &pj, int 
 // --------------------------------------------------------------------------------------------------
 // Launch 2: the chunked scan.
 // --------------------------------------------------------------------------------------------------
-// HALFP: the model's headdim is P / 2.  The CTA still moves 64-channel tiles (the second half is padding that never
-// leaves it), but the conv, the state hand-over and the epilogue work on the 32 real channels only, split over the
-// same threads; the padded halves of the w o x' tile and of the state copy are zeroed once, so the padded state
-// columns stay zero.
-template <bool HALFP>
+// HM = 0: heads of P = 64 channels, one per CTA.
+// HM = 1 (HALFP): the model's headdim is P / 2 and the CTA carries one head.  It still moves 64-channel tiles (the second half is
+// padding that never leaves it), but the conv, the state hand-over and the epilogue work on the 32 real channels only, split over
+// the same threads; the padded halves of the w o x' tile and of the state copy are zeroed once, so the padded state columns stay zero.
+// HM = 2 (PAIR): headdim P / 2 and an even number of heads: the CTA carries two neighbouring heads in its 64 channels.  They share
+// the B', C' tiles and S; each has its own Lambda, Lambda' (two per stage), its own mask W (mask group g builds head g's W, the second
+// one in the TMEM columns the other modes leave unused) and its own 32-wide Ya = W x' product; Yb, St, the state (two 32-column halves)
+// and the tiles are those of a 64-channel head, with the decay factors taken per column half.
+template <int HM>
 __global__ void __launch_bounds__(NTHREADS, 1)
 ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_z,
                 const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_c,
@@ -436,11 +442,14 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    Misc *misc = reinterpret_cast<Misc *>(smem + OFF_MISC);
+    constexpr bool HALFP = HM == 1, PAIR = HM == 2;
+    constexpr int NH = PAIR ? 2 : 1;                               // heads per CTA
+    constexpr uint32_t DL_STAGE = NH * DL_HEAD;                    // bytes of one (Lambda, Lambda') stage
+    Misc *misc = reinterpret_cast<Misc *>(smem + OFF_DL + NDL * DL_STAGE);
     volatile int *abort_flag = &misc->abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    int item = blockIdx.x;                     // (batch row, direction, head), heads fastest
+    int item = blockIdx.x;                     // (batch row, direction, head or head pair), heads fastest
     if (pj.sync) {
         if (tid == 0) misc->ticket = atomicAdd(pj.sync, 1);
         __syncthreads();
@@ -448,7 +457,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         if (ticket < pj.nprep) { prep_role(a, pj, ticket, dir0, smem); return; }
         item = ticket - pj.nprep;
     }
-    const int h = item % a.H, b = item / (a.H * pj.ndir), dir = dir0 + (item / a.H) % pj.ndir;
+    const int HC = a.H / NH;                   // CTAs per (batch row, direction)
+    const int h = (item % HC) * NH, b = item / (HC * pj.ndir), dir = dir0 + (item / HC) % pj.ndir;     // h: the CTA's (first) head
     const bool rev = dir == 1;
     const int *ready = pj.sync ? pj.sync + 1 + ((int64_t)dir * a.B + b) * a.nch : nullptr;     // per chunk: units of its B', C', Lambda that are in memory
     const int L = a.L, nch = a.nch;
@@ -474,7 +484,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         mbar_fence_init();
     }
     const int Pr = a.Pr;                 // channels of this head; the tile's remaining P - Pr columns are padding and never leave the CTA
-    if (tid < P) misc->norm_w[tid] = (norm_on && w.norm_w && tid < Pr) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * Pr + tid]) : 1.f;
+    if (tid < P) misc->norm_w[tid] = (norm_on && w.norm_w && tid < NH * Pr) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.norm_w)[h * Pr + tid]) : 1.f;
     if (warp == 1) tmem_alloc(&misc->tmem_base, TM_COLS);
     fence_before();
     __syncthreads();
@@ -499,9 +509,12 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!WAIT2(&misc->empty_x[sx], ((c / NX) & 1) ^ 1, &misc->empty_dl[sd], ((c / NDL) & 1) ^ 1)) break;
                 mbar_expect_tx(&misc->full_x[sx], XTILE);
                 tma_load_3d(smem + OFF_X + sx * XTILE, &map_x, a.d_inner + h * Pr, rev ? pc * Q : pc * Q - HALO, zseq, &misc->full_x[sx]);
-                mbar_expect_tx(&misc->full_dl[sd], 2 * Q * 4);
-                bulk_load(smem + OFF_DL + sd * 2 * Q * 4, dA_head + pc * Q, Q * 4, &misc->full_dl[sd]);
-                bulk_load(smem + OFF_DL + sd * 2 * Q * 4 + Q * 4, dA_head + a.Lp + pc * Q, Q * 4, &misc->full_dl[sd]);
+                mbar_expect_tx(&misc->full_dl[sd], DL_STAGE);
+#pragma unroll
+                for (int hh = 0; hh < NH; ++hh) {                  // stage layout: [head][Lambda | Lambda'][Q]
+                    bulk_load(smem + OFF_DL + sd * DL_STAGE + hh * DL_HEAD, dA_head + (int64_t)hh * 2 * a.Lp + pc * Q, Q * 4, &misc->full_dl[sd]);
+                    bulk_load(smem + OFF_DL + sd * DL_STAGE + hh * DL_HEAD + Q * 4, dA_head + (int64_t)hh * 2 * a.Lp + a.Lp + pc * Q, Q * 4, &misc->full_dl[sd]);
+                }
                 issued = c + 1;
             }
             if (*abort_flag)            // aborting: bounded wait for the loads still in flight
@@ -565,14 +578,29 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const uint32_t dBk0 = desc_lo_k(smem_u32(smem + OFF_B)), dBm0 = desc_lo_mn(smem_u32(smem + OFF_B), T16);
             const uint32_t dX0 = desc_lo_mn(smem_u32(smem + OFF_X) + (rev ? 0 : HALO * 128), T16);
             constexpr uint32_t I128 = idesc_bf16(128, 128, 0, 0), I64 = idesc_bf16(128, 64, 0, 1), I64T = idesc_bf16(128, 64, 1, 1);
+            constexpr uint32_t I32 = idesc_bf16(128, 32, 0, 1);
             auto issue_ya = [&](int c) -> bool {       // Ya = W x'  (A = W from TMEM, B = x' [j][p] MN-major)
                 const int sx = c % NX;
                 if (!WAIT2(&misc->w_full, c & 1, &misc->ya_empty, (c & 1) ^ 1)) return false;
                 fence_after();
                 const uint32_t dX = dX0 + (uint32_t)sx * (XTILE >> 4);
-                if (leader) umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
+                if constexpr (PAIR) {
+                    // two products of 32 channels: head 0 = W x'[:, 0:32], head 1 = W1 x'[:, 32:64] (the operand starts 64 bytes into the 128-byte rows)
 #pragma unroll
-                for (int kk = 1; kk < 8; ++kk) if (leader) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
+                    for (int kk = 0; kk < 8; ++kk) {
+                        if (kk == 0) { if (leader) umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I32); }
+                        else if (leader) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I32);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        if (kk == 0) { if (leader) umma_ts<0>(tmem + TM_YA + 32, tmem + TM_W1, dX + 4, I32); }
+                        else if (leader) umma_ts<1>(tmem + TM_YA + 32, tmem + TM_W1 + 8 * kk, dX + kk * 128 + 4, I32);
+                    }
+                } else {
+                    if (leader) umma_ts<0>(tmem + TM_YA, tmem + TM_W, dX, I64);
+#pragma unroll
+                    for (int kk = 1; kk < 8; ++kk) if (leader) umma_ts<1>(tmem + TM_YA, tmem + TM_W + 8 * kk, dX + kk * 128, I64);
+                }
                 if (leader) umma_commit(&misc->y_full);              // Yb of the same chunk was issued earlier: it has completed as well; also frees W
                 if (leader) umma_commit(&misc->empty_x[sx]);
                 return true;
@@ -656,7 +684,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
         // incoming state -> TMEM (fp32)
         {
-            const float *h0 = (!rev && a.ssm_in && srow < a.Nr && sh * 32 < Pr) ? a.ssm_in + (((int64_t)b * a.H + h) * Pr) * a.Nr + srow : nullptr;
+            const float *h0 = (!rev && a.ssm_in && srow < a.Nr && sh * 32 < NH * Pr) ? a.ssm_in + (((int64_t)b * a.H + h) * Pr) * a.Nr + srow : nullptr;
             uint32_t hs[32];
 #pragma unroll
             for (int p = 0; p < 32; ++p) hs[p] = h0 ? __float_as_uint(h0[(int64_t)(sh * 32 + p) * a.Nr]) : 0u;
@@ -699,7 +727,8 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const uint32_t par = c & 1;
             if (ok) ok = WAIT3(&misc->full_x[sx], (c / NX) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->st_full, par ^ 1);
             if (!named_all(1, ROLE, ok)) { ok = false; break; }
-            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
+            // (Lambda, Lambda') of the head whose state columns this thread hands over (two heads per CTA: the column half sh)
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * DL_STAGE + (PAIR ? sh : 0) * DL_HEAD), *lamp = lam + Q;
             // St of the previous chunk has completed (so has its Yb, issued before it): hand the state over first, Yb and St wait for it
             state_prepare(ex2f(lam[rev ? 0 : Q - 1]));
             // ---- conv.  The three rows before the block (in time) belong to a neighbour, who overwrites them in
@@ -721,7 +750,10 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 h2[0] = bf2_to_f2(hr[1].x); h2[1] = bf2_to_f2(hr[1].y);
                 h3[0] = bf2_to_f2(hr[2].x); h3[1] = bf2_to_f2(hr[2].y);
             }
-            if (t < Q) misc->wbuf[t] = ex2f(lam[rev ? 0 : Q - 1] - lamp[t]);
+            if (t < NH * Q) {                              // w_j of every head: thread t = (head t / Q, row t % Q); with two heads t / Q == sh
+                const int tr = t & (Q - 1);
+                misc->wbuf[PAIR ? sh : 0][tr] = ex2f(lam[rev ? 0 : Q - 1] - lamp[tr]);
+            }
             mbar_arrive(&misc->empty_dl[sd]);
             named_sync(1, ROLE);                           // halo rows are in registers; wbuf is visible
             // Row j of the block sits at j * 128 + ((colx ^ (j & 7)) << 4) in both tiles; with j & 7 = jx this is
@@ -729,7 +761,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             constexpr int R8 = 8 / RB;                          // blocks per group of eight rows
             const int r8 = (rb / R8) * 8, rlo = (rb % R8) * RB;  // the block starts rlo rows into the eight rows at r8
             uint8_t *bx = xt + (toff + r8) * 128 + sub, *bs = smem + OFF_XS + r8 * 128 + sub;
-            const uint8_t *wp = reinterpret_cast<const uint8_t *>(misc->wbuf + rb * RB + (rev ? RB - 1 : 0));
+            const uint8_t *wp = reinterpret_cast<const uint8_t *>(misc->wbuf[PAIR ? cg >> 3 : 0] + rb * RB + (rev ? RB - 1 : 0));      // the head of this thread's channels
             uint32_t k = (uint32_t)(rlo + (rev ? RB - 1 : 0)) * 144u;
 #pragma unroll 2
             for (int tau = 0; tau < RB; ++tau) {
@@ -768,7 +800,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             uint32_t hs[32];
             tmem_ld_x32(tlane + TM_HS + half * 32, hs);          // warp-wide: every lane takes part
             tmem_wait_ld();
-            if (srow < a.Nr && half * 32 < Pr) {                 // rows beyond the model's d_state and columns beyond its headdim are padding
+            if (srow < a.Nr && half * 32 < NH * Pr) {            // rows beyond the model's d_state and columns beyond the CTA's channels are padding
 #pragma unroll
                 for (int p = 0; p < 32; ++p) ho[(int64_t)(half * 32 + p) * a.Nr] = __uint_as_float(hs[p]);
             }
@@ -780,7 +812,9 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int mg = (warp - 4 - 4 * NWG) >> 2;       // group index
         const int row = (tid - (4 + 4 * NWG) * 32) & (WG - 1);      // token row i (mask) / state row n (state)
         const int q = warp & 3;
-        const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
+        // two heads per CTA: group mg builds the whole mask of head h + mg (its own Lambda, D and W columns) instead of half of one mask
+        const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h + (PAIR ? mg : 0)] : 0.f;
+        const uint32_t tm_w = (PAIR && mg) ? TM_W1 : TM_W;
         float *cbuf = misc->cbuf[mg][q];
         bool ok = true;
         for (int c = 0; c < nch; ++c) {
@@ -789,7 +823,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // the decay factors depend on Lambda only: they are prepared while S of this chunk is still being computed
             if (ok) ok = WAIT(&misc->full_dl[sd], (c / NDL) & 1);
             if (!named_all(3 + mg, WG, ok)) { ok = false; break; }
-            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4), *lamp = lam + Q;
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * DL_STAGE + (PAIR ? mg : 0) * DL_HEAD), *lamp = lam + Q;
             const float li = lam[row];
             // ---- W_ij = S_ij 2^(Lambda_i - Lambda'_j) for j not after i in time, + D on the diagonal; 0 elsewhere.
             // Blocks of 32 x 32: the block on the diagonal takes one exponential per entry; a block before it (in
@@ -813,7 +847,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (!WAIT2(&misc->s_full, par, &misc->y_full, par ^ 1)) { ok = false; continue; }
             fence_after();
 #pragma unroll 1
-            for (int gi = mg; gi < 8; gi += NWG) {        // this group's share of the 8 groups of 16 columns
+            for (int gi = PAIR ? 0 : mg; gi < 8; gi += PAIR ? 1 : NWG) {        // this group's share of the 8 groups of 16 columns
                 const int jb = gi >> 1, j0 = gi * 16;
                 uint32_t out[8];
                 if (rev ? jb > q : jb < q) {
@@ -850,7 +884,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 #pragma unroll
                     for (int i = 0; i < 8; ++i) out[i] = 0u;
                 }
-                tmem_st_x8(tlane + TM_W + gi * 8, out);
+                tmem_st_x8(tlane + tm_w + gi * 8, out);
             }
             fence_before();
             mbar_arrive(&misc->s_empty);                 // every read of S has completed (wait::ld above)
@@ -871,7 +905,7 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (ok) ok = WAIT3(&misc->full_z[sz], (c / NZ) & 1, &misc->full_dl[sd], (c / NDL) & 1, &misc->y_full, par);
             if (!named_all(2, ROLE, ok)) { ok = false; break; }
             fence_after();
-            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * 2 * Q * 4);
+            const float *lam = reinterpret_cast<const float *>(smem + OFF_DL + sd * DL_STAGE + (PAIR ? eg : 0) * DL_HEAD);      // two heads per CTA: group eg = head h + eg
             const float ei = ex2f(lam[row]);
             mbar_arrive(&misc->empty_dl[sd]);
             const int t = pc * Q + row;
@@ -906,13 +940,15 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             float ss, ss_hi;
             upk2(ss2, ss, ss_hi);
             ss += ss_hi;
-            if (eg == 1) misc->ssq_part[row] = ss;
+            if (!PAIR && eg == 1) misc->ssq_part[row] = ss;
             fence_proxy_async();
             named_sync(2, ROLE);
-            if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + misc->ssq_part[row];
+            if (PAIR) {                                    // each group's channels are one head
+                if (t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h + eg] = ss;
+            } else if (eg == 0 && t < L && a.ssq) a.ssq[((int64_t)seq * L + t) * a.H + h] = ss + misc->ssq_part[row];
             if (eg == 0 && row == 0) {
                 if (!HALFP) {
-                    tma_store_3d(&map_g, zt, h * P, pc * Q, seq);    // rows past the end of the sequence are clipped
+                    tma_store_3d(&map_g, zt, h * Pr, pc * Q, seq);   // rows past the end of the sequence are clipped
                     bulk_commit();
                     bulk_wait_read0();
                 }
@@ -1273,7 +1309,8 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     // the first PRE_CHUNKS chunks of every sequence and direction, which a small prep launch of their own has ready by the time the
     // scan starts (a prep CTA inside the scan launch needs about 20 us for its first chunk; the scan would stand idle that long).
     constexpr int PRE_CHUNKS = 8;
-    const int nscan = a.H * ndir * a.B;
+    const bool pair = a.P == P / 2 && a.H % 2 == 0;        // two half-width heads per scan CTA
+    const int nscan = (pair ? a.H / 2 : a.H) * ndir * a.B;
     PrepJob pj{Bp, Cp, dA, nullptr, 0, ndir, 0};
     int n_pre = l.nch;                              // chunks (in time order) done by the prep launch
     if (!blk && nscan < sm_count() && a.N % 8 == 0 && l.nch > PRE_CHUNKS) {
@@ -1321,10 +1358,11 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     }
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
-    auto kern = a.P == P ? ssd_scan_kernel<false> : ssd_scan_kernel<true>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    auto kern = a.P == P ? ssd_scan_kernel<0> : pair ? ssd_scan_kernel<2> : ssd_scan_kernel<1>;
+    const uint32_t smem_bytes = pair ? SMEM_BYTES_PAIR : SMEM_BYTES;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) return e;
-    kern<<<nscan + pj.nprep, NTHREADS, SMEM_BYTES, s>>>(mx, mz, mb, mc, mg, k, pj, dir0, status);
+    kern<<<nscan + pj.nprep, NTHREADS, smem_bytes, s>>>(mx, mz, mb, mc, mg, k, pj, dir0, status);
     count_launch();
     return cudaGetLastError();
 }

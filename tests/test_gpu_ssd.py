@@ -163,3 +163,22 @@ def test_seeded_mix_of_shapes_and_options(G, seed):
     else:
         _check(G, G.run_forward(shape, I.BF16, wf, wr, x, flags=flags, dir_mask=dir_mask),
                O.bimamba_forward(x, wf, wr, dir_mask=dir_mask, **kw))
+
+
+@pytest.mark.parametrize("H,L", [(5, 300), (6, 300), (2, 129)])
+def test_half_width_heads_single_and_paired(G, H, L):
+    """Heads of 32 channels: an even head count puts two neighbouring heads into one CTA of the tensor-core scan (shared B', C' and
+    S, one mask and one 32-wide product each), an odd one keeps one head per CTA with half of the tile as padding."""
+    shape = I.MixerShape(2, L, 16 * H, 2, 128, 4, H)
+    assert shape.headdim == 32
+    wf, wr = I.make_mixer_weights(shape, 60 + H, I.BF16, perturb=True)
+    x = I.make_activations(shape, 60 + H, I.BF16)
+    got = G.run_forward(shape, I.BF16, wf, wr, x, chunk=128)
+    _check(G, got, O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape)))
+    # carried state in and out through the same kernel
+    blk = I.MixerShape(2, L, 16 * H, 2, 128, 4, H)
+    ssm_in, conv_in = I.make_states(blk, 61, I.BF16)
+    y, s_out, c_out = G.run_block_step(blk, I.BF16, wf, wr, x, ssm_in, conv_in, chunk=128)
+    y_o, s_o, c_o = O.bimamba_block_step(x, wf, wr, ssm_state_in=ssm_in, conv_state_in=conv_in, **G.oracle_kwargs(blk))
+    _check(G, y, y_o)
+    assert G.rel_l2(s_out, s_o) <= BF16_REL and G.rel_l2(c_out, c_o) <= BF16_REL
