@@ -360,6 +360,14 @@ int dm_bimamba_forward_static(const dm_mixer_cfg *cfg, const dm_dir_weights w[2]
  * and the nanoseconds the second one waited. */
 int dm_selftest_wait_timeout(uint32_t limit_us, uint64_t *out, void *cuda_stream);
 
+/* Self-test switch for the same failure path inside the tensor-core scan (no counterpart in the paper).  While on, a mixer call
+ * whose scan would do its prep work inside the scan launch (one long sequence: fewer scan CTAs than SMs, more than eight chunks)
+ * launches the scan without the CTAs of that role: the flags its load warps wait for from the ninth chunk on are never raised,
+ * the waits run out after their regular limit (2 s), and every role of every CTA has to leave through the abort path -- loads in
+ * flight waited for, TMEM freed.  The call itself returns DM_OK; dm_check then reports DM_ERR_TIMEOUT; y is unspecified.  Nothing
+ * faults or hangs.  Process-wide; switch it off again. */
+int dm_selftest_withhold_prep(int on);
+
 /* Number of kernels this library has launched from this process since load (for benchmarks). */
 uint64_t dm_kernel_launch_count(void);
 

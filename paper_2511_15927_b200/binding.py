@@ -145,7 +145,7 @@ EXPORTS = ("dm_status_string", "dm_last_error_message", "dm_kernel_launch_count"
            "dm_bimamba_block_step", "dm_denoise_step", "dm_profile_enable", "dm_profile_read", "dm_linear", "dm_bimamba_forward_static",
            "dm_denoise_cond_workspace_bytes", "dm_denoise_step_cond", "dm_denoise_sample_workspace_bytes", "dm_denoise_sample_step",
            "dm_attention_workspace_bytes", "dm_attention_forward", "dm_denoise_hybrid_workspace_bytes", "dm_denoise_step_hybrid",
-           "dm_denoise_step_hybrid_block", "dm_attention_block_step", "dm_generate_workspace_bytes", "dm_generate", "dm_selftest_wait_timeout")
+           "dm_denoise_step_hybrid_block", "dm_attention_block_step", "dm_generate_workspace_bytes", "dm_generate", "dm_selftest_wait_timeout", "dm_selftest_withhold_prep")
 DM_STATIC_WORKSPACE_BYTES = 32 << 20
 DM_STAGE_IN_PROJ, DM_STAGE_SCAN, DM_STAGE_OUT_PROJ, DM_STAGE_COUNT = 0, 1, 2, 3
 
@@ -268,6 +268,12 @@ def dm_denoise_sample_step(cfg, blk, weights, block_weights, tokens_in: int, tau
     _ok(_lib.dm_denoise_sample_step(C.byref(cfg), C.byref(blk) if blk is not None else None, C.byref(weights), block_weights,
                                     _vp(tokens_in), _vp(tau or None), C.byref(sample), _vp(u_keep), _vp(u_cat), _vp(tokens_out),
                                     states, _vp(workspace), _sz(workspace_bytes), _vp(cuda_stream)))
+
+
+def dm_selftest_withhold_prep(on: bool) -> None:
+    _lib.dm_selftest_withhold_prep.argtypes = [C.c_int]
+    _lib.dm_selftest_withhold_prep.restype = C.c_int
+    _ok(_lib.dm_selftest_withhold_prep(1 if on else 0))
 
 
 def dm_selftest_wait_timeout(limit_us: int, out: int, cuda_stream: int = 0) -> None:

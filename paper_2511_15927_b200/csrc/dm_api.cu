@@ -860,6 +860,11 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
     return DM_OK;
 }
 
+int dm_selftest_withhold_prep(int on) {
+    scan_ssd_selftest_withhold(on);
+    return DM_OK;
+}
+
 int dm_selftest_wait_timeout(uint32_t limit_us, uint64_t *out, void *cuda_stream) {
     if (!out) return fail(DM_ERR_INVALID_ARG, "out is NULL");
     if (limit_us == 0 || limit_us > 1000000u) return fail(DM_ERR_INVALID_ARG, "limit_us must be in [1, 1000000]");

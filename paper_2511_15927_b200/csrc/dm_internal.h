@@ -78,6 +78,7 @@ cudaError_t scan_sequential(const ScanArgs &a, void *ws, cudaStream_t s);
 bool scan_ssd_supports(const ScanArgs &a);
 // chunk values the chunked bf16 path takes (0 = default, 32 = CUDA-core kernel, 128 = tensor-core kernel); other paths take any chunk > 0
 bool scan_ssd_chunk_ok(int dtype, int d_state, int chunk);
+void scan_ssd_selftest_withhold(int on);
 size_t scan_ssd_workspace_bytes(const ScanArgs &a);
 cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s);
 

@@ -1271,6 +1271,11 @@ bool shape_ok(const ScanArgs &a) {
 
 }  // namespace
 
+// Self-test switch: the scan launch keeps its prep role's flags but gets no prep CTA, so the load warps' bounded waits for the
+// ninth chunk run out and every role of every CTA leaves through the abort path (dm_selftest_withhold_prep).
+static int g_withhold_prep = 0;
+void scan_ssd_selftest_withhold(int on) { g_withhold_prep = on ? 1 : 0; }
+
 bool scan_ssd_chunk_ok(int dtype, int d_state, int chunk) {
     return !(dtype == DM_BF16 && d_state <= N) || chunk == 0 || chunk == QB || chunk == Q;
 }
@@ -1322,6 +1327,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
             pj.c0 = n_pre = PRE_CHUNKS;
         }
     }
+    if (pj.sync && g_withhold_prep) pj.nprep = 0;
     cudaError_t e;
     if (pj.sync && (e = cudaMemsetAsync(pj.sync, 0, ((size_t)2 * a.B * l.nch + 1) * sizeof(int), s)) != cudaSuccess) return e;
     ssd_prep_kernel<<<dim3(n_pre * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);

@@ -40,6 +40,34 @@ def test_a_wait_that_runs_out_is_reported_and_the_library_stays_usable(G):
     assert G.rel_l2(got, O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape))) <= 1e-2
 
 
+def test_the_scan_kernel_leaves_through_its_abort_path_when_its_prep_never_comes(G):
+    """The tensor-core scan itself: with the prep role withheld, its load warps wait (bounded, 2 s) for flags nothing raises; the
+    whole pipeline -- 28 warps in six roles per CTA -- has to unwind through the abort flag, wait for its loads in flight and free
+    its TMEM.  The status comes back as DM_ERR_TIMEOUT, and the same call with the switch off is correct again."""
+    import time
+    import torch
+    from oracle import bimamba_oracle as O
+    from paper_2511_15927_b200 import binding as dm
+    shape = I.MixerShape(1, 9 * 128 + 5, 128, 2, 128, 4, 4)    # 10 chunks, 8 scan CTAs: the configuration that fuses the prep work
+    wf, wr = I.make_mixer_weights(shape, 4, I.BF16)
+    x = I.make_activations(shape, 4, I.BF16)
+    st = torch.cuda.current_stream().cuda_stream
+    dm.dm_check(st)
+    dm.dm_selftest_withhold_prep(True)
+    try:
+        t0 = time.time()
+        with pytest.raises(dm.DmError) as e:
+            G.run_forward(shape, I.BF16, wf, wr, x, chunk=128)
+        waited = time.time() - t0
+    finally:
+        dm.dm_selftest_withhold_prep(False)
+    assert e.value.status == dm.DM_ERR_TIMEOUT
+    assert 1.5 < waited < 20.0                                  # the waits' own limit, not a hang
+    dm.dm_check(st)
+    got = G.run_forward(shape, I.BF16, wf, wr, x, chunk=128)
+    assert G.rel_l2(got, O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape))) <= 1e-2
+
+
 def test_selftest_argument_checks(G):
     from paper_2511_15927_b200 import binding as dm
     before = dm.dm_kernel_launch_count()
