@@ -985,12 +985,16 @@ ssd_scan_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 constexpr int NLD = N + 8;             // row pitch (bf16) of the C', B' and state tiles: 16-byte rows, conflict-free ldmatrix
 constexpr int SLD = QB + 4;            // row pitch (fp32) of S
 constexpr int WTL = QB + 8;            // row pitch (bf16) of W
+// The tiles only the state update reads (B', w o x') come last: a launch that carries no state out of its single sub-chunk
+// (KEEP = false: the denoising passes of block decoding) asks for the bytes before them only.  The fp32 y tile reuses the
+// bytes of S and of the raw x rows, both dead once the conv and mask phase is over.
 template <int PP> struct BlockSmem {
     static constexpr int XLD = PP + 8;             // row pitch (bf16) of x' and w o x'
-    static constexpr size_t ct = 0, bt = ct + QB * NLD * 2, ht = bt + QB * NLD * 2, xt = ht + PP * NLD * 2, wxt = xt + QB * XLD * 2,
-                            wt = wxt + QB * XLD * 2, xr = wt + QB * WTL * 2, ys = xr + (QB + 4) * PP * 2, ss = ys + QB * PP * 4,
-                            lam = ss + QB * SLD * 4, total = lam + (2 * QB + 4) * 4;
-    static_assert(ht % 16 == 0 && xt % 16 == 0 && wxt % 16 == 0 && wt % 16 == 0 && xr % 16 == 0 && ys % 16 == 0 && ss % 16 == 0 && lam % 16 == 0, "16-byte tiles");
+    static constexpr size_t ct = 0, ht = ct + QB * NLD * 2, xt = ht + PP * NLD * 2, wt = xt + QB * XLD * 2, ss = wt + QB * WTL * 2,
+                            xr = ss + QB * SLD * 4, lam = xr + (QB + 4) * PP * 2, total_nokeep = lam + (2 * QB + 4) * 4,
+                            bt = total_nokeep, wxt = bt + QB * NLD * 2, total = wxt + QB * XLD * 2, ys = ss;
+    static_assert(ht % 16 == 0 && xt % 16 == 0 && wt % 16 == 0 && ss % 16 == 0 && xr % 16 == 0 && lam % 16 == 0 && bt % 16 == 0 && wxt % 16 == 0, "16-byte tiles");
+    static_assert(QB * PP * 4 <= lam - ss, "the y tile fits the bytes of S and the raw x rows");
 };
 __device__ __forceinline__ void ldmatrix_x4_t(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, const void *p) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(smem_u32(p)));
@@ -999,19 +1003,21 @@ __device__ __forceinline__ void ldmatrix_x2_t(uint32_t &r0, uint32_t &r1, const 
     asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(smem_u32(p)));
 }
 
-template <int PP>
-__global__ void __launch_bounds__(4 * PP, 3)
+// KEEP: the fp32 state lives in the accumulators (several sub-chunks, or a state to write out); without it the launch is a
+// single sub-chunk whose state nobody reads, the accumulators and the update's tiles are gone and more CTAs fit an SM.
+template <int PP, bool KEEP>
+__global__ void __launch_bounds__(4 * PP, (KEEP ? 192 : 256) / PP)
 ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __nv_bfloat16 *__restrict__ Cp, const float *__restrict__ Sb, int dir0) {
-    constexpr int NT = 4 * PP, U8 = PP / 8, MT = PP / 16, XLD = BlockSmem<PP>::XLD;
+    constexpr int NT = 4 * PP, U8 = PP / 8, MT = PP / 16, XLD = BlockSmem<PP>::XLD, CP2 = PP / 2;
     extern __shared__ __align__(16) uint8_t bsm[];
     __nv_bfloat16 (*Ct)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::ct);      // C' rows [i][n]
-    __nv_bfloat16 (*Bt)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::bt);      // B' rows [j][n]
+    __nv_bfloat16 (*Bt)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::bt);      // B' rows [j][n]               (KEEP only)
     __nv_bfloat16 (*Ht)[NLD] = reinterpret_cast<__nv_bfloat16 (*)[NLD]>(bsm + BlockSmem<PP>::ht);      // incoming state [p][n]
     __nv_bfloat16 (*Xt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::xt);      // x' [j][p]
-    __nv_bfloat16 (*WXt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::wxt);    // w_j x'_j [j][p]
+    __nv_bfloat16 (*WXt)[XLD] = reinterpret_cast<__nv_bfloat16 (*)[XLD]>(bsm + BlockSmem<PP>::wxt);    // w_j x'_j [j][p]              (KEEP only)
     __nv_bfloat16 (*Wt)[WTL] = reinterpret_cast<__nv_bfloat16 (*)[WTL]>(bsm + BlockSmem<PP>::wt);      // W [i][j]
     __nv_bfloat16 (*xr)[PP] = reinterpret_cast<__nv_bfloat16 (*)[PP]>(bsm + BlockSmem<PP>::xr);        // raw x rows and conv history
-    float (*ys)[PP] = reinterpret_cast<float (*)[PP]>(bsm + BlockSmem<PP>::ys);                        // the sub-chunk's y
+    float (*ys)[PP] = reinterpret_cast<float (*)[PP]>(bsm + BlockSmem<PP>::ys);                        // the sub-chunk's y (over S and the raw rows)
     float (*Ss)[SLD] = reinterpret_cast<float (*)[SLD]>(bsm + BlockSmem<PP>::ss);
     float *lam = reinterpret_cast<float *>(bsm + BlockSmem<PP>::lam), *lamp = lam + QB, *sc = lamp + QB;
 
@@ -1023,34 +1029,37 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
     const ScanDir &w = a.dir[dir];
     const __nv_bfloat16 *zx = a.zx + ((int64_t)(a.zx_tied ? 0 : dir) * a.B + b) * L * a.d_in_proj;
     const float *dA_head = a.dA + ((seq * a.H + h) * 2) * a.Lp;
-    const int nsub = (L + QB - 1) / QB, nsub_all = a.nch * PREP_PARTS;
+    const int nsub = KEEP ? (L + QB - 1) / QB : 1, nsub_all = a.nch * PREP_PARTS;
     const float Dh = (a.flags & DM_FLAG_D_SKIP) ? w.D[h] : 0.f;
     const bool norm_on = (a.flags & DM_FLAG_GATED_RMSNORM) != 0;
-    const bool keep_state = nsub > 1 || (!rev && a.ssm_out != nullptr);        // the fp32 state is carried in the accumulators
 
-    // per-thread constants: conv taps of channel tid % PP (wl[m] multiplies the row m steps back in time), norm weights of the epilogue's 8 channels
-    const int cch = tid % PP, crg = tid / PP;
-    float wl[4], cbias;
+    // per-thread constants: conv taps of the channel pair 2 cp2, 2 cp2 + 1 (wl2[m] multiplies the row m steps back in time; halved, the
+    // SiLU below wants v / 2), norm weights of the epilogue's 8 channels
+    const int cp2 = tid % CP2, rg = tid / CP2;         // conv: channel pair, group of four rows
+    f32x2 wl2[4], cb2;
     {
-        const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)(h * PP + cch) * k;
+        const __nv_bfloat16 *cw = static_cast<const __nv_bfloat16 *>(w.conv_w) + (int64_t)(h * PP + 2 * cp2) * k;
+        float w0[4], w1[4];
 #pragma unroll
-        for (int m = 0; m < 4; ++m) wl[m] = m < k ? __bfloat162float(cw[k - 1 - m]) : 0.f;
-        cbias = ((a.flags & DM_FLAG_CONV_BIAS) && w.conv_b) ? __bfloat162float(static_cast<const __nv_bfloat16 *>(w.conv_b)[h * PP + cch]) : 0.f;
+        for (int m = 0; m < 4; ++m) {
+            w0[m] = m < k ? 0.5f * __bfloat162float(cw[k - 1 - m]) : 0.f;
+            w1[m] = m < k ? 0.5f * __bfloat162float(cw[k + k - 1 - m]) : 0.f;
+            wl2[m] = pk2(w0[m], w1[m]);
+        }
+        const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
+        const __nv_bfloat16 *cb = static_cast<const __nv_bfloat16 *>(w.conv_b) + h * PP + 2 * cp2;
+        cb2 = has_bias ? pk2(0.5f * __bfloat162float(cb[0]), 0.5f * __bfloat162float(cb[1])) : pk2(0.f, 0.f);
     }
     const int ei = tid / U8, ec = (tid % U8) * 8;      // epilogue: token row of the sub-chunk, first of 8 channels
-    uint32_t nwp[4];                                   // norm weights of those channels as bf16 pairs (ones when the norm is off)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat16 *nwq = static_cast<const __nv_bfloat16 *>(w.norm_w) + h * PP + ec + 2 * e;
-        nwp[e] = (norm_on && w.norm_w) ? pack_bf16(__bfloat162float(nwq[0]), __bfloat162float(nwq[1])) : 0x3F803F80u;
-    }
+    uint4 nwp = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);      // norm weights of those channels as bf16 pairs (ones when the norm is off)
+    if (norm_on && w.norm_w) nwp = __ldg(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(w.norm_w) + h * PP + ec));
 
     // state accumulators: warp = channels [16 smt, +16) x states [64 snh, +64): tile t covers states 64 snh + 8 t .. + 7;
     // a thread holds rows p = 16 smt + gr (+8), columns n = 64 snh + 8 t + 2 qc (+1)
     const int smt = warp % MT, snh = warp / MT;
-    float hacc[8][4];
+    float hacc[KEEP ? 8 : 1][4];
     const float *h_in = (!rev && a.ssm_in) ? a.ssm_in + ((int64_t)b * a.H + h) * PP * a.Nr : nullptr;
-    if (keep_state) {
+    if constexpr (KEEP) {
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
             const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
@@ -1066,8 +1075,9 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
     for (int si = 0; si < nsub; ++si) {
         const int sub = rev ? nsub - 1 - si : si, r0 = sub * QB;
         const bool have_state = si > 0 || h_in != nullptr;
-        const bool need_update = si + 1 < nsub || (!rev && a.ssm_out != nullptr);
-        __syncthreads();                                   // the previous sub-chunk's readers are done with the tiles
+        const bool need_update = KEEP && (si + 1 < nsub || (!rev && a.ssm_out != nullptr));
+        const int nvalid = min(QB, L - r0);                // tokens of the sub-chunk inside the sequence
+        if (KEEP) __syncthreads();                         // the previous sub-chunk's readers are done with the tiles
         // ---- load
         if (tid < QB) {
             lam[tid] = dA_head[r0 + tid];
@@ -1089,12 +1099,15 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             }
             cp_async16(&xr[rr][c], src, nb);
         }
-        for (int u = tid; u < QB * (N / 8); u += NT) {
-            const int i = u / (N / 8), c = (u % (N / 8)) * 8;
-            const int64_t off = (seq * L + min(r0 + i, L - 1)) * N + c;
-            const uint32_t nb = r0 + i < L ? 16 : 0;
-            if (have_state) cp_async16(&Ct[i][c], Cp + off, nb);
-            if (need_update) cp_async16(&Bt[i][c], Bp + off, nb);
+        if (have_state || need_update) {
+            const __nv_bfloat16 *Cs = Cp + (seq * L + r0) * N, *Bs = Bp + (seq * L + r0) * N;
+            for (int u = tid; u < QB * (N / 8); u += NT) {
+                const int i = u / (N / 8), c = (u % (N / 8)) * 8;
+                const int off = min(i, nvalid - 1) * N + c;
+                const uint32_t nb = i < nvalid ? 16 : 0;
+                if (have_state) cp_async16(&Ct[i][c], Cs + off, nb);
+                if (need_update) cp_async16(&Bt[i][c], Bs + off, nb);
+            }
         }
         {
             const float *S = Sb + (seq * nsub_all + sub) * (QB * QB);
@@ -1114,7 +1127,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
                     }
                     *reinterpret_cast<uint4 *>(&Ht[p][n0]) = make_uint4(pack_bf16(v0.x, v0.y), pack_bf16(v0.z, v0.w), pack_bf16(v1.x, v1.y), pack_bf16(v1.z, v1.w));
                 }
-            } else {
+            } else if constexpr (KEEP) {
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {              // from the accumulators of the previous sub-chunk
                     const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
@@ -1125,31 +1138,48 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
         }
         // the gate's z (it holds SiLU(z): the in_proj epilogue applied it), fetched now so that its latency hides behind the products
         uint4 zv = make_uint4(0u, 0u, 0u, 0u);
-        if (r0 + ei < L) zv = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)(r0 + ei) * a.d_in_proj + h * PP + ec));
+        if (ei < nvalid) zv = __ldg(reinterpret_cast<const uint4 *>(zx + (int64_t)(r0 + ei) * a.d_in_proj + h * PP + ec));
         cp_async_wait_all();
         __syncthreads();
-        // ---- conv + SiLU: thread = channel cch, rows 8 crg .. 8 crg + 7;  mask: W from S
+        // ---- conv + SiLU: thread = channel pair cp2, four rows in time order with the three rows before them carried in registers
         const float lam_last = lam[rev ? 0 : QB - 1], lam0 = sc[0];      // rows past the end of the sequence have Delta = 0: Lambda stays put there
+        {
+            auto raw = [&](int rr) { return bf2_to_f2(*reinterpret_cast<const uint32_t *>(&xr[rr][2 * cp2])); };
+            const int i0 = 4 * rg;
+            // the raw row of chunk row i sits at xr[i + 3] (->) or xr[i] (<-); one step back in time is one row down (->) or up (<-)
+            f32x2 h1 = raw(rev ? i0 + 4 : i0 + 2), h2 = raw(rev ? i0 + 5 : i0 + 1), h3 = raw(rev ? i0 + 6 : i0);
 #pragma unroll
-        for (int ii = 0; ii < QB * PP / NT; ++ii) {
-            const int i = crg * (QB * PP / NT) + ii;
-            float v = cbias;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) v = fmaf(wl[m], __bfloat162float(xr[rev ? i + m : i + 3 - m][cch]), v);
-            const float xv = v / (1.f + __expf(-v));
-            Xt[i][cch] = __float2bfloat16_rn(xv);
-            WXt[i][cch] = __float2bfloat16_rn(r0 + i < L ? ex2f(lam_last - lamp[i]) * xv : 0.f);
-        }
-        for (int e = tid; e < QB * QB / 2; e += NT) {
-            const int i = e / (QB / 2), j = (e % (QB / 2)) * 2;
-            float wv[2];
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int jj = j + q;
-                const bool ok = (rev ? jj >= i : jj <= i) && r0 + i < L && r0 + jj < L;
-                wv[q] = ok ? fmaf(Ss[i][jj], ex2f(lam[i] - lamp[jj]), i == jj ? Dh : 0.f) : 0.f;
+            for (int t = 0; t < 4; ++t) {
+                const int i = rev ? i0 + 3 - t : i0 + t;
+                const f32x2 cur = raw(rev ? i : i + 3);
+                f32x2 hh = fma2(wl2[3], h3, cb2);                   // half of the conv output
+                hh = fma2(wl2[2], h2, hh); hh = fma2(wl2[1], h1, hh); hh = fma2(wl2[0], cur, hh);
+                float ha, hb;
+                upk2(hh, ha, hb);
+                const f32x2 o = fma2(hh, pk2(tanh_fast(ha), tanh_fast(hb)), hh);      // SiLU(v) = v/2 + v/2 tanh(v/2)
+                *reinterpret_cast<uint32_t *>(&Xt[i][2 * cp2]) = f2_to_bf2(o);
+                if (need_update) {
+                    const float wj = i < nvalid ? ex2f(lam_last - lamp[i]) : 0.f;
+                    *reinterpret_cast<uint32_t *>(&WXt[i][2 * cp2]) = f2_to_bf2(mul2(o, pk2(wj, wj)));
+                }
+                h3 = h2; h2 = h1; h1 = cur;
             }
-            *reinterpret_cast<uint32_t *>(&Wt[i][j]) = pack_bf16(wv[0], wv[1]);
+        }
+        // ---- mask: W_ij = S_ij 2^(Lambda_i - Lambda'_j) [+ D on the diagonal] for j not after i in time and inside the sequence, else 0;
+        // thread = (row i, four columns)
+        for (int u = tid; u < QB * QB / 4; u += NT) {
+            const int i = u >> 3, j0 = (u & 7) * 4;
+            const float li = lam[i];
+            const float4 s4 = *reinterpret_cast<const float4 *>(&Ss[i][j0]), lp4 = *reinterpret_cast<const float4 *>(lamp + j0);
+            const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, lpv[4] = {lp4.x, lp4.y, lp4.z, lp4.w};
+            float wv[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int jj = j0 + q;
+                const bool ok = (rev ? jj >= i : jj <= i) && jj < nvalid;
+                wv[q] = fmaf(sv[q], ex2f(ok ? li - lpv[q] : -INFINITY), (ok && i == jj) ? Dh : 0.f);      // 2^-inf = 0: no branch around the exponential
+            }
+            *reinterpret_cast<uint2 *>(&Wt[i][j0]) = make_uint2(pack_bf16(wv[0], wv[1]), pack_bf16(wv[2], wv[3]));
         }
         __syncthreads();
         // ---- y: warp = tokens [16 ymt, +16) x channels [16 ynh, +16)
@@ -1183,6 +1213,7 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
                     mma_bf16_16816(acc[nt], a0, a1, a2, a3, b0, b1);
                 }
             }
+            // S and the raw rows were last read before the barrier above: their bytes take y
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
                 const int col = 16 * ynh + 8 * nt + 2 * qc, row = 16 * ymt + gr;
@@ -1191,28 +1222,29 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             }
         }
         // ---- state after the sub-chunk: h <- dec h + (w o x')^T B'
-        if (need_update) {
-            const float dec = ex2f(lam_last - lam0);
+        if constexpr (KEEP) {
+            if (need_update) {
+                const float dec = ex2f(lam_last - lam0);
 #pragma unroll
-            for (int t = 0; t < 8; ++t) { hacc[t][0] *= dec; hacc[t][1] *= dec; hacc[t][2] *= dec; hacc[t][3] *= dec; }
+                for (int t = 0; t < 8; ++t) { hacc[t][0] *= dec; hacc[t][1] *= dec; hacc[t][2] *= dec; hacc[t][3] *= dec; }
 #pragma unroll
-            for (int k0 = 0; k0 < QB; k0 += 16) {
-                uint32_t a0, a1, a2, a3;                    // A = (w o x')^T [p][j] read transposed from [j][p]
-                ldmatrix_x4_t(a0, a1, a2, a3, &WXt[k0 + (lane & 7) + ((lane >> 4) & 1) * 8][16 * smt + ((lane >> 3) & 1) * 8]);
+                for (int k0 = 0; k0 < QB; k0 += 16) {
+                    uint32_t a0, a1, a2, a3;                    // A = (w o x')^T [p][j] read transposed from [j][p]
+                    ldmatrix_x4_t(a0, a1, a2, a3, &WXt[k0 + (lane & 7) + ((lane >> 4) & 1) * 8][16 * smt + ((lane >> 3) & 1) * 8]);
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    uint32_t b0, b1;                        // B = B' [j][n] read transposed
-                    ldmatrix_x2_t(b0, b1, &Bt[k0 + (lane & 15)][64 * snh + 8 * t]);
-                    mma_bf16_16816(hacc[t], a0, a1, a2, a3, b0, b1);
+                    for (int t = 0; t < 8; ++t) {
+                        uint32_t b0, b1;                        // B = B' [j][n] read transposed
+                        ldmatrix_x2_t(b0, b1, &Bt[k0 + (lane & 15)][64 * snh + 8 * t]);
+                        mma_bf16_16816(hacc[t], a0, a1, a2, a3, b0, b1);
+                    }
                 }
             }
         }
         __syncthreads();
         // ---- gate: thread = (token ei, channels ec .. ec + 7)
         {
-            const int row = r0 + ei;
             const float zf[8] = {bf16_lo(zv.x), bf16_hi(zv.x), bf16_lo(zv.y), bf16_hi(zv.y), bf16_lo(zv.z), bf16_hi(zv.z), bf16_lo(zv.w), bf16_hi(zv.w)};
-            const float nw[8] = {bf16_lo(nwp[0]), bf16_hi(nwp[0]), bf16_lo(nwp[1]), bf16_hi(nwp[1]), bf16_lo(nwp[2]), bf16_hi(nwp[2]), bf16_lo(nwp[3]), bf16_hi(nwp[3])};
+            const float nw[8] = {bf16_lo(nwp.x), bf16_hi(nwp.x), bf16_lo(nwp.y), bf16_hi(nwp.y), bf16_lo(nwp.z), bf16_hi(nwp.z), bf16_lo(nwp.w), bf16_hi(nwp.w)};
             const float4 y0 = *reinterpret_cast<const float4 *>(&ys[ei][ec]), y1 = *reinterpret_cast<const float4 *>(&ys[ei][ec + 4]);
             const float yv[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
             float g[8], ss = 0.f;
@@ -1220,21 +1252,23 @@ ssd_block_kernel(const SsdArgs a, const __nv_bfloat16 *__restrict__ Bp, const __
             for (int e = 0; e < 8; ++e) { g[e] = yv[e] * zf[e]; ss = fmaf(g[e], g[e], ss); g[e] *= nw[e]; }
 #pragma unroll
             for (int off = 1; off < U8; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-            if (row < L) {
-                *reinterpret_cast<uint4 *>(a.g + (seq * L + row) * a.d_inner + h * PP + ec) =
+            if (ei < nvalid) {
+                *reinterpret_cast<uint4 *>(a.g + (seq * L + r0 + ei) * a.d_inner + h * PP + ec) =
                     make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]), pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
-                if (a.ssq && ec == 0) a.ssq[(seq * L + row) * a.H + h] = ss;
+                if (a.ssq && ec == 0) a.ssq[(seq * L + r0 + ei) * a.H + h] = ss;
             }
         }
     }
-    if (!rev && a.ssm_out) {
-        float *ho = a.ssm_out + ((int64_t)b * a.H + h) * PP * a.Nr;
+    if constexpr (KEEP) {
+        if (!rev && a.ssm_out) {
+            float *ho = a.ssm_out + ((int64_t)b * a.H + h) * PP * a.Nr;
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
-            if (n < a.Nr) {
-                *reinterpret_cast<float2 *>(ho + (int64_t)p0 * a.Nr + n) = make_float2(hacc[t][0], hacc[t][1]);
-                *reinterpret_cast<float2 *>(ho + (int64_t)(p0 + 8) * a.Nr + n) = make_float2(hacc[t][2], hacc[t][3]);
+            for (int t = 0; t < 8; ++t) {
+                const int n = 64 * snh + 8 * t + 2 * qc, p0 = 16 * smt + gr;
+                if (n < a.Nr) {
+                    *reinterpret_cast<float2 *>(ho + (int64_t)p0 * a.Nr + n) = make_float2(hacc[t][0], hacc[t][1]);
+                    *reinterpret_cast<float2 *>(ho + (int64_t)(p0 + 8) * a.Nr + n) = make_float2(hacc[t][2], hacc[t][3]);
+                }
             }
         }
     }
@@ -1334,8 +1368,12 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (blk) {
-        auto kern = a.P == P ? ssd_block_kernel<P> : ssd_block_kernel<P / 2>;
-        const size_t smem = a.P == P ? BlockSmem<P>::total : BlockSmem<P / 2>::total;
+        // the state is carried in registers when there are several sub-chunks or someone reads it afterwards
+        const bool keep = a.L > QB || a.ssm_out != nullptr;
+        auto kern = a.P == P ? (keep ? ssd_block_kernel<P, true> : ssd_block_kernel<P, false>)
+                             : (keep ? ssd_block_kernel<P / 2, true> : ssd_block_kernel<P / 2, false>);
+        const size_t smem = a.P == P ? (keep ? BlockSmem<P>::total : BlockSmem<P>::total_nokeep)
+                                     : (keep ? BlockSmem<P / 2>::total : BlockSmem<P / 2>::total_nokeep);
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<dim3(a.H, ndir, a.B), 4 * a.P, smem, s>>>(k, Bp, Cp, Sb, dir0);
