@@ -139,7 +139,7 @@ static MixerWs mixer_ws(const dm_mixer_cfg *c, const Dims &m) {
     w.g = off;    off += align_up((size_t)2 * m.T * m.d_inner * m.es);
     w.ssq = off;  off += align_up((size_t)2 * m.T * m.H * sizeof(float));
     w.rstd = off; off += align_up((size_t)2 * m.T * sizeof(float));
-    w.ytmp = off; off += align_up((size_t)(m.T <= PAIR_OUT_MAX_T ? 2 : 1) * m.T * m.d * sizeof(float));      // short inputs: one fp32 partial per direction
+    w.ytmp = off; off += align_up((size_t)(m.T <= PAIR_OUT_MAX_T ? 4 : 1) * m.T * m.d * sizeof(float));      // short inputs: up to two fp32 partials per direction
     ScanArgs sa{};
     sa.B = m.B; sa.L = m.L; sa.d_inner = m.d_inner; sa.H = m.H; sa.P = m.P; sa.N = m.N; sa.k = m.k;
     sa.d_in_proj = m.ldz; sa.conv_ch = m.conv_ch; sa.dtype = c->dtype; sa.flags = c->flags; sa.dir_mask = c->dir_mask; sa.chunk = c->chunk;
@@ -159,6 +159,8 @@ static cudaError_t gemm(const GemmArgs &a, cudaStream_t s) {
 struct MixerOut {
     void *y; int y_dtype; const float *addend; int64_t ld_add;
     const float *col_scale = nullptr; int cs_rows = 0; int64_t ld_cs = 0;   // per-sequence gate on the mixer's output (App. A.1), or NULL
+    // The caller's next step is u = RMSNorm(y; next_norm_w): a mixer that sums its directions in a pass of its own applies it there and sets *next_done
+    const void *next_norm_w = nullptr; void *next_u = nullptr; float next_eps = 0.f; bool *next_done = nullptr;
 };
 
 // in_proj -> fused conv/scan/gate -> out_proj of both directions, summed (Sec. 3.2).
@@ -223,6 +225,36 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         e = conv_state_update(zx, conv_in, conv_out, c->dtype, m.B, m.L, m.k, m.d_inner, m.conv_ch, m.ldz, s);
         if (e != cudaSuccess) return cuda_fail(e, "conv_state_update");
     }
+    if (!tied && c->dir_mask == DM_DIR_BOTH && m.T <= PAIR_OUT_MAX_T && sum_partials_norm_supports(m.d)) {
+        // short inputs (block decoding): both out_proj in one launch, each into its own fp32 partial (gated by col_scale, not yet scaled by the
+        // gated norm); one pass then scales, sums, adds the residual and applies the caller's next norm
+        GemmArgs ga[2];
+        for (int dir = 0; dir < 2; ++dir) {
+            GemmArgs a{};
+            a.A = g + (size_t)dir * m.T * m.d_inner * m.es; a.lda = m.d_inner;
+            a.B = w[dir].w_out; a.ldb = m.d_inner;
+            a.in_dtype = c->dtype; a.M = (int)m.T; a.N = m.d; a.K = m.d_inner;
+            a.col_scale = out.col_scale; a.cs_rows = out.cs_rows; a.ld_cs = out.ld_cs;
+            a.C = ytmp + (size_t)dir * m.T * m.d; a.ldc = m.d; a.c_dtype = DM_F32;
+            ga[dir] = a;
+        }
+        if (gemm_tcgen05_pair_supports(ga[0], ga[1])) {
+            {
+                StageTimer tm(DM_STAGE_OUT_PROJ, s);
+                const size_t part = (size_t)m.T * m.d;
+                const bool split = gemm_tcgen05_pair_splitk_pays(ga[0], ga[1]);
+                e = split ? gemm_tcgen05_pair_splitk(ga[0], ga[1], ytmp + 2 * part, ytmp + 3 * part, s) : gemm_tcgen05_pair(ga[0], ga[1], s);
+                if (e != cudaSuccess) return cuda_fail(e, "out_proj");
+                const bool next = out.next_norm_w && out.next_u;
+                e = sum_partials_norm(ytmp, ytmp + part, split ? ytmp + 2 * part : nullptr, split ? ytmp + 3 * part : nullptr, norm_on ? ssq : nullptr, norm_on ? ssq + (size_t)m.T * m.H : nullptr, m.H, m.d_inner,
+                                      c->norm_eps, out.addend, out.ld_add, out.y, out.y_dtype, next ? out.next_norm_w : nullptr, next ? out.next_u : nullptr,
+                                      c->dtype, m.T, m.d, out.next_eps, s);
+                if (next && out.next_done) *out.next_done = true;
+            }
+            if (e != cudaSuccess) return cuda_fail(e, "out_proj sum");
+            return DM_OK;
+        }
+    }
     if (norm_on) {
         e = rstd_from_ssq(ssq, rstd, (int)(2 * m.T), m.H, m.d_inner, c->norm_eps, s);
         if (e != cudaSuccess) return cuda_fail(e, "rstd");
@@ -241,30 +273,6 @@ static int run_mixer(const dm_mixer_cfg *c, const Dims &m, const dm_dir_weights 
         a.C = out.y; a.ldc = m.d; a.c_dtype = out.y_dtype;
         if ((e = gemm(a, s)) != cudaSuccess) return cuda_fail(e, "out_proj");
         return DM_OK;
-    }
-    if (c->dir_mask == DM_DIR_BOTH && m.T <= PAIR_OUT_MAX_T && (m.T * m.d) % 4 == 0) {
-        // short inputs (block decoding): both out_proj in one launch, each into its own fp32 partial, then their sum
-        GemmArgs ga[2];
-        for (int dir = 0; dir < 2; ++dir) {
-            GemmArgs a{};
-            a.A = g + (size_t)dir * m.T * m.d_inner * m.es; a.lda = m.d_inner;
-            a.B = w[dir].w_out; a.ldb = m.d_inner;
-            a.in_dtype = c->dtype; a.M = (int)m.T; a.N = m.d; a.K = m.d_inner;
-            a.row_scale = norm_on ? rstd + (size_t)dir * m.T : nullptr;
-            if (dir == 0) { a.addend = out.addend; a.ld_add = out.ld_add; }
-            a.col_scale = out.col_scale; a.cs_rows = out.cs_rows; a.ld_cs = out.ld_cs;
-            a.C = ytmp + (size_t)dir * m.T * m.d; a.ldc = m.d; a.c_dtype = DM_F32;
-            ga[dir] = a;
-        }
-        if (gemm_tcgen05_pair_supports(ga[0], ga[1])) {
-            {
-                StageTimer tm(DM_STAGE_OUT_PROJ, s);
-                if ((e = gemm_tcgen05_pair(ga[0], ga[1], s)) != cudaSuccess) return cuda_fail(e, "out_proj");
-                e = add_partials(ytmp, ytmp + (size_t)m.T * m.d, out.y, out.y_dtype, (size_t)m.T * m.d, s);
-            }
-            if (e != cudaSuccess) return cuda_fail(e, "out_proj sum");
-            return DM_OK;
-        }
     }
     // out_proj of each direction; the second one adds the first (Mamba(x) = h-> + h<-)
     const float *carry = out.addend;
@@ -585,6 +593,7 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
     cudaError_t e;
 
     if ((e = embed_gather(weights->embed, dtype, tokens, r, (int)m.T, m.d, cfg->vocab, s)) != cudaSuccess) return cuda_fail(e, "embed");
+    bool u_ready = false;                         // u already holds the norm of r (applied by the previous layer's last pass)
     for (int i = 0; i < cfg->n_layers; ++i) {
         const dm_layer_weights &lw = weights->layers[i];
         MixerOut out{r, DM_F32, r, m.d};          // r <- r + Mamba(u): the residual add rides in the out_proj epilogue
@@ -594,8 +603,12 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
             if ((e = adaln_rows(r, mod + m.d, mod, ldm, u, dtype, (int)m.T, m.L, m.d, blk->ln_eps, s)) != cudaSuccess) return cuda_fail(e, "adaln");
             out.col_scale = mod + 2 * m.d; out.cs_rows = m.L; out.ld_cs = ldm;
         } else {
-            if ((e = rmsnorm_rows(r, lw.norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "rmsnorm");
+            if (!u_ready && (e = rmsnorm_rows(r, lw.norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "rmsnorm");
+            // what follows this layer's mixer is the next layer's (or the final) RMSNorm of r
+            out.next_norm_w = i + 1 < cfg->n_layers ? weights->layers[i + 1].norm_w : weights->final_norm_w;
+            out.next_u = u; out.next_eps = cfg->rms_eps; out.next_done = &u_ready;
         }
+        u_ready = false;
         if (period > 0 && i % period == 0) {
             // attention mixer (Sec. 3.3): r <- r + [gate *] Attn(u); gate and residual ride in the output projection's epilogue
             void *qkv = ws + l.qkv, *att = ws + l.att;
@@ -633,7 +646,7 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
             if ((e = gemm(dn, s)) != cudaSuccess) return cuda_fail(e, "mlp down");
         }
     }
-    if ((e = rmsnorm_rows(r, weights->final_norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "final norm");
+    if (!u_ready && (e = rmsnorm_rows(r, weights->final_norm_w, u, dtype, (int)m.T, m.d, cfg->rms_eps, s)) != cudaSuccess) return cuda_fail(e, "final norm");
     if (smp) {
         // Eq. 3: only the positions drawn this step go through the vocabulary projection; how many there are stays on the device
         int32_t *idx = reinterpret_cast<int32_t *>(ws + l.idx);

@@ -50,6 +50,10 @@ bool gemm_tcgen05_supports(const GemmArgs &a);
 // of each other: neither reads what the other writes.
 bool gemm_tcgen05_pair_supports(const GemmArgs &a, const GemmArgs &b);
 cudaError_t gemm_tcgen05_pair(const GemmArgs &a, const GemmArgs &b, cudaStream_t s);
+// The same pair with each product cut in two along K (fp32 outputs only): the first half of a's product goes to a.C (with its addend and bias),
+// the second half to a_hi (same pitch), likewise b; the caller adds the halves.  _pays: the shapes for which that fills the GPU better.
+bool gemm_tcgen05_pair_splitk_pays(const GemmArgs &a, const GemmArgs &b);
+cudaError_t gemm_tcgen05_pair_splitk(const GemmArgs &a, const GemmArgs &b, float *a_hi, float *b_hi, cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
 // Fused conv + SiLU + discretisation + selective scan + gate, both directions in one launch.
@@ -116,7 +120,12 @@ cudaError_t draw_rows(const void *logits, int64_t ld, int dtype, const int32_t *
 // out[t] = argmax_v logits[t, v], lowest index on ties
 cudaError_t argmax_rows(const void *logits, int dtype, int32_t *out, int T, int V, cudaStream_t s);
 // y[i] = (dtype) (a[i] + b[i])
-cudaError_t add_partials(const float *a, const float *b, void *y, int dtype, size_t n, cudaStream_t s);
+// y[t, :] = addend[t, :] + s0[t] (p0[t, :] + q0[t, :]) + s1[t] (p1[t, :] + q1[t, :])  (q0, q1: second halves of a product split along K, or NULL) with s_dir[t] = rsqrt(sum_h ssq_dir[t, h] / d_inner + eps_g) (1 when ssq_dir is NULL);
+// u != NULL: also u[t, :] = w * y[t, :] * rsqrt(mean(y[t, :]^2) + eps).  One block per token; sum_partials_norm_supports(d) says whether d fits.
+bool sum_partials_norm_supports(int d);
+cudaError_t sum_partials_norm(const float *p0, const float *p1, const float *q0, const float *q1, const float *ssq0, const float *ssq1, int H, int d_inner, float eps_g,
+                              const float *addend, int64_t ld_add, void *y, int y_dtype, const void *w, void *u, int u_dtype, int64_t T, int d,
+                              float eps, cudaStream_t s);
 // Tied projections: g0[t, :] = s0[t] * g0[t, :] + s1[t] * g1[t, :]  (s = rstd of each direction, or 1 when rstd is NULL), in place over g0
 cudaError_t combine_directions(void *g0, const void *g1, const float *rstd0, const float *rstd1, int dtype, int64_t T, int d_inner, cudaStream_t s);
 // conv_out[b] = last k-1 rows of concat(conv_in[b] (or zeros), xBC columns of zx[b, 0..L-1])

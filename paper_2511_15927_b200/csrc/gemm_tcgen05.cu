@@ -17,11 +17,14 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BK = 64;
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 6;
+// pipeline depth: as many (A, B) stages as shared memory holds -- 4 x 48 KB with 256-column tiles, 6 x 32 KB with 128-column tiles (whose
+// lower arithmetic intensity needs more bytes in flight per MMA clock)
+__host__ __device__ constexpr int stages_for(int bn) { return bn == 128 ? 6 : 4; }
 constexpr int NUM_THREADS = 192;
 
 struct __align__(8) PipeBars {
-    uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort;
 };
@@ -34,11 +37,13 @@ struct EpiArgs {
     const float *col_bias; int gelu; const float *col_scale; int cs_rows; int64_t ld_cs;   // see GemmArgs
     const int *m_dev; int m_off;
     int n_fast;      // tile order: consecutive tiles step along N (the A rows are streamed once, B stays in L2) or along M
+    int k_off;       // first element along K of this problem's share (split K: the second half of a product is a problem of its own)
 };
 
-// Up to two problems of the same M, N, K in one launch (the two directions' in_proj, or their out_proj on short inputs): the tile
+// Up to two products of the same M, N, K in one launch (the two directions' in_proj, or their out_proj on short inputs), each optionally
+// cut in two along K (ksplit: problems 2 i and 2 i + 1 are the halves of product i, each with an output of its own that the caller adds): the tile
 // loop runs over both, so that they share one tail round and -- for in_proj, whose A operand is the same x -- the rows of A in L2.
-struct EpiPair { EpiArgs p[2]; int nprob; };
+struct EpiPair { EpiArgs p[4]; int nprob; int ksplit; };
 
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -49,6 +54,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    constexpr int STAGES = stages_for(BN);
     constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
     PipeBars *bars = reinterpret_cast<PipeBars *>(smem + STAGES * STAGE_BYTES);
     volatile int *abort_flag = &bars->abort;
@@ -87,14 +93,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int cb = tile_cb(tile), prob = cb / tiles_n;
                 const int m0 = tile_mb(tile) * BM, n0 = (cb - prob * tiles_n) * BN;
-                const CUtensorMap *ma = prob ? &map_a1 : &map_a0, *mb = prob ? &map_b1 : &map_b0;
+                const int prod = epp.ksplit ? prob >> 1 : prob, k_off = epp.p[prob].k_off;
+                const CUtensorMap *ma = prod ? &map_a1 : &map_a0, *mb = prod ? &map_b1 : &map_b0;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!(ok = mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, status))) break;
                     uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_BYTES;
                     mbar_expect_tx(&bars->full[s], STAGE_BYTES);
-                    tma_load_2d(sa, ma, kb * BK, m0, &bars->full[s]);
-                    tma_load_2d(sb, mb, kb * BK, n0, &bars->full[s]);
+                    tma_load_2d(sa, ma, k_off + kb * BK, m0, &bars->full[s]);
+                    tma_load_2d(sb, mb, k_off + kb * BK, n0, &bars->full[s]);
                 }
             }
             if (!ok) {
@@ -282,25 +289,38 @@ bool make_map(CUtensorMap *m, const void *base, int64_t rows, int64_t cols, int6
 EpiArgs epi_of(const GemmArgs &a) {
     // The operand with more rows is streamed from HBM once; the other one is re-read by every wave of CTAs and should stay in L2.
     return EpiArgs{a.C, a.ldc, a.c_dtype == DM_F32 ? 1 : 0, a.row_scale, a.addend, a.ld_add, a.M, a.N, a.K, a.silu_cols,
-                   a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.m_dev, a.m_off, a.M > a.N ? 1 : 0};
+                   a.col_bias, a.gelu, a.col_scale, a.cs_rows > 0 ? a.cs_rows : 1, a.ld_cs > 0 ? a.ld_cs : (int64_t)a.N, a.m_dev, a.m_off, a.M > a.N ? 1 : 0, 0};
 }
 
-// b == NULL: one problem
+// b == NULL: one product.  hi != NULL (two products, fp32 outputs): each product is cut in two along K; the first half goes to the
+// product's own C with its addend and bias, the second half to hi[i] (same pitch), scaled like the first (the scales are linear).
 template <int BN>
-cudaError_t launch(const GemmArgs &a, const GemmArgs *b, cudaStream_t s) {
+cudaError_t launch(const GemmArgs &a, const GemmArgs *b, float *const *hi, cudaStream_t s) {
     CUtensorMap ma[2], mb[2];
     if (!make_map(&ma[0], a.A, a.M, a.K, a.lda, BM) || !make_map(&mb[0], a.B, a.N, a.K, a.ldb, BN)) return cudaErrorInvalidValue;
     ma[1] = ma[0]; mb[1] = mb[0];
     if (b && (!make_map(&ma[1], b->A, b->M, b->K, b->lda, BM) || !make_map(&mb[1], b->B, b->N, b->K, b->ldb, BN))) return cudaErrorInvalidValue;
-    constexpr size_t smem = STAGES * (size_t)(BM * BK * 2 + BN * BK * 2) + sizeof(PipeBars) + 1024;
+    constexpr size_t smem = stages_for(BN) * (size_t)(BM * BK * 2 + BN * BK * 2) + sizeof(PipeBars) + 1024;
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
     EpiPair epp{};
-    epp.p[0] = epi_of(a);
-    epp.p[1] = b ? epi_of(*b) : epp.p[0];
-    epp.nprob = b ? 2 : 1;
+    if (hi) {
+        const GemmArgs *prod[2] = {&a, b};
+        for (int i = 0; i < 2; ++i) {
+            EpiArgs lo = epi_of(*prod[i]), up = lo;
+            lo.K = up.K = prod[i]->K / 2;
+            up.k_off = lo.K;
+            up.C = hi[i]; up.addend = nullptr; up.col_bias = nullptr;
+            epp.p[2 * i] = lo; epp.p[2 * i + 1] = up;
+        }
+        epp.nprob = 4; epp.ksplit = 1;
+    } else {
+        epp.p[0] = epi_of(a);
+        epp.p[1] = b ? epi_of(*b) : epp.p[0];
+        epp.nprob = b ? 2 : 1;
+    }
     const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * epp.nprob;
     const int grid = tiles < sm_count() ? tiles : sm_count();
     gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma[0], mb[0], ma[1], mb[1], epp, status);
@@ -332,7 +352,7 @@ bool gemm_tcgen05_supports(const GemmArgs &a) {
 
 cudaError_t gemm_tcgen05(const GemmArgs &a, cudaStream_t s) {
     if (!gemm_tcgen05_supports(a)) return cudaErrorNotSupported;
-    return wide_tile(a, 1) ? launch<256>(a, nullptr, s) : launch<128>(a, nullptr, s);
+    return wide_tile(a, 1) ? launch<256>(a, nullptr, nullptr, s) : launch<128>(a, nullptr, nullptr, s);
 }
 
 bool gemm_tcgen05_pair_supports(const GemmArgs &a, const GemmArgs &b) {
@@ -342,7 +362,23 @@ bool gemm_tcgen05_pair_supports(const GemmArgs &a, const GemmArgs &b) {
 
 cudaError_t gemm_tcgen05_pair(const GemmArgs &a, const GemmArgs &b, cudaStream_t s) {
     if (!gemm_tcgen05_pair_supports(a, b)) return cudaErrorNotSupported;
-    return wide_tile(a, 2) ? launch<256>(a, &b, s) : launch<128>(a, &b, s);
+    return wide_tile(a, 2) ? launch<256>(a, &b, nullptr, s) : launch<128>(a, &b, nullptr, s);
+}
+
+// Few rows and a long K (the out_proj pair of block decoding): two products of 128 x 256 tiles fill less than half of the SMs, and 128 x 128
+// tiles run their MMAs at about half rate (their operand traffic per product is twice that of the wide tile).  Halving K instead doubles
+// the number of wide tiles.
+bool gemm_tcgen05_pair_splitk_pays(const GemmArgs &a, const GemmArgs &b) {
+    if (!gemm_tcgen05_pair_supports(a, b) || a.c_dtype != DM_F32 || a.K % (2 * BK) || a.gelu || b.gelu || a.silu_cols || b.silu_cols) return false;
+    const int tiles = ((a.M + BM - 1) / BM) * ((a.N + 255) / 256) * 2;
+    return a.N > 128 && 2 * tiles <= sm_count();
+}
+
+cudaError_t gemm_tcgen05_pair_splitk(const GemmArgs &a, const GemmArgs &b, float *a_hi, float *b_hi, cudaStream_t s) {
+    if (!gemm_tcgen05_pair_splitk_pays(a, b) || !a_hi || !b_hi || ((reinterpret_cast<uintptr_t>(a_hi) | reinterpret_cast<uintptr_t>(b_hi)) & 15u))
+        return cudaErrorNotSupported;
+    float *const hi[2] = {a_hi, b_hi};
+    return launch<256>(a, &b, hi, s);
 }
 
 }  // namespace dm

@@ -207,11 +207,58 @@ __global__ void conv_state_kernel(const T *__restrict__ zx, const T *__restrict_
     conv_out[((int64_t)b * (k - 1) + r) * conv_ch + c] = v;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(256) add_partials_kernel(const float *__restrict__ a, const float *__restrict__ b, T *__restrict__ y, size_t n4) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
-        const float4 u = __ldg(reinterpret_cast<const float4 *>(a) + i), v = __ldg(reinterpret_cast<const float4 *>(b) + i);
-        st4(y + 4 * i, u.x + v.x, u.y + v.y, u.z + v.z, u.w + v.w);
+// Short inputs (block decoding), one block of threads per token: the two directions' out_proj partials are summed with the gated norm's
+// row scale of each direction applied here (the scale of a row commutes with the projection: Mamba(x) = s-> (g-> W->^T) + s<- (g<- W<-^T),
+// Sec. 3.2), the residual is added, and -- when the caller's next step is an RMSNorm of the result -- that norm is applied to the row
+// while it is still in registers.  ssq0/ssq1 = per-head sums of squares of the directions' gated outputs (NULL: no gated norm);
+// q0, q1 = the second halves of the partials when the products were split along K (both or neither); addend may alias y; u = NULL: no norm.  Needs d % 4 == 0 and d <= 4 * ROW_THREADS * ROW_K.
+template <typename TY, typename TU>
+__global__ void __launch_bounds__(ROW_THREADS)
+sum_partials_norm_kernel(const float *__restrict__ p0, const float *__restrict__ p1, const float *__restrict__ q0, const float *__restrict__ q1,
+                         const float *__restrict__ ssq0, const float *__restrict__ ssq1,
+                         int H, float inv_n, float eps_g, const float *addend, int64_t ld_add, TY *y, const TU *__restrict__ w, TU *__restrict__ u,
+                         int d, float eps) {
+    __shared__ float red[32];
+    __shared__ float sc[2];
+    const int64_t t = blockIdx.x;
+    if (threadIdx.x < 64) {                      // warps 0 and 1: the two directions' scales, summed in the order of rstd_kernel
+        const int dir = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        const float *q = dir ? ssq1 : ssq0;
+        float v = 0.f;
+        if (q) for (int h = lane; h < H; h += 32) v += q[t * H + h];
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (lane == 0) sc[dir] = q ? rsqrtf(v * inv_n + eps_g) : 1.f;
+    }
+    __syncthreads();
+    const float s0 = sc[0], s1 = sc[1];
+    float4 v[ROW_K];
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < ROW_K; ++k) {
+        const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < d) {
+            float4 a = __ldg(reinterpret_cast<const float4 *>(p0 + t * d + c)), b = __ldg(reinterpret_cast<const float4 *>(p1 + t * d + c));
+            if (q0) {                            // products split along K: the second halves
+                const float4 a2 = __ldg(reinterpret_cast<const float4 *>(q0 + t * d + c)), b2 = __ldg(reinterpret_cast<const float4 *>(q1 + t * d + c));
+                a.x += a2.x; a.y += a2.y; a.z += a2.z; a.w += a2.w;
+                b.x += b2.x; b.y += b2.y; b.z += b2.z; b.w += b2.w;
+            }
+            float4 r = addend ? *reinterpret_cast<const float4 *>(addend + t * ld_add + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            r.x = fmaf(s1, b.x, fmaf(s0, a.x, r.x)); r.y = fmaf(s1, b.y, fmaf(s0, a.y, r.y));
+            r.z = fmaf(s1, b.z, fmaf(s0, a.z, r.z)); r.w = fmaf(s1, b.w, fmaf(s0, a.w, r.w));
+            st4(y + t * d + c, r.x, r.y, r.z, r.w);
+            v[k] = r;
+            ss = fmaf(r.x, r.x, ss); ss = fmaf(r.y, r.y, ss); ss = fmaf(r.z, r.z, ss); ss = fmaf(r.w, r.w, ss);
+        }
+    }
+    if (!u) return;
+    ss = block_sum(ss, red);
+    const float rs = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+    for (int k = 0; k < ROW_K; ++k) {
+        const int c = 4 * (threadIdx.x + ROW_THREADS * k);
+        if (c < d) st4(u + t * d + c, v[k].x * rs * ldf(w + c), v[k].y * rs * ldf(w + c + 1), v[k].z * rs * ldf(w + c + 2), v[k].w * rs * ldf(w + c + 3));
     }
 }
 
@@ -308,12 +355,19 @@ cudaError_t conv_state_update(const void *zx_fwd, const void *conv_in, void *con
     return cudaGetLastError();
 }
 
-cudaError_t add_partials(const float *a, const float *b, void *y, int dtype, size_t n, cudaStream_t s) {
-    if (n % 4) return cudaErrorInvalidValue;
-    const size_t n4 = n / 4;
-    const int blocks = (int)((n4 + 255) / 256 > 148 * 8 ? 148 * 8 : (n4 + 255) / 256);
-    if (dtype == DM_BF16) add_partials_kernel<<<blocks, 256, 0, s>>>(a, b, static_cast<__nv_bfloat16 *>(y), n4);
-    else add_partials_kernel<<<blocks, 256, 0, s>>>(a, b, static_cast<float *>(y), n4);
+bool sum_partials_norm_supports(int d) { return d % 4 == 0 && d <= 4 * ROW_THREADS * ROW_K; }
+
+cudaError_t sum_partials_norm(const float *p0, const float *p1, const float *q0, const float *q1, const float *ssq0, const float *ssq1, int H, int d_inner, float eps_g,
+                              const float *addend, int64_t ld_add, void *y, int y_dtype, const void *w, void *u, int u_dtype, int64_t T, int d,
+                              float eps, cudaStream_t s) {
+    if (!sum_partials_norm_supports(d) || (q0 == nullptr) != (q1 == nullptr)) return cudaErrorInvalidValue;
+    const float inv_n = 1.f / (float)d_inner;
+    const int grid = (int)T;
+#define DM_SPN(TY, TU) sum_partials_norm_kernel<TY, TU><<<grid, ROW_THREADS, 0, s>>>(p0, p1, q0, q1, ssq0, ssq1, H, inv_n, eps_g, addend, ld_add, \
+        static_cast<TY *>(y), static_cast<const TU *>(w), static_cast<TU *>(u), d, eps)
+    if (y_dtype == DM_F32) { if (u_dtype == DM_BF16) DM_SPN(float, __nv_bfloat16); else DM_SPN(float, float); }
+    else { if (u_dtype == DM_BF16) DM_SPN(__nv_bfloat16, __nv_bfloat16); else DM_SPN(__nv_bfloat16, float); }
+#undef DM_SPN
     count_launch();
     return cudaGetLastError();
 }
