@@ -246,6 +246,9 @@ STACKS = {
     # B = 8, L = 1024 throughput point (App. D): one reverse step with p = 16 tokens drawn per sequence, K = L / 16 steps per generation
     "paper_b8_1k_sample": dict(shape=I.MixerShape(8, 1024, 1920, 2, 128, 4, 120), layers=24, vocab=50304,
                                cond=dict(d_ff=3840, d_cond=128), sample=dict(p=16)),
+    # the paper's 1.3B hybrid (Sec. 3.3, App. A.3: the same blocks with an attention mixer of 24 heads x 80 channels in every fifth layer)
+    "paper_b8_1k_hybrid": dict(shape=I.MixerShape(8, 1024, 1920, 2, 128, 4, 120), layers=24, vocab=50304,
+                               cond=dict(d_ff=3840, d_cond=128), hybrid=dict(period=5, heads=24)),
     "cfg2_stack_cond": dict(shape=I.MixerShape(4, 4096, 1024, 2, 16, 4, 32), layers=24, vocab=50304, cond=dict(d_ff=2048, d_cond=128)),
     # block-autoregressive decoding as stated: a 2048-token prefix committed once, then 64 blocks of 32 tokens, each with 8 denoising
     # passes that read the carried state and one commit pass that writes the next block's state (ping-pong); step = one block
@@ -566,8 +569,8 @@ def run_stack(args, rank, local_rank, world):
                             "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T * npass / (ms_step * 1e-3),
                             "parallelism": "replicas only" if world > 1 else "1 GPU",
                             "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
-                           **({"hybrid": "attention mixer (%d heads of 64) in every %dth layer, %d Mamba layers; the attention layers are inside rest_of_step_ms"
-                                         % (hyb["heads"], hyb["period"], n_mamba)} if hyb else {}),
+                           **({"hybrid": "attention mixer (%d heads of %d) in every %dth layer, %d Mamba layers; the attention layers are inside rest_of_step_ms"
+                                         % (hyb["heads"], shape.d_model // hyb["heads"], hyb["period"], n_mamba)} if hyb else {}),
                            **({"sample": "half of the positions masked, p = %d drawn per sequence and step" % smp["p"],
                                "generated_tokens_per_s_at_K_eq_L_over_p": world * T / ((Lb // smp["p"]) * ms_step * 1e-3)} if smp else {}),
                            **({"loop": "step = one block of %d tokens per sequence: %d denoising passes reading the carried state + 1 commit pass; "

@@ -252,8 +252,8 @@ int dm_generate(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const dm_stack
  * (bidirectional, unmasked) multi-head self-attention over each sequence, no position encoding,
  *     y = concat_h softmax(Q_h K_h^T / sqrt(d_h)) V_h  W_o^T,   [Q | K | V] = x W_qkv^T.
  * x, y [B, L, d_model] dtype (y != x); w_qkv [3 * d_model, d_model] with rows [Q | K | V], each split into
- * n_heads consecutive blocks of d_h = d_model / n_heads; w_o [d_model, d_model].  bf16 only, d_h = 64 only
- * (DM_ERR_UNSUPPORTED otherwise).  The scores never leave the SM (running-maximum softmax over key tiles);
+ * n_heads consecutive blocks of d_h = d_model / n_heads; w_o [d_model, d_model].  bf16 only, d_h = 64 or 80 (the
+ * paper's 1.3B hybrid: 24 heads at d_model = 1920) only (DM_ERR_UNSUPPORTED otherwise).  The scores never leave the SM (running-maximum softmax over key tiles);
  * P is rounded to bf16 before P V, accumulation is fp32.  The hybrid stack (which layers are attention) is
  * dm_denoise_step_hybrid below. */
 int dm_attention_workspace_bytes(int32_t batch, int32_t seqlen, int32_t d_model, int32_t dtype, size_t *bytes);
@@ -267,10 +267,10 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
  * the RMSNorm pre-norm + residual of dm_denoise_step (blk == NULL) or the timestep-conditioned block of
  * dm_denoise_step_cond (blk, block_weights, tau given).  attn_weights: HOST array of cfg->n_layers entries, read
  * only where the layer is attention (the Mamba weights of those layers are not read).  Full-sequence mode; block
- * mode is dm_denoise_step_hybrid_block.  bf16, attention heads of width 64. */
+ * mode is dm_denoise_step_hybrid_block.  bf16, attention heads of width 64 or 80. */
 typedef struct {
     int32_t attn_period;   /* N: layers 0, N, 2N, ... are attention; 0 = none */
-    int32_t attn_heads;    /* d_model = 64 * attn_heads */
+    int32_t attn_heads;    /* d_model = 64 * attn_heads or 80 * attn_heads */
 } dm_hybrid_cfg;
 typedef struct {
     const void *w_qkv;     /* [3 * d_model, d_model] dtype, rows [Q | K | V] */

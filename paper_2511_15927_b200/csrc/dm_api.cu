@@ -561,8 +561,8 @@ static int denoise_impl(const dm_stack_cfg *cfg, const dm_block_cfg *blk, const 
                         return fail(DM_ERR_INVALID_ARG, "layer %d: key/value caches must be non-NULL and 16-byte aligned", i);
                     if (q.len < 0 || q.len + m.L > q.cap) return fail(DM_ERR_INVALID_ARG, "layer %d: cache length + block length exceeds its capacity", i);
                 }
-            if (hyb->cfg->attn_heads <= 0 || m.d != 64 * hyb->cfg->attn_heads || !attention_supports(cfg->mixer.dtype, m.d, hyb->cfg->attn_heads))
-                return fail(DM_ERR_UNSUPPORTED, "attention layers need bf16 and heads of width 64 (d_model = 64 * attn_heads)");
+            if (hyb->cfg->attn_heads <= 0 || !attention_supports(cfg->mixer.dtype, m.d, hyb->cfg->attn_heads))
+                return fail(DM_ERR_UNSUPPORTED, "attention layers need bf16 and heads of width 64 or 80 (d_model = 64 or 80 * attn_heads)");
             for (int i = 0; i < cfg->n_layers; i += period)
                 if (!hyb->aw[i].w_qkv || !hyb->aw[i].w_o || !aligned16(hyb->aw[i].w_qkv) || !aligned16(hyb->aw[i].w_o))
                     return fail(DM_ERR_INVALID_ARG, "layer %d: attention weights must be non-NULL and 16-byte aligned", i);
@@ -814,7 +814,8 @@ int dm_attention_block_step(int32_t batch, int32_t block_len, int32_t d_model, i
     if (x_blk == y_blk) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
     if (!aligned16(w_qkv) || !aligned16(w_o) || !aligned16(x_blk) || !aligned16(y_blk) || !aligned16(k_cache) || !aligned16(v_cache))
         return fail(DM_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
-    if (n_heads <= 0 || d_model != n_heads * 64) return fail(DM_ERR_UNSUPPORTED, "the attention mixer needs heads of width 64 (d_model = 64 * n_heads)");
+    if (n_heads <= 0 || (d_model != n_heads * 64 && d_model != n_heads * 80))
+        return fail(DM_ERR_UNSUPPORTED, "the attention mixer needs heads of width 64 or 80 (d_model = 64 or 80 * n_heads)");
     if (batch > 65535 || n_heads > 65535) return fail(DM_ERR_UNSUPPORTED, "batch and n_heads must be below 65536");
     if (cache_len < 0 || cache_len + block_len > cache_cap) return fail(DM_ERR_INVALID_ARG, "cache length + block length exceeds the cache's capacity");
     if (!attention_supports(dtype, d_model, n_heads)) return fail(DM_ERR_UNSUPPORTED, "the attention mixer is not available for this configuration");
@@ -852,7 +853,8 @@ int dm_attention_forward(int32_t batch, int32_t seqlen, int32_t d_model, int32_t
     if (!w_qkv || !w_o || !x || !y) return fail(DM_ERR_INVALID_ARG, "NULL pointer");
     if (x == y) return fail(DM_ERR_INVALID_ARG, "y must not alias x");
     if (!aligned16(w_qkv) || !aligned16(w_o) || !aligned16(x) || !aligned16(y)) return fail(DM_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
-    if (n_heads <= 0 || d_model != n_heads * 64) return fail(DM_ERR_UNSUPPORTED, "the attention mixer needs heads of width 64 (d_model = 64 * n_heads)");
+    if (n_heads <= 0 || (d_model != n_heads * 64 && d_model != n_heads * 80))
+        return fail(DM_ERR_UNSUPPORTED, "the attention mixer needs heads of width 64 or 80 (d_model = 64 or 80 * n_heads)");
     if (batch > 65535 || n_heads > 65535) return fail(DM_ERR_UNSUPPORTED, "batch and n_heads must be below 65536");
     if (!attention_supports(dtype, d_model, n_heads)) return fail(DM_ERR_UNSUPPORTED, "the attention mixer is not available for this configuration");
     if ((st = check_ws(workspace, workspace_bytes, need)) != DM_OK) return st;

@@ -32,8 +32,8 @@ def _run(G, x, w_qkv, w_o, H):
     return yd.float().cpu().numpy().astype(np.float64)
 
 
-def _case(B, L, H, seed, w_scale):
-    d = 64 * H
+def _case(B, L, H, seed, w_scale, dh=64):
+    d = dh * H
     r = np.random.default_rng(seed)
     x = I.round_to_bf16(r.standard_normal((B, L, d), dtype=np.float32))
     w_qkv = I.round_to_bf16((w_scale / np.sqrt(d)) * r.standard_normal((3 * d, d), dtype=np.float32))
@@ -60,6 +60,27 @@ def test_flat_and_peaked_scores_many_heads(G, w_scale):
     x, wq, wo = _case(3, 400, 8, 11, w_scale)
     got = _run(G, x, wq, wo, 8)
     want = O.attention_mixer(x, wq, wo, 8)
+    assert np.all(np.isfinite(got))
+    assert G.rel_l2(got, want) <= BF16_REL, G.rel_l2(got, want)
+    assert G.max_abs(got, want) <= BF16_ABS * max(1.0, np.abs(want).max()), G.max_abs(got, want)
+
+
+@pytest.mark.parametrize("L", [5, 129, 300, 1000])
+def test_heads_of_80_channels(G, L):
+    """The head width of the paper's 1.3B hybrid (d_model 1920 = 24 heads of 80): three heads, so that the first, a middle and the
+    last head (whose second sub-tile runs past the end of the row) are all there."""
+    x, wq, wo = _case(2, L, 3, 40 + L, 1.0, dh=80)
+    got = _run(G, x, wq, wo, 3)
+    want = O.attention_mixer(x, wq, wo, 3)
+    assert np.all(np.isfinite(got))
+    assert G.rel_l2(got, want) <= BF16_REL, G.rel_l2(got, want)
+    assert G.max_abs(got, want) <= BF16_ABS, G.max_abs(got, want)
+
+
+def test_heads_of_80_channels_peaked_scores(G):
+    x, wq, wo = _case(2, 400, 6, 17, 2.0, dh=80)
+    got = _run(G, x, wq, wo, 6)
+    want = O.attention_mixer(x, wq, wo, 6)
     assert np.all(np.isfinite(got))
     assert G.rel_l2(got, want) <= BF16_REL, G.rel_l2(got, want)
     assert G.max_abs(got, want) <= BF16_ABS * max(1.0, np.abs(want).max()), G.max_abs(got, want)
@@ -99,6 +120,18 @@ def _hybrid_stack(shape, layers, V, seed, cond):
     return sw, tau, d_ff
 
 
+def test_hybrid_stack_with_heads_of_80(G):
+    """d_model 160 = 2 attention heads of 80 beside Mamba layers of 5 heads x 64 channels."""
+    shape = I.MixerShape(2, 150, 160, 2, 128, 4, 5)
+    V = 504
+    sw, tau, d_ff = _hybrid_stack(shape, 4, V, 23, False)
+    tok = I.make_tokens(2, 150, V - 1, V - 1, seed=23)
+    want = O.denoise_step_hybrid(tok, sw, attn_period=3, attn_heads=2, tau=tau, **G.oracle_kwargs(shape))
+    got = G.run_denoise_hybrid(shape, I.BF16, sw, tok, V, 3, 2, tau=tau, d_ff=d_ff)
+    assert np.all(np.isfinite(got))
+    assert G.rel_l2(got, want) <= 1e-2, G.rel_l2(got, want)
+
+
 @pytest.mark.parametrize("cond", [False, True])
 def test_hybrid_stack_against_the_oracle(G, cond):
     """Attention mixer in layers 0 and 3 of a 5-layer stack (period 3), bidirectional Mamba elsewhere."""
@@ -116,14 +149,15 @@ def test_hybrid_stack_against_the_oracle(G, cond):
     assert np.any(got != plain)
 
 
-def test_attention_block_step_with_cache(G):
+@pytest.mark.parametrize("dh", [64, 80])
+def test_attention_block_step_with_cache(G, dh):
     """Prefix of 200 tokens through the block entry point with an empty cache, then a block of 40 that attends to the cached
     prefix and to itself: outputs and cache contents against the oracle; rows past the valid keys of the cache hold NaN on
     purpose (the kernel must not let them in)."""
     from paper_2511_15927_b200 import binding as dm
     B, H, cap = 2, 2, 300
-    d = 64 * H
-    x, wq, wo = _case(B, 240, H, 31, 1.0)
+    d = dh * H
+    x, wq, wo = _case(B, 240, H, 31, 1.0, dh=dh)
     wqd, wod = G.dev(wq, I.BF16), G.dev(wo, I.BF16)
     kc = torch.full((B, cap, d), float("nan"), device="cuda", dtype=torch.bfloat16)
     vc = torch.full((B, cap, d), float("nan"), device="cuda", dtype=torch.bfloat16)
