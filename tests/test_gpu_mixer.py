@@ -74,6 +74,24 @@ def test_bf16_parity_small(G, dims):
     _check(got, O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape)), I.BF16)
 
 
+@pytest.mark.parametrize("B,L,d,H", [(1, 1500, 1024, 32), (3, 400, 512, 16), (2, 60, 256, 8)])
+def test_short_input_out_proj_paths_bf16(G, B, L, d, H):
+    """Up to 2048 tokens the two out_proj run as one launch into fp32 partials that one pass scales and sums: 1500 tokens at d_model 1024
+    fill the GPU with whole products (256 tiles), the two smaller cases cut each product in two along K (four partials)."""
+    shape = I.MixerShape(B, L, d, 2, 128, 4, H)
+    wf, wr, x = _case(shape, I.BF16, seed=9)
+    got = G.run_forward(shape, I.BF16, wf, wr, x)
+    _check(got, O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape)), I.BF16)
+    # without the gated norm the partials are summed unscaled
+    got0 = G.run_forward(shape, I.BF16, wf, wr, x, flags=dm_flags_no_norm())
+    _check(got0, O.bimamba_forward(x, wf, wr, **G.oracle_kwargs(shape, flags=dm_flags_no_norm())), I.BF16)
+
+
+def dm_flags_no_norm():
+    from paper_2511_15927_b200 import binding as dm
+    return dm.DM_FLAGS_DEFAULT & ~dm.DM_FLAG_GATED_RMSNORM
+
+
 def test_direction_masks_and_reversal_invariant(G):
     shape = I.MixerShape(2, 77, 64, 2, 16, 4, 4)
     wf, wr, x = _case(shape, I.F32, seed=5)
