@@ -4,6 +4,9 @@
 // Persistent kernel, one CTA per SM, CTA tile 128 x BN, K step 64.  Warp roles: warp 0 issues the TMA
 // loads, warp 1 owns TMEM and issues the MMAs, warps 2-5 drain the accumulator (double-buffered in
 // TMEM, so the epilogue of one tile overlaps the main loop of the next).
+// Tall tiles (MB = 2: 256 x 256, two 128-row accumulator blocks that share the B stage, all 512 TMEM columns as one buffer, eight
+// epilogue warps) are for few rows and many columns, where every CTA has one tile anyway: each weight tile is then fetched by
+// half as many CTAs, and what L2 delivers to the SMs is what bounds such a product.
 //
 // Every wait on an mbarrier is bounded by wall time; when one gives up the CTA raises an abort flag,
 // stores DM_ERR_TIMEOUT in the device status word, waits (bounded) for its own TMA loads, frees its
@@ -20,8 +23,8 @@ constexpr int BM = 128, BK = 64;
 constexpr int MAX_STAGES = 6;
 // pipeline depth: as many (A, B) stages as shared memory holds -- 4 x 48 KB with 256-column tiles, 6 x 32 KB with 128-column tiles (whose
 // lower arithmetic intensity needs more bytes in flight per MMA clock)
-__host__ __device__ constexpr int stages_for(int bn) { return bn == 128 ? 6 : 4; }
-constexpr int NUM_THREADS = 192;
+__host__ __device__ constexpr int stages_for(int bn, int mb) { return mb == 2 ? 3 : bn == 128 ? 6 : 4; }
+__host__ __device__ constexpr int threads_for(int mb) { return 64 + 128 * mb; }      // TMA warp, MMA warp, 4 epilogue warps per row block
 
 struct __align__(8) PipeBars {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
@@ -45,8 +48,8 @@ struct EpiArgs {
 // loop runs over both, so that they share one tail round and -- for in_proj, whose A operand is the same x -- the rows of A in L2.
 struct EpiPair { EpiArgs p[4]; int nprob; int ksplit; };
 
-template <int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int BN, int MB>
+__global__ void __launch_bounds__(threads_for(MB), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_b0,
                const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ EpiPair epp, int *status) {
@@ -54,26 +57,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte aligned base, derived by offsetting the __shared__ array so that accesses stay shared-space loads and stores
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    constexpr int STAGES = stages_for(BN);
-    constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    constexpr int STAGES = stages_for(BN, MB);
+    constexpr uint32_t A_BLOCK = BM * BK * 2, A_BYTES = MB * A_BLOCK, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    constexpr int NBUF = MB == 1 ? 2 : 1;            // accumulator buffers
     PipeBars *bars = reinterpret_cast<PipeBars *>(smem + STAGES * STAGE_BYTES);
     volatile int *abort_flag = &bars->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // rows to compute: all of them, or the count another kernel left on the device (tiles beyond it are skipped)
     const int M_eff = ep.m_dev ? min(ep.M, max(0, *ep.m_dev - ep.m_off)) : ep.M;
-    const int tiles_m = (M_eff + BM - 1) / BM, tiles_n = (ep.N + BN - 1) / BN;
+    const int tiles_m = (M_eff + MB * BM - 1) / (MB * BM), tiles_n = (ep.N + BN - 1) / BN;
     const int np = epp.nprob, tiles_np = tiles_n * np;         // the problems sit side by side along N
     const int num_tiles = tiles_m * tiles_np;
     // tile -> (row block, column block over both problems); the column block's problem is cb / tiles_n
     auto tile_mb = [&](int tile) { return ep.n_fast ? tile / tiles_np : tile % tiles_m; };
     auto tile_cb = [&](int tile) { return ep.n_fast ? tile % tiles_np : tile / tiles_m; };
     const int kblocks = (ep.K + BK - 1) / BK;
-    constexpr uint32_t TMEM_COLS = 2 * BN;          // two accumulator buffers; 256 or 512 columns
+    constexpr uint32_t TMEM_COLS = 2 * BN;          // two accumulator buffers, or the two row blocks of a tall tile; 256 or 512 columns
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bars->tmem_full[i], 1); mbar_init(&bars->tmem_empty[i], 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&bars->tmem_full[i], 1); mbar_init(&bars->tmem_empty[i], 4 * MB); }
         bars->abort = 0;
         mbar_fence_init();
     }
@@ -92,7 +96,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int cb = tile_cb(tile), prob = cb / tiles_n;
-                const int m0 = tile_mb(tile) * BM, n0 = (cb - prob * tiles_n) * BN;
+                const int m0 = tile_mb(tile) * MB * BM, n0 = (cb - prob * tiles_n) * BN;
                 const int prod = epp.ksplit ? prob >> 1 : prob, k_off = epp.p[prob].k_off;
                 const CUtensorMap *ma = prod ? &map_a1 : &map_a0, *mb = prod ? &map_b1 : &map_b0;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -100,7 +104,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     if (!(ok = mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, status))) break;
                     uint8_t *sa = smem + s * STAGE_BYTES, *sb = sa + A_BYTES;
                     mbar_expect_tx(&bars->full[s], STAGE_BYTES);
-                    tma_load_2d(sa, ma, k_off + kb * BK, m0, &bars->full[s]);
+#pragma unroll
+                    for (int i = 0; i < MB; ++i) tma_load_2d(sa + i * A_BLOCK, ma, k_off + kb * BK, m0 + i * BM, &bars->full[s]);
                     tma_load_2d(sb, mb, k_off + kb * BK, n0, &bars->full[s]);
                 }
             }
@@ -119,7 +124,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
-                const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
+                const uint32_t buf = NBUF == 2 ? tcount & 1u : 0u, bph = (NBUF == 2 ? tcount >> 1 : tcount) & 1u;
                 if (!(ok = mbar_wait(&bars->tmem_empty[buf], bph ^ 1u, abort_flag, status))) break;
                 fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
@@ -128,26 +133,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     if (!(ok = mbar_wait(&bars->full[s], ph, abort_flag, status))) break;
                     fence_after();
                     const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
-                    const uint64_t da = desc_k_sw128(sa), db = desc_k_sw128(sb);
+                    const uint64_t db = desc_k_sw128(sb);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)      // 32 bytes along K per MMA: +2 in 16-byte units
-                        umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    for (int i = 0; i < MB; ++i) {          // row block i accumulates into columns [i BN, (i + 1) BN)
+                        const uint64_t da = desc_k_sw128(sa + i * A_BLOCK);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)      // 32 bytes along K per MMA: +2 in 16-byte units
+                            umma_bf16(d_tmem + i * BN, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    }
                     umma_commit(&bars->empty[s]);          // frees the stage when these MMAs have read it
                 }
                 if (ok) umma_commit(&bars->tmem_full[buf]);
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue: 4 warps, one TMEM lane quarter each
+        // ------------------------------------------------------------ epilogue: 4 warps per row block, one TMEM lane quarter each
         const int q = warp & 3;                            // warps 2,3,4,5 -> quarters 2,3,0,1
+        const int rb = MB == 1 ? 0 : (warp - 2) >> 2;      // row block of a tall tile
         // 32-byte stores and loads (one full sector per thread) when every row of C / of the addend starts on a 32-byte boundary
         const int c_es = ep.c_is_f32 ? 4 : 2;
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
-            const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
+            const uint32_t buf = NBUF == 2 ? tcount & 1u : 0u, bph = (NBUF == 2 ? tcount >> 1 : tcount) & 1u;
             const int cb = tile_cb(tile), prob = cb / tiles_n;
-            const int m0 = tile_mb(tile) * BM, n0 = (cb - prob * tiles_n) * BN;
+            const int m0 = tile_mb(tile) * MB * BM + rb * BM, n0 = (cb - prob * tiles_n) * BN;
             const EpiArgs &ep = epp.p[prob];               // this tile's problem: its output, scales and addend
             const bool wide_c = (reinterpret_cast<uintptr_t>(ep.C) & 31u) == 0 && ((ep.ldc * c_es) & 31) == 0;
             const bool wide_add = ep.addend && (reinterpret_cast<uintptr_t>(ep.addend) & 31u) == 0 && ((ep.ld_add * 4) & 31) == 0;
@@ -162,7 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld_x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + c0, r);
+                tmem_ld_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (MB == 1 ? buf : rb) * BN + c0, r);
                 tmem_wait_ld();
                 const int col = n0 + c0;
                 if (!row_ok || col >= ep.N) continue;
@@ -294,14 +304,14 @@ EpiArgs epi_of(const GemmArgs &a) {
 
 // b == NULL: one product.  hi != NULL (two products, fp32 outputs): each product is cut in two along K; the first half goes to the
 // product's own C with its addend and bias, the second half to hi[i] (same pitch), scaled like the first (the scales are linear).
-template <int BN>
+template <int BN, int MB = 1>
 cudaError_t launch(const GemmArgs &a, const GemmArgs *b, float *const *hi, cudaStream_t s) {
     CUtensorMap ma[2], mb[2];
     if (!make_map(&ma[0], a.A, a.M, a.K, a.lda, BM) || !make_map(&mb[0], a.B, a.N, a.K, a.ldb, BN)) return cudaErrorInvalidValue;
     ma[1] = ma[0]; mb[1] = mb[0];
     if (b && (!make_map(&ma[1], b->A, b->M, b->K, b->lda, BM) || !make_map(&mb[1], b->B, b->N, b->K, b->ldb, BN))) return cudaErrorInvalidValue;
-    constexpr size_t smem = stages_for(BN) * (size_t)(BM * BK * 2 + BN * BK * 2) + sizeof(PipeBars) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    constexpr size_t smem = stages_for(BN, MB) * (size_t)(MB * BM * BK * 2 + BN * BK * 2) + sizeof(PipeBars) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int *status = device_status_ptr();
     if (!status) return cudaErrorUnknown;
@@ -321,9 +331,9 @@ cudaError_t launch(const GemmArgs &a, const GemmArgs *b, float *const *hi, cudaS
         epp.p[1] = b ? epi_of(*b) : epp.p[0];
         epp.nprob = b ? 2 : 1;
     }
-    const int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN) * epp.nprob;
+    const int tiles = ((a.M + MB * BM - 1) / (MB * BM)) * ((a.N + BN - 1) / BN) * epp.nprob;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    gemm_tc_kernel<BN><<<grid, NUM_THREADS, smem, s>>>(ma[0], mb[0], ma[1], mb[1], epp, status);
+    gemm_tc_kernel<BN, MB><<<grid, threads_for(MB), smem, s>>>(ma[0], mb[0], ma[1], mb[1], epp, status);
     count_launch();
     return cudaGetLastError();
 }
@@ -334,6 +344,13 @@ bool wide_tile(const GemmArgs &a, int nprob) {
     const int tm = (a.M + BM - 1) / BM, sms = sm_count();
     const int rounds128 = (tm * ((a.N + 127) / 128) * nprob + sms - 1) / sms, rounds256 = (tm * ((a.N + 255) / 256) * nprob + sms - 1) / sms;
     return !(a.N <= 128 || 10 * rounds128 <= 16 * rounds256);
+}
+
+// Tall tiles pay when the wide tiles would need a second, partly filled round of CTAs and the tall ones fit in one: every CTA then has
+// one tile either way, and the tall tile moves a third less operand data per product.
+bool tall_tile(const GemmArgs &a, int nprob) {
+    const int sms = sm_count(), cols = (a.N + 255) / 256;
+    return a.M > BM && !a.m_dev && ((a.M + BM - 1) / BM) * cols * nprob > sms && ((a.M + 2 * BM - 1) / (2 * BM)) * cols * nprob <= sms;
 }
 
 }  // namespace
@@ -352,6 +369,7 @@ bool gemm_tcgen05_supports(const GemmArgs &a) {
 
 cudaError_t gemm_tcgen05(const GemmArgs &a, cudaStream_t s) {
     if (!gemm_tcgen05_supports(a)) return cudaErrorNotSupported;
+    if (tall_tile(a, 1)) return launch<256, 2>(a, nullptr, nullptr, s);
     return wide_tile(a, 1) ? launch<256>(a, nullptr, nullptr, s) : launch<128>(a, nullptr, nullptr, s);
 }
 
@@ -362,6 +380,7 @@ bool gemm_tcgen05_pair_supports(const GemmArgs &a, const GemmArgs &b) {
 
 cudaError_t gemm_tcgen05_pair(const GemmArgs &a, const GemmArgs &b, cudaStream_t s) {
     if (!gemm_tcgen05_pair_supports(a, b)) return cudaErrorNotSupported;
+    if (tall_tile(a, 2)) return launch<256, 2>(a, &b, nullptr, s);
     return wide_tile(a, 2) ? launch<256>(a, &b, nullptr, s) : launch<128>(a, &b, nullptr, s);
 }
 

@@ -26,7 +26,9 @@ def _rand(shape, seed, dtype, scale=1.0):
 
 @pytest.mark.parametrize("dtype", [I.BF16, I.F32])
 @pytest.mark.parametrize("M,N,K", [(1, 8, 8), (300, 520, 200), (129, 257, 72), (1000, 1288, 256), (2048, 2048, 1024), (77, 100, 64),
-                                   (512, 50304 // 16, 128)])
+                                   (512, 50304 // 16, 128),
+                                   # few rows, many columns: two rounds of 128 x 256 tiles or one of 256 x 256 -- the tall tile (ragged rows and columns)
+                                   (300, 13000, 192), (512, 17024, 256), (130, 18000, 64)])
 def test_linear_parity(dm, dtype, M, N, K):
     from paper_2511_15927_b200.torch_io import dev, dm_dtype, tdtype
     x = _rand((M, K), 1, dtype); w = _rand((N, K), 2, dtype, 0.05)
@@ -45,9 +47,10 @@ def test_linear_parity(dm, dtype, M, N, K):
 
 
 @pytest.mark.parametrize("dtype", [I.BF16, I.F32])
-def test_linear_epilogue_scale_addend_inplace(dm, dtype):
+@pytest.mark.parametrize("shape", [(333, 300, 136), (300, 13000, 136)])
+def test_linear_epilogue_scale_addend_inplace(dm, dtype, shape):
     from paper_2511_15927_b200.torch_io import dev, dm_dtype
-    M, N, K = 333, 300, 136
+    M, N, K = shape                                         # the second shape takes the tall tile on the tensor-core path
     x = _rand((M, K), 3, dtype); w = _rand((N, K), 4, dtype, 0.05)
     sc = np.random.default_rng(5).uniform(0.5, 2.0, M).astype(np.float32)
     add = np.random.default_rng(6).standard_normal((M, N)).astype(np.float32)
