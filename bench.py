@@ -446,20 +446,24 @@ def run_stack(args, rank, local_rank, world):
         D.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        timed.launches0 = dm.dm_kernel_launch_count()
         e0.record()
         for i in range(n):
             fn(i)
         e1.record()
+        timed.launches = dm.dm_kernel_launch_count() - timed.launches0      # kernels enqueued inside the timed region
         D.barrier()
         torch.cuda.synchronize()
         return D.max_over_ranks(e0.elapsed_time(e1), "cuda")
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms_total = timed(step, args.steps)
+    launches = timed.launches
+    # per-stage times: the same steps once more with the library's stage events switched on (a step of a stack records some 150 of them, which
+    # costs a short-kernel workload a third of its time: they stay out of the region `value` is taken from)
     dm.dm_profile_enable(True)
     dm.dm_profile_read()
-    launches0 = dm.dm_kernel_launch_count()
-    ms_total = timed(step, args.steps)
-    launches = dm.dm_kernel_launch_count() - launches0
+    ms_staged = timed(step, args.steps) / args.steps
     stage_ms, stage_n = dm.dm_profile_read()          # includes the warm-up steps
     dm.dm_profile_enable(False)
     clocks = sampler.stop() if sampler else None
@@ -567,6 +571,7 @@ def run_stack(args, rank, local_rank, world):
             "dtype": "bf16", "data": "synthetic",
             "config": dict({"workload": args.workload, "batch": B, "seq_len": Lb, "d_model": shape.d_model, "d_state": shape.d_state,
                             "heads": shape.n_heads, "layers": layers, "vocab": vocab, "block": "AdaLN + mixer + MLP (d_ff %d, d_cond %d)" % (cond["d_ff"], cond["d_cond"]) if cond else "RMSNorm pre-norm + mixer", "tokens_per_s_whole_stack": world * T * npass / (ms_step * 1e-3),
+                            "ms_per_step_with_stage_events": ms_staged,
                             "parallelism": "replicas only" if world > 1 else "1 GPU",
                             "l2": "weights of 24 layers and the vocabulary projection exceed the 126 MB L2; token ids rotate over 4 buffers"},
                            **({"hybrid": "attention mixer (%d heads of %d) in every %dth layer, %d Mamba layers; the attention layers are inside rest_of_step_ms"
