@@ -179,9 +179,11 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 // `part` of chunk pc of (direction, batch row): QB rows of B' and C', PREP_HEADS of every 64 heads for the decays.
 // dsm: the group's [Q][PREP_HEADS + 1] floats.  Sb != NULL (short-block mode, with bct = the group's [2][QB][BCT_LD] words): the unit
 // also writes S[i][j] = C'_i . B'_j over its rows, fp32, to Sb[seq][pc * PREP_PARTS + part][QB][QB].
+// what: PREP_BC = the B', C' (and S) half of the unit, PREP_DECAY = its decays, or both.
+constexpr int PREP_BC = 1, PREP_DECAY = 2;
 __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA,
                                           float *__restrict__ Sb, int dir, int b, int pc, int part, int tid, int bar, float *dsm,
-                                          uint32_t (*bct)[QB][BCT_LD]) {
+                                          uint32_t (*bct)[QB][BCT_LD], int what) {
     const bool rev = dir == 1;
     const int L = a.L, k = a.k;
     const ScanDir &w = a.dir[dir];
@@ -191,7 +193,9 @@ __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__res
     const bool has_bias = (a.flags & DM_FLAG_CONV_BIAS) && w.conv_b;
 
     // ---- B and C channels: thread = channel pair, over this unit's block of 32 rows; the 35-row window is loaded up front
-    {
+    // (a block past the end of the sequence has nothing to write and nobody reads its S)
+    const bool bc_live = (what & PREP_BC) && r0 + part * 32 < L;
+    if (bc_live) {
         const int cp = tid, rg = part;
         const bool isC = cp >= N / 2;
         const int pi = cp & (N / 2 - 1);                                 // pair index inside B or C
@@ -229,7 +233,7 @@ __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__res
             if (Sb) bct[isC ? 1 : 0][rev ? QB - 1 - i : i][pi] = pk;          // row of the tile = physical row inside the block
         }
     }
-    if (Sb) {
+    if (Sb && bc_live) {
         // S = C' B'^T of this block's 32 rows on the legacy tensor path: warp = 16 rows i x 16 columns j, K = d_state
         named_sync(bar, PREP_THREADS);
         const int warp = tid >> 5, lane = tid & 31;
@@ -256,6 +260,7 @@ __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__res
         }
     }
     // ---- Delta, then the inclusive cumulative log-decay of every head in the direction's time order
+    if (!(what & PREP_DECAY)) return;
     for (int h0 = 0; h0 < a.H; h0 += 64) {
         named_sync(bar, PREP_THREADS);
 #pragma unroll 4
@@ -272,14 +277,18 @@ __device__ __forceinline__ void prep_unit(const SsdArgs &a, __nv_bfloat16 *__res
     }
 }
 
-// grid.x covers the chunks the direction visits first: blockIdx.x / PREP_PARTS is the chunk's index in time order
+// grid.x covers the chunks the direction visits first: blockIdx.x / PREP_PARTS is the chunk's index in time order.  With split set (short
+// blocks, where the launch is a handful of CTAs and its latency is what counts) grid.x is twice that: the first half of the CTAs take the
+// B', C', S halves of the units, the second half their decays.
 __global__ void __launch_bounds__(PREP_THREADS)
 ssd_prep_kernel(const SsdArgs a, __nv_bfloat16 *__restrict__ Bp, __nv_bfloat16 *__restrict__ Cp, float *__restrict__ dA, float *__restrict__ Sb,
-                int dir0) {
+                int dir0, int split) {
     __shared__ float dsm[Q * (PREP_HEADS + 1)];
     __shared__ __align__(16) uint32_t bct[2][QB][BCT_LD];     // short-block mode: this CTA's rows of B' ([0]) and C' ([1]) as bf16 pairs
-    const int dir = dir0 + blockIdx.z, c = blockIdx.x / PREP_PARTS;
-    prep_unit(a, Bp, Cp, dA, Sb, dir, blockIdx.y, dir == 1 ? a.nch - 1 - c : c, blockIdx.x % PREP_PARTS, threadIdx.x, 0, dsm, bct);
+    const int units = split ? gridDim.x / 2 : gridDim.x, u = blockIdx.x % units;
+    const int what = !split ? (PREP_BC | PREP_DECAY) : blockIdx.x < units ? PREP_BC : PREP_DECAY;
+    const int dir = dir0 + blockIdx.z, c = u / PREP_PARTS;
+    prep_unit(a, Bp, Cp, dA, Sb, dir, blockIdx.y, dir == 1 ? a.nch - 1 - c : c, u % PREP_PARTS, threadIdx.x, 0, dsm, bct, what);
 }
 
 // --------------------------------------------------------------------------------------------------
@@ -1364,7 +1373,7 @@ cudaError_t scan_ssd(const ScanArgs &a, void *ws, cudaStream_t s) {
     if (pj.sync && g_withhold_prep) pj.nprep = 0;
     cudaError_t e;
     if (pj.sync && (e = cudaMemsetAsync(pj.sync, 0, ((size_t)2 * a.B * l.nch + 1) * sizeof(int), s)) != cudaSuccess) return e;
-    ssd_prep_kernel<<<dim3(n_pre * PREP_PARTS, a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0);
+    ssd_prep_kernel<<<dim3(n_pre * PREP_PARTS * (blk ? 2 : 1), a.B, ndir), PREP_THREADS, 0, s>>>(k, Bp, Cp, dA, Sb, dir0, blk ? 1 : 0);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (blk) {
